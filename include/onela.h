@@ -1,0 +1,172 @@
+/*
+ * onela.h - C ABI of the beam-shared Gated DeltaNet (GDN) decode library for NVIDIA B200 (sm_100a).
+ *
+ * The library holds, for every request, ONE post-prefill recurrent state S_0 per (layer, head)
+ * ("stores S_ctx only once", paper Section 3.2), an append-only arena of per-token transition
+ * records, and an ancestry index that maps every live beam to the records on its lineage
+ * (Section 3.3, Eq. 5).  A decode call evaluates the GDN output of Eq. 1,
+ *
+ *        S_t = alpha_t S_{t-1} + beta_t (v_t - alpha_t S_{t-1} k_t) k_t^T ,    o_t = S_t q_t ,
+ *
+ * for every (beam, head) WITHOUT materialising any per-beam state: with
+ * A_j = alpha_j (I - beta_j k_j k_j^T), Eq. 1 reads S_j = S_{j-1} A_j + beta_j v_j k_j^T, hence for any r
+ * S_j r = S_{j-1} (A_j r) + beta_j (k_j . r) v_j.  Folding the query through the beam's records from
+ * the newest to the oldest,
+ *        r <- q ;   for j = t ... 0:   c = k_j . r ;  corr += beta_j c v_j ;  r <- alpha_j (r - beta_j c k_j) ,
+ * gives o = S_0 r + corr, so all beams of a request meet S_0 in one dense [dv x dk] . [dk x W]
+ * contraction per head.  (This is the adjoint of the paper's forward projection replay, Eq. 3-4;
+ * the record kept here is the raw token (k, v, alpha, beta) rather than (alpha, delta, k).)
+ *
+ * Conventions
+ *  - Every pointer whose name ends in _dev is DEVICE memory owned by the caller; *_host is host memory.
+ *    The library allocates no device memory: the caller passes one workspace of
+ *    onela_workspace_bytes() bytes (1024-byte aligned) at onela_create(); the library carves it into the
+ *    S_0 store, the record arena, the ancestry tables and a status word.  The context itself is a small
+ *    host object released by onela_destroy(), which never touches the workspace.
+ *  - `stream` is a cudaStream_t passed as void*.  Every call is asynchronous and ordered on that
+ *    stream; inputs may be reused as soon as the stream has passed the call.  Only
+ *    onela_poll_device_status() synchronises.
+ *  - Tensors are dense, row-major, last index contiguous.  q, k, v use cfg.rec_dtype, outputs
+ *    cfg.out_dtype, gates and S_0 are fp32.  All tensor pointers must be 16-byte aligned.
+ *  - Errors the host can see return a negative status and launch nothing.  Errors only the device can
+ *    see (a parent index outside the previous beam) set a sticky status word, the offending index is
+ *    clamped to 0, and nothing traps.
+ *  - Call order per request:  init/prefill_shared_state for each layer used (restarts the request at
+ *    depth 0)  ->  repeat {  reorder_beams (once per decode call; shared by all layers and heads)  ->
+ *    per layer { append_records exactly once  ->  decode_step any number of times } }.
+ *    Violations return ONELA_E_ORDER.
+ *  - Slot numbering: one bump cursor per context.  reorder_beams over requests [b, b+n) assigns, in
+ *    request order, base(req, t) = cursor, cursor += W_new.  The record of beam i at decode call t lives
+ *    at global slot base(req, t) + i in every layer ("written once to the physical slots of the current
+ *    decoding step and never relocated", Section 3.3).
+ *  - Batched calls (req_count > 1) need the same beam width and depth on every request of the batch,
+ *    and at most ONELA_MAX_BATCH requests.
+ */
+#ifndef ONELA_H
+#define ONELA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct onela_ctx onela_ctx;
+typedef int32_t onela_status;
+
+#define ONELA_OK 0
+#define ONELA_E_INVAL (-1)        /* null / shape / dtype / alignment / range */
+#define ONELA_E_CAPACITY (-2)     /* arena, max_steps or max_beam exhausted */
+#define ONELA_E_ORDER (-3)        /* call sequence violated */
+#define ONELA_E_CUDA (-4)         /* a CUDA runtime call or launch failed */
+#define ONELA_E_UNSUPPORTED (-5)  /* (dk, dv, dtype) combination not compiled */
+#define ONELA_E_DEVICE_CHECK (-6) /* the device found a bad parent index (sticky) */
+#define ONELA_E_TIMEOUT (-7)      /* a bounded device-side wait expired (sticky) */
+
+#define ONELA_DTYPE_F32 0
+#define ONELA_DTYPE_BF16 1
+
+#define ONELA_MAX_BATCH 64
+
+/* flags */
+#define ONELA_FLAG_DRY_RUN 1u       /* validate and advance host bookkeeping, launch nothing (host-logic tests) */
+#define ONELA_FLAG_FORCE_GENERIC 2u /* use the CUDA-core decode kernel even where the tensor-core kernel applies */
+
+typedef struct onela_config {
+    int32_t num_requests; /* request slots */
+    int32_t num_layers;   /* GDN layers sharing the ancestry index */
+    int32_t num_heads;    /* key heads == value heads */
+    int32_t dk, dv;       /* head dimensions of k/q and of v/o */
+    int32_t max_beam;     /* largest beam width W_t */
+    int32_t max_steps;    /* largest number of decode calls per request (chain depth) */
+    int32_t rec_dtype;    /* dtype of q, k, v: ONELA_DTYPE_* */
+    int32_t out_dtype;    /* dtype of o */
+    int64_t arena_slots;  /* record slots per layer, shared by all requests (< 2^31) */
+    uint32_t flags;
+} onela_config;
+
+/* Bytes of device workspace the configuration needs; 0 if the configuration is invalid. */
+size_t onela_workspace_bytes(const onela_config* cfg);
+
+/* Build a context over a caller-owned workspace (device pointer, 1024-byte aligned, at least
+ * onela_workspace_bytes(cfg) bytes).  Pure host work: nothing is launched; the first call that takes
+ * a stream clears the status word on that stream.  The workspace must outlive the context. */
+onela_status onela_create(const onela_config* cfg, void* workspace_dev, size_t workspace_bytes, onela_ctx** out);
+onela_status onela_destroy(onela_ctx* ctx);
+
+/* Forget every request and rewind the arena cursor to 0 (records are never reclaimed one by one:
+ * the arena is append-only, Section 3.3). */
+onela_status onela_reset(onela_ctx* ctx, void* stream);
+
+/* Shared-state store (Section 3.2: the post-prefill state S_ctx is stored once per request).
+ * Copies S0_dev [num_heads][dv][dk] fp32 into the store slot of (request, layer); the caller may free
+ * S0_dev once the stream has passed the call.  Restarts the request at depth 0 if it had decoded. */
+onela_status onela_init_shared_state(onela_ctx* ctx, int32_t request, int32_t layer, const float* S0_dev,
+                                     void* stream);
+
+/* Same store slot, filled by running Eq. 1 from the zero state over n_tokens prompt tokens in fp32:
+ * k_dev [n_tokens][H][dk], v_dev [n_tokens][H][dv] in rec_dtype, alpha_dev, beta_dev [n_tokens][H] fp32. */
+onela_status onela_prefill_shared_state(onela_ctx* ctx, int32_t request, int32_t layer, const void* k_dev,
+                                        const void* v_dev, const float* alpha_dev, const float* beta_dev,
+                                        int32_t n_tokens, void* stream);
+
+/* Read the store slot of (request, layer) back as S0_out_dev [num_heads][dv][dk] fp32 row-major (the
+ * values the decode kernels consume: identical to what was stored, except that the tensor-core path
+ * keeps S_0 rounded to TF32, 10 mantissa bits). */
+onela_status onela_export_shared_state(onela_ctx* ctx, int32_t request, int32_t layer, float* S0_out_dev,
+                                       void* stream);
+
+/* Ancestry index update, Eq. 5 (Section 3.3): open decode call t for requests
+ * [req_begin, req_begin+req_count) with W_new beams each.  parents_dev [req_count][W_new] int32 gives
+ * pi_t(b), the parent of beam b in the previous beam; it must be NULL exactly when the requests are
+ * at depth 0 (every beam's parent is S_0).  Writes indices only: new row b = parent's row, plus the
+ * slot base(req, t) + b of the record about to be appended.  No record is moved or copied. */
+onela_status onela_reorder_beams(onela_ctx* ctx, int32_t req_begin, int32_t req_count, const int32_t* parents_dev,
+                                 int32_t W_new, void* stream);
+
+/* Append this call's transition records for one layer ("appends only the compact record ... rather
+ * than writing back a full recurrent state", Section 3.4): k_dev [req_count][W][H][dk],
+ * v_dev [req_count][W][H][dv] in rec_dtype, alpha_dev, beta_dev [req_count][W][H] fp32.  Values are
+ * stored bit-exactly and never modified afterwards. */
+onela_status onela_append_records(onela_ctx* ctx, int32_t req_begin, int32_t req_count, int32_t layer,
+                                  const void* k_dev, const void* v_dev, const float* alpha_dev,
+                                  const float* beta_dev, void* stream);
+
+/* Fused decode (Eq. 1 output through the backward fold described at the top): q_dev
+ * [req_count][W][H][dk] in rec_dtype -> out_dev [req_count][W][H][dv] in out_dtype.  The chain of a beam
+ * includes the record appended in this call (o_t reads the UPDATED state, Eq. 1). */
+onela_status onela_decode_step(onela_ctx* ctx, int32_t req_begin, int32_t req_count, int32_t layer,
+                               const void* q_dev, void* out_dev, void* stream);
+
+/* Copy the ancestry rows of one request to slots_dev [W][depth] int32 (global slot ids, oldest first;
+ * the last column is the beam's own record).  depth_host / width_host (host pointers, may be NULL)
+ * receive the shape immediately. */
+onela_status onela_export_chains(onela_ctx* ctx, int32_t request, int32_t* slots_dev, int32_t* depth_host,
+                                 int32_t* width_host, void* stream);
+
+/* Synchronise the device and read the sticky status word: *code_host is ONELA_OK,
+ * ONELA_E_DEVICE_CHECK or ONELA_E_TIMEOUT; *detail_host the offending value.  Clears the word. */
+onela_status onela_poll_device_status(onela_ctx* ctx, int32_t* code_host, int32_t* detail_host);
+
+/* Resident bytes (host bookkeeping; Section 4.4 reports the same three quantities): the stored S_0
+ * matrices, the records appended so far (slots * heads * record bytes * layers), and the live
+ * ancestry rows. */
+onela_status onela_get_stats(const onela_ctx* ctx, int64_t* s0_bytes_host, int64_t* arena_bytes_used_host,
+                             int64_t* index_bytes_host);
+
+/* First global slot of the records request `request` appended at decode call `step` (host bookkeeping). */
+onela_status onela_get_step_base(const onela_ctx* ctx, int32_t request, int32_t step, int32_t* base_host);
+
+/* Kernels this context has launched since creation (host counter; for launch accounting). */
+int64_t onela_launch_count(const onela_ctx* ctx);
+
+/* 1 if decode_step of this context runs the tcgen05 tensor-core kernel, 0 if the CUDA-core kernel. */
+int32_t onela_uses_tensor_core_path(const onela_ctx* ctx);
+
+const char* onela_status_string(onela_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ONELA_H */

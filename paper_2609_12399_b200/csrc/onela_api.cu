@@ -1,0 +1,420 @@
+// Host side of the C ABI: context, workspace carve-up, per-request state machine, slot allocation and
+// kernel dispatch.  No device memory is allocated here; every launch goes to the caller's stream.
+#include <algorithm>
+#include <new>
+#include <vector>
+
+#include "onela_internal.h"
+
+using namespace onela;
+
+namespace {
+
+constexpr size_t kAlign = 1024;
+size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct ReqState {
+    int32_t depth = 0;  // decode calls opened so far (reorder_beams calls since the last restart)
+    int32_t W = 0;      // beam width of the current call
+    std::vector<uint8_t> has_state;      // per layer: S_0 stored
+    std::vector<int32_t> appended_depth; // per layer: depth at which records were last appended
+    std::vector<int32_t> step_base;      // per decode call: first slot
+    std::vector<int32_t> step_width;     // per decode call: beam width
+};
+
+bool config_sane(const onela_config* c) {
+    if (!c) return false;
+    if (c->num_requests < 1 || c->num_layers < 1 || c->num_heads < 1) return false;
+    if (c->dk < 1 || c->dv < 1 || c->max_beam < 1 || c->max_steps < 1) return false;
+    if ((c->rec_dtype != ONELA_DTYPE_F32 && c->rec_dtype != ONELA_DTYPE_BF16) ||
+        (c->out_dtype != ONELA_DTYPE_F32 && c->out_dtype != ONELA_DTYPE_BF16))
+        return false;
+    if (c->arena_slots < 1 || c->arena_slots > 0x7fffffffLL - c->max_beam) return false;
+    const int es = c->rec_dtype == ONELA_DTYPE_BF16 ? 2 : 4;
+    if ((c->dk * es) % 16 != 0 || (c->dv * es) % 16 != 0) return false;  // 16-byte vector rows
+    return true;
+}
+
+// Carve the workspace.  `base` may be null (size query only).
+Layout carve(const onela_config& c, char* base) {
+    const size_t es = c.rec_dtype == ONELA_DTYPE_BF16 ? 2 : 4;
+    size_t off = 0;
+    Layout l{};
+    auto take = [&](size_t bytes) {
+        char* p = base ? base + off : nullptr;
+        off += align_up(bytes);
+        return p;
+    };
+    l.status = reinterpret_cast<int32_t*>(take(4 * sizeof(int32_t)));
+    l.tables = reinterpret_cast<int32_t*>(take((size_t)c.num_requests * 2 * c.max_steps * c.max_beam * sizeof(int32_t)));
+    l.s0 = reinterpret_cast<float*>(take((size_t)c.num_requests * c.num_layers * c.num_heads * c.dv * c.dk * sizeof(float)));
+    l.gates = reinterpret_cast<float2*>(take((size_t)c.num_layers * c.num_heads * (size_t)c.arena_slots * sizeof(float2)));
+    l.kv = take((size_t)c.num_layers * c.num_heads * (size_t)c.arena_slots * (c.dk + c.dv) * es);
+    l.total_bytes = off;
+    return l;
+}
+
+}  // namespace
+
+struct onela_ctx {
+    onela_config cfg;
+    Layout lay;
+    std::vector<ReqState> req;
+    int64_t cursor = 0;        // next free arena slot
+    int64_t launches = 0;
+    bool status_cleared = false;
+    bool tensor_core = false;  // decode_step runs the tcgen05 kernel; S_0 is stored as its operand image
+    int32_t elem_bytes = 4;
+
+    bool dry() const { return cfg.flags & ONELA_FLAG_DRY_RUN; }
+    long long table_req_stride() const { return 2LL * cfg.max_steps * cfg.max_beam; }
+    long long s0_layer_floats() const { return (long long)cfg.num_heads * cfg.dv * cfg.dk; }
+    float* s0_slot(int r, int l) const { return lay.s0 + ((long long)r * cfg.num_layers + l) * s0_layer_floats(); }
+    int32_t* table_cur(int r) const {
+        const int d = req[r].depth;
+        return lay.tables + r * table_req_stride() + (long long)((d - 1) & 1) * cfg.max_steps * cfg.max_beam;
+    }
+    size_t plane_rows() const { return (size_t)cfg.num_heads * (size_t)cfg.arena_slots; }
+    char* kv_plane(int l) const { return lay.kv + (size_t)l * plane_rows() * (cfg.dk + cfg.dv) * elem_bytes; }
+    float2* gate_plane(int l) const { return lay.gates + (size_t)l * plane_rows(); }
+
+    onela_status prepare(cudaStream_t s) {
+        if (dry() || status_cleared) return ONELA_OK;
+        if (cudaMemsetAsync(lay.status, 0, 4 * sizeof(int32_t), s) != cudaSuccess) return ONELA_E_CUDA;
+        status_cleared = true;
+        return ONELA_OK;
+    }
+    void restart(ReqState& r) {
+        r.depth = 0;
+        r.W = 0;
+        std::fill(r.appended_depth.begin(), r.appended_depth.end(), -1);
+        r.step_base.clear();
+        r.step_width.clear();
+    }
+};
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+// Requests of a batched call must exist and share beam width and depth.
+onela_status check_batch(const onela_ctx* ctx, int32_t req_begin, int32_t req_count) {
+    if (!ctx) return ONELA_E_INVAL;
+    if (req_count < 1 || req_count > ONELA_MAX_BATCH || req_begin < 0 ||
+        (int64_t)req_begin + req_count > ctx->cfg.num_requests)
+        return ONELA_E_INVAL;
+    const ReqState& r0 = ctx->req[req_begin];
+    for (int i = 1; i < req_count; ++i) {
+        const ReqState& r = ctx->req[req_begin + i];
+        if (r.depth != r0.depth || r.W != r0.W) return ONELA_E_INVAL;
+    }
+    return ONELA_OK;
+}
+
+onela_status begin_state_write(onela_ctx* ctx, int32_t request, int32_t layer) {
+    if (!ctx || request < 0 || request >= ctx->cfg.num_requests || layer < 0 || layer >= ctx->cfg.num_layers)
+        return ONELA_E_INVAL;
+    return ONELA_OK;
+}
+
+void finish_state_write(onela_ctx* ctx, int32_t request, int32_t layer) {
+    ReqState& r = ctx->req[request];
+    if (r.depth > 0) {  // a new prompt in this request slot: forget the old beams and every layer's state
+        ctx->restart(r);
+        std::fill(r.has_state.begin(), r.has_state.end(), 0);
+    }
+    r.has_state[layer] = 1;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t onela_workspace_bytes(const onela_config* cfg) {
+    if (!config_sane(cfg)) return 0;
+    return carve(*cfg, nullptr).total_bytes;
+}
+
+onela_status onela_create(const onela_config* cfg, void* workspace_dev, size_t workspace_bytes, onela_ctx** out) {
+    if (!out) return ONELA_E_INVAL;
+    *out = nullptr;
+    if (!config_sane(cfg) || !workspace_dev) return ONELA_E_INVAL;
+    if (reinterpret_cast<uintptr_t>(workspace_dev) % kAlign != 0) return ONELA_E_INVAL;
+    if (!decode_generic_supported(cfg->dk, cfg->dv, cfg->rec_dtype)) return ONELA_E_UNSUPPORTED;
+    const Layout lay = carve(*cfg, static_cast<char*>(workspace_dev));
+    if (workspace_bytes < lay.total_bytes) return ONELA_E_CAPACITY;
+    onela_ctx* ctx = new (std::nothrow) onela_ctx();
+    if (!ctx) return ONELA_E_INVAL;
+    ctx->cfg = *cfg;
+    ctx->lay = lay;
+    ctx->elem_bytes = cfg->rec_dtype == ONELA_DTYPE_BF16 ? 2 : 4;
+    ctx->req.resize(cfg->num_requests);
+    for (auto& r : ctx->req) {
+        r.has_state.assign(cfg->num_layers, 0);
+        r.appended_depth.assign(cfg->num_layers, -1);
+    }
+    ctx->tensor_core = false;
+    *out = ctx;
+    return ONELA_OK;
+}
+
+onela_status onela_destroy(onela_ctx* ctx) {
+    delete ctx;
+    return ONELA_OK;
+}
+
+onela_status onela_reset(onela_ctx* ctx, void* stream) {
+    if (!ctx) return ONELA_E_INVAL;
+    for (auto& r : ctx->req) {
+        ctx->restart(r);
+        std::fill(r.has_state.begin(), r.has_state.end(), 0);
+    }
+    ctx->cursor = 0;
+    ctx->status_cleared = false;
+    return ctx->prepare(static_cast<cudaStream_t>(stream));
+}
+
+onela_status onela_init_shared_state(onela_ctx* ctx, int32_t request, int32_t layer, const float* S0_dev,
+                                     void* stream) {
+    onela_status st = begin_state_write(ctx, request, layer);
+    if (st != ONELA_OK) return st;
+    if (!S0_dev || !aligned16(S0_dev)) return ONELA_E_INVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if ((st = ctx->prepare(s)) != ONELA_OK) return st;
+    if (!ctx->dry()) {
+        if (launch_store_state(S0_dev, ctx->s0_slot(request, layer), ctx->cfg.num_heads, ctx->cfg.dk, ctx->cfg.dv,
+                               ctx->tensor_core, s) != cudaSuccess)
+            return ONELA_E_CUDA;
+        ctx->launches++;
+    }
+    finish_state_write(ctx, request, layer);
+    return ONELA_OK;
+}
+
+onela_status onela_prefill_shared_state(onela_ctx* ctx, int32_t request, int32_t layer, const void* k_dev,
+                                        const void* v_dev, const float* alpha_dev, const float* beta_dev,
+                                        int32_t n_tokens, void* stream) {
+    onela_status st = begin_state_write(ctx, request, layer);
+    if (st != ONELA_OK) return st;
+    if (n_tokens < 0) return ONELA_E_INVAL;
+    if (n_tokens > 0 && (!k_dev || !v_dev || !alpha_dev || !beta_dev || !aligned16(k_dev) || !aligned16(v_dev)))
+        return ONELA_E_INVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if ((st = ctx->prepare(s)) != ONELA_OK) return st;
+    if (!ctx->dry()) {
+        bool supported = true;
+        const cudaError_t e = launch_prefill(k_dev, v_dev, alpha_dev, beta_dev, ctx->s0_slot(request, layer), n_tokens,
+                                             ctx->cfg.num_heads, ctx->cfg.dk, ctx->cfg.dv, ctx->cfg.rec_dtype,
+                                             ctx->tensor_core, &supported, s);
+        if (!supported) return ONELA_E_UNSUPPORTED;
+        if (e != cudaSuccess) return ONELA_E_CUDA;
+        ctx->launches++;
+    }
+    finish_state_write(ctx, request, layer);
+    return ONELA_OK;
+}
+
+onela_status onela_export_shared_state(onela_ctx* ctx, int32_t request, int32_t layer, float* S0_out_dev,
+                                       void* stream) {
+    onela_status st = begin_state_write(ctx, request, layer);
+    if (st != ONELA_OK) return st;
+    if (!S0_out_dev || !aligned16(S0_out_dev)) return ONELA_E_INVAL;
+    if (!ctx->req[request].has_state[layer]) return ONELA_E_ORDER;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if ((st = ctx->prepare(s)) != ONELA_OK) return st;
+    if (ctx->dry()) return ONELA_OK;
+    if (launch_export_state(ctx->s0_slot(request, layer), S0_out_dev, ctx->cfg.num_heads, ctx->cfg.dk, ctx->cfg.dv,
+                            ctx->tensor_core, s) != cudaSuccess)
+        return ONELA_E_CUDA;
+    ctx->launches++;
+    return ONELA_OK;
+}
+
+onela_status onela_reorder_beams(onela_ctx* ctx, int32_t req_begin, int32_t req_count, const int32_t* parents_dev,
+                                 int32_t W_new, void* stream) {
+    onela_status st = check_batch(ctx, req_begin, req_count);
+    if (st != ONELA_OK) return st;
+    const onela_config& c = ctx->cfg;
+    if (W_new < 1) return ONELA_E_INVAL;
+    if (W_new > c.max_beam) return ONELA_E_CAPACITY;
+    const int32_t depth_old = ctx->req[req_begin].depth, W_prev = ctx->req[req_begin].W;
+    if ((depth_old == 0) != (parents_dev == nullptr)) return ONELA_E_ORDER;
+    for (int i = 0; i < req_count; ++i) {
+        const ReqState& r = ctx->req[req_begin + i];
+        bool any_state = false;
+        for (uint8_t hs : r.has_state) any_state |= hs != 0;
+        if (!any_state) return ONELA_E_ORDER;  // no shared state stored for this request yet
+        // the previous call must have appended its records in every layer that holds a state
+        if (depth_old > 0)
+            for (int l = 0; l < c.num_layers; ++l)
+                if (r.has_state[l] && r.appended_depth[l] != depth_old) return ONELA_E_ORDER;
+    }
+    if (depth_old >= c.max_steps) return ONELA_E_CAPACITY;
+    if (ctx->cursor + (int64_t)req_count * W_new > c.arena_slots) return ONELA_E_CAPACITY;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if ((st = ctx->prepare(s)) != ONELA_OK) return st;
+    BatchBases bases{};
+    for (int i = 0; i < req_count; ++i) bases.base[i] = (int32_t)(ctx->cursor + (int64_t)i * W_new);
+    if (!ctx->dry()) {
+        if (launch_reorder(ctx->lay.tables + req_begin * ctx->table_req_stride(), ctx->table_req_stride(), req_count,
+                           parents_dev, W_new, W_prev, depth_old, c.max_beam, c.max_steps, bases, ctx->lay.status,
+                           s) != cudaSuccess)
+            return ONELA_E_CUDA;
+        ctx->launches++;
+    }
+    for (int i = 0; i < req_count; ++i) {
+        ReqState& r = ctx->req[req_begin + i];
+        r.depth = depth_old + 1;
+        r.W = W_new;
+        r.step_base.push_back(bases.base[i]);
+        r.step_width.push_back(W_new);
+    }
+    ctx->cursor += (int64_t)req_count * W_new;
+    return ONELA_OK;
+}
+
+onela_status onela_append_records(onela_ctx* ctx, int32_t req_begin, int32_t req_count, int32_t layer,
+                                  const void* k_dev, const void* v_dev, const float* alpha_dev,
+                                  const float* beta_dev, void* stream) {
+    onela_status st = check_batch(ctx, req_begin, req_count);
+    if (st != ONELA_OK) return st;
+    const onela_config& c = ctx->cfg;
+    if (layer < 0 || layer >= c.num_layers) return ONELA_E_INVAL;
+    if (!k_dev || !v_dev || !alpha_dev || !beta_dev || !aligned16(k_dev) || !aligned16(v_dev)) return ONELA_E_INVAL;
+    const int32_t depth = ctx->req[req_begin].depth, W = ctx->req[req_begin].W;
+    if (depth < 1) return ONELA_E_ORDER;
+    for (int i = 0; i < req_count; ++i) {
+        const ReqState& r = ctx->req[req_begin + i];
+        if (!r.has_state[layer] || r.appended_depth[layer] == depth) return ONELA_E_ORDER;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if ((st = ctx->prepare(s)) != ONELA_OK) return st;
+    BatchBases bases{};
+    for (int i = 0; i < req_count; ++i) bases.base[i] = ctx->req[req_begin + i].step_base.back();
+    if (!ctx->dry()) {
+        if (launch_append(k_dev, v_dev, alpha_dev, beta_dev, ctx->kv_plane(layer), ctx->gate_plane(layer),
+                          c.arena_slots, req_count, W, c.num_heads, c.dk, c.dv, ctx->elem_bytes, bases,
+                          s) != cudaSuccess)
+            return ONELA_E_CUDA;
+        ctx->launches++;
+    }
+    for (int i = 0; i < req_count; ++i) ctx->req[req_begin + i].appended_depth[layer] = depth;
+    return ONELA_OK;
+}
+
+onela_status onela_decode_step(onela_ctx* ctx, int32_t req_begin, int32_t req_count, int32_t layer,
+                               const void* q_dev, void* out_dev, void* stream) {
+    onela_status st = check_batch(ctx, req_begin, req_count);
+    if (st != ONELA_OK) return st;
+    const onela_config& c = ctx->cfg;
+    if (layer < 0 || layer >= c.num_layers) return ONELA_E_INVAL;
+    if (!q_dev || !out_dev || !aligned16(q_dev) || !aligned16(out_dev)) return ONELA_E_INVAL;
+    const int32_t depth = ctx->req[req_begin].depth, W = ctx->req[req_begin].W;
+    if (depth < 1) return ONELA_E_ORDER;
+    for (int i = 0; i < req_count; ++i) {
+        const ReqState& r = ctx->req[req_begin + i];
+        if (!r.has_state[layer] || r.appended_depth[layer] != depth) return ONELA_E_ORDER;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if ((st = ctx->prepare(s)) != ONELA_OK) return st;
+    if (ctx->dry()) return ONELA_OK;
+    DecodeArgs a{};
+    a.q = q_dev;
+    a.out = out_dev;
+    a.s0 = ctx->s0_slot(req_begin, layer);
+    a.kv = ctx->kv_plane(layer);
+    a.gates = ctx->gate_plane(layer);
+    a.table = ctx->table_cur(req_begin);
+    a.status = ctx->lay.status;
+    a.s0_req_stride = (long long)c.num_layers * ctx->s0_layer_floats();
+    a.table_req_stride = ctx->table_req_stride();
+    a.arena_slots = c.arena_slots;
+    a.req_count = req_count;
+    a.W = W;
+    a.H = c.num_heads;
+    a.depth = depth;
+    a.max_beam = c.max_beam;
+    a.s0_swizzled = ctx->tensor_core;
+    for (int i = 0; i < req_count; ++i) a.bases.base[i] = ctx->req[req_begin + i].step_base.back();
+    bool supported = true;
+    const cudaError_t e = launch_decode_generic(a, c.dk, c.dv, c.rec_dtype, c.out_dtype, &supported, s);
+    if (!supported) return ONELA_E_UNSUPPORTED;
+    if (e != cudaSuccess) return ONELA_E_CUDA;
+    ctx->launches++;
+    return ONELA_OK;
+}
+
+onela_status onela_export_chains(onela_ctx* ctx, int32_t request, int32_t* slots_dev, int32_t* depth_host,
+                                 int32_t* width_host, void* stream) {
+    if (!ctx || request < 0 || request >= ctx->cfg.num_requests) return ONELA_E_INVAL;
+    const ReqState& r = ctx->req[request];
+    if (depth_host) *depth_host = r.depth;
+    if (width_host) *width_host = r.W;
+    if (r.depth < 1) return ONELA_E_ORDER;
+    if (!slots_dev) return ONELA_E_INVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    onela_status st = ctx->prepare(s);
+    if (st != ONELA_OK) return st;
+    if (ctx->dry()) return ONELA_OK;
+    if (launch_export_chains(ctx->table_cur(request), r.W, r.depth, ctx->cfg.max_beam, slots_dev, s) != cudaSuccess)
+        return ONELA_E_CUDA;
+    ctx->launches++;
+    return ONELA_OK;
+}
+
+onela_status onela_poll_device_status(onela_ctx* ctx, int32_t* code_host, int32_t* detail_host) {
+    if (!ctx) return ONELA_E_INVAL;
+    int32_t w[4] = {0, 0, 0, 0};
+    if (!ctx->dry() && ctx->status_cleared) {
+        if (cudaDeviceSynchronize() != cudaSuccess) return ONELA_E_CUDA;
+        if (cudaMemcpy(w, ctx->lay.status, sizeof(w), cudaMemcpyDeviceToHost) != cudaSuccess) return ONELA_E_CUDA;
+        if (w[0] != ONELA_OK && cudaMemset(ctx->lay.status, 0, sizeof(w)) != cudaSuccess) return ONELA_E_CUDA;
+    }
+    if (code_host) *code_host = w[0];
+    if (detail_host) *detail_host = w[1];
+    return ONELA_OK;
+}
+
+onela_status onela_get_stats(const onela_ctx* ctx, int64_t* s0_bytes_host, int64_t* arena_bytes_used_host,
+                             int64_t* index_bytes_host) {
+    if (!ctx) return ONELA_E_INVAL;
+    const onela_config& c = ctx->cfg;
+    int64_t states = 0, index = 0;
+    for (const auto& r : ctx->req) {
+        for (uint8_t hs : r.has_state) states += hs;
+        index += (int64_t)r.W * r.depth * (int64_t)sizeof(int32_t);
+    }
+    const int64_t rec_bytes = (int64_t)(c.dk + c.dv) * ctx->elem_bytes + 2 * (int64_t)sizeof(float);
+    if (s0_bytes_host) *s0_bytes_host = states * ctx->s0_layer_floats() * (int64_t)sizeof(float);
+    if (arena_bytes_used_host) *arena_bytes_used_host = ctx->cursor * c.num_heads * rec_bytes * c.num_layers;
+    if (index_bytes_host) *index_bytes_host = index;
+    return ONELA_OK;
+}
+
+onela_status onela_get_step_base(const onela_ctx* ctx, int32_t request, int32_t step, int32_t* base_host) {
+    if (!ctx || !base_host || request < 0 || request >= ctx->cfg.num_requests) return ONELA_E_INVAL;
+    const ReqState& r = ctx->req[request];
+    if (step < 0 || step >= (int32_t)r.step_base.size()) return ONELA_E_INVAL;
+    *base_host = r.step_base[step];
+    return ONELA_OK;
+}
+
+int64_t onela_launch_count(const onela_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int32_t onela_uses_tensor_core_path(const onela_ctx* ctx) { return ctx && ctx->tensor_core ? 1 : 0; }
+
+const char* onela_status_string(onela_status s) {
+    switch (s) {
+        case ONELA_OK: return "ok";
+        case ONELA_E_INVAL: return "invalid argument";
+        case ONELA_E_CAPACITY: return "capacity exhausted";
+        case ONELA_E_ORDER: return "call order violated";
+        case ONELA_E_CUDA: return "CUDA runtime error";
+        case ONELA_E_UNSUPPORTED: return "unsupported head dimensions or dtype";
+        case ONELA_E_DEVICE_CHECK: return "device found an out-of-range parent index";
+        case ONELA_E_TIMEOUT: return "bounded device-side wait expired";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,69 @@
+// Internal declarations shared by the host-side context (onela_api.cu) and the kernel files.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "onela.h"
+
+namespace onela {
+
+// Device addresses of the sub-buffers carved out of the caller's workspace.
+struct Layout {
+    int32_t* status;   // [4]: code, detail, spare, spare
+    int32_t* tables;   // [request][2][max_steps][max_beam] global slot ids (double-buffered per request)
+    float* s0;         // [request][layer][head][dv*dk] fp32
+    float2* gates;     // [layer][head][arena_slots] (alpha, beta)
+    char* kv;          // [layer][head][arena_slots][dk + dv] in rec_dtype: one row = k | v of one record
+    size_t total_bytes;
+};
+
+struct BatchBases {
+    int32_t base[ONELA_MAX_BATCH];  // first slot of this call's records, per request of the batch
+};
+
+// Everything a decode kernel needs, passed by value as the kernel parameter.
+struct DecodeArgs {
+    const void* q;          // [req_count][W][H][dk]
+    void* out;              // [req_count][W][H][dv]
+    const float* s0;        // store slot of (req_begin, layer)
+    const char* kv;         // arena plane of this layer
+    const float2* gates;    // gate plane of this layer
+    const int32_t* table;   // current ancestry buffer of req_begin: [level][max_beam]
+    int32_t* status;
+    long long s0_req_stride;     // floats between consecutive requests' store slots (same layer)
+    long long table_req_stride;  // ints between consecutive requests' tables
+    long long arena_slots;
+    int32_t req_count, W, H, depth, max_beam, s0_swizzled;
+    BatchBases bases;
+};
+
+// index kernels
+cudaError_t launch_reorder(int32_t* tables_req0, long long table_req_stride, int32_t req_count,
+                           const int32_t* parents, int32_t W_new, int32_t W_prev, int32_t depth_old,
+                           int32_t max_beam, int32_t max_steps, const BatchBases& bases, int32_t* status,
+                           cudaStream_t stream);
+cudaError_t launch_export_chains(const int32_t* table_cur, int32_t W, int32_t depth, int32_t max_beam,
+                                 int32_t* slots_out, cudaStream_t stream);
+
+// record / state kernels
+cudaError_t launch_append(const void* k, const void* v, const float* alpha, const float* beta, char* kv_plane,
+                          float2* gate_plane, long long arena_slots, int32_t req_count, int32_t W, int32_t H,
+                          int32_t dk, int32_t dv, int32_t elem_bytes, const BatchBases& bases,
+                          cudaStream_t stream);
+cudaError_t launch_store_state(const float* S0_in, float* slot, int32_t H, int32_t dk, int32_t dv,
+                               int32_t swizzled, cudaStream_t stream);
+cudaError_t launch_export_state(const float* slot, float* S0_out, int32_t H, int32_t dk, int32_t dv,
+                                int32_t swizzled, cudaStream_t stream);
+// returns cudaErrorInvalidValue with *supported = false when (dk, dv, dtype) has no instantiation
+cudaError_t launch_prefill(const void* k, const void* v, const float* alpha, const float* beta, float* slot,
+                           int32_t n_tokens, int32_t H, int32_t dk, int32_t dv, int32_t rec_dtype,
+                           int32_t swizzled, bool* supported, cudaStream_t stream);
+
+// decode kernels
+cudaError_t launch_decode_generic(const DecodeArgs& a, int32_t dk, int32_t dv, int32_t rec_dtype,
+                                  int32_t out_dtype, bool* supported, cudaStream_t stream);
+bool decode_generic_supported(int32_t dk, int32_t dv, int32_t rec_dtype);
+
+}  // namespace onela

@@ -1,0 +1,56 @@
+// Device helpers shared by the kernel files: the shared-state image layout and bf16 unpacking.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace onela {
+
+// Shared-state image for the tensor-core kernel (dk = dv = 128): the [dv][dk] fp32 matrix of one head
+// stored as the K-major, 128-byte-swizzled shared-memory operand the tcgen05 MMA reads, so that the
+// decode kernel brings a head in with ONE contiguous 64 KiB bulk copy.  K is split into 4 blocks of
+// 32 floats (128 bytes); inside a block row i holds its 32 floats as eight 16-byte chunks, chunk c
+// stored at position c ^ (i & 7).  Returns the float offset of element (i, k) inside the head image.
+__host__ __device__ __forceinline__ int s0_image_index(int i, int k) {
+    const int kb = k >> 5, kk = k & 31;
+    return kb * (128 * 32) + i * 32 + ((((kk >> 2) ^ (i & 7)) << 2) | (kk & 3));
+}
+
+// Round to the nearest TF32 value (10 explicit mantissa bits), ties away from zero.  The tensor core
+// reads only the upper 19 bits of an fp32 operand; rounding once when the state is stored makes that
+// read unbiased instead of a truncation.
+__device__ __forceinline__ float round_tf32(float x) {
+    uint32_t u;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(x));
+    return __uint_as_float(u);
+}
+
+// Two packed bf16 (little endian: element 0 in the low half) -> two fp32, exactly.
+__device__ __forceinline__ void unpack_bf16x2(uint32_t w, float& lo, float& hi) {
+    lo = __uint_as_float(w << 16);
+    hi = __uint_as_float(w & 0xffff0000u);
+}
+
+template <typename T>
+struct Vec16;  // one 16-byte vector of T, unpacked to fp32
+template <>
+struct Vec16<float> {
+    static constexpr int N = 4;
+    static __device__ __forceinline__ void load(const float* p, float* out) {
+        const float4 x = __ldg(reinterpret_cast<const float4*>(p));
+        out[0] = x.x; out[1] = x.y; out[2] = x.z; out[3] = x.w;
+    }
+};
+template <>
+struct Vec16<__nv_bfloat16> {
+    static constexpr int N = 8;
+    static __device__ __forceinline__ void load(const __nv_bfloat16* p, float* out) {
+        const uint4 x = __ldg(reinterpret_cast<const uint4*>(p));
+        unpack_bf16x2(x.x, out[0], out[1]);
+        unpack_bf16x2(x.y, out[2], out[3]);
+        unpack_bf16x2(x.z, out[4], out[5]);
+        unpack_bf16x2(x.w, out[6], out[7]);
+    }
+};
+
+}  // namespace onela

@@ -1,0 +1,186 @@
+// Shared-state store and record arena kernels.
+//  - append: copy one decode call's (k, v, alpha, beta) into the append-only arena (paper Section 3.3:
+//    records are written once to the slots of the current step and never relocated).
+//  - store_state / prefill: fill the store slot of one (request, layer) with S_0 (Section 3.2: the
+//    post-prefill state is stored once per request), either from a caller tensor or by running Eq. 1
+//    from the zero state over the prompt.
+#include "onela_internal.h"
+#include "onela_layout.cuh"
+
+namespace onela {
+
+namespace {
+
+// One warp per (request, beam, head) row.  The arena is head-major ([head][slot][k | v]) so that the
+// records one decode tile reads - consecutive beams of one head - are contiguous.
+__global__ void __launch_bounds__(256) append_kernel(const char* __restrict__ k, const char* __restrict__ v,
+                                                     const float* __restrict__ alpha, const float* __restrict__ beta,
+                                                     char* __restrict__ kv_plane, float2* __restrict__ gate_plane,
+                                                     long long arena_slots, int32_t req_count, int32_t W, int32_t H,
+                                                     int32_t k_bytes, int32_t v_bytes, BatchBases bases) {
+    const long long row = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    const long long rows = (long long)req_count * W * H;
+    if (row >= rows) return;
+    const int h = (int)(row % H);
+    const long long rb = row / H;
+    const int b = (int)(rb % W), r = (int)(rb / W);
+    const long long slot = (long long)bases.base[r] + b;
+    const long long dst_row = (long long)h * arena_slots + slot;
+    const uint4* ksrc = reinterpret_cast<const uint4*>(k + row * k_bytes);
+    const uint4* vsrc = reinterpret_cast<const uint4*>(v + row * v_bytes);
+    uint4* dst = reinterpret_cast<uint4*>(kv_plane + dst_row * (k_bytes + v_bytes));
+    const int nk = k_bytes >> 4, nv = v_bytes >> 4;
+    for (int c = lane; c < nk + nv; c += 32) dst[c] = (c < nk) ? __ldg(ksrc + c) : __ldg(vsrc + (c - nk));
+    if (lane == 0) gate_plane[dst_row] = make_float2(__ldg(alpha + row), __ldg(beta + row));
+}
+
+__global__ void __launch_bounds__(256) store_state_swizzled_kernel(const float* __restrict__ in, float* __restrict__ slot,
+                                                                   int32_t n) {
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= n) return;
+    const int h = e >> 14, i = (e >> 7) & 127, k = e & 127;
+    slot[(h << 14) + s0_image_index(i, k)] = round_tf32(__ldg(in + e));
+}
+
+__global__ void __launch_bounds__(256) export_state_swizzled_kernel(const float* __restrict__ slot, float* __restrict__ out,
+                                                                    int32_t n) {
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= n) return;
+    const int h = e >> 14, i = (e >> 7) & 127, k = e & 127;
+    out[e] = __ldg(slot + (h << 14) + s0_image_index(i, k));
+}
+
+template <typename T>
+__device__ __forceinline__ float to_float(T x);
+template <>
+__device__ __forceinline__ float to_float<float>(float x) { return x; }
+template <>
+__device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+// Eq. 1 from the zero state over the prompt, one CTA per head, thread i owns row i of S in registers.
+template <int DK, int DV, typename T>
+__global__ void __launch_bounds__(DV) prefill_kernel(const T* __restrict__ k, const T* __restrict__ v,
+                                                     const float* __restrict__ alpha, const float* __restrict__ beta,
+                                                     float* __restrict__ slot, int32_t n_tokens, int32_t H,
+                                                     int32_t swizzled) {
+    __shared__ __align__(16) float k_s[2][DK];
+    const int h = blockIdx.x, i = threadIdx.x;
+    float S[DK];
+#pragma unroll
+    for (int j = 0; j < DK; ++j) S[j] = 0.f;
+    constexpr int KPT = (DK + DV - 1) / DV;  // k elements each thread stages per token
+    float kn[KPT], vn = 0.f, an = 1.f, bn = 0.f;
+    auto fetch = [&](int t) {
+        const long long row = (long long)t * H + h;
+#pragma unroll
+        for (int c = 0; c < KPT; ++c) {
+            const int j = i + c * DV;
+            kn[c] = (j < DK) ? to_float(k[row * DK + j]) : 0.f;
+        }
+        vn = to_float(v[row * DV + i]);
+        an = __ldg(alpha + row);
+        bn = __ldg(beta + row);
+    };
+    auto stage = [&](int buf) {
+#pragma unroll
+        for (int c = 0; c < KPT; ++c) {
+            const int j = i + c * DV;
+            if (j < DK) k_s[buf][j] = kn[c];
+        }
+    };
+    if (n_tokens > 0) { fetch(0); stage(0); }
+    __syncthreads();
+    for (int t = 0; t < n_tokens; ++t) {
+        const float vt = vn, a = an, b = bn;
+        if (t + 1 < n_tokens) fetch(t + 1);
+        const float4* kk = reinterpret_cast<const float4*>(k_s[t & 1]);
+        float u0 = 0.f, u1 = 0.f, u2 = 0.f, u3 = 0.f;
+#pragma unroll
+        for (int j = 0; j < DK / 4; ++j) {
+            const float4 x = kk[j];
+            u0 = fmaf(S[4 * j + 0], x.x, u0);
+            u1 = fmaf(S[4 * j + 1], x.y, u1);
+            u2 = fmaf(S[4 * j + 2], x.z, u2);
+            u3 = fmaf(S[4 * j + 3], x.w, u3);
+        }
+        const float u = (u0 + u1) + (u2 + u3);
+        const float delta = b * (vt - a * u);   // Eq. 2's delta_t
+#pragma unroll
+        for (int j = 0; j < DK / 4; ++j) {
+            const float4 x = kk[j];
+            S[4 * j + 0] = fmaf(a, S[4 * j + 0], delta * x.x);
+            S[4 * j + 1] = fmaf(a, S[4 * j + 1], delta * x.y);
+            S[4 * j + 2] = fmaf(a, S[4 * j + 2], delta * x.z);
+            S[4 * j + 3] = fmaf(a, S[4 * j + 3], delta * x.w);
+        }
+        if (t + 1 < n_tokens) stage((t + 1) & 1);
+        __syncthreads();
+    }
+    float* dst = slot + (long long)h * DV * DK;
+    if (swizzled) {
+#pragma unroll
+        for (int j = 0; j < DK; ++j) dst[s0_image_index(i, j)] = round_tf32(S[j]);
+    } else {
+#pragma unroll
+        for (int j = 0; j < DK; ++j) dst[(long long)i * DK + j] = S[j];
+    }
+}
+
+template <int DK, int DV>
+cudaError_t prefill_dispatch(const void* k, const void* v, const float* alpha, const float* beta, float* slot,
+                             int32_t n_tokens, int32_t H, int32_t rec_dtype, int32_t swizzled, cudaStream_t stream) {
+    if (rec_dtype == ONELA_DTYPE_BF16)
+        prefill_kernel<DK, DV, __nv_bfloat16><<<H, DV, 0, stream>>>(
+            static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(v), alpha, beta, slot, n_tokens, H, swizzled);
+    else
+        prefill_kernel<DK, DV, float><<<H, DV, 0, stream>>>(static_cast<const float*>(k), static_cast<const float*>(v),
+                                                           alpha, beta, slot, n_tokens, H, swizzled);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_append(const void* k, const void* v, const float* alpha, const float* beta, char* kv_plane,
+                          float2* gate_plane, long long arena_slots, int32_t req_count, int32_t W, int32_t H,
+                          int32_t dk, int32_t dv, int32_t elem_bytes, const BatchBases& bases,
+                          cudaStream_t stream) {
+    const long long rows = (long long)req_count * W * H;
+    const int warps_per_block = 8;
+    const long long blocks = (rows + warps_per_block - 1) / warps_per_block;
+    append_kernel<<<(unsigned)blocks, warps_per_block * 32, 0, stream>>>(
+        static_cast<const char*>(k), static_cast<const char*>(v), alpha, beta, kv_plane, gate_plane, arena_slots,
+        req_count, W, H, dk * elem_bytes, dv * elem_bytes, bases);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_store_state(const float* S0_in, float* slot, int32_t H, int32_t dk, int32_t dv,
+                               int32_t swizzled, cudaStream_t stream) {
+    const long long n = (long long)H * dk * dv;
+    if (!swizzled)
+        return cudaMemcpyAsync(slot, S0_in, n * sizeof(float), cudaMemcpyDeviceToDevice, stream);
+    store_state_swizzled_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(S0_in, slot, (int32_t)n);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_export_state(const float* slot, float* S0_out, int32_t H, int32_t dk, int32_t dv,
+                                int32_t swizzled, cudaStream_t stream) {
+    const long long n = (long long)H * dk * dv;
+    if (!swizzled)
+        return cudaMemcpyAsync(S0_out, slot, n * sizeof(float), cudaMemcpyDeviceToDevice, stream);
+    export_state_swizzled_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(slot, S0_out, (int32_t)n);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_prefill(const void* k, const void* v, const float* alpha, const float* beta, float* slot,
+                           int32_t n_tokens, int32_t H, int32_t dk, int32_t dv, int32_t rec_dtype,
+                           int32_t swizzled, bool* supported, cudaStream_t stream) {
+    *supported = true;
+    if (dk == 32 && dv == 32) return prefill_dispatch<32, 32>(k, v, alpha, beta, slot, n_tokens, H, rec_dtype, swizzled, stream);
+    if (dk == 64 && dv == 64) return prefill_dispatch<64, 64>(k, v, alpha, beta, slot, n_tokens, H, rec_dtype, swizzled, stream);
+    if (dk == 128 && dv == 128) return prefill_dispatch<128, 128>(k, v, alpha, beta, slot, n_tokens, H, rec_dtype, swizzled, stream);
+    *supported = false;
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace onela

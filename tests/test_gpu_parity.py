@@ -1,0 +1,173 @@
+"""Parity of the CUDA path against the CPU oracle, element by element, through the C ABI.
+
+Bar: ancestry chains and slot ids bit-exact; outputs within 5e-3 relative L2 per (beam, head) vector
+of the fp64 oracle.  Where the arithmetic allows a much tighter bound (fp32 fold and contraction with
+fp32 output: rounding only), that bound is asserted as well so a regression cannot hide under the bar.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2609_12399_b200 as P
+from paper_2609_12399_b200 import binding, inputs
+
+from _cases import (REL_L2_BAR, check_parity, expected_slots, make_case, rel_l2, run_library, run_oracle)
+
+pytestmark = pytest.mark.gpu
+
+CFG0, CFG1 = inputs.WORKLOADS[0], inputs.WORKLOADS[1]
+
+
+def _small(base, **kw):
+    return base.scaled(**kw)
+
+
+def _full_check(case, out_dtype, flags=0, batched=True, tight=None):
+    ref, chains = run_oracle(case)
+    outs, slots, ctx = run_library(case, out_dtype=out_dtype, flags=flags, batched=batched)
+    want = expected_slots(case, chains)
+    for key in want:
+        assert np.array_equal(slots[key], want[key]), f"ancestry rows of {key} differ"
+    worst = check_parity(case, outs, ref, tight=tight)
+    assert ctx.onela_poll_device_status() == (0, 0)
+    return worst, ctx
+
+
+def test_config0_tiny_reference():
+    """1 request, 1 layer, 2 heads, dk = dv = 32, fp32, beam 8, 3 calls, uniform parents."""
+    worst, ctx = _full_check(make_case(CFG0), "fp32", tight=2e-6)
+    assert not ctx.onela_uses_tensor_core_path()
+
+
+@pytest.mark.parametrize("out_dtype,tight", [("fp32", None), ("bf16", None)])
+def test_config1_beam128(out_dtype, tight):
+    """16 heads, dk = dv = 128, bf16 records, beam 128, depth 4, uniform parents; every call, every unit."""
+    _full_check(make_case(CFG1), out_dtype, tight=tight)
+
+
+def test_config1_cuda_core_kernel_is_fp32_accurate():
+    _full_check(make_case(CFG1.scaled(prompt_len=256)), "fp32", flags=P.FLAG_FORCE_GENERIC, tight=5e-6)
+
+
+@pytest.mark.parametrize("W", [1, 31, 33, 77, 200])
+def test_ragged_beam_widths(W):
+    """Beam widths that are not a multiple of any tile: a partial tail tile, and tiles of one beam."""
+    wl = CFG1.scaled(H=3, W=W, D=3, prompt_len=64, seed=500 + W)
+    _full_check(make_case(wl), "fp32")
+    _full_check(make_case(wl), "fp32", flags=P.FLAG_FORCE_GENERIC, tight=5e-6)
+
+
+def test_multi_request_multi_layer_batched_and_unbatched():
+    wl = CFG1.scaled(R=3, L=2, H=4, W=40, D=3, prompt_len=96, parents="zipf", zipf_s=1.3, seed=77)
+    case = make_case(wl)
+    _full_check(case, "bf16", batched=True)
+    _full_check(case, "fp32", batched=False)
+
+
+def test_varying_beam_width_between_calls():
+    wl = CFG1.scaled(H=2, W=96, D=4, prompt_len=64, seed=91)
+    _full_check(make_case(wl, widths=[96, 17, 64, 5]), "fp32")
+
+
+def test_depth_one_and_max_depth():
+    _full_check(make_case(CFG1.scaled(H=2, W=64, D=1, prompt_len=64)), "fp32")
+    _full_check(make_case(CFG1.scaled(H=2, W=48, D=12, prompt_len=64, parents="zipf", zipf_s=1.5)), "fp32")
+
+
+@pytest.mark.parametrize("dk,dv,dtype", [(64, 64, "bf16"), (64, 64, "fp32"), (128, 128, "fp32"), (128, 256, "bf16"),
+                                         (256, 256, "bf16"), (32, 32, "bf16")])
+def test_other_geometries(dk, dv, dtype):
+    wl = CFG1.scaled(H=2, dk=dk, dv=dv, dtype=dtype, W=37, D=3, prompt_len=48, seed=dk + dv)
+    _full_check(make_case(wl), "fp32")
+
+
+def test_alpha1_beta0_reduces_to_matvec_on_gpu():
+    wl = CFG1.scaled(H=2, W=64, D=3, prompt_len=64)
+    case = make_case(wl)
+    for tk in case["tok"].values():
+        tk["alpha"].fill_(1.0)
+        tk["beta"].zero_()
+    outs, _, _ = run_library(case, out_dtype="fp32")
+    for (r, l, t), o in outs.items():
+        want = np.einsum("hij,bhj->bhi", case["S0"][(r, l)].double().numpy(), case["q"][(r, l, t)].double().numpy())
+        assert rel_l2(o.numpy(), want).max() <= REL_L2_BAR
+
+
+def test_shared_chains_give_identical_outputs_on_gpu():
+    wl = CFG1.scaled(H=2, W=64, D=3, prompt_len=64)
+    case = make_case(wl)
+    case["parents"][(0, 2)] = torch.full((64,), 5, dtype=torch.int32)
+    for n in ("k", "v", "alpha", "beta"):
+        x = case["tok"][(0, 0, 2)][n]
+        x[:] = x[0]
+    case["q"][(0, 0, 2)][:] = case["q"][(0, 0, 2)][0]
+    outs, _, _ = run_library(case, out_dtype="fp32")
+    o = outs[(0, 0, 2)]
+    assert torch.equal(o, o[0:1].expand_as(o))
+
+
+def test_records_are_stored_bit_exactly_and_never_rewritten():
+    """The arena planes hold exactly the appended bytes at slot base(req, t) + beam, head-major, and a
+    later reorder/append leaves earlier records untouched (read straight out of the workspace)."""
+    wl = CFG1.scaled(R=2, H=3, W=20, D=3, prompt_len=32, seed=5)
+    case = make_case(wl)
+    outs, slots, ctx = run_library(case, out_dtype="fp32")
+    c = ctx.cfg
+    al = lambda n: (n + 1023) // 1024 * 1024
+    off_tables = al(16)
+    off_s0 = off_tables + al(c.num_requests * 2 * c.max_steps * c.max_beam * 4)
+    off_gates = off_s0 + al(c.num_requests * c.num_layers * c.num_heads * c.dv * c.dk * 4)
+    off_kv = off_gates + al(c.num_layers * c.num_heads * c.arena_slots * 8)
+    ws = ctx.workspace[ctx.workspace_ptr - ctx.workspace.data_ptr():]
+    gates = ws[off_gates:off_gates + c.num_heads * c.arena_slots * 8].view(torch.float32).view(c.num_heads, c.arena_slots, 2).cpu()
+    kv = ws[off_kv:off_kv + c.num_heads * c.arena_slots * 512].view(torch.bfloat16).view(c.num_heads, c.arena_slots, 256).cpu()
+    for r in range(wl.R):
+        for t in range(wl.D):
+            base = ctx.onela_get_step_base(r, t)
+            tk = case["tok"][(r, 0, t)]
+            for h in range(wl.H):
+                assert torch.equal(kv[h, base:base + wl.W, :128], tk["k"][:, h])
+                assert torch.equal(kv[h, base:base + wl.W, 128:], tk["v"][:, h])
+                assert torch.equal(gates[h, base:base + wl.W, 0], tk["alpha"][:, h])
+                assert torch.equal(gates[h, base:base + wl.W, 1], tk["beta"][:, h])
+
+
+def test_out_of_range_parent_is_reported_not_trapped():
+    wl = CFG1.scaled(H=2, W=16, D=2, prompt_len=32)
+    case = make_case(wl)
+    bad = case["parents"][(0, 1)].clone()
+    bad[3] = 16          # one past the previous beam
+    case["parents"][(0, 1)] = bad
+    outs, slots, ctx = run_library(case, out_dtype="fp32")
+    code, detail = ctx.onela_poll_device_status()
+    assert code == binding.E_DEVICE_CHECK and detail == 16
+    assert ctx.onela_poll_device_status() == (0, 0)          # reading clears the sticky word
+    assert slots[(0, 1)][3, 0] == 0                          # the offending index was clamped to parent 0
+    assert torch.isfinite(outs[(0, 0, 1)]).all()
+
+
+def test_prefill_kernel_matches_oracle_prefill():
+    for wl in (CFG0, CFG1.scaled(H=4, prompt_len=300)):
+        cfg = P.make_config(1, 1, wl.H, wl.dk, wl.dv, 8, 2, wl.dtype, "fp32", 16)
+        ctx = P.Onela(cfg)
+        p = inputs.prompt_tokens(wl, 0, 0)
+        ctx.onela_prefill_shared_state(0, 0, *(p[n].cuda() for n in ("k", "v", "alpha", "beta")))
+        got = ctx.onela_export_shared_state(0, 0).cpu().double().numpy()
+        want = oracle.prefill(p["k"], p["v"], p["alpha"], p["beta"])
+        err = np.linalg.norm(got - want, axis=(1, 2)) / np.linalg.norm(want, axis=(1, 2))
+        # fp32 recurrence (plus TF32 storage, 2^-11 per element, on the tensor-core path)
+        assert err.max() < (6e-4 if ctx.onela_uses_tensor_core_path() else 1e-5), err
+
+
+def test_init_then_export_round_trip():
+    wl = CFG1.scaled(H=2)
+    ctx = P.Onela(P.make_config(1, 1, 2, 128, 128, 8, 2, "bf16", "fp32", 16))
+    S = torch.randn(2, 128, 128, generator=torch.Generator().manual_seed(1))
+    ctx.onela_init_shared_state(0, 0, S.cuda())
+    back = ctx.onela_export_shared_state(0, 0).cpu()
+    if ctx.onela_uses_tensor_core_path():
+        assert ((back - S).abs() <= S.abs() * 2.0 ** -11 + 1e-30).all()      # rounded to TF32, nothing more
+        assert torch.equal(back.view(torch.int32) & 0x1FFF, torch.zeros_like(back, dtype=torch.int32))
+    else:
+        assert torch.equal(back, S)

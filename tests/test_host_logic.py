@@ -1,0 +1,221 @@
+"""Host-side bookkeeping of the library, exercised without a GPU through ONELA_FLAG_DRY_RUN
+(validate and advance the state machine, launch nothing): call order, slot numbering, capacity
+limits, workspace carve-up and the resident-byte statistics."""
+import json
+from pathlib import Path
+
+import numpy as np
+import pytest
+
+import paper_2609_12399_b200 as P
+from paper_2609_12399_b200 import accounting, binding, build
+
+GOLDEN = Path(__file__).parent / "golden"
+FAKE = 4096  # a non-null, 16-byte aligned fake device address; dry runs never dereference it
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+
+
+def ctx(R=2, L=2, H=4, dk=32, dv=32, W=8, steps=3, slots=64, rec="fp32", out="fp32"):
+    cfg = P.make_config(R, L, H, dk, dv, W, steps, rec, out, slots, P.FLAG_DRY_RUN)
+    return P.Onela(cfg, device="cpu")
+
+
+def raises(status):
+    class _Ctx:
+        def __enter__(self):
+            return self
+        def __exit__(self, et, ev, tb):
+            assert et is binding.OnelaError, f"expected OnelaError({status}), got {et}"
+            assert ev.status == status, f"expected {status}, got {ev.status}"
+            return True
+    return _Ctx()
+
+
+def full_step(o, req_begin, req_count, W, parents, layers):
+    o.onela_reorder_beams(req_begin, req_count, parents, W)
+    for l in layers:
+        o.onela_append_records(req_begin, req_count, l, FAKE, FAKE, FAKE, FAKE)
+        o.onela_decode_step(req_begin, req_count, l, FAKE, FAKE)
+
+
+def test_invalid_configs():
+    bad = [dict(num_requests=0), dict(dk=0), dict(max_beam=0), dict(arena_slots=0), dict(rec_dtype=7),
+           dict(arena_slots=2 ** 31), dict(dk=36)]   # dk=36 fp32 is fine (144 B); bf16 would not be
+    base = dict(num_requests=1, num_layers=1, num_heads=1, dk=32, dv=32, max_beam=4, max_steps=2, rec_dtype=0,
+                out_dtype=0, arena_slots=8, flags=1)
+    for i, b in enumerate(bad):
+        cfg = binding.OnelaConfig(**{**base, **b})
+        n = P.onela_workspace_bytes(cfg)
+        if "dk" in b and b["dk"] == 36:
+            assert n > 0
+        else:
+            assert n == 0, b
+    cfg = binding.OnelaConfig(**{**base, "dk": 36, "rec_dtype": 1})   # 72-byte bf16 rows: not 16-byte vectors
+    assert P.onela_workspace_bytes(cfg) == 0
+    with raises(binding.E_UNSUPPORTED):                                  # sane but not compiled
+        P.Onela(binding.OnelaConfig(**{**base, "dk": 48, "dv": 48}), device="cpu")
+    with raises(binding.E_INVAL):                                        # misaligned workspace
+        P.Onela(binding.OnelaConfig(**base), device="cpu", workspace_ptr=1024 + 16)
+
+
+def test_workspace_carve_up_size():
+    cfg = P.make_config(4, 16, 32, 128, 128, 512, 8, "bf16", "bf16", 4 * 512 * 8)
+    n = P.onela_workspace_bytes(cfg)
+    s0 = 4 * 16 * 32 * 128 * 128 * 4
+    arena = 16 * 32 * (4 * 512 * 8) * 520
+    tables = 4 * 2 * 8 * 512 * 4
+    assert s0 + arena + tables <= n <= s0 + arena + tables + 8 * 1024
+
+
+def test_call_order_is_enforced():
+    o = ctx()
+    with raises(binding.E_ORDER):
+        o.onela_reorder_beams(0, 1, None, 8)                 # no shared state yet
+    o.onela_init_shared_state(0, 0, FAKE)
+    with raises(binding.E_ORDER):
+        o.onela_append_records(0, 1, 0, FAKE, FAKE, FAKE, FAKE)   # no decode call opened
+    with raises(binding.E_ORDER):
+        o.onela_reorder_beams(0, 1, FAKE, 8)                 # depth 0 must pass parents = NULL
+    o.onela_reorder_beams(0, 1, None, 8)
+    with raises(binding.E_ORDER):
+        o.onela_decode_step(0, 1, 0, FAKE, FAKE)             # records not appended yet
+    with raises(binding.E_ORDER):
+        o.onela_append_records(0, 1, 1, FAKE, FAKE, FAKE, FAKE)   # layer 1 holds no state
+    o.onela_append_records(0, 1, 0, FAKE, FAKE, FAKE, FAKE)
+    with raises(binding.E_ORDER):
+        o.onela_append_records(0, 1, 0, FAKE, FAKE, FAKE, FAKE)   # exactly once per call
+    o.onela_decode_step(0, 1, 0, FAKE, FAKE)
+    o.onela_decode_step(0, 1, 0, FAKE, FAKE)                 # any number of times
+    with raises(binding.E_ORDER):
+        o.onela_reorder_beams(0, 1, None, 8)                 # depth 1 needs parents
+    o.onela_reorder_beams(0, 1, FAKE, 5)                     # the beam may shrink
+    with raises(binding.E_ORDER):
+        o.onela_reorder_beams(0, 1, FAKE, 5)                 # previous call never appended
+    assert o.depth_and_width(0) == (2, 5)
+
+
+def test_every_layer_with_state_must_append_before_next_call():
+    o = ctx()
+    o.onela_init_shared_state(0, 0, FAKE)
+    o.onela_init_shared_state(0, 1, FAKE)
+    o.onela_reorder_beams(0, 1, None, 4)
+    o.onela_append_records(0, 1, 0, FAKE, FAKE, FAKE, FAKE)
+    with raises(binding.E_ORDER):
+        o.onela_reorder_beams(0, 1, FAKE, 4)                 # layer 1 would have a hole in its chains
+    o.onela_append_records(0, 1, 1, FAKE, FAKE, FAKE, FAKE)
+    o.onela_reorder_beams(0, 1, FAKE, 4)
+
+
+def test_slot_numbering_bump_cursor():
+    o = ctx(R=3, slots=200)
+    for r in range(3):
+        o.onela_init_shared_state(r, 0, FAKE)
+    full_step(o, 0, 2, 8, None, [0])          # requests 0,1 batched: bases 0, 8
+    full_step(o, 2, 1, 6, None, [0])          # request 2 alone: base 16
+    full_step(o, 0, 2, 4, FAKE, [0])          # bases 22, 26
+    full_step(o, 2, 1, 6, FAKE, [0])          # base 30
+    assert [o.onela_get_step_base(0, t) for t in (0, 1)] == [0, 22]
+    assert [o.onela_get_step_base(1, t) for t in (0, 1)] == [8, 26]
+    assert [o.onela_get_step_base(2, t) for t in (0, 1)] == [16, 30]
+    with raises(binding.E_INVAL):
+        o.onela_get_step_base(0, 2)
+    st = o.onela_get_stats()
+    assert st["arena_bytes_used"] == 36 * 4 * 264 * 2         # slots * heads * record bytes * layers
+    assert st["index_bytes"] == (4 * 2 + 4 * 2 + 6 * 2) * 4
+    assert st["s0_bytes"] == 3 * 4 * 32 * 32 * 4
+
+
+def test_batches_must_be_uniform_and_bounded():
+    o = ctx(R=3, slots=200)
+    for r in range(3):
+        o.onela_init_shared_state(r, 0, FAKE)
+    full_step(o, 0, 1, 8, None, [0])
+    with raises(binding.E_INVAL):
+        o.onela_reorder_beams(0, 2, FAKE, 8)      # request 1 is at depth 0, request 0 at depth 1
+    with raises(binding.E_INVAL):
+        o.onela_reorder_beams(2, 2, None, 8)      # runs past the last request
+    with raises(binding.E_INVAL):
+        o.onela_reorder_beams(0, 0, None, 8)
+    with raises(binding.E_INVAL):
+        o.onela_decode_step(0, 1, 5, FAKE, FAKE)  # no such layer
+    with raises(binding.E_INVAL):
+        o.onela_decode_step(0, 1, 0, FAKE + 4, FAKE)   # misaligned pointer
+    with raises(binding.E_INVAL):
+        o.onela_decode_step(0, 1, 0, None, FAKE)
+
+
+def test_capacity_limits():
+    o = ctx(R=1, W=8, steps=2, slots=12)
+    o.onela_init_shared_state(0, 0, FAKE)
+    with raises(binding.E_CAPACITY):
+        o.onela_reorder_beams(0, 1, None, 9)      # wider than max_beam
+    full_step(o, 0, 1, 8, None, [0])
+    with raises(binding.E_CAPACITY):
+        o.onela_reorder_beams(0, 1, FAKE, 8)      # 8 + 8 > 12 arena slots
+    full_step(o, 0, 1, 4, FAKE, [0])
+    with raises(binding.E_CAPACITY):
+        o.onela_reorder_beams(0, 1, FAKE, 1)      # max_steps reached (checked before the arena)
+    o.onela_reset()
+    assert o.onela_get_stats() == {"s0_bytes": 0, "arena_bytes_used": 0, "index_bytes": 0}
+    with raises(binding.E_ORDER):
+        o.onela_reorder_beams(0, 1, None, 8)      # reset forgot the shared state too
+    o.onela_init_shared_state(0, 0, FAKE)
+    full_step(o, 0, 1, 8, None, [0])
+    assert o.onela_get_step_base(0, 0) == 0       # the cursor was rewound
+
+
+def test_new_prompt_restarts_a_request():
+    o = ctx(R=1, slots=100)
+    o.onela_init_shared_state(0, 0, FAKE)
+    o.onela_init_shared_state(0, 1, FAKE)
+    full_step(o, 0, 1, 8, None, [0, 1])
+    full_step(o, 0, 1, 8, FAKE, [0, 1])
+    o.onela_init_shared_state(0, 0, FAKE)         # a new prompt arrives in this slot
+    assert o.depth_and_width(0) == (0, 0)
+    o.onela_reorder_beams(0, 1, None, 8)          # depth 0 again: parents = NULL
+    with raises(binding.E_ORDER):
+        o.onela_append_records(0, 1, 1, FAKE, FAKE, FAKE, FAKE)   # layer 1's old state was dropped
+    assert o.onela_get_step_base(0, 0) == 16      # the arena is append-only: no slot is reused
+
+
+def test_storage_arithmetic_matches_section_4_4():
+    """The resident-byte arithmetic reproduces the capacities and write volumes the paper prints, with
+    the paper's 516-byte record; the raw (k, v, alpha, beta) record kept here is 520 bytes."""
+    g = json.loads((GOLDEN / "storage_section44.json").read_text())
+    geo = g["geometry"]
+    MiB = 2.0 ** 20
+    for case in g["cases"]:
+        p = accounting.persistent_bytes(T=case["T"], rec_bytes=g["paper_record_bytes"], **geo)
+        # printed to three significant figures (36.25 -> 36.3, 100.75 -> 101, 32.25 -> 32.3, 96.75 -> 96.8)
+        assert p["total"] / MiB == pytest.approx(case["capacity_MiB"], abs=0.0501 if case["capacity_MiB"] < 100 else 0.501)
+        assert p["writes"] / MiB == pytest.approx(case["writes_MiB"], abs=0.0501)
+        assert p["fullstate"] / p["total"] == pytest.approx(case["capacity_reduction"], rel=5e-3)
+        assert p["fullstate_writes"] / p["writes"] == pytest.approx(case["write_reduction"], rel=5e-3)
+        # the library's own statistics for the same geometry with its 520-byte records
+        o = ctx(R=geo["R"], L=1, H=geo["H"], dk=128, dv=128, W=geo["W"], steps=case["T"],
+                slots=geo["R"] * geo["W"] * case["T"], rec="bf16", out="bf16")
+        for r in range(geo["R"]):
+            o.onela_init_shared_state(r, 0, FAKE)
+        for t in range(case["T"]):
+            full_step(o, 0, geo["R"], geo["W"], None if t == 0 else FAKE, [0])
+        st = o.onela_get_stats()
+        assert st["s0_bytes"] == 4 * 2 ** 20
+        assert st["arena_bytes_used"] == int(case["T"] * 16.25 * 2 ** 20)
+        mine = accounting.persistent_bytes(T=case["T"], rec_bytes=accounting.record_bytes(128, 128, 2), **geo)
+        assert st["s0_bytes"] + st["arena_bytes_used"] == mine["total"]
+        assert st["index_bytes"] == geo["R"] * geo["W"] * case["T"] * 4
+
+
+def test_distinct_record_count():
+    parents = [None, np.array([0, 0, 2, 2]), np.array([1, 1, 1, 3])]
+    assert accounting.distinct_records(parents, [4, 4, 4]) == [2, 2, 4]
+    rows = accounting.chain_table(parents, [4, 4, 4])
+    assert rows.tolist() == [[0, 1, 0], [0, 1, 1], [0, 1, 2], [2, 3, 3]]
+    b = accounting.decode_bytes(R=1, H=2, dk=128, dv=128, W=4, depth=3, elem_bytes=2, out_bytes=2,
+                                distinct_per_request=[8])
+    assert b["algorithmic"] == 2 * 128 * 128 * 4 + 4 * 2 * 512 + 4 * 3 * 4 + 8 * 2 * 520
+    assert b["undeduplicated"] == 2 * 128 * 128 * 4 + 4 * 2 * 512 + 4 * 3 * 4 + 12 * 2 * 520
