@@ -1,0 +1,399 @@
+#!/usr/bin/env python
+"""Benchmark of the beam-shared GDN decode path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg4]
+
+One STEP is one whole generation of the workload through the C ABI: reset, store every shared state
+(a1), then for every decode call: reorder_beams (a2) and, per layer, append_records (a3) and the fused
+decode_step (a4-a6).  The default workload is the 16-layer beam-512 decode stack (benchmark config 4:
+4 requests x 16 layers x 32 heads, dk = dv = 128, depth 8, Zipf(1.5) parents, bf16 records, fp32 S_0),
+whose per-step inputs (4.6 GiB) are far larger than L2.
+
+Printed JSON line: `value` = beam-head decodes/s with inputs resident in HBM (CUDA-graph replay of the
+step, timed with CUDA events, max over ranks); `e2e` = the same metric with every input copied from
+pinned host memory and every output copied back inside the timed region; `roofline` = algorithmic bytes
+of the decode launches / their CUDA-event durations against the measured HBM peak; `cpu_baseline` = the
+fp64 oracle timed on the host cores on a bounded sample of the same workload.
+
+`--impl reference` times the CPU oracle alone (there is no other reference implementation).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+import torch
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+from paper_2609_12399_b200 import accounting, inputs  # noqa: E402
+
+METRIC = "beam-head GDN decodes/s per layer at beam 512"
+UNIT = "decodes/s"
+FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes per decode launch of the deepest call, from the ncu capture summarised in
+# profiles/ (filled in once a capture exists; None = not captured)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def workload_by_name(name: str) -> inputs.Workload:
+    for i, wl in enumerate(inputs.WORKLOADS):
+        if name in (wl.name, f"cfg{i}"):
+            return wl
+    raise SystemExit(f"unknown workload {name!r}")
+
+
+def describe(wl: inputs.Workload) -> str:
+    idx = inputs.WORKLOADS.index(wl) if wl in inputs.WORKLOADS else -1
+    return (f"configs[{idx}] {wl.name}: {wl.R} requests x {wl.L} layers x {wl.H} heads, dk=dv={wl.dk}, "
+            f"{wl.prompt_len}-token prompts, beam {wl.W}, depth {wl.D}, {wl.parents} parents"
+            + (f"(s={wl.zipf_s})" if wl.parents == "zipf" else "") + f", {wl.dtype} records, fp32 S_0")
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=lambda: self.lines.extend(self.proc.stdout), daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+            self.thread.join(timeout=5)
+
+    def summary(self) -> dict:
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------------
+def launch_bytes(wl: inputs.Workload, out_bytes: int) -> list:
+    """Algorithmic / un-deduplicated bytes of one decode launch (all requests, one layer) per call depth."""
+    res = []
+    par = {r: [None] + [inputs.parents(wl, r, t).numpy() for t in range(1, wl.D)] for r in range(wl.R)}
+    for t in range(wl.D):
+        distinct = [sum(accounting.distinct_records(par[r][:t + 1], [wl.W] * (t + 1))) for r in range(wl.R)]
+        res.append(accounting.decode_bytes(R=wl.R, H=wl.H, dk=wl.dk, dv=wl.dv, W=wl.W, depth=t + 1,
+                                           elem_bytes=wl.elem_bytes, out_bytes=out_bytes,
+                                           distinct_per_request=distinct))
+    return res
+
+
+def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
+    from paper_2609_12399_b200.runner import WorkloadRun
+
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    wl = workload_by_name(args.workload)
+    out_dtype = args.out_dtype or wl.dtype
+    out_bytes = 4 if out_dtype == "fp32" else 2
+    run = WorkloadRun(wl, dev, out_dtype)
+    ctx = run.ctx
+    run.prefill_states()
+    S0 = {(r, l): ctx.onela_export_shared_state(r, l) for r in range(wl.R) for l in range(wl.L)}
+    calls = [run.generate_call(t) for t in range(wl.D)]
+    outs = run.alloc_outputs()
+    torch.cuda.synchronize()
+    units_per_step = wl.R * wl.W * wl.H * wl.L * wl.D
+    per_depth = launch_bytes(wl, out_bytes)
+
+    def generation(decode_events=None, stream=None):
+        ctx.onela_reset(stream)
+        for (r, l), S in S0.items():
+            ctx.onela_init_shared_state(r, l, S, stream)
+        for call in calls:
+            run.run_call(call, outs, stream, decode_events)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    # ---- A. whole-step throughput, inputs resident: CUDA-graph replay of one generation -----------
+    side = torch.cuda.Stream()
+    launches_before = ctx.onela_launch_count()
+    with torch.cuda.stream(side):
+        generation()                      # eager once: primes lazy kernel attributes outside capture
+    torch.cuda.synchronize()
+    launches_per_step = ctx.onela_launch_count() - launches_before
+    graph, mode = None, "eager"
+    if not args.no_graph:
+        try:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                generation()
+            mode = "cuda_graph"
+        except Exception as e:  # capture unavailable: fall back to plain launches, and say so
+            graph, mode = None, f"eager (graph capture failed: {type(e).__name__})"
+            torch.cuda.synchronize()
+
+    def step():
+        if graph is not None:
+            graph.replay()
+        else:
+            generation()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    with ClockSampler(local_rank) as clocks:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+        barrier()
+        ms_total = e0.elapsed_time(e1)
+
+        # ---- B. per-launch decode durations for the roofline (eager, GPU kept ahead of the CPU) ------
+        pairs = []
+        torch.cuda._sleep(int(2.0e7))      # ~10 ms of spin so event timestamps are paced by the GPU, not by Python
+        for _ in range(args.steps):
+            generation(decode_events=pairs)
+        torch.cuda.synchronize()
+    dur_ms = np.array([a.elapsed_time(b) for a, b in pairs]).reshape(args.steps, wl.D, -1)   # [step, call, launches]
+    ms_depth = dur_ms.mean(axis=(0, 2))                                                     # mean per launch at each depth
+    n_per_depth = dur_ms.shape[2]
+    alg_total = sum(per_depth[t]["algorithmic"] for t in range(wl.D)) * n_per_depth * args.steps
+    und_total = sum(per_depth[t]["undeduplicated"] for t in range(wl.D)) * n_per_depth * args.steps
+    achieved_gbs = alg_total / (dur_ms.sum() * 1e-3) / 1e9
+
+    # ---- C. end to end: host buffers in, host buffers out, copies inside the timed region ----------
+    e2e = run_e2e(args, run, S0, calls, outs, units_per_step, barrier)
+
+    if world > 1:
+        t = torch.tensor([ms_total, e2e["ms_per_step"]], device=dev, dtype=torch.float64)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        ms_total, e2e["ms_per_step"] = float(t[0]), float(t[1])
+        e2e["value"] = world * units_per_step / (e2e["ms_per_step"] * 1e-3)
+
+    peaks_file = ROOT / "MEASURED_PEAKS.json"
+    if peaks_file.exists():
+        peak, peak_src = float(json.loads(peaks_file.read_text())["hbm_gbs"]), "of measured (MEASURED_PEAKS.json hbm_gbs)"
+    else:
+        peak, peak_src = FALLBACK_HBM_GBS, "of fallback"
+    ms_per_step = ms_total / args.steps
+    line = {
+        "metric": METRIC, "value": world * units_per_step / (ms_per_step * 1e-3), "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": describe(wl), "step": "one whole generation: reset, store S_0, then per decode call "
+                   "reorder + per layer append + decode", "units_per_step": units_per_step,
+                   "l2": "inputs larger than L2 (%.1f GiB of records, queries and states per step)" %
+                         ((wl.R * wl.W * wl.H * wl.L * wl.D * (wl.record_bytes + wl.dk * wl.elem_bytes)
+                           + wl.R * wl.L * wl.H * wl.dk * wl.dv * 4) / 2 ** 30),
+                   "out_dtype": out_dtype, "launch": mode, "parallelism": f"replicas x{world} (requests are independent)",
+                   "tensor_core_path": bool(ctx.onela_uses_tensor_core_path())},
+        "clocks": clocks.summary(),
+        "e2e": {"value": e2e["value"], "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                "ms_per_step": e2e["ms_per_step"]},
+        "gpu_launches": int(launches_per_step * args.steps),
+        "roofline": {"bound": "hbm", "achieved": achieved_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": achieved_gbs / peak, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "peak_source": peak_src,
+                     "kernel": "decode_step (all requests of one layer per launch)",
+                     "bytes": "algorithmic: S_0 once + each distinct record once + q + o + ancestry rows",
+                     "undeduplicated_gbs": und_total / (dur_ms.sum() * 1e-3) / 1e9,
+                     "per_depth": [{"depth": t + 1, "us": float(ms_depth[t] * 1e3),
+                                    "algorithmic_MB": per_depth[t]["algorithmic"] / 1e6,
+                                    "frac": per_depth[t]["algorithmic"] / (ms_depth[t] * 1e-3) / 1e9 / peak}
+                                   for t in range(wl.D)]},
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(wl, reps=1, gen_device=dev)
+    return line
+
+
+def run_e2e(args, run, S0, calls, outs, units_per_step, barrier) -> dict:
+    """The same generation with every input starting in pinned host memory and every output read back."""
+    ctx, wl = run.ctx, run.wl
+    pin = lambda t: t.cpu().pin_memory()
+    hS0 = {k: pin(v) for k, v in S0.items()}
+    hcalls = [{"parents": None if c["parents"] is None else pin(c["parents"]),
+               "layers": [{n: pin(x) for n, x in lay.items()} for lay in c["layers"]]} for c in calls]
+    houts = [torch.empty(o.shape, dtype=o.dtype).pin_memory() for o in outs]
+    dS0 = next(iter(S0.values())).clone()
+    dcall = {"parents": torch.empty_like(calls[-1]["parents"]) if wl.D > 1 else None,
+             "layers": [{n: torch.empty_like(x) for n, x in lay.items()} for lay in calls[0]["layers"]]}
+    h2d = sum(v.numel() * v.element_size() for v in hS0.values())
+    for c in hcalls:
+        h2d += 0 if c["parents"] is None else c["parents"].numel() * 4
+        h2d += sum(x.numel() * x.element_size() for lay in c["layers"] for x in lay.values())
+    d2h = sum(o.numel() * o.element_size() for o in houts) * wl.D
+
+    def generation():
+        ctx.onela_reset()
+        for key, hS in hS0.items():
+            dS0.copy_(hS, non_blocking=True)
+            ctx.onela_init_shared_state(key[0], key[1], dS0)
+        for hc in hcalls:
+            stage = {"parents": None, "layers": dcall["layers"]}
+            if hc["parents"] is not None:
+                dcall["parents"].copy_(hc["parents"], non_blocking=True)
+                stage["parents"] = dcall["parents"]
+            for dl, hl in zip(dcall["layers"], hc["layers"]):
+                for n in dl:
+                    dl[n].copy_(hl[n], non_blocking=True)
+            run.run_call(stage, outs)
+            for ho, o in zip(houts, outs):
+                ho.copy_(o, non_blocking=True)
+
+    for _ in range(max(1, min(args.warmup, 2))):
+        generation()
+    barrier()
+    n = max(1, min(args.steps, 3))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(n):
+        generation()
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1) / n
+    return {"value": units_per_step / (ms * 1e-3), "ms_per_step": ms, "h2d": int(h2d), "d2h": int(d2h)}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle timing (the reported baseline, and the whole of --impl reference)
+# ------------------------------------------------------------------------------------------------
+def cpu_sample(wl: inputs.Workload, gen_device) -> dict:
+    """Inputs of the bounded sample: every (beam, head) unit of every decode call of TWO (request,
+    layer) pairs of the workload - the first and the last - with their true S_0 (oracle prefill)."""
+    import oracle
+    pairs = sorted({(0, 0), (wl.R - 1, wl.L - 1)})
+    sample = []
+    for (r, l) in pairs:
+        parts = [inputs.prompt_tokens(wl, r, l, a, min(a + 2048, wl.prompt_len), device=gen_device)
+                 for a in range(0, wl.prompt_len, 2048)]
+        p = {n: torch.cat([x[n] for x in parts]).cpu() for n in ("k", "v", "alpha", "beta")}
+        S0 = oracle.prefill(p["k"], p["v"], p["alpha"], p["beta"]).astype(np.float32)
+        steps = [{n: x.cpu().float().numpy() for n, x in inputs.decode_token(wl, r, l, t, device=gen_device).items()}
+                 for t in range(wl.D)]
+        qs = [inputs.decode_query(wl, r, l, t, device=gen_device).cpu().float().numpy() for t in range(wl.D)]
+        par = [None] + [inputs.parents(wl, r, t).numpy() for t in range(1, wl.D)]
+        sample.append((S0, steps, par, qs))
+    return {"pairs": pairs, "data": sample, "units": len(pairs) * wl.D * wl.W * wl.H}
+
+
+def time_cpu_sample(sample) -> float:
+    import oracle
+    t0 = time.perf_counter()
+    for (S0, steps, par, qs) in sample["data"]:
+        for t in range(len(steps)):
+            oracle.decode(S0, steps[:t + 1], par[:t + 1], qs[t])
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(wl: inputs.Workload, reps: int, gen_device) -> dict:
+    import oracle
+    sample = cpu_sample(wl, gen_device)
+    secs = min(time_cpu_sample(sample) for _ in range(max(1, reps)))
+    return {"value": sample["units"] / secs, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "seconds": secs,
+            "sample": f"all {wl.W}x{wl.H} (beam, head) units of all {wl.D} decode calls of (request, layer) pairs "
+                      f"{sample['pairs']} = {sample['units']} decodes, fp64 full-state replay (OpenMP)"}
+
+
+def run_reference(args) -> dict:
+    import oracle
+    wl = workload_by_name(args.workload)
+    gen_device = torch.device("cuda", 0) if torch.cuda.is_available() else torch.device("cpu")
+    sample = cpu_sample(wl, gen_device)
+    for _ in range(args.warmup):
+        time_cpu_sample(sample)
+    secs = [time_cpu_sample(sample) for _ in range(args.steps)]
+    per = sum(secs) / len(secs)
+    value = sample["units"] / per
+    desc = {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"each step = all {wl.W}x{wl.H} units of all {wl.D} decode calls of (request, layer) pairs "
+                      f"{sample['pairs']} = {sample['units']} decodes"}
+    return {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": per * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": describe(wl), "note": "CPU fp64 oracle (full-state replay) on the host cores; "
+                       "the paper ships no code, so the oracle is the reference arm"},
+            "cpu_baseline": desc,
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg4")
+    ap.add_argument("--out-dtype", default=None, choices=[None, "fp32", "bf16"])
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            print(json.dumps(run_reference(args)), flush=True)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    line = run_ours(args, rank, world, local_rank)
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
