@@ -153,7 +153,7 @@ onela_status onela_create(const onela_config* cfg, void* workspace_dev, size_t w
         r.has_state.assign(cfg->num_layers, 0);
         r.appended_depth.assign(cfg->num_layers, -1);
     }
-    ctx->tensor_core = false;
+    ctx->tensor_core = decode_sm100_supported(cfg->dk, cfg->dv, cfg->rec_dtype) && !(cfg->flags & ONELA_FLAG_FORCE_GENERIC);
     *out = ctx;
     return ONELA_OK;
 }
@@ -337,7 +337,8 @@ onela_status onela_decode_step(onela_ctx* ctx, int32_t req_begin, int32_t req_co
     a.s0_swizzled = ctx->tensor_core;
     for (int i = 0; i < req_count; ++i) a.bases.base[i] = ctx->req[req_begin + i].step_base.back();
     bool supported = true;
-    const cudaError_t e = launch_decode_generic(a, c.dk, c.dv, c.rec_dtype, c.out_dtype, &supported, s);
+    const cudaError_t e = ctx->tensor_core ? launch_decode_sm100(a, c.out_dtype, s)
+                                           : launch_decode_generic(a, c.dk, c.dv, c.rec_dtype, c.out_dtype, &supported, s);
     if (!supported) return ONELA_E_UNSUPPORTED;
     if (e != cudaSuccess) return ONELA_E_CUDA;
     ctx->launches++;
