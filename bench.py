@@ -129,9 +129,11 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
     wl = workload_by_name(args.workload)
+    if args.layers:
+        wl = wl.scaled(L=args.layers)
     out_dtype = args.out_dtype or wl.dtype
     out_bytes = 4 if out_dtype == "fp32" else 2
-    run = WorkloadRun(wl, dev, out_dtype)
+    run = WorkloadRun(wl, dev, out_dtype, flags=2 if args.force_generic else 0)
     ctx = run.ctx
     run.prefill_states()
     S0 = {(r, l): ctx.onela_export_shared_state(r, l) for r in range(wl.R) for l in range(wl.L)}
@@ -153,6 +155,13 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
         if world > 1:
             torch.distributed.barrier()
         torch.cuda.synchronize()
+
+    if args.profile:   # plain eager generations for a profiler to attach to: no graph, no timing legs
+        for _ in range(args.steps):
+            generation()
+        torch.cuda.synchronize()
+        return {"profile": True, "workload": describe(wl), "generations": args.steps,
+                "launches": int(ctx.onela_launch_count()), "decode_bytes_per_depth": per_depth}
 
     # ---- A. whole-step throughput, inputs resident: CUDA-graph replay of one generation -----------
     side = torch.cuda.Stream()
@@ -204,13 +213,16 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     achieved_gbs = alg_total / (dur_ms.sum() * 1e-3) / 1e9
 
     # ---- C. end to end: host buffers in, host buffers out, copies inside the timed region ----------
-    e2e = run_e2e(args, run, S0, calls, outs, units_per_step, barrier)
+    if args.no_e2e:
+        e2e = {"value": None, "ms_per_step": 0.0, "h2d": 0, "d2h": 0}
+    else:
+        e2e = run_e2e(args, run, S0, calls, outs, units_per_step, barrier)
 
     if world > 1:
         t = torch.tensor([ms_total, e2e["ms_per_step"]], device=dev, dtype=torch.float64)
         torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
         ms_total, e2e["ms_per_step"] = float(t[0]), float(t[1])
-        e2e["value"] = world * units_per_step / (e2e["ms_per_step"] * 1e-3)
+        e2e["value"] = None if args.no_e2e else world * units_per_step / (e2e["ms_per_step"] * 1e-3)
 
     peaks_file = ROOT / "MEASURED_PEAKS.json"
     if peaks_file.exists():
@@ -370,9 +382,13 @@ def main():
     ap.add_argument("--workload", default="cfg4")
     ap.add_argument("--out-dtype", default=None, choices=[None, "fp32", "bf16"])
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling)")
+    ap.add_argument("--force-generic", action="store_true", help="run the CUDA-core decode kernel")
+    ap.add_argument("--profile", action="store_true", help="eager generations only, for ncu")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (kernel experiments)")
     args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" and not args.profile else args.warmup
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

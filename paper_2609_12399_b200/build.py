@@ -15,7 +15,7 @@ OBJ = PKG / "build"
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-I", str(ROOT / "include"), "-I", str(CSRC),
-]
+] + os.environ.get("ONELA_NVCC_EXTRA", "").split()   # extra flags (e.g. -D switches) for experiments
 
 
 def _nvcc() -> str:

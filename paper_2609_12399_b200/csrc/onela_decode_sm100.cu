@@ -15,6 +15,8 @@
 //              memory, the fold groups add their corr registers and store coalesced rows.
 // Every wait is bounded: on expiry the CTA records ONELA_E_TIMEOUT in the status word, stops taking
 // tiles, releases its tensor memory and returns.
+#include <cstdio>
+
 #include "onela_internal.h"
 #include "onela_layout.cuh"
 
@@ -120,21 +122,51 @@ struct Rec {           // one lane's share of a record: 2 x 8 elements of k, 2 x
     float2 gate;
 };
 
-__device__ __forceinline__ Rec load_rec(const __nv_bfloat16* kv, const float2* gates, long long row, int g) {
-    const uint4* p = reinterpret_cast<const uint4*>(kv + row * (DK + DV));
+__device__ __forceinline__ Rec load_rec(const char* kv, const float2* gates, long long row, int g) {
+    const uint4* p = reinterpret_cast<const uint4*>(kv + row * ((DK + DV) * 2)) + g;
     Rec r;
-    r.k0 = __ldg(p + g);
-    r.k1 = __ldg(p + 8 + g);
-    r.v0 = __ldg(p + 16 + g);
-    r.v1 = __ldg(p + 24 + g);
+    r.k0 = __ldg(p);
+    r.k1 = __ldg(p + 8);
+    r.v0 = __ldg(p + 16);
+    r.v1 = __ldg(p + 24);
     r.gate = __ldg(gates + row);
     return r;
 }
-__device__ __forceinline__ void unpack8(const uint4& x, float* o) {
-    unpack_bf16x2(x.x, o[0], o[1]);
-    unpack_bf16x2(x.y, o[2], o[3]);
-    unpack_bf16x2(x.z, o[4], o[5]);
-    unpack_bf16x2(x.w, o[6], o[7]);
+// two packed bf16 -> float2 {element 0, element 1}, exactly
+__device__ __forceinline__ float2 up2(uint32_t w) {
+    return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
+__device__ __forceinline__ void unpack8(const uint4& x, float2* o) {
+    o[0] = up2(x.x); o[1] = up2(x.y); o[2] = up2(x.z); o[3] = up2(x.w);
+}
+
+// One fold step on this lane's 16 elements (packed fp32x2 FMAs), with the 8-lane dot reduction:
+//   c~ = k . r~ ;  corr += (decay beta c~) v ;  r~ -= (beta c~) k ;  decay *= alpha
+__device__ __forceinline__ void fold_step(const Rec& rec, float2* r, float2* corr, float& decay) {
+    float2 kx[8];
+    unpack8(rec.k0, kx);
+    unpack8(rec.k1, kx + 4);
+    float2 d0 = make_float2(0.f, 0.f), d1 = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int e = 0; e < 8; e += 2) {
+        d0 = __ffma2_rn(kx[e], r[e], d0);
+        d1 = __ffma2_rn(kx[e + 1], r[e + 1], d1);
+    }
+    float dot = (d0.x + d0.y) + (d1.x + d1.y);
+    dot += __shfl_xor_sync(0xffffffffu, dot, 4);
+    dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+    dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+    const float bc = rec.gate.y * dot;
+    const float wv = decay * bc;
+    const float2 nbc2 = make_float2(-bc, -bc), wv2 = make_float2(wv, wv);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) r[e] = __ffma2_rn(kx[e], nbc2, r[e]);
+    float2 vx[8];
+    unpack8(rec.v0, vx);
+    unpack8(rec.v1, vx + 4);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) corr[e] = __ffma2_rn(vx[e], wv2, corr[e]);
+    decay *= rec.gate.x;
 }
 
 template <typename OutT>
@@ -173,14 +205,47 @@ __global__ void __launch_bounds__(THREADS, 2) decode_sm100_kernel(const DecodeAr
     const int t_begin = (int)(((long long)blockIdx.x * total_tiles) / gridDim.x);
     const int t_end = (int)(((long long)(blockIdx.x + 1) * total_tiles) / gridDim.x);
 
-    const __nv_bfloat16* kv = reinterpret_cast<const __nv_bfloat16*>(a.kv);
+    const char* kv = a.kv;
+    const __nv_bfloat16* qbase = static_cast<const __nv_bfloat16*>(a.q);
     int cur_pair = -1;
     uint32_t s0_phase = 0, mma_phase = 0;
     int failed = 0;
 
-    for (int tile = t_begin; tile < t_end; ++tile) {
+    // Decompose a tile index and fetch what its fold needs first: the query and the beam's own record.
+    struct TileHead {
+        int req, h, b, bb;
+        bool active;
+        uint4 q0, q1;
+        Rec own;
+    };
+    auto open_tile = [&](int tile) {
+        TileHead t;
         const int pair = tile / tiles_per_pair, tb = tile - pair * tiles_per_pair;
-        const int req = pair / a.H, h = pair - req * a.H;
+        t.req = pair / a.H;
+        t.h = pair - t.req * a.H;
+        t.b = tb * NT + grp;
+        t.active = t.b < a.W;
+        t.bb = t.active ? t.b : a.W - 1;   // idle groups shadow a live beam: loads and shuffles stay uniform
+        const uint4* qp = reinterpret_cast<const uint4*>(qbase + (((long long)t.req * a.W + t.bb) * a.H + t.h) * DK) + g;
+        t.q0 = __ldg(qp);
+        t.q1 = __ldg(qp + 8);
+        t.own = load_rec(kv, a.gates, (long long)t.h * a.arena_slots + a.bases.base[t.req] + t.bb, g);
+        return t;
+    };
+
+#ifdef ONELA_TIMING
+    long long tph[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+    long long tk = clock64();
+    const long long tstart = tk;
+#define ONELA_TICK(i) { const long long now = clock64(); tph[i] += now - tk; tk = now; }
+#else
+#define ONELA_TICK(i)
+#endif
+    TileHead th = open_tile(t_begin);
+    for (int tile = t_begin; tile < t_end; ++tile) {
+        const int req = th.req, h = th.h, b = th.b, bb = th.bb;
+        const bool active = th.active;
+        const int pair = req * a.H + h;
         bool s0_pending = false;
         if (pair != cur_pair) {
             cur_pair = pair;
@@ -192,83 +257,90 @@ __global__ void __launch_bounds__(THREADS, 2) decode_sm100_kernel(const DecodeAr
         }
 
         // ---- 1. fold ------------------------------------------------------------------------------
-        const int b = tb * NT + grp;
-        const bool active = b < a.W;
-        const int bb = active ? b : a.W - 1;
         const long long plane_row0 = (long long)h * a.arena_slots;
-        const int32_t* table = a.table + req * a.table_req_stride;
+        const int32_t* table = a.table + req * a.table_req_stride + bb;
+        const int old = a.depth - 1;          // records older than the beam's own: levels old-1 .. 0
+        // lane g keeps the slot of level g (levels 0..7); deeper chains read the rest on demand
+        const int32_t my_slot = (g < old) ? __ldg(table + (long long)g * a.max_beam) : 0;
+        auto slot_of = [&](int level) -> int32_t {
+            const int32_t s = __shfl_sync(0xffffffffu, my_slot, level & 7, 8);
+            return level < 8 ? s : __ldg(table + (long long)level * a.max_beam);
+        };
+        auto load_level = [&](int level) { return load_rec(kv, a.gates, plane_row0 + slot_of(level), g); };
 
-        float r[16], corr[16];
-        {
-            const uint4* qp = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(a.q) +
-                                                             (((long long)req * a.W + bb) * a.H + h) * DK);
-            const uint4 q0 = __ldg(qp + g), q1 = __ldg(qp + 8 + g);
-            unpack8(q0, r);
-            unpack8(q1, r + 8);
-        }
+        float2 r[8], corr[8];
+        unpack8(th.q0, r);
+        unpack8(th.q1, r + 4);
 #pragma unroll
-        for (int e = 0; e < 16; ++e) corr[e] = 0.f;
+        for (int e = 0; e < 8; ++e) corr[e] = make_float2(0.f, 0.f);
         float decay = 1.f;
-        Rec next = load_rec(kv, a.gates, plane_row0 + a.bases.base[req] + bb, g);
-        for (int level = a.depth - 1; level >= 0; --level) {
-            const Rec cur = next;
-            if (level > 0) {
-                const int32_t slot = __ldg(table + (long long)(level - 1) * a.max_beam + bb);
-                next = load_rec(kv, a.gates, plane_row0 + slot, g);
-            }
-            float kx[16];
-            unpack8(cur.k0, kx);
-            unpack8(cur.k1, kx + 8);
-            float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
-#pragma unroll
-            for (int e = 0; e < 16; e += 4) {
-                d0 = fmaf(kx[e], r[e], d0);
-                d1 = fmaf(kx[e + 1], r[e + 1], d1);
-                d2 = fmaf(kx[e + 2], r[e + 2], d2);
-                d3 = fmaf(kx[e + 3], r[e + 3], d3);
-            }
-            float dot = (d0 + d1) + (d2 + d3);
-            dot += __shfl_xor_sync(0xffffffffu, dot, 4);
-            dot += __shfl_xor_sync(0xffffffffu, dot, 2);
-            dot += __shfl_xor_sync(0xffffffffu, dot, 1);
-            const float bc = cur.gate.y * dot;
-            const float wv = decay * bc;
-            float vx[16];
-            unpack8(cur.v0, vx);
-            unpack8(cur.v1, vx + 8);
-#pragma unroll
-            for (int e = 0; e < 16; ++e) {
-                corr[e] = fmaf(wv, vx[e], corr[e]);
-                r[e] = fmaf(-bc, kx[e], r[e]);
-            }
-            decay *= cur.gate.x;
+
+#ifndef ONELA_PF1
+        // three record buffers rotate: while one is folded the next two are in flight
+        Rec A = th.own, B, C;
+        int level = old;                       // level being folded; level == old is the own record
+        if (level >= 1) B = load_level(level - 1);
+        while (true) {
+            if (level >= 2) C = load_level(level - 2);
+            fold_step(A, r, corr, decay);
+            if (--level < 0) break;
+            if (level >= 2) A = load_level(level - 2);
+            fold_step(B, r, corr, decay);
+            if (--level < 0) break;
+            if (level >= 2) B = load_level(level - 2);
+            fold_step(C, r, corr, decay);
+            if (--level < 0) break;
         }
+#else
+        // two record buffers: while one is folded the next is in flight
+        Rec A = th.own, B;
+        int level = old;
+        while (true) {
+            if (level >= 1) B = load_level(level - 1);
+            fold_step(A, r, corr, decay);
+            if (--level < 0) break;
+            if (level >= 1) A = load_level(level - 1);
+            fold_step(B, r, corr, decay);
+            if (--level < 0) break;
+        }
+#endif
+
+        ONELA_TICK(0)   // fold
 
         // ---- 2. meet S_0 ----------------------------------------------------------------------------
         // lane g holds elements [8g, 8g+8) and [64+8g, 64+8g+8) of the folded query of beam `grp`
         {
             const int sw = grp & 7;
+            const float2 dc = make_float2(decay, decay);
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 const int kb = 2 * c + (g >> 2);            // K block of 32 floats
                 const int ch = 2 * (g & 3);                 // first of two 16-byte chunks inside the 128-byte row
                 uint8_t* row = R_s + kb * R_KB_STRIDE + grp * 128;
-                const float* x = r + 8 * c;
+                float2 x[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) x[e] = __fmul2_rn(r[4 * c + e], dc);
                 *reinterpret_cast<float4*>(row + (((ch) ^ sw) << 4)) =
-                    make_float4(round_tf32(decay * x[0]), round_tf32(decay * x[1]), round_tf32(decay * x[2]), round_tf32(decay * x[3]));
+                    make_float4(round_tf32(x[0].x), round_tf32(x[0].y), round_tf32(x[1].x), round_tf32(x[1].y));
                 *reinterpret_cast<float4*>(row + (((ch + 1) ^ sw) << 4)) =
-                    make_float4(round_tf32(decay * x[4]), round_tf32(decay * x[5]), round_tf32(decay * x[6]), round_tf32(decay * x[7]));
+                    make_float4(round_tf32(x[2].x), round_tf32(x[2].y), round_tf32(x[3].x), round_tf32(x[3].y));
             }
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        ONELA_TICK(1)   // R write
         if (__syncthreads_or(failed)) break;
+        ONELA_TICK(2)   // barrier A
+        // The next tile's query and own record start their trip now and land during the MMA and the
+        // epilogue.  (Issued after the proxy fence above: that fence waits for loads in flight.)
+#ifndef ONELA_NO_XTILE
+        if (tile + 1 < t_end) th = open_tile(tile + 1);
+#endif
+        ONELA_TICK(6)   // open next tile
 
         if (tid == 0) {
             bool ok = true;
-            if (s0_pending) {
-                ok = mbar_wait(bar_s0, s0_phase);
-            }
+            if (s0_pending) ok = mbar_wait(bar_s0, s0_phase);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             if (ok) {
 #pragma unroll
@@ -283,11 +355,13 @@ __global__ void __launch_bounds__(THREADS, 2) decode_sm100_kernel(const DecodeAr
             umma_commit(bar_mma);   // arrives when the MMAs above (if any) have completed
         }
         if (s0_pending) s0_phase ^= 1;
+        ONELA_TICK(7)   // S0 wait + MMA issue (thread 0)
 
         // ---- 3. finish --------------------------------------------------------------------------------
         if (!mbar_wait(bar_mma, mma_phase)) failed = 1;
         mma_phase ^= 1;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        ONELA_TICK(3)   // MMA issue + wait
         {
             // warp w reads accumulator rows (dv) 32*(w&3) + lane, beams 16*(w>>2) .. +16
             const int col0 = (warp >> 2) * 16;
@@ -300,6 +374,7 @@ __global__ void __launch_bounds__(THREADS, 2) decode_sm100_kernel(const DecodeAr
         }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         if (__syncthreads_or(failed)) break;
+        ONELA_TICK(4)   // tmem ld + transpose + barrier B
 
         if (active) {
             OutT* out = static_cast<OutT*>(a.out) + (((long long)req * a.W + b) * a.H + h) * DV;
@@ -308,12 +383,22 @@ __global__ void __launch_bounds__(THREADS, 2) decode_sm100_kernel(const DecodeAr
                 const int e0 = (c * 8 + g) * 8;
                 const float4 x0 = *reinterpret_cast<const float4*>(O_s + grp * OP + e0);
                 const float4 x1 = *reinterpret_cast<const float4*>(O_s + grp * OP + e0 + 4);
-                float o[8] = {x0.x + corr[8 * c], x0.y + corr[8 * c + 1], x0.z + corr[8 * c + 2], x0.w + corr[8 * c + 3],
-                              x1.x + corr[8 * c + 4], x1.y + corr[8 * c + 5], x1.z + corr[8 * c + 6], x1.w + corr[8 * c + 7]};
+                const float2* cc = corr + 4 * c;
+                float o[8] = {x0.x + cc[0].x, x0.y + cc[0].y, x0.z + cc[1].x, x0.w + cc[1].y,
+                              x1.x + cc[2].x, x1.y + cc[2].y, x1.z + cc[3].x, x1.w + cc[3].y};
                 store8<OutT>(out + e0, o);
             }
         }
+#ifdef ONELA_NO_XTILE
+        if (tile + 1 < t_end) th = open_tile(tile + 1);
+#endif
+        ONELA_TICK(5)   // store
     }
+#ifdef ONELA_TIMING
+    if ((tid == 0 || tid == 255) && (blockIdx.x == 0 || blockIdx.x == 150 || blockIdx.x == gridDim.x - 1))
+        printf("cta %d tid %d depth %d tiles %d total %lld | fold %lld Rwrite %lld barA %lld mmawait %lld ld+barB %lld store %lld open %lld issue %lld\n",
+               (int)blockIdx.x, tid, a.depth, t_end - t_begin, clock64() - tstart, tph[0], tph[1], tph[2], tph[3], tph[4], tph[5], tph[6], tph[7]);
+#endif
 
     if (failed && tid == 0) {
         if (atomicCAS(a.status, ONELA_OK, ONELA_E_TIMEOUT) == ONELA_OK) a.status[1] = (int32_t)blockIdx.x;
