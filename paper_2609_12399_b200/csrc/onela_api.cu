@@ -47,6 +47,9 @@ Layout carve(const onela_config& c, char* base) {
     };
     l.status = reinterpret_cast<int32_t*>(take(4 * sizeof(int32_t)));
     l.tables = reinterpret_cast<int32_t*>(take((size_t)c.num_requests * 2 * c.max_steps * c.max_beam * sizeof(int32_t)));
+    l.sidx = reinterpret_cast<int32_t*>(take((size_t)c.num_requests * c.max_steps * c.max_beam * sizeof(int32_t)));
+    l.ulist = reinterpret_cast<int32_t*>(take((size_t)c.num_requests * c.max_steps * c.max_beam * sizeof(int32_t)));
+    l.uoff = reinterpret_cast<int32_t*>(take((size_t)c.num_requests * (c.max_steps + 1) * sizeof(int32_t)));
     l.s0 = reinterpret_cast<float*>(take((size_t)c.num_requests * c.num_layers * c.num_heads * c.dv * c.dk * sizeof(float)));
     l.gates = reinterpret_cast<float2*>(take((size_t)c.num_layers * c.num_heads * (size_t)c.arena_slots * sizeof(float2)));
     l.kv = take((size_t)c.num_layers * c.num_heads * (size_t)c.arena_slots * (c.dk + c.dv) * es);
@@ -74,6 +77,8 @@ struct onela_ctx {
         const int d = req[r].depth;
         return lay.tables + r * table_req_stride() + (long long)((d - 1) & 1) * cfg.max_steps * cfg.max_beam;
     }
+    long long sidx_req_stride() const { return (long long)cfg.max_steps * cfg.max_beam; }
+    long long uoff_req_stride() const { return cfg.max_steps + 1; }
     size_t plane_rows() const { return (size_t)cfg.num_heads * (size_t)cfg.arena_slots; }
     char* kv_plane(int l) const { return lay.kv + (size_t)l * plane_rows() * (cfg.dk + cfg.dv) * elem_bytes; }
     float2* gate_plane(int l) const { return lay.gates + (size_t)l * plane_rows(); }
@@ -262,6 +267,18 @@ onela_status onela_reorder_beams(onela_ctx* ctx, int32_t req_begin, int32_t req_
             return ONELA_E_CUDA;
         ctx->launches++;
     }
+    if (!ctx->dry() && ctx->tensor_core && depth_old >= 1) {
+        // distinct-record index of the table just written (buffer depth_old & 1), for the decode kernel's
+        // shared-ancestor staging
+        const int32_t* cur = ctx->lay.tables + req_begin * ctx->table_req_stride() +
+                             (long long)(depth_old & 1) * c.max_steps * c.max_beam;
+        if (launch_dedupe(cur, ctx->table_req_stride(), ctx->lay.sidx + req_begin * ctx->sidx_req_stride(),
+                          ctx->sidx_req_stride(), ctx->lay.ulist + req_begin * ctx->sidx_req_stride(),
+                          ctx->sidx_req_stride(), ctx->lay.uoff + req_begin * ctx->uoff_req_stride(),
+                          ctx->uoff_req_stride(), req_count, W_new, depth_old + 1, c.max_beam, s) != cudaSuccess)
+            return ONELA_E_CUDA;
+        ctx->launches++;
+    }
     for (int i = 0; i < req_count; ++i) {
         ReqState& r = ctx->req[req_begin + i];
         r.depth = depth_old + 1;
@@ -329,6 +346,12 @@ onela_status onela_decode_step(onela_ctx* ctx, int32_t req_begin, int32_t req_co
     a.s0_req_stride = (long long)c.num_layers * ctx->s0_layer_floats();
     a.table_req_stride = ctx->table_req_stride();
     a.arena_slots = c.arena_slots;
+    a.sidx = ctx->lay.sidx + req_begin * ctx->sidx_req_stride();
+    a.ulist = ctx->lay.ulist + req_begin * ctx->sidx_req_stride();
+    a.uoff = ctx->lay.uoff + req_begin * ctx->uoff_req_stride();
+    a.sidx_req_stride = ctx->sidx_req_stride();
+    a.ulist_req_stride = ctx->sidx_req_stride();
+    a.uoff_req_stride = ctx->uoff_req_stride();
     a.req_count = req_count;
     a.W = W;
     a.H = c.num_heads;

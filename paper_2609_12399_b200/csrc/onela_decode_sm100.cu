@@ -1,20 +1,27 @@
 // Fused decode kernel for B200 (sm_100a): dk = dv = 128, bf16 records.
 //
-// Persistent CTAs (two per SM) walk a contiguous range of work items (request, head, tile of 32 beams).
-// For every tile:
+// One persistent CTA per SM (512 threads) walks a contiguous range of work items (request, head, tile of
+// TN beams).  Consecutive tiles of one (request, head) form a segment; per segment the CTA brings in,
+// with bulk async copies signalled on mbarriers,
+//   - the head's S_0 (the pre-swizzled TF32 image kept in the store): ONE contiguous 64 KiB copy,
+//   - the DISTINCT ancestor records of the oldest chain levels (as many whole levels as fit): beams of a
+//     request share ancestors, so each shared record crosses L2 -> SM once per segment instead of once
+//     per beam, and the fold reads it from shared memory at shared-memory latency.
+// The CTA is split into NP independent pipelines of TN*8 threads, each working on its own tiles with its
+// own named barrier, operand buffers, mbarrier and tensor-memory columns, so one pipeline's waits
+// (DRAM, MMA completion) are filled by the others.  Per tile a pipeline does:
 //   1. fold  - a group of 8 lanes owns one (beam, head) unit and folds its query through the unit's
-//              records newest -> oldest (c = k.r; corr += beta c v; r -= beta c k, decay kept as a scalar).
-//              Records are read with coalesced 16-byte read-only loads (8 lanes cover 128 contiguous
-//              bytes), one level prefetched ahead; shared ancestors are served by L1/L2.
-//   2. meet  - the 32 folded queries are written to shared memory as a K-major, 128-byte-swizzled
-//              operand; the head's S_0 (pre-swizzled, TF32-rounded image in the store) arrives by ONE
-//              64 KiB bulk async copy that was issued before the fold and stays resident while
-//              consecutive tiles belong to the same head; one thread issues 16 tcgen05.mma
-//              (kind::tf32, M = dv = 128, N = 32 beams, K = 8) accumulating fp32 in tensor memory.
-//   3. finish- tcgen05.ld brings the [dv x 32] accumulator back, it is transposed through shared
-//              memory, the fold groups add their corr registers and store coalesced rows.
-// Every wait is bounded: on expiry the CTA records ONELA_E_TIMEOUT in the status word, stops taking
-// tiles, releases its tensor memory and returns.
+//              records newest -> oldest (c = k.r; corr += beta c v; r -= beta c k; decay kept as a scalar;
+//              packed fp32x2 FMAs).  The beam's own record and query were prefetched during the previous
+//              tile; records of levels that are not staged are gathered with coalesced 16-byte read-only
+//              loads, one level ahead; staged levels come from shared memory.
+//   2. meet  - the TN folded queries go to shared memory as a K-major, 128-byte-swizzled operand; one
+//              thread issues 16 tcgen05.mma (kind::tf32, M = dv = 128, N = TN, K = 8), fp32 accumulation
+//              in tensor memory.
+//   3. finish- tcgen05.ld brings the [dv x TN] accumulator back, it is transposed through shared memory,
+//              the fold groups add their corr registers and store coalesced rows.
+// Every wait is bounded: on expiry the pipeline records ONELA_E_TIMEOUT in the status word and stops
+// working (it still joins the CTA-wide barriers), and the CTA releases its tensor memory and returns.
 #include <cstdio>
 
 #include "onela_internal.h"
@@ -24,16 +31,17 @@ namespace onela {
 
 namespace {
 
-constexpr int NT = 32;              // beams per tile (= MMA N)
-constexpr int THREADS = NT * 8;     // 8 lanes per unit
 constexpr int DK = 128, DV = 128;
+constexpr int REC_BYTES = (DK + DV) * 2;       // 512: k | v in bf16
 constexpr int S0_BYTES = DV * DK * 4;          // 65536
-constexpr int R_KB_STRIDE = NT * 128;          // bytes between K blocks of the R operand
-constexpr int R_BYTES = 4 * R_KB_STRIDE;       // 16384
 constexpr int OP = DV + 4;                     // pitch (floats) of the transposed accumulator
-constexpr int O_BYTES = NT * OP * 4;           // 16896
-constexpr int SMEM_BYTES = S0_BYTES + R_BYTES + O_BYTES + 64 + 1024;  // + barriers + alignment slack
-constexpr uint32_t TMEM_COLS = 32;
+constexpr int R_TOTAL = 64 * 128 * 4;          // all pipelines' folded-query operands: 64 beams x 512 B
+constexpr int O_TOTAL = 64 * OP * 4;           // all pipelines' transposed accumulators
+constexpr int STAGE_CAP = 184;                 // distinct ancestor records staged per segment
+constexpr int STAGE_BYTES = STAGE_CAP * REC_BYTES;
+constexpr int GATE_BYTES = STAGE_CAP * 8;
+constexpr int SMEM_BYTES = S0_BYTES + R_TOTAL + O_TOTAL + STAGE_BYTES + GATE_BYTES + 128 + 1024;
+constexpr uint32_t TMEM_COLS = 256;            // 64 beams x 4 partial accumulators (one per K block)
 constexpr int WAIT_LIMIT = 1 << 20;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -67,6 +75,20 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                  : "memory");
 }
 
+// Named barrier over `count` threads that also ORs a predicate across them.
+__device__ __forceinline__ int bar_or(int id, int count, int pred) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "barrier.cta.red.or.pred p, %2, %3, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out)
+        : "r"(pred), "r"(id), "r"(count)
+        : "memory");
+    return (int)out;
+}
+
 // Shared-memory matrix descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
     uint64_t d = 0;
@@ -77,15 +99,27 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
     d |= (uint64_t)2 << 61;                            // SWIZZLE_128B
     return d;
 }
-// Instruction descriptor: D fp32, A and B TF32, both K-major, M = 128, N = NT.
-constexpr uint32_t IDESC = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(NT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+// Instruction descriptor: D fp32, A and B TF32, both K-major, M = 128, N = n.
+__host__ __device__ constexpr uint32_t idesc_tf32(int n) {
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
 
-__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
-        "l"(adesc), "l"(bdesc), "r"(IDESC), "r"(accumulate)
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_tf32_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
@@ -169,25 +203,68 @@ __device__ __forceinline__ void fold_step(const Rec& rec, float2* r, float2* cor
     decay *= rec.gate.x;
 }
 
-template <typename OutT>
-__global__ void __launch_bounds__(THREADS, 2) decode_sm100_kernel(const DecodeArgs a, int total_tiles, int tiles_per_pair) {
+__device__ __forceinline__ Rec load_rec_smem(const uint8_t* stage, const float2* gates_s, int idx, int g) {
+    const uint4* p = reinterpret_cast<const uint4*>(stage + idx * REC_BYTES) + g;
+    Rec r;
+    r.k0 = p[0];
+    r.k1 = p[8];
+    r.v0 = p[16];
+    r.v1 = p[24];
+    r.gate = gates_s[idx];
+    return r;
+}
+
+// Fold `first` (already in registers) and then levels hi .. lo (newest first) fetched by `load`, keeping
+// one record in flight while the previous one is folded.  Two buffers alternate so no record is moved.
+template <class LoadFn>
+__device__ __forceinline__ void fold_chain(const Rec& first, int hi, int lo, LoadFn load, float2* r, float2* corr,
+                                           float& decay) {
+    Rec A = first, B;
+    int level = hi + 1;   // level of the record held in A
+    while (true) {
+        if (level - 1 >= lo) B = load(level - 1);
+        fold_step(A, r, corr, decay);
+        if (--level < lo) break;
+        if (level - 1 >= lo) A = load(level - 1);
+        fold_step(B, r, corr, decay);
+        if (--level < lo) break;
+    }
+}
+
+template <typename OutT, int TN, int NP>
+__global__ void __launch_bounds__(TN * 8 * NP, 1) decode_sm100_kernel(const DecodeArgs a, int total_tiles, int tiles_per_pair) {
+    constexpr int PT = TN * 8;            // threads per pipeline
+    constexpr int R_BYTES = TN * 128 * 4, R_KB_STRIDE = TN * 128;
+    constexpr int O_FLOATS = TN * OP;
+    static_assert(NP * TN <= 64, "at most 64 beams in flight per CTA (operand buffers and tensor-memory columns)");
+
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;            // swizzle atoms need 1024-byte alignment
     uint8_t* smem = smem_raw + (base - raw);
-    const uint32_t s0_addr = base, r_addr = base + S0_BYTES;
-    uint8_t* R_s = smem + S0_BYTES;
-    float* O_s = reinterpret_cast<float*>(smem + S0_BYTES + R_BYTES);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S0_BYTES + R_BYTES + O_BYTES);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2);
-    const uint32_t bar_s0 = smem_u32(bars), bar_mma = smem_u32(bars + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int grp = tid >> 3, g = tid & 7;
+    const int pipe = tid / PT, ptid = tid - pipe * PT;
+    const int grp = ptid >> 3, g = ptid & 7;
+
+    const uint32_t s0_addr = base;
+    const uint32_t r_addr = base + S0_BYTES + pipe * R_BYTES;
+    uint8_t* R_s = smem + S0_BYTES + pipe * R_BYTES;
+    float* O_s = reinterpret_cast<float*>(smem + S0_BYTES + R_TOTAL) + pipe * O_FLOATS;
+    uint8_t* stage = smem + S0_BYTES + R_TOTAL + O_TOTAL;
+    float2* gates_s = reinterpret_cast<float2*>(stage + STAGE_BYTES);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(stage + STAGE_BYTES + GATE_BYTES);
+    // bars[0] S_0 image, bars[1] staged records, bars[2 + p] pipeline p's MMA; then the tmem slot and the abort flag
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 + NP);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    const uint32_t bar_s0 = smem_u32(bars), bar_stage = smem_u32(bars + 1), bar_mma = smem_u32(bars + 2 + pipe);
+    const int bar_id = 1 + pipe;
 
     if (tid == 0) {
         mbar_init(bar_s0, 1);
-        mbar_init(bar_mma, 1);
+        mbar_init(bar_stage, 32);
+        for (int p = 0; p < NP; ++p) mbar_init(smem_u32(bars + 2 + p), 4);   // four issuing threads per tile
+        *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
@@ -199,7 +276,8 @@ __global__ void __launch_bounds__(THREADS, 2) decode_sm100_kernel(const DecodeAr
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t tmem_base = *tmem_slot;
+    // this pipeline's accumulator columns: four partial sums (one per 32-wide K block), TN columns each
+    const uint32_t tmem_acc = *tmem_slot + (uint32_t)(pipe * 4 * TN);
 
     // contiguous range of tiles for this CTA
     const int t_begin = (int)(((long long)blockIdx.x * total_tiles) / gridDim.x);
@@ -207,31 +285,9 @@ __global__ void __launch_bounds__(THREADS, 2) decode_sm100_kernel(const DecodeAr
 
     const char* kv = a.kv;
     const __nv_bfloat16* qbase = static_cast<const __nv_bfloat16*>(a.q);
-    int cur_pair = -1;
-    uint32_t s0_phase = 0, mma_phase = 0;
-    int failed = 0;
-
-    // Decompose a tile index and fetch what its fold needs first: the query and the beam's own record.
-    struct TileHead {
-        int req, h, b, bb;
-        bool active;
-        uint4 q0, q1;
-        Rec own;
-    };
-    auto open_tile = [&](int tile) {
-        TileHead t;
-        const int pair = tile / tiles_per_pair, tb = tile - pair * tiles_per_pair;
-        t.req = pair / a.H;
-        t.h = pair - t.req * a.H;
-        t.b = tb * NT + grp;
-        t.active = t.b < a.W;
-        t.bb = t.active ? t.b : a.W - 1;   // idle groups shadow a live beam: loads and shuffles stay uniform
-        const uint4* qp = reinterpret_cast<const uint4*>(qbase + (((long long)t.req * a.W + t.bb) * a.H + t.h) * DK) + g;
-        t.q0 = __ldg(qp);
-        t.q1 = __ldg(qp + 8);
-        t.own = load_rec(kv, a.gates, (long long)t.h * a.arena_slots + a.bases.base[t.req] + t.bb, g);
-        return t;
-    };
+    const int old = a.depth - 1;          // records older than a beam's own: levels old-1 .. 0
+    uint32_t seg_phase = 0, mma_phase = 0;
+    bool dead = false;                    // this pipeline gave up after a timeout (uniform across the pipeline)
 
 #ifdef ONELA_TIMING
     long long tph[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
@@ -241,172 +297,235 @@ __global__ void __launch_bounds__(THREADS, 2) decode_sm100_kernel(const DecodeAr
 #else
 #define ONELA_TICK(i)
 #endif
-    TileHead th = open_tile(t_begin);
-    for (int tile = t_begin; tile < t_end; ++tile) {
-        const int req = th.req, h = th.h, b = th.b, bb = th.bb;
-        const bool active = th.active;
-        const int pair = req * a.H + h;
-        bool s0_pending = false;
-        if (pair != cur_pair) {
-            cur_pair = pair;
-            s0_pending = true;
-            if (tid == 0) {   // every MMA that read the previous image has completed (bar_mma was waited on)
+
+    // What a tile's fold needs first: the query and the beam's own record (both contiguous per tile).
+    struct TileHead {
+        int b, bb;
+        bool active;
+        uint4 q0, q1;
+        Rec own;
+    };
+
+    for (int seg_begin = t_begin, seg_end; seg_begin < t_end; seg_begin = seg_end) {
+        const int pair = seg_begin / tiles_per_pair;
+        seg_end = min(t_end, (pair + 1) * tiles_per_pair);
+        const int req = pair / a.H, h = pair - req * a.H;
+        const long long plane_row0 = (long long)h * a.arena_slots;
+
+        // How many of the oldest levels fit in the staging buffer (whole levels only; uniform over the CTA).
+        int staged_levels = 0, n_staged = 0;
+        {
+            const int32_t* uoff = a.uoff + req * a.uoff_req_stride;
+            for (int l = 0; l < old; ++l) {
+                const int e = __ldg(uoff + l + 1);
+                if (e > STAGE_CAP) break;
+                staged_levels = l + 1;
+                n_staged = e;
+            }
+        }
+
+        // Everything of the previous segment has been consumed: each pipeline waited for its last MMA
+        // (the S_0 image is free) and finished its last fold (the staged records are free).
+        __syncthreads();
+        if (warp == 0) {
+            if (lane == 0) {
                 mbar_expect_tx(bar_s0, S0_BYTES);
                 bulk_load(s0_addr, a.s0 + req * a.s0_req_stride + (long long)h * (DV * DK), S0_BYTES, bar_s0);
             }
-        }
-
-        // ---- 1. fold ------------------------------------------------------------------------------
-        const long long plane_row0 = (long long)h * a.arena_slots;
-        const int32_t* table = a.table + req * a.table_req_stride + bb;
-        const int old = a.depth - 1;          // records older than the beam's own: levels old-1 .. 0
-        // lane g keeps the slot of level g (levels 0..7); deeper chains read the rest on demand
-        const int32_t my_slot = (g < old) ? __ldg(table + (long long)g * a.max_beam) : 0;
-        auto slot_of = [&](int level) -> int32_t {
-            const int32_t s = __shfl_sync(0xffffffffu, my_slot, level & 7, 8);
-            return level < 8 ? s : __ldg(table + (long long)level * a.max_beam);
-        };
-        auto load_level = [&](int level) { return load_rec(kv, a.gates, plane_row0 + slot_of(level), g); };
-
-        float2 r[8], corr[8];
-        unpack8(th.q0, r);
-        unpack8(th.q1, r + 4);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) corr[e] = make_float2(0.f, 0.f);
-        float decay = 1.f;
-
-#ifndef ONELA_PF1
-        // three record buffers rotate: while one is folded the next two are in flight
-        Rec A = th.own, B, C;
-        int level = old;                       // level being folded; level == old is the own record
-        if (level >= 1) B = load_level(level - 1);
-        while (true) {
-            if (level >= 2) C = load_level(level - 2);
-            fold_step(A, r, corr, decay);
-            if (--level < 0) break;
-            if (level >= 2) A = load_level(level - 2);
-            fold_step(B, r, corr, decay);
-            if (--level < 0) break;
-            if (level >= 2) B = load_level(level - 2);
-            fold_step(C, r, corr, decay);
-            if (--level < 0) break;
-        }
-#else
-        // two record buffers: while one is folded the next is in flight
-        Rec A = th.own, B;
-        int level = old;
-        while (true) {
-            if (level >= 1) B = load_level(level - 1);
-            fold_step(A, r, corr, decay);
-            if (--level < 0) break;
-            if (level >= 1) A = load_level(level - 1);
-            fold_step(B, r, corr, decay);
-            if (--level < 0) break;
-        }
-#endif
-
-        ONELA_TICK(0)   // fold
-
-        // ---- 2. meet S_0 ----------------------------------------------------------------------------
-        // lane g holds elements [8g, 8g+8) and [64+8g, 64+8g+8) of the folded query of beam `grp`
-        {
-            const int sw = grp & 7;
-            const float2 dc = make_float2(decay, decay);
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                const int kb = 2 * c + (g >> 2);            // K block of 32 floats
-                const int ch = 2 * (g & 3);                 // first of two 16-byte chunks inside the 128-byte row
-                uint8_t* row = R_s + kb * R_KB_STRIDE + grp * 128;
-                float2 x[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) x[e] = __fmul2_rn(r[4 * c + e], dc);
-                *reinterpret_cast<float4*>(row + (((ch) ^ sw) << 4)) =
-                    make_float4(round_tf32(x[0].x), round_tf32(x[0].y), round_tf32(x[1].x), round_tf32(x[1].y));
-                *reinterpret_cast<float4*>(row + (((ch + 1) ^ sw) << 4)) =
-                    make_float4(round_tf32(x[2].x), round_tf32(x[2].y), round_tf32(x[3].x), round_tf32(x[3].y));
+            const int32_t* ulist = a.ulist + req * a.ulist_req_stride;
+            const int mine = (n_staged > lane) ? (n_staged - lane + 31) / 32 : 0;
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_stage), "r"(mine * REC_BYTES)
+                         : "memory");
+            for (int i = lane; i < n_staged; i += 32) {
+                const long long row = plane_row0 + __ldg(ulist + i);
+                bulk_load(smem_u32(stage + i * REC_BYTES), kv + row * REC_BYTES, REC_BYTES, bar_stage);
             }
         }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        ONELA_TICK(1)   // R write
-        if (__syncthreads_or(failed)) break;
-        ONELA_TICK(2)   // barrier A
-        // The next tile's query and own record start their trip now and land during the MMA and the
-        // epilogue.  (Issued after the proxy fence above: that fence waits for loads in flight.)
-#ifndef ONELA_NO_XTILE
-        if (tile + 1 < t_end) th = open_tile(tile + 1);
-#endif
-        ONELA_TICK(6)   // open next tile
+        // the gates of the staged records: plain loads by everybody, published by the pipeline barrier below
+        // (each pipeline reads only after its own barrier; all pipelines write the same values)
+        if (ptid < n_staged || n_staged > PT) {
+            const int32_t* ulist = a.ulist + req * a.ulist_req_stride;
+            for (int i = ptid; i < n_staged; i += PT) gates_s[i] = __ldg(a.gates + plane_row0 + __ldg(ulist + i));
+        }
 
-        if (tid == 0) {
-            bool ok = true;
-            if (s0_pending) ok = mbar_wait(bar_s0, s0_phase);
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            if (ok) {
+        auto open_tile = [&](int tile) {
+            TileHead t;
+            const int tb = tile - pair * tiles_per_pair;
+            t.b = tb * TN + grp;
+            t.active = t.b < a.W;
+            t.bb = t.active ? t.b : a.W - 1;   // idle groups shadow a live beam: loads and shuffles stay uniform
+            const uint4* qp = reinterpret_cast<const uint4*>(qbase + (((long long)req * a.W + t.bb) * a.H + h) * DK) + g;
+            t.q0 = __ldg(qp);
+            t.q1 = __ldg(qp + 8);
+            t.own = load_rec(kv, a.gates, plane_row0 + a.bases.base[req] + t.bb, g);
+            return t;
+        };
+
+        int tile = seg_begin + pipe;
+        TileHead th;
+        if (tile < seg_end && !dead) th = open_tile(tile);
+        bool first_in_seg = true;
+        for (; tile < seg_end && !dead; tile += NP) {
+            const int b = th.b, bb = th.bb;
+            const bool active = th.active;
+
+            // ---- 1. fold --------------------------------------------------------------------------
+            // lane g keeps the index of level g (levels 0..7): the position in the staged list for staged
+            // levels, the arena slot otherwise; deeper chains read the rest on demand
+            const int32_t* table = a.table + req * a.table_req_stride + bb;
+            const int32_t* sidx = a.sidx + req * a.sidx_req_stride + bb;
+            int32_t my_idx = 0;
+            if (g < old) my_idx = __ldg((g < staged_levels ? sidx : table) + (long long)g * a.max_beam);
+            auto idx_of = [&](int level) -> int32_t {
+                const int32_t s = __shfl_sync(0xffffffffu, my_idx, level & 7, 8);
+                return level < 8 ? s : __ldg((level < staged_levels ? sidx : table) + (long long)level * a.max_beam);
+            };
+
+            float2 r[8], corr[8];
+            unpack8(th.q0, r);
+            unpack8(th.q1, r + 4);
 #pragma unroll
-                for (int kb = 0; kb < 4; ++kb)
+            for (int e = 0; e < 8; ++e) corr[e] = make_float2(0.f, 0.f);
+            float decay = 1.f;
+
+            // own record, then the gathered levels old-1 .. staged_levels from global memory
+            fold_chain(th.own, old - 1, staged_levels,
+                       [&](int level) { return load_rec(kv, a.gates, plane_row0 + idx_of(level), g); }, r, corr, decay);
+            int failed = 0;
+            if (staged_levels > 0) {
+                if (first_in_seg) {
+                    // the pipeline barrier publishes the staged gates written above; the mbarrier the records
+                    failed |= bar_or(bar_id, PT, 0);
+                    if (!mbar_wait(bar_stage, seg_phase)) failed = 1;
+                }
+                const Rec newest = load_rec_smem(stage, gates_s, idx_of(staged_levels - 1), g);
+                fold_chain(newest, staged_levels - 2, 0,
+                           [&](int level) { return load_rec_smem(stage, gates_s, idx_of(level), g); }, r, corr, decay);
+            }
+            ONELA_TICK(0)   // fold
+
+            // ---- 2. meet S_0 ------------------------------------------------------------------------
+            // lane g holds elements [8g, 8g+8) and [64+8g, 64+8g+8) of the folded query of beam `grp`
+            {
+                const int sw = grp & 7;
+                const float2 dc = make_float2(decay, decay);
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const int kb = 2 * c + (g >> 2);            // K block of 32 floats
+                    const int ch = 2 * (g & 3);                 // first of two 16-byte chunks inside the 128-byte row
+                    uint8_t* row = R_s + kb * R_KB_STRIDE + grp * 128;
+                    float2 x[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) x[e] = __fmul2_rn(r[4 * c + e], dc);
+                    *reinterpret_cast<float4*>(row + (((ch) ^ sw) << 4)) =
+                        make_float4(round_tf32(x[0].x), round_tf32(x[0].y), round_tf32(x[1].x), round_tf32(x[1].y));
+                    *reinterpret_cast<float4*>(row + (((ch + 1) ^ sw) << 4)) =
+                        make_float4(round_tf32(x[2].x), round_tf32(x[2].y), round_tf32(x[3].x), round_tf32(x[3].y));
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            ONELA_TICK(1)   // R write
+            failed |= *abort_flag;
+            failed = bar_or(bar_id, PT, failed);
+            ONELA_TICK(2)   // barrier A
+            if (failed) {
+                dead = true;
+                break;
+            }
+
+            // The next tile's query and own record start their trip now and land during the MMA and the
+            // epilogue.  (Issued after the proxy fence above: that fence waits for loads in flight.)
+            const int b_out = b;
+            const bool active_out = active;
+            if (tile + NP < seg_end) th = open_tile(tile + NP);
+            ONELA_TICK(6)   // open next tile
+
+            // Issuing a tcgen05.mma costs its thread ~90 cycles, so the 16 K steps are spread over four
+            // threads (lane 0 of the pipeline's first four warps), one 32-wide K block and one partial
+            // accumulator each; the epilogue adds the four partials.
+            if ((ptid & 31) == 0 && (ptid >> 5) < 4) {
+                const int kb = ptid >> 5;
+                bool ok = mbar_wait(bar_s0, seg_phase);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                ONELA_TICK(6)   // S0 wait (added to "open")
+                if (ok) {
+                    constexpr uint32_t idesc = idesc_tf32(TN);
+                    const uint64_t ad = umma_desc(s0_addr + kb * (DV * 128)), bd = umma_desc(r_addr + kb * R_KB_STRIDE);
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)
-                        umma_tf32(tmem_base, umma_desc(s0_addr + kb * (DV * 128) + ks * 32),
-                                  umma_desc(r_addr + kb * R_KB_STRIDE + ks * 32), (kb | ks) ? 1u : 0u);
-            } else {
-                failed = 1;
-            }
-            umma_commit(bar_mma);   // arrives when the MMAs above (if any) have completed
-        }
-        if (s0_pending) s0_phase ^= 1;
-        ONELA_TICK(7)   // S0 wait + MMA issue (thread 0)
-
-        // ---- 3. finish --------------------------------------------------------------------------------
-        if (!mbar_wait(bar_mma, mma_phase)) failed = 1;
-        mma_phase ^= 1;
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        ONELA_TICK(3)   // MMA issue + wait
-        {
-            // warp w reads accumulator rows (dv) 32*(w&3) + lane, beams 16*(w>>2) .. +16
-            const int col0 = (warp >> 2) * 16;
-            uint32_t v[16];
-            tmem_ld16(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)col0, v);
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            const int i = (warp & 3) * 32 + lane;
-#pragma unroll
-            for (int j = 0; j < 16; ++j) O_s[(col0 + j) * OP + i] = __uint_as_float(v[j]);
-        }
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        if (__syncthreads_or(failed)) break;
-        ONELA_TICK(4)   // tmem ld + transpose + barrier B
-
-        if (active) {
-            OutT* out = static_cast<OutT*>(a.out) + (((long long)req * a.W + b) * a.H + h) * DV;
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                const int e0 = (c * 8 + g) * 8;
-                const float4 x0 = *reinterpret_cast<const float4*>(O_s + grp * OP + e0);
-                const float4 x1 = *reinterpret_cast<const float4*>(O_s + grp * OP + e0 + 4);
-                const float2* cc = corr + 4 * c;
-                float o[8] = {x0.x + cc[0].x, x0.y + cc[0].y, x0.z + cc[1].x, x0.w + cc[1].y,
-                              x1.x + cc[2].x, x1.y + cc[2].y, x1.z + cc[3].x, x1.w + cc[3].y};
-                store8<OutT>(out + e0, o);
-            }
-        }
-#ifdef ONELA_NO_XTILE
-        if (tile + 1 < t_end) th = open_tile(tile + 1);
+                        umma_tf32(tmem_acc + kb * TN, ad + (uint64_t)(ks * 2), bd + (uint64_t)(ks * 2), idesc, ks ? 1u : 0u);
+                } else {
+                    failed = 1;
+                }
+#ifdef ONELA_TIMING
+                { const long long now = clock64(); tph[8] += now - tk; tk = now; }
 #endif
-        ONELA_TICK(5)   // store
+                umma_commit(bar_mma);   // arrives when this thread's MMAs (if any) have completed
+            }
+            ONELA_TICK(7)   // S0 wait + MMA issue (issuing thread)
+
+            // ---- 3. finish ----------------------------------------------------------------------------
+            if (!mbar_wait(bar_mma, mma_phase)) failed = 1;
+            mma_phase ^= 1;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            ONELA_TICK(3)   // MMA wait
+            {
+                // a warp reads accumulator rows (dv) 32*(warp&3) + lane and 16 of the tile's beams
+                const int col0 = ((ptid >> 5) >> 2) * 16;
+                const uint32_t taddr = tmem_acc + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)col0;
+                uint32_t v0[16], v1[16], v2[16], v3[16];
+                tmem_ld16(taddr, v0);
+                tmem_ld16(taddr + TN, v1);
+                tmem_ld16(taddr + 2 * TN, v2);
+                tmem_ld16(taddr + 3 * TN, v3);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                const int i = (warp & 3) * 32 + lane;
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    O_s[(col0 + j) * OP + i] = (__uint_as_float(v0[j]) + __uint_as_float(v1[j])) +
+                                               (__uint_as_float(v2[j]) + __uint_as_float(v3[j]));
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            failed = bar_or(bar_id, PT, failed);
+            ONELA_TICK(4)   // tmem ld + transpose + barrier B
+            if (failed) {
+                dead = true;
+                break;
+            }
+
+            if (active_out) {
+                OutT* out = static_cast<OutT*>(a.out) + (((long long)req * a.W + b_out) * a.H + h) * DV;
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const int e0 = (c * 8 + g) * 8;
+                    const float4 x0 = *reinterpret_cast<const float4*>(O_s + grp * OP + e0);
+                    const float4 x1 = *reinterpret_cast<const float4*>(O_s + grp * OP + e0 + 4);
+                    const float2* cc = corr + 4 * c;
+                    float o[8] = {x0.x + cc[0].x, x0.y + cc[0].y, x0.z + cc[1].x, x0.w + cc[1].y,
+                                  x1.x + cc[2].x, x1.y + cc[2].y, x1.z + cc[3].x, x1.w + cc[3].y};
+                    store8<OutT>(out + e0, o);
+                }
+            }
+            first_in_seg = false;
+            ONELA_TICK(5)   // store
+        }
+        if (dead && ptid == 0) {
+            *abort_flag = 1;
+            if (atomicCAS(a.status, ONELA_OK, ONELA_E_TIMEOUT) == ONELA_OK) a.status[1] = (int32_t)blockIdx.x;
+        }
+        seg_phase ^= 1;
     }
 #ifdef ONELA_TIMING
-    if ((tid == 0 || tid == 255) && (blockIdx.x == 0 || blockIdx.x == 150 || blockIdx.x == gridDim.x - 1))
-        printf("cta %d tid %d depth %d tiles %d total %lld | fold %lld Rwrite %lld barA %lld mmawait %lld ld+barB %lld store %lld open %lld issue %lld\n",
-               (int)blockIdx.x, tid, a.depth, t_end - t_begin, clock64() - tstart, tph[0], tph[1], tph[2], tph[3], tph[4], tph[5], tph[6], tph[7]);
+    if ((ptid == 0 || ptid == PT - 1) && pipe == NP - 1 && (blockIdx.x == 0 || blockIdx.x == gridDim.x / 2 || blockIdx.x == gridDim.x - 1))
+        printf("cta %d tid %d depth %d tiles %d total %lld | fold %lld Rwrite %lld barA %lld mmawait %lld ld+barB %lld store %lld open %lld issue+commit %lld mmaissue %lld\n",
+               (int)blockIdx.x, tid, a.depth, t_end - t_begin, clock64() - tstart, tph[0], tph[1], tph[2], tph[3], tph[4], tph[5], tph[6], tph[7], tph[8]);
 #endif
 
-    if (failed && tid == 0) {
-        if (atomicCAS(a.status, ONELA_OK, ONELA_E_TIMEOUT) == ONELA_OK) a.status[1] = (int32_t)blockIdx.x;
-    }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 0) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(*tmem_slot), "r"(TMEM_COLS) : "memory");
     }
 }
 
@@ -422,21 +541,30 @@ int sm_count() {
     return cached[dev];
 }
 
-template <typename OutT>
+template <typename OutT, int TN, int NP>
 cudaError_t launch_t(const DecodeArgs& a, cudaStream_t stream) {
-    auto kern = decode_sm100_kernel<OutT>;
+    auto kern = decode_sm100_kernel<OutT, TN, NP>;
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    const int tiles_per_pair = (a.W + NT - 1) / NT;
+    const int tiles_per_pair = (a.W + TN - 1) / TN;
     const int total_tiles = a.req_count * a.H * tiles_per_pair;
-    const int grid = total_tiles < 2 * sm_count() ? total_tiles : 2 * sm_count();
-    kern<<<grid, THREADS, SMEM_BYTES, stream>>>(a, total_tiles, tiles_per_pair);
+    // one CTA per SM; a CTA needs at least one tile per pipeline to keep all its threads busy
+    const int want = (total_tiles + NP - 1) / NP;
+    const int grid = want < sm_count() ? (want < 1 ? 1 : want) : sm_count();
+    kern<<<grid, TN * 8 * NP, SMEM_BYTES, stream>>>(a, total_tiles, tiles_per_pair);
     return cudaGetLastError();
 }
+
+#ifndef ONELA_TILE_N
+#define ONELA_TILE_N 16
+#endif
+#ifndef ONELA_PIPES
+#define ONELA_PIPES 3
+#endif
 
 }  // namespace
 
@@ -445,7 +573,8 @@ bool decode_sm100_supported(int32_t dk, int32_t dv, int32_t rec_dtype) {
 }
 
 cudaError_t launch_decode_sm100(const DecodeArgs& a, int32_t out_dtype, cudaStream_t stream) {
-    return out_dtype == ONELA_DTYPE_BF16 ? launch_t<__nv_bfloat16>(a, stream) : launch_t<float>(a, stream);
+    return out_dtype == ONELA_DTYPE_BF16 ? launch_t<__nv_bfloat16, ONELA_TILE_N, ONELA_PIPES>(a, stream)
+                                         : launch_t<float, ONELA_TILE_N, ONELA_PIPES>(a, stream);
 }
 
 }  // namespace onela

@@ -46,7 +46,101 @@ __global__ void __launch_bounds__(256) export_chains_kernel(const int32_t* __res
     out[i] = table[(long long)level * max_beam + b];
 }
 
+// One CTA per request.  For every level older than the beams' own records: mark which slots of that
+// level some live chain refers to (slots of one level of one request are consecutive, so slot - min is a
+// dense key < max_beam), prefix-sum the marks, and emit the distinct slots in increasing order plus each
+// beam's position in the request's concatenated list.
+__global__ void __launch_bounds__(1024) dedupe_kernel(const int32_t* __restrict__ tables_cur_req0, long long table_req_stride,
+                                                      int32_t* __restrict__ sidx_req0, long long sidx_req_stride,
+                                                      int32_t* __restrict__ ulist_req0, long long ulist_req_stride,
+                                                      int32_t* __restrict__ uoff_req0, long long uoff_req_stride,
+                                                      int32_t W, int32_t depth, int32_t max_beam) {
+    extern __shared__ int32_t marks[];          // [max_beam] marks, then their exclusive prefix sums
+    __shared__ int32_t warp_part[32];
+    __shared__ int32_t s_min, s_total;
+    const int r = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int32_t* table = tables_cur_req0 + r * table_req_stride;
+    int32_t* sidx = sidx_req0 + r * sidx_req_stride;
+    int32_t* ulist = ulist_req0 + r * ulist_req_stride;
+    int32_t* uoff = uoff_req0 + r * uoff_req_stride;
+    const int ipt = (max_beam + 1023) / 1024;   // marks per thread in the scan
+    int32_t off = 0;
+    if (tid == 0) uoff[0] = 0;
+    for (int level = 0; level < depth - 1; ++level) {
+        const int32_t* row = table + (long long)level * max_beam;
+        int32_t mn = 0x7fffffff;
+        for (int b = tid; b < W; b += 1024) mn = min(mn, row[b]);
+        for (int o = 16; o > 0; o >>= 1) mn = min(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        if (lane == 0) warp_part[warp] = mn;
+        for (int i = tid; i < max_beam; i += 1024) marks[i] = 0;
+        __syncthreads();
+        if (warp == 0) {
+            int32_t m = warp_part[lane];
+            for (int o = 16; o > 0; o >>= 1) m = min(m, __shfl_xor_sync(0xffffffffu, m, o));
+            if (lane == 0) s_min = m;
+        }
+        __syncthreads();
+        mn = s_min;
+        for (int b = tid; b < W; b += 1024) marks[row[b] - mn] = 1;
+        __syncthreads();
+        // exclusive scan of marks: thread t owns marks [t*ipt, (t+1)*ipt)
+        int32_t local = 0;
+        for (int j = 0; j < ipt; ++j) {
+            const int i = tid * ipt + j;
+            if (i < max_beam) local += marks[i];
+        }
+        int32_t incl = local;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        __syncthreads();                       // warp_part is reused
+        if (lane == 31) warp_part[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            int32_t w = warp_part[lane], wi = w;
+            for (int o = 1; o < 32; o <<= 1) {
+                const int32_t t = __shfl_up_sync(0xffffffffu, wi, o);
+                if (lane >= o) wi += t;
+            }
+            warp_part[lane] = wi - w;          // exclusive prefix of the warp totals
+            if (lane == 31) s_total = wi;
+        }
+        __syncthreads();
+        int32_t pos = warp_part[warp] + incl - local;
+        for (int j = 0; j < ipt; ++j) {
+            const int i = tid * ipt + j;
+            if (i < max_beam) {
+                const int32_t m = marks[i];
+                marks[i] = pos;                // now the rank of slot mn + i among the distinct slots
+                if (m) ulist[off + pos] = mn + i;
+                pos += m;
+            }
+        }
+        __syncthreads();
+        for (int b = tid; b < W; b += 1024) sidx[(long long)level * max_beam + b] = off + marks[row[b] - mn];
+        off += s_total;
+        if (tid == 0) uoff[level + 1] = off;
+        __syncthreads();
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_dedupe(const int32_t* tables_cur_req0, long long table_req_stride, int32_t* sidx_req0,
+                          long long sidx_req_stride, int32_t* ulist_req0, long long ulist_req_stride,
+                          int32_t* uoff_req0, long long uoff_req_stride, int32_t req_count, int32_t W,
+                          int32_t depth, int32_t max_beam, cudaStream_t stream) {
+    const size_t smem = sizeof(int32_t) * (size_t)max_beam;
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(dedupe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    dedupe_kernel<<<req_count, 1024, smem, stream>>>(tables_cur_req0, table_req_stride, sidx_req0, sidx_req_stride,
+                                                     ulist_req0, ulist_req_stride, uoff_req0, uoff_req_stride, W, depth,
+                                                     max_beam);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_reorder(int32_t* tables_req0, long long table_req_stride, int32_t req_count,
                            const int32_t* parents, int32_t W_new, int32_t W_prev, int32_t depth_old,

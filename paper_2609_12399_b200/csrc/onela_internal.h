@@ -13,6 +13,9 @@ namespace onela {
 struct Layout {
     int32_t* status;   // [4]: code, detail, spare, spare
     int32_t* tables;   // [request][2][max_steps][max_beam] global slot ids (double-buffered per request)
+    int32_t* sidx;     // [request][max_steps][max_beam] per (level, beam): index into the request's distinct-record list
+    int32_t* ulist;    // [request][max_steps*max_beam] distinct record slots of the live chains, oldest level first
+    int32_t* uoff;     // [request][max_steps+1] start of each level inside ulist (uoff[level+1] = end)
     float* s0;         // [request][layer][head][dv*dk] fp32
     float2* gates;     // [layer][head][arena_slots] (alpha, beta)
     char* kv;          // [layer][head][arena_slots][dk + dv] in rec_dtype: one row = k | v of one record
@@ -35,6 +38,10 @@ struct DecodeArgs {
     long long s0_req_stride;     // floats between consecutive requests' store slots (same layer)
     long long table_req_stride;  // ints between consecutive requests' tables
     long long arena_slots;
+    const int32_t* sidx;    // distinct-record index of req_begin (see Layout)
+    const int32_t* ulist;
+    const int32_t* uoff;
+    long long sidx_req_stride, ulist_req_stride, uoff_req_stride;
     int32_t req_count, W, H, depth, max_beam, s0_swizzled;
     BatchBases bases;
 };
@@ -44,6 +51,13 @@ cudaError_t launch_reorder(int32_t* tables_req0, long long table_req_stride, int
                            const int32_t* parents, int32_t W_new, int32_t W_prev, int32_t depth_old,
                            int32_t max_beam, int32_t max_steps, const BatchBases& bases, int32_t* status,
                            cudaStream_t stream);
+// Distinct-record index of the CURRENT ancestry table (levels 0 .. depth-2; the newest level is the
+// beams' own records, all distinct): per level the sorted distinct slots and, per beam, where its
+// ancestor sits in the request's concatenated list.  Integer work only.
+cudaError_t launch_dedupe(const int32_t* tables_cur_req0, long long table_req_stride, int32_t* sidx_req0,
+                          long long sidx_req_stride, int32_t* ulist_req0, long long ulist_req_stride,
+                          int32_t* uoff_req0, long long uoff_req_stride, int32_t req_count, int32_t W,
+                          int32_t depth, int32_t max_beam, cudaStream_t stream);
 cudaError_t launch_export_chains(const int32_t* table_cur, int32_t W, int32_t depth, int32_t max_beam,
                                  int32_t* slots_out, cudaStream_t stream);
 

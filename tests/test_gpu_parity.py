@@ -116,7 +116,10 @@ def test_records_are_stored_bit_exactly_and_never_rewritten():
     c = ctx.cfg
     al = lambda n: (n + 1023) // 1024 * 1024
     off_tables = al(16)
-    off_s0 = off_tables + al(c.num_requests * 2 * c.max_steps * c.max_beam * 4)
+    n_idx = c.num_requests * c.max_steps * c.max_beam * 4
+    off_s0 = (off_tables + al(2 * n_idx)                    # ancestry tables (double-buffered)
+              + al(n_idx) + al(n_idx)                       # distinct-record index: per-beam positions, slot list
+              + al(c.num_requests * (c.max_steps + 1) * 4)) # ... and per-level offsets
     off_gates = off_s0 + al(c.num_requests * c.num_layers * c.num_heads * c.dv * c.dk * 4)
     off_kv = off_gates + al(c.num_layers * c.num_heads * c.arena_slots * 8)
     ws = ctx.workspace[ctx.workspace_ptr - ctx.workspace.data_ptr():]
