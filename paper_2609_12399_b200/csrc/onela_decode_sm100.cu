@@ -35,13 +35,13 @@ constexpr int DK = 128, DV = 128;
 constexpr int REC_BYTES = (DK + DV) * 2;       // 512: k | v in bf16
 constexpr int S0_BYTES = DV * DK * 4;          // 65536
 constexpr int OP = DV + 4;                     // pitch (floats) of the transposed accumulator
-constexpr int R_TOTAL = 64 * 128 * 4;          // all pipelines' folded-query operands: 64 beams x 512 B
-constexpr int O_TOTAL = 64 * OP * 4;           // all pipelines' transposed accumulators
-constexpr int STAGE_CAP = 184;                 // distinct ancestor records staged per segment
+constexpr int R_TOTAL = 96 * 128 * 4;          // all pipelines' folded-query operands: up to 96 beams x 512 B
+constexpr int O_TOTAL = 96 * OP * 4;           // all pipelines' output tiles (corr, then corr + accumulator)
+constexpr int STAGE_CAP = 120;                 // distinct ancestor records staged per segment
 constexpr int STAGE_BYTES = STAGE_CAP * REC_BYTES;
 constexpr int GATE_BYTES = STAGE_CAP * 8;
 constexpr int SMEM_BYTES = S0_BYTES + R_TOTAL + O_TOTAL + STAGE_BYTES + GATE_BYTES + 128 + 1024;
-constexpr uint32_t TMEM_COLS = 256;            // 64 beams x 4 partial accumulators (one per K block)
+constexpr uint32_t TMEM_COLS = 128;            // accumulator columns: one per beam in flight
 constexpr int WAIT_LIMIT = 1 << 20;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -113,15 +113,6 @@ __device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t adesc, uint6
         "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-__device__ __forceinline__ void umma_tf32_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc,
-                                             uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}" ::"r"(tmem_d),
-        "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -151,21 +142,13 @@ __device__ __forceinline__ void store8<__nv_bfloat16>(__nv_bfloat16* p, const fl
                                               pack_bf16x2(x[6], x[7]));
 }
 
-struct Rec {           // one lane's share of a record: 2 x 8 elements of k, 2 x 8 of v, and the gates
-    uint4 k0, k1, v0, v1;
+// One lane's share of a record: NCH x 8 elements of k, NCH x 8 of v (packed bf16), and the gates.
+template <int NCH>
+struct Rec {
+    uint4 k[NCH], v[NCH];
     float2 gate;
 };
 
-__device__ __forceinline__ Rec load_rec(const char* kv, const float2* gates, long long row, int g) {
-    const uint4* p = reinterpret_cast<const uint4*>(kv + row * ((DK + DV) * 2)) + g;
-    Rec r;
-    r.k0 = __ldg(p);
-    r.k1 = __ldg(p + 8);
-    r.v0 = __ldg(p + 16);
-    r.v1 = __ldg(p + 24);
-    r.gate = __ldg(gates + row);
-    return r;
-}
 // two packed bf16 -> float2 {element 0, element 1}, exactly
 __device__ __forceinline__ float2 up2(uint32_t w) {
     return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
@@ -174,69 +157,105 @@ __device__ __forceinline__ void unpack8(const uint4& x, float2* o) {
     o[0] = up2(x.x); o[1] = up2(x.y); o[2] = up2(x.z); o[3] = up2(x.w);
 }
 
-// One fold step on this lane's 16 elements (packed fp32x2 FMAs), with the 8-lane dot reduction:
-//   c~ = k . r~ ;  corr += (decay beta c~) v ;  r~ -= (beta c~) k ;  decay *= alpha
-__device__ __forceinline__ void fold_step(const Rec& rec, float2* r, float2* corr, float& decay) {
-    float2 kx[8];
-    unpack8(rec.k0, kx);
-    unpack8(rec.k1, kx + 4);
-    float2 d0 = make_float2(0.f, 0.f), d1 = make_float2(0.f, 0.f);
+// LPU lanes share one (beam, head) unit; lane g owns the 16-byte chunks c*LPU + g (c < NCH) of every
+// 256-byte vector, i.e. elements [(c*LPU + g)*8, +8): LPU consecutive lanes cover contiguous memory.
+template <int LPU>
+struct Lanes {
+    static constexpr int NCH = 16 / LPU;     // 16-byte chunks per lane per 128-element bf16 vector
+    static constexpr int NP2 = 4 * NCH;      // float2 pairs per lane
+    using R = Rec<NCH>;
+
+    static __device__ __forceinline__ R load_global(const char* kv, const float2* gates, long long row, int g) {
+        const uint4* p = reinterpret_cast<const uint4*>(kv + row * REC_BYTES) + g;
+        R r;
 #pragma unroll
-    for (int e = 0; e < 8; e += 2) {
-        d0 = __ffma2_rn(kx[e], r[e], d0);
-        d1 = __ffma2_rn(kx[e + 1], r[e + 1], d1);
+        for (int c = 0; c < NCH; ++c) {
+            r.k[c] = __ldg(p + c * LPU);
+            r.v[c] = __ldg(p + 16 + c * LPU);
+        }
+        r.gate = __ldg(gates + row);
+        return r;
     }
-    float dot = (d0.x + d0.y) + (d1.x + d1.y);
-    dot += __shfl_xor_sync(0xffffffffu, dot, 4);
-    dot += __shfl_xor_sync(0xffffffffu, dot, 2);
-    dot += __shfl_xor_sync(0xffffffffu, dot, 1);
-    const float bc = rec.gate.y * dot;
-    const float wv = decay * bc;
-    const float2 nbc2 = make_float2(-bc, -bc), wv2 = make_float2(wv, wv);
+    static __device__ __forceinline__ R load_shared(const uint8_t* stage, const float2* gates_s, int idx, int g) {
+        const uint4* p = reinterpret_cast<const uint4*>(stage + idx * REC_BYTES) + g;
+        R r;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) r[e] = __ffma2_rn(kx[e], nbc2, r[e]);
-    float2 vx[8];
-    unpack8(rec.v0, vx);
-    unpack8(rec.v1, vx + 4);
-#pragma unroll
-    for (int e = 0; e < 8; ++e) corr[e] = __ffma2_rn(vx[e], wv2, corr[e]);
-    decay *= rec.gate.x;
-}
-
-__device__ __forceinline__ Rec load_rec_smem(const uint8_t* stage, const float2* gates_s, int idx, int g) {
-    const uint4* p = reinterpret_cast<const uint4*>(stage + idx * REC_BYTES) + g;
-    Rec r;
-    r.k0 = p[0];
-    r.k1 = p[8];
-    r.v0 = p[16];
-    r.v1 = p[24];
-    r.gate = gates_s[idx];
-    return r;
-}
-
-// Fold `first` (already in registers) and then levels hi .. lo (newest first) fetched by `load`, keeping
-// one record in flight while the previous one is folded.  Two buffers alternate so no record is moved.
-template <class LoadFn>
-__device__ __forceinline__ void fold_chain(const Rec& first, int hi, int lo, LoadFn load, float2* r, float2* corr,
-                                           float& decay) {
-    Rec A = first, B;
-    int level = hi + 1;   // level of the record held in A
-    while (true) {
-        if (level - 1 >= lo) B = load(level - 1);
-        fold_step(A, r, corr, decay);
-        if (--level < lo) break;
-        if (level - 1 >= lo) A = load(level - 1);
-        fold_step(B, r, corr, decay);
-        if (--level < lo) break;
+        for (int c = 0; c < NCH; ++c) {
+            r.k[c] = p[c * LPU];
+            r.v[c] = p[16 + c * LPU];
+        }
+        r.gate = gates_s[idx];
+        return r;
     }
+    // One fold step on this lane's elements (packed fp32x2 FMAs), with the LPU-lane dot reduction:
+    //   c~ = k . r~ ;  corr += (decay beta c~) v ;  r~ -= (beta c~) k ;  decay *= alpha
+    static __device__ __forceinline__ void fold_step(const R& rec, float2* r, float2* corr, float& decay) {
+        float2 kx[NP2];
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) unpack8(rec.k[c], kx + 4 * c);
+        float2 d0 = make_float2(0.f, 0.f), d1 = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int e = 0; e < NP2; e += 2) {
+            d0 = __ffma2_rn(kx[e], r[e], d0);
+            d1 = __ffma2_rn(kx[e + 1], r[e + 1], d1);
+        }
+        float dot = (d0.x + d0.y) + (d1.x + d1.y);
+#pragma unroll
+        for (int o = LPU / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+        const float bc = rec.gate.y * dot;
+        const float wv = decay * bc;
+        const float2 nbc2 = make_float2(-bc, -bc), wv2 = make_float2(wv, wv);
+#pragma unroll
+        for (int e = 0; e < NP2; ++e) r[e] = __ffma2_rn(kx[e], nbc2, r[e]);
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) {
+            float2 vx[4];
+            unpack8(rec.v[c], vx);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) corr[4 * c + e] = __ffma2_rn(vx[e], wv2, corr[4 * c + e]);
+        }
+        decay *= rec.gate.x;
+    }
+    // Fold `first` (already in registers) and then levels hi .. lo (newest first) fetched by `load`, keeping
+    // one record in flight while the previous one is folded.  Two buffers alternate so no record is moved.
+    template <class LoadFn>
+    static __device__ __forceinline__ void fold_chain(const R& first, int hi, int lo, LoadFn load, float2* r,
+                                                      float2* corr, float& decay) {
+        R A = first, B;
+        int level = hi + 1;   // level of the record held in A
+        while (true) {
+            if (level - 1 >= lo) B = load(level - 1);
+            fold_step(A, r, corr, decay);
+            if (--level < lo) break;
+            if (level - 1 >= lo) A = load(level - 1);
+            fold_step(B, r, corr, decay);
+            if (--level < lo) break;
+        }
+    }
+};
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async8(uint32_t dst, const void* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
 }
 
-template <typename OutT, int TN, int NP>
-__global__ void __launch_bounds__(TN * 8 * NP, 1) decode_sm100_kernel(const DecodeArgs a, int total_tiles, int tiles_per_pair) {
-    constexpr int PT = TN * 8;            // threads per pipeline
-    constexpr int R_BYTES = TN * 128 * 4, R_KB_STRIDE = TN * 128;
-    constexpr int O_FLOATS = TN * OP;
-    static_assert(NP * TN <= 64, "at most 64 beams in flight per CTA (operand buffers and tensor-memory columns)");
+// LPU lanes per unit, PT threads per pipeline (TU = PT/LPU units folded at a time), RND rounds of units per
+// tile (one MMA group per tile over N = RND * TU beams: issuing a tcgen05.mma costs ~90 cycles whatever its N,
+// so tiles are wide), NP pipelines per CTA.
+template <typename OutT, int LPU, int PT, int RND, int NP>
+__global__ void __launch_bounds__(PT* NP, 1) decode_sm100_kernel(const DecodeArgs a, int total_tiles, int tiles_per_pair) {
+    using L = Lanes<LPU>;
+    using RecT = typename L::R;
+    constexpr int NCH = L::NCH, NP2 = L::NP2;
+    constexpr int TU = PT / LPU;          // units per round
+    constexpr int N = TU * RND;           // beams per tile = MMA N
+    constexpr int R_BYTES = N * 128 * 4, R_KB_STRIDE = N * 128;
+    constexpr int O_FLOATS = N * OP;
+    static_assert(N % 16 == 0 && N <= 256 && (R_KB_STRIDE % 1024) == 0, "MMA N and swizzle-atom alignment");
+    static_assert(NP * R_BYTES <= R_TOTAL && NP * O_FLOATS * 4 <= O_TOTAL && NP * N <= (int)TMEM_COLS, "buffers");
+    static_assert(PT % 128 == 0 || PT >= 128, "a pipeline needs four warps on the four tensor-memory lane quadrants");
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -244,8 +263,8 @@ __global__ void __launch_bounds__(TN * 8 * NP, 1) decode_sm100_kernel(const Deco
     uint8_t* smem = smem_raw + (base - raw);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int pipe = tid / PT, ptid = tid - pipe * PT;
-    const int grp = ptid >> 3, g = ptid & 7;
+    const int pipe = tid / PT, ptid = tid - pipe * PT, pwarp = ptid >> 5;
+    const int grp = ptid / LPU, g = ptid % LPU;
 
     const uint32_t s0_addr = base;
     const uint32_t r_addr = base + S0_BYTES + pipe * R_BYTES;
@@ -263,7 +282,7 @@ __global__ void __launch_bounds__(TN * 8 * NP, 1) decode_sm100_kernel(const Deco
     if (tid == 0) {
         mbar_init(bar_s0, 1);
         mbar_init(bar_stage, 32);
-        for (int p = 0; p < NP; ++p) mbar_init(smem_u32(bars + 2 + p), 4);   // four issuing threads per tile
+        for (int p = 0; p < NP; ++p) mbar_init(smem_u32(bars + 2 + p), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -276,8 +295,7 @@ __global__ void __launch_bounds__(TN * 8 * NP, 1) decode_sm100_kernel(const Deco
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    // this pipeline's accumulator columns: four partial sums (one per 32-wide K block), TN columns each
-    const uint32_t tmem_acc = *tmem_slot + (uint32_t)(pipe * 4 * TN);
+    const uint32_t tmem_acc = *tmem_slot + (uint32_t)(pipe * N);   // this pipeline's accumulator columns
 
     // contiguous range of tiles for this CTA
     const int t_begin = (int)(((long long)blockIdx.x * total_tiles) / gridDim.x);
@@ -290,7 +308,10 @@ __global__ void __launch_bounds__(TN * 8 * NP, 1) decode_sm100_kernel(const Deco
     bool dead = false;                    // this pipeline gave up after a timeout (uniform across the pipeline)
 
 #ifdef ONELA_TIMING
-    long long tph[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+    unsigned long long gt0; unsigned smid;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt0));
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+    long long tph[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     long long tk = clock64();
     const long long tstart = tk;
 #define ONELA_TICK(i) { const long long now = clock64(); tph[i] += now - tk; tk = now; }
@@ -298,12 +319,10 @@ __global__ void __launch_bounds__(TN * 8 * NP, 1) decode_sm100_kernel(const Deco
 #define ONELA_TICK(i)
 #endif
 
-    // What a tile's fold needs first: the query and the beam's own record (both contiguous per tile).
-    struct TileHead {
-        int b, bb;
-        bool active;
-        uint4 q0, q1;
-        Rec own;
+    // What a unit's fold needs first: the query and the beam's own record.
+    struct UnitHead {
+        uint4 q[NCH];
+        RecT own;
     };
 
     for (int seg_begin = t_begin, seg_end; seg_begin < t_end; seg_begin = seg_end) {
@@ -311,6 +330,9 @@ __global__ void __launch_bounds__(TN * 8 * NP, 1) decode_sm100_kernel(const Deco
         seg_end = min(t_end, (pair + 1) * tiles_per_pair);
         const int req = pair / a.H, h = pair - req * a.H;
         const long long plane_row0 = (long long)h * a.arena_slots;
+        const long long own_row0 = plane_row0 + a.bases.base[req];
+        const int32_t* table_r = a.table + req * a.table_req_stride;
+        const int32_t* sidx_r = a.sidx + req * a.sidx_req_stride;
 
         // How many of the oldest levels fit in the staging buffer (whole levels only; uniform over the CTA).
         int staged_levels = 0, n_staged = 0;
@@ -334,181 +356,216 @@ __global__ void __launch_bounds__(TN * 8 * NP, 1) decode_sm100_kernel(const Deco
             }
             const int32_t* ulist = a.ulist + req * a.ulist_req_stride;
             const int mine = (n_staged > lane) ? (n_staged - lane + 31) / 32 : 0;
-            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_stage), "r"(mine * REC_BYTES)
-                         : "memory");
+            mbar_expect_tx(bar_stage, mine * REC_BYTES);   // one arrival per lane, with the bytes it is about to request
             for (int i = lane; i < n_staged; i += 32) {
                 const long long row = plane_row0 + __ldg(ulist + i);
                 bulk_load(smem_u32(stage + i * REC_BYTES), kv + row * REC_BYTES, REC_BYTES, bar_stage);
             }
         }
-        // the gates of the staged records: plain loads by everybody, published by the pipeline barrier below
-        // (each pipeline reads only after its own barrier; all pipelines write the same values)
-        if (ptid < n_staged || n_staged > PT) {
+        // the gates of the staged records: plain loads by every pipeline (same values), published to the
+        // pipeline by the barrier each pipeline takes before its first staged read
+        {
             const int32_t* ulist = a.ulist + req * a.ulist_req_stride;
             for (int i = ptid; i < n_staged; i += PT) gates_s[i] = __ldg(a.gates + plane_row0 + __ldg(ulist + i));
         }
 
-        auto open_tile = [&](int tile) {
-            TileHead t;
-            const int tb = tile - pair * tiles_per_pair;
-            t.b = tb * TN + grp;
-            t.active = t.b < a.W;
-            t.bb = t.active ? t.b : a.W - 1;   // idle groups shadow a live beam: loads and shuffles stay uniform
-            const uint4* qp = reinterpret_cast<const uint4*>(qbase + (((long long)req * a.W + t.bb) * a.H + h) * DK) + g;
-            t.q0 = __ldg(qp);
-            t.q1 = __ldg(qp + 8);
-            t.own = load_rec(kv, a.gates, plane_row0 + a.bases.base[req] + t.bb, g);
-            return t;
+        auto beam_of = [&](int tile, int rnd) { return (tile - pair * tiles_per_pair) * N + rnd * TU + grp; };
+        auto open_unit = [&](int bb) {
+            UnitHead u;
+            const uint4* qp = reinterpret_cast<const uint4*>(qbase + (((long long)req * a.W + bb) * a.H + h) * DK) + g;
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) u.q[c] = __ldg(qp + c * LPU);
+            u.own = L::load_global(kv, a.gates, own_row0 + bb, g);
+            return u;
         };
 
-        int tile = seg_begin + pipe;
-        TileHead th;
-        if (tile < seg_end && !dead) th = open_tile(tile);
+        // tiles go to the pipelines round-robin over the CTA's whole range, so the pipelines stay within one
+        // tile of each other however the range is cut into segments
+        int tile = seg_begin + (pipe - (seg_begin - t_begin) % NP + NP) % NP;
+        UnitHead th;
+        if (tile < seg_end && !dead) th = open_unit(min(beam_of(tile, 0), a.W - 1));
         bool first_in_seg = true;
         for (; tile < seg_end && !dead; tile += NP) {
-            const int b = th.b, bb = th.bb;
-            const bool active = th.active;
-
-            // ---- 1. fold --------------------------------------------------------------------------
-            // lane g keeps the index of level g (levels 0..7): the position in the staged list for staged
-            // levels, the arena slot otherwise; deeper chains read the rest on demand
-            const int32_t* table = a.table + req * a.table_req_stride + bb;
-            const int32_t* sidx = a.sidx + req * a.sidx_req_stride + bb;
-            int32_t my_idx = 0;
-            if (g < old) my_idx = __ldg((g < staged_levels ? sidx : table) + (long long)g * a.max_beam);
-            auto idx_of = [&](int level) -> int32_t {
-                const int32_t s = __shfl_sync(0xffffffffu, my_idx, level & 7, 8);
-                return level < 8 ? s : __ldg((level < staged_levels ? sidx : table) + (long long)level * a.max_beam);
-            };
-
-            float2 r[8], corr[8];
-            unpack8(th.q0, r);
-            unpack8(th.q1, r + 4);
+            // Heads of the later rounds: copied asynchronously into those rounds' own, still unused, operand
+            // rows (record chunks into the R row's four 128-byte pieces, query and gates into the O row).
 #pragma unroll
-            for (int e = 0; e < 8; ++e) corr[e] = make_float2(0.f, 0.f);
-            float decay = 1.f;
+            for (int rnd = 1; rnd < RND; ++rnd) {
+                const int bb = min(beam_of(tile, rnd), a.W - 1);
+                const int u = rnd * TU + grp;
+                const char* rec = kv + (own_row0 + bb) * REC_BYTES;
+                const char* qrow = reinterpret_cast<const char*>(qbase + (((long long)req * a.W + bb) * a.H + h) * DK);
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    const int ci = c * LPU + g;   // 16-byte chunk of a 256-byte vector
+                    cp_async16(smem_u32(R_s + (ci >> 3) * R_KB_STRIDE + u * 128 + (ci & 7) * 16), rec + ci * 16);
+                    cp_async16(smem_u32(R_s + (2 + (ci >> 3)) * R_KB_STRIDE + u * 128 + (ci & 7) * 16), rec + 256 + ci * 16);
+                    cp_async16(smem_u32(O_s + u * OP) + ci * 16, qrow + ci * 16);
+                }
+                if (g == 0) cp_async8(smem_u32(O_s + u * OP) + 256, a.gates + own_row0 + bb);
+            }
+            if (RND > 1) asm volatile("cp.async.commit_group;" ::: "memory");
 
-            // own record, then the gathered levels old-1 .. staged_levels from global memory
-            fold_chain(th.own, old - 1, staged_levels,
-                       [&](int level) { return load_rec(kv, a.gates, plane_row0 + idx_of(level), g); }, r, corr, decay);
             int failed = 0;
-            if (staged_levels > 0) {
-                if (first_in_seg) {
-                    // the pipeline barrier publishes the staged gates written above; the mbarrier the records
-                    failed |= bar_or(bar_id, PT, 0);
-                    if (!mbar_wait(bar_stage, seg_phase)) failed = 1;
-                }
-                const Rec newest = load_rec_smem(stage, gates_s, idx_of(staged_levels - 1), g);
-                fold_chain(newest, staged_levels - 2, 0,
-                           [&](int level) { return load_rec_smem(stage, gates_s, idx_of(level), g); }, r, corr, decay);
-            }
-            ONELA_TICK(0)   // fold
+#pragma unroll
+            for (int rnd = 0; rnd < RND; ++rnd) {
+                const int bb = min(beam_of(tile, rnd), a.W - 1);   // idle groups shadow a live beam: uniform control flow
+                const int u = rnd * TU + grp;                      // row of this unit in the tile's operand buffers
 
-            // ---- 2. meet S_0 ------------------------------------------------------------------------
-            // lane g holds elements [8g, 8g+8) and [64+8g, 64+8g+8) of the folded query of beam `grp`
-            {
-                const int sw = grp & 7;
-                const float2 dc = make_float2(decay, decay);
+                // ---- 1. fold ----------------------------------------------------------------------
+                // lane g keeps the index of level g: the position in the staged list for staged levels, the
+                // arena slot otherwise; chains deeper than LPU read the rest on demand
+                int32_t my_idx = 0;
+                if (g < old) my_idx = __ldg((g < staged_levels ? sidx_r : table_r) + (long long)g * a.max_beam + bb);
+                auto idx_of = [&](int level) -> int32_t {
+                    const int32_t s = __shfl_sync(0xffffffffu, my_idx, level & (LPU - 1), LPU);
+                    return level < LPU ? s
+                                       : __ldg((level < staged_levels ? sidx_r : table_r) + (long long)level * a.max_beam + bb);
+                };
+                UnitHead uh;
+                if (rnd == 0) {
+                    uh = th;
+                } else {
+                    if (rnd == 1) {
+                        asm volatile("cp.async.wait_all;" ::: "memory");
+                        __syncwarp();
+                    }
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    const int kb = 2 * c + (g >> 2);            // K block of 32 floats
-                    const int ch = 2 * (g & 3);                 // first of two 16-byte chunks inside the 128-byte row
-                    uint8_t* row = R_s + kb * R_KB_STRIDE + grp * 128;
-                    float2 x[4];
+                    for (int c = 0; c < NCH; ++c) {
+                        const int ci = c * LPU + g;
+                        uh.own.k[c] = *reinterpret_cast<const uint4*>(R_s + (ci >> 3) * R_KB_STRIDE + u * 128 + (ci & 7) * 16);
+                        uh.own.v[c] = *reinterpret_cast<const uint4*>(R_s + (2 + (ci >> 3)) * R_KB_STRIDE + u * 128 + (ci & 7) * 16);
+                        uh.q[c] = reinterpret_cast<const uint4*>(O_s + u * OP)[ci];
+                    }
+                    uh.own.gate = *reinterpret_cast<const float2*>(O_s + u * OP + 64);
+                    __syncwarp();   // every lane has read the scratch before any lane overwrites it below
+                }
+
+                float2 r[NP2], corr[NP2];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) x[e] = __fmul2_rn(r[4 * c + e], dc);
-                    *reinterpret_cast<float4*>(row + (((ch) ^ sw) << 4)) =
-                        make_float4(round_tf32(x[0].x), round_tf32(x[0].y), round_tf32(x[1].x), round_tf32(x[1].y));
-                    *reinterpret_cast<float4*>(row + (((ch + 1) ^ sw) << 4)) =
-                        make_float4(round_tf32(x[2].x), round_tf32(x[2].y), round_tf32(x[3].x), round_tf32(x[3].y));
+                for (int c = 0; c < NCH; ++c) unpack8(uh.q[c], r + 4 * c);
+#pragma unroll
+                for (int e = 0; e < NP2; ++e) corr[e] = make_float2(0.f, 0.f);
+                float decay = 1.f;
+
+                // own record, then the gathered levels old-1 .. staged_levels from global memory
+                L::fold_chain(uh.own, old - 1, staged_levels,
+                              [&](int level) { return L::load_global(kv, a.gates, plane_row0 + idx_of(level), g); }, r, corr,
+                              decay);
+                if (staged_levels > 0) {
+                    if (first_in_seg) {
+                        // the pipeline barrier publishes the staged gates written above; the mbarrier the records
+                        failed |= bar_or(bar_id, PT, 0);
+                        if (!mbar_wait(bar_stage, seg_phase)) failed = 1;
+                        first_in_seg = false;
+                    }
+                    const RecT newest = L::load_shared(stage, gates_s, idx_of(staged_levels - 1), g);
+                    L::fold_chain(newest, staged_levels - 2, 0,
+                                  [&](int level) { return L::load_shared(stage, gates_s, idx_of(level), g); }, r, corr, decay);
+                }
+
+                // ---- 2. operands: folded query -> K-major swizzled row u; corr -> row u of the output tile
+                {
+                    const int sw = u & 7;
+                    const float2 dc = make_float2(decay, decay);
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) {
+                        const int ci = c * LPU + g;                 // elements [8 ci, 8 ci + 8)
+                        const int kb = ci >> 2;                     // K block of 32 floats
+                        const int ch = 2 * (ci & 3);                // first of two 16-byte chunks inside the 128-byte row
+                        uint8_t* row = R_s + kb * R_KB_STRIDE + u * 128;
+                        float2 x[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) x[e] = __fmul2_rn(r[4 * c + e], dc);
+                        *reinterpret_cast<float4*>(row + (((ch) ^ sw) << 4)) =
+                            make_float4(round_tf32(x[0].x), round_tf32(x[0].y), round_tf32(x[1].x), round_tf32(x[1].y));
+                        *reinterpret_cast<float4*>(row + (((ch + 1) ^ sw) << 4)) =
+                            make_float4(round_tf32(x[2].x), round_tf32(x[2].y), round_tf32(x[3].x), round_tf32(x[3].y));
+                        float* orow = O_s + u * OP + ci * 8;
+                        *reinterpret_cast<float4*>(orow) = make_float4(corr[4 * c].x, corr[4 * c].y, corr[4 * c + 1].x, corr[4 * c + 1].y);
+                        *reinterpret_cast<float4*>(orow + 4) =
+                            make_float4(corr[4 * c + 2].x, corr[4 * c + 2].y, corr[4 * c + 3].x, corr[4 * c + 3].y);
+                    }
                 }
             }
+            ONELA_TICK(0)   // folds + operand writes
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            ONELA_TICK(1)   // R write
             failed |= *abort_flag;
             failed = bar_or(bar_id, PT, failed);
-            ONELA_TICK(2)   // barrier A
+            ONELA_TICK(1)   // barrier A
             if (failed) {
                 dead = true;
                 break;
             }
 
-            // The next tile's query and own record start their trip now and land during the MMA and the
+            // The next tile's first query and record start their trip now and land during the MMA and the
             // epilogue.  (Issued after the proxy fence above: that fence waits for loads in flight.)
-            const int b_out = b;
-            const bool active_out = active;
-            if (tile + NP < seg_end) th = open_tile(tile + NP);
-            ONELA_TICK(6)   // open next tile
+            if (tile + NP < seg_end) th = open_unit(min(beam_of(tile + NP, 0), a.W - 1));
 
-            // Issuing a tcgen05.mma costs its thread ~90 cycles, so the 16 K steps are spread over four
-            // threads (lane 0 of the pipeline's first four warps), one 32-wide K block and one partial
-            // accumulator each; the epilogue adds the four partials.
-            if ((ptid & 31) == 0 && (ptid >> 5) < 4) {
-                const int kb = ptid >> 5;
+            if (ptid == 0) {
                 bool ok = mbar_wait(bar_s0, seg_phase);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                ONELA_TICK(6)   // S0 wait (added to "open")
+                ONELA_TICK(2)   // S0 wait
                 if (ok) {
-                    constexpr uint32_t idesc = idesc_tf32(TN);
-                    const uint64_t ad = umma_desc(s0_addr + kb * (DV * 128)), bd = umma_desc(r_addr + kb * R_KB_STRIDE);
+                    constexpr uint32_t idesc = idesc_tf32(N);
+                    const uint64_t ad = umma_desc(s0_addr), bd = umma_desc(r_addr);
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        umma_tf32(tmem_acc + kb * TN, ad + (uint64_t)(ks * 2), bd + (uint64_t)(ks * 2), idesc, ks ? 1u : 0u);
+                    for (int kb = 0; kb < 4; ++kb)
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks)
+                            umma_tf32(tmem_acc, ad + (uint64_t)((kb * (DV * 128) + ks * 32) >> 4),
+                                      bd + (uint64_t)((kb * R_KB_STRIDE + ks * 32) >> 4), idesc, (kb | ks) ? 1u : 0u);
                 } else {
                     failed = 1;
                 }
-#ifdef ONELA_TIMING
-                { const long long now = clock64(); tph[8] += now - tk; tk = now; }
-#endif
-                umma_commit(bar_mma);   // arrives when this thread's MMAs (if any) have completed
+                umma_commit(bar_mma);   // arrives when the MMAs above (if any) have completed
             }
-            ONELA_TICK(7)   // S0 wait + MMA issue (issuing thread)
+            ONELA_TICK(3)   // MMA issue (issuing thread)
 
             // ---- 3. finish ----------------------------------------------------------------------------
             if (!mbar_wait(bar_mma, mma_phase)) failed = 1;
             mma_phase ^= 1;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            ONELA_TICK(3)   // MMA wait
-            {
-                // a warp reads accumulator rows (dv) 32*(warp&3) + lane and 16 of the tile's beams
-                const int col0 = ((ptid >> 5) >> 2) * 16;
-                const uint32_t taddr = tmem_acc + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)col0;
-                uint32_t v0[16], v1[16], v2[16], v3[16];
-                tmem_ld16(taddr, v0);
-                tmem_ld16(taddr + TN, v1);
-                tmem_ld16(taddr + 2 * TN, v2);
-                tmem_ld16(taddr + 3 * TN, v3);
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            ONELA_TICK(4)   // MMA wait
+            if (pwarp < 4) {
+                // the pipeline's first four warps sit on the four lane quadrants of tensor memory: each adds
+                // accumulator rows (dv) 32*(warp&3) + lane of every beam of the tile onto the stored corr
                 const int i = (warp & 3) * 32 + lane;
+                const uint32_t taddr = tmem_acc + ((uint32_t)((warp & 3) * 32) << 16);
 #pragma unroll
-                for (int j = 0; j < 16; ++j)
-                    O_s[(col0 + j) * OP + i] = (__uint_as_float(v0[j]) + __uint_as_float(v1[j])) +
-                                               (__uint_as_float(v2[j]) + __uint_as_float(v3[j]));
+                for (int c0 = 0; c0 < N; c0 += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(taddr + c0, v);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) O_s[(c0 + j) * OP + i] += __uint_as_float(v[j]);
+                }
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             failed = bar_or(bar_id, PT, failed);
-            ONELA_TICK(4)   // tmem ld + transpose + barrier B
+            ONELA_TICK(5)   // tmem ld + add + barrier B
             if (failed) {
                 dead = true;
                 break;
             }
 
-            if (active_out) {
-                OutT* out = static_cast<OutT*>(a.out) + (((long long)req * a.W + b_out) * a.H + h) * DV;
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    const int e0 = (c * 8 + g) * 8;
-                    const float4 x0 = *reinterpret_cast<const float4*>(O_s + grp * OP + e0);
-                    const float4 x1 = *reinterpret_cast<const float4*>(O_s + grp * OP + e0 + 4);
-                    const float2* cc = corr + 4 * c;
-                    float o[8] = {x0.x + cc[0].x, x0.y + cc[0].y, x0.z + cc[1].x, x0.w + cc[1].y,
-                                  x1.x + cc[2].x, x1.y + cc[2].y, x1.z + cc[3].x, x1.w + cc[3].y};
-                    store8<OutT>(out + e0, o);
+            for (int rnd = 0; rnd < RND; ++rnd) {
+                const int b = beam_of(tile, rnd);
+                const int u = rnd * TU + grp;
+                if (b < a.W) {
+                    OutT* out = static_cast<OutT*>(a.out) + (((long long)req * a.W + b) * a.H + h) * DV;
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) {
+                        const int e0 = (c * LPU + g) * 8;
+                        const float4 x0 = *reinterpret_cast<const float4*>(O_s + u * OP + e0);
+                        const float4 x1 = *reinterpret_cast<const float4*>(O_s + u * OP + e0 + 4);
+                        const float o[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+                        store8<OutT>(out + e0, o);
+                    }
                 }
             }
-            first_in_seg = false;
-            ONELA_TICK(5)   // store
+            ONELA_TICK(6)   // store
         }
         if (dead && ptid == 0) {
             *abort_flag = 1;
@@ -517,9 +574,14 @@ __global__ void __launch_bounds__(TN * 8 * NP, 1) decode_sm100_kernel(const Deco
         seg_phase ^= 1;
     }
 #ifdef ONELA_TIMING
+    if (tid == 0 && (a.depth == 1)) {
+        unsigned long long gt1;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt1));
+        printf("span cta %d sm %u start %llu end %llu\n", (int)blockIdx.x, smid, gt0 % 100000000ull, gt1 % 100000000ull);
+    }
     if ((ptid == 0 || ptid == PT - 1) && pipe == NP - 1 && (blockIdx.x == 0 || blockIdx.x == gridDim.x / 2 || blockIdx.x == gridDim.x - 1))
-        printf("cta %d tid %d depth %d tiles %d total %lld | fold %lld Rwrite %lld barA %lld mmawait %lld ld+barB %lld store %lld open %lld issue+commit %lld mmaissue %lld\n",
-               (int)blockIdx.x, tid, a.depth, t_end - t_begin, clock64() - tstart, tph[0], tph[1], tph[2], tph[3], tph[4], tph[5], tph[6], tph[7], tph[8]);
+        printf("cta %d tid %d depth %d tiles %d total %lld | folds %lld barA %lld s0wait %lld mmaissue %lld mmawait %lld ld+barB %lld store %lld\n",
+               (int)blockIdx.x, tid, a.depth, t_end - t_begin, clock64() - tstart, tph[0], tph[1], tph[2], tph[3], tph[4], tph[5], tph[6]);
 #endif
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -541,29 +603,36 @@ int sm_count() {
     return cached[dev];
 }
 
-template <typename OutT, int TN, int NP>
+template <typename OutT, int LPU, int PT, int RND, int NP>
 cudaError_t launch_t(const DecodeArgs& a, cudaStream_t stream) {
-    auto kern = decode_sm100_kernel<OutT, TN, NP>;
+    auto kern = decode_sm100_kernel<OutT, LPU, PT, RND, NP>;
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    const int tiles_per_pair = (a.W + TN - 1) / TN;
+    constexpr int N = PT / LPU * RND;
+    const int tiles_per_pair = (a.W + N - 1) / N;
     const int total_tiles = a.req_count * a.H * tiles_per_pair;
-    // one CTA per SM; a CTA needs at least one tile per pipeline to keep all its threads busy
+    // one CTA per SM; a CTA wants at least one tile per pipeline
     const int want = (total_tiles + NP - 1) / NP;
     const int grid = want < sm_count() ? (want < 1 ? 1 : want) : sm_count();
-    kern<<<grid, TN * 8 * NP, SMEM_BYTES, stream>>>(a, total_tiles, tiles_per_pair);
+    kern<<<grid, PT * NP, SMEM_BYTES, stream>>>(a, total_tiles, tiles_per_pair);
     return cudaGetLastError();
 }
 
-#ifndef ONELA_TILE_N
-#define ONELA_TILE_N 16
+#ifndef ONELA_LPU
+#define ONELA_LPU 8
+#endif
+#ifndef ONELA_PT
+#define ONELA_PT 192
+#endif
+#ifndef ONELA_RND
+#define ONELA_RND 2
 #endif
 #ifndef ONELA_PIPES
-#define ONELA_PIPES 3
+#define ONELA_PIPES 2
 #endif
 
 }  // namespace
@@ -573,8 +642,8 @@ bool decode_sm100_supported(int32_t dk, int32_t dv, int32_t rec_dtype) {
 }
 
 cudaError_t launch_decode_sm100(const DecodeArgs& a, int32_t out_dtype, cudaStream_t stream) {
-    return out_dtype == ONELA_DTYPE_BF16 ? launch_t<__nv_bfloat16, ONELA_TILE_N, ONELA_PIPES>(a, stream)
-                                         : launch_t<float, ONELA_TILE_N, ONELA_PIPES>(a, stream);
+    return out_dtype == ONELA_DTYPE_BF16 ? launch_t<__nv_bfloat16, ONELA_LPU, ONELA_PT, ONELA_RND, ONELA_PIPES>(a, stream)
+                                         : launch_t<float, ONELA_LPU, ONELA_PT, ONELA_RND, ONELA_PIPES>(a, stream);
 }
 
 }  // namespace onela
