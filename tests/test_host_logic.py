@@ -68,7 +68,8 @@ def test_workspace_carve_up_size():
     s0 = 4 * 16 * 32 * 128 * 128 * 4
     arena = 16 * 32 * (4 * 512 * 8) * 520
     tables = 4 * 2 * 8 * 512 * 4
-    assert s0 + arena + tables <= n <= s0 + arena + tables + 8 * 1024
+    index = 2 * (4 * 8 * 512 * 4) + 4 * 9 * 4          # distinct-record index: positions, slot list, level offsets
+    assert s0 + arena + tables + index <= n <= s0 + arena + tables + index + 8 * 1024
 
 
 def test_call_order_is_enforced():
