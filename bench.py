@@ -35,14 +35,16 @@ import torch
 ROOT = Path(__file__).resolve().parent
 sys.path.insert(0, str(ROOT))
 
-from paper_2609_12399_b200 import accounting, inputs  # noqa: E402
+from paper_2609_12399_b200 import accounting, inputs, replicas  # noqa: E402
 
 METRIC = "beam-head GDN decodes/s per layer at beam 512"
 UNIT = "decodes/s"
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes per decode launch of the deepest call, from the ncu capture summarised in
-# profiles/ (filled in once a capture exists; None = not captured)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE decode launch of the default workload at its deepest
+# call (depth 8, all 4 requests of one layer), from the ncu capture summarised in
+# profiles/decode_sm100_cfg4_ncu.md; the algorithmic bytes of that same launch are 84.6 MB (the 16.8 MB of
+# outputs were still in L2 when the kernel ended, so DRAM saw the 67.8 MB of reads and little else).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 72.66e6
 
 
 def workload_by_name(name: str) -> inputs.Workload:
@@ -152,8 +154,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
 
     def barrier():
         torch.cuda.synchronize()
-        if world > 1:
-            torch.distributed.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
 
     if args.profile:   # plain eager generations for a profiler to attach to: no graph, no timing legs
@@ -187,10 +188,14 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
         else:
             generation()
 
-    for _ in range(args.warmup):
-        step()
-    barrier()
     with ClockSampler(local_rank) as clocks:
+        for _ in range(args.warmup):
+            step()
+        t_warm = time.perf_counter()          # keep the GPU busy a little longer so clocks settle under load
+        while time.perf_counter() - t_warm < args.settle_seconds:
+            step()
+            torch.cuda.synchronize()
+        barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(args.steps):
@@ -202,14 +207,15 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
         # ---- B. per-launch decode durations for the roofline (eager, GPU kept ahead of the CPU) ------
         pairs = []
         torch.cuda._sleep(int(2.0e7))      # ~10 ms of spin so event timestamps are paced by the GPU, not by Python
-        for _ in range(args.steps):
+        n_b = max(1, min(args.steps, 5))
+        for _ in range(n_b):
             generation(decode_events=pairs)
         torch.cuda.synchronize()
-    dur_ms = np.array([a.elapsed_time(b) for a, b in pairs]).reshape(args.steps, wl.D, -1)   # [step, call, launches]
+    dur_ms = np.array([a.elapsed_time(b) for a, b in pairs]).reshape(n_b, wl.D, -1)   # [step, call, launches]
     ms_depth = dur_ms.mean(axis=(0, 2))                                                     # mean per launch at each depth
     n_per_depth = dur_ms.shape[2]
-    alg_total = sum(per_depth[t]["algorithmic"] for t in range(wl.D)) * n_per_depth * args.steps
-    und_total = sum(per_depth[t]["undeduplicated"] for t in range(wl.D)) * n_per_depth * args.steps
+    alg_total = sum(per_depth[t]["algorithmic"] for t in range(wl.D)) * n_per_depth * n_b
+    und_total = sum(per_depth[t]["undeduplicated"] for t in range(wl.D)) * n_per_depth * n_b
     achieved_gbs = alg_total / (dur_ms.sum() * 1e-3) / 1e9
 
     # ---- C. end to end: host buffers in, host buffers out, copies inside the timed region ----------
@@ -218,11 +224,9 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     else:
         e2e = run_e2e(args, run, S0, calls, outs, units_per_step, barrier)
 
-    if world > 1:
-        t = torch.tensor([ms_total, e2e["ms_per_step"]], device=dev, dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms_total, e2e["ms_per_step"] = float(t[0]), float(t[1])
-        e2e["value"] = None if args.no_e2e else world * units_per_step / (e2e["ms_per_step"] * 1e-3)
+    ms_total, e2e["ms_per_step"] = replicas.max_over_ranks([ms_total, e2e["ms_per_step"]], device=dev)
+    if not args.no_e2e:
+        e2e["value"] = replicas.aggregate_throughput(units_per_step, e2e["ms_per_step"], world)
 
     peaks_file = ROOT / "MEASURED_PEAKS.json"
     if peaks_file.exists():
@@ -231,7 +235,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
         peak, peak_src = FALLBACK_HBM_GBS, "of fallback"
     ms_per_step = ms_total / args.steps
     line = {
-        "metric": METRIC, "value": world * units_per_step / (ms_per_step * 1e-3), "unit": UNIT,
+        "metric": METRIC, "value": replicas.aggregate_throughput(units_per_step, ms_per_step, world), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
@@ -242,12 +246,15 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
                            + wl.R * wl.L * wl.H * wl.dk * wl.dv * 4) / 2 ** 30),
                    "out_dtype": out_dtype, "launch": mode, "parallelism": f"replicas x{world} (requests are independent)",
                    "tensor_core_path": bool(ctx.onela_uses_tensor_core_path())},
-        "clocks": clocks.summary(),
+        "clocks": {**clocks.summary(), "window": "sampled from the warm-up to the end of the timed legs"},
         "e2e": {"value": e2e["value"], "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                 "ms_per_step": e2e["ms_per_step"]},
         "gpu_launches": int(launches_per_step * args.steps),
         "roofline": {"bound": "hbm", "achieved": achieved_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": achieved_gbs / peak, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "peak_source": peak_src,
+                     "frac": achieved_gbs / peak, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                     "traffic_note": "ncu DRAM read+write bytes of one launch at the deepest call (depth %d), whose "
+                                     "algorithmic bytes are %.1f MB; see profiles/" % (wl.D, per_depth[-1]["algorithmic"] / 1e6),
+                     "peak_source": peak_src,
                      "kernel": "decode_step (all requests of one layer per launch)",
                      "bytes": "algorithmic: S_0 once + each distinct record once + q + o + ancestry rows",
                      "undeduplicated_gbs": und_total / (dur_ms.sum() * 1e-3) / 1e9,
@@ -376,12 +383,13 @@ def run_reference(args) -> dict:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4")
     ap.add_argument("--out-dtype", default=None, choices=[None, "fp32", "bf16"])
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--settle-seconds", type=float, default=1.0, help="extra untimed warm-up after the W steps")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling)")
     ap.add_argument("--force-generic", action="store_true", help="run the CUDA-core decode kernel")
     ap.add_argument("--profile", action="store_true", help="eager generations only, for ncu")

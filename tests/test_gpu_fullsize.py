@@ -1,0 +1,100 @@
+"""Parity at the benchmark configs' FULL sizes, in the launch configuration bench.py times (all requests
+of a layer in one batched call, bf16 outputs, the tensor-core kernel).
+
+The oracle cannot replay every unit of these sizes in seconds, so it computes a seeded sample of
+(beam, head) units one by one for a few (request, layer) pairs at several call depths; for those pairs
+S_0 comes from the oracle's fp64 prefill of the seeded prompt (all other pairs: the library's own prefill
+kernel), so both sides consume identical inputs.  Integer work is checked everywhere: the ancestry rows of
+every request at every call against Eq. 5.  One more property holds at any size and is checked on every
+unit: the tensor-core kernel and the CUDA-core kernel, which share no device code, agree.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import evaluators as ev
+import paper_2609_12399_b200 as P
+from paper_2609_12399_b200 import inputs
+from paper_2609_12399_b200.runner import WorkloadRun
+
+from _cases import REL_L2_BAR, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+
+def _oracle_state(wl, r, l):
+    parts = [inputs.prompt_tokens(wl, r, l, a, min(a + 2048, wl.prompt_len), device="cuda")
+             for a in range(0, wl.prompt_len, 2048)]
+    p = {n: torch.cat([x[n] for x in parts]).cpu() for n in ("k", "v", "alpha", "beta")}
+    return torch.from_numpy(oracle.prefill(p["k"], p["v"], p["alpha"], p["beta"]).astype(np.float32))
+
+
+def _run_and_check(wl, pairs, check_calls, n_units=384, flags=0, keep_all_outputs=False):
+    run = WorkloadRun(wl, "cuda", "bf16", flags=flags)
+    S0 = {pr: _oracle_state(wl, *pr) for pr in pairs}
+    run.prefill_states(overrides=S0)
+    outs = run.alloc_outputs()
+    rng = np.random.default_rng(wl.seed)
+    hist = {pr: {"tok": [], "par": [None]} for pr in pairs}
+    parents_all = {r: [None] for r in range(wl.R)}
+    worst, kept = 0.0, {}
+    for t in range(wl.D):
+        call = run.generate_call(t)
+        run.run_call(call, outs)
+        torch.cuda.synchronize()
+        if t > 0:
+            par = call["parents"].cpu().numpy()
+            for r in range(wl.R):
+                parents_all[r].append(par[r])
+        # ancestry rows of EVERY request: Eq. 5 table + the slot rule (base(req, t) = t*R*W + r*W here)
+        for r in range(wl.R):
+            rows = ev.ancestry_table(parents_all[r], [wl.W] * (t + 1))
+            want = rows + np.array([j * wl.R * wl.W + r * wl.W for j in range(t + 1)])[None, :]
+            got = run.ctx.onela_export_chains(r).cpu().numpy()
+            assert np.array_equal(got, want), f"ancestry rows of request {r} at call {t}"
+        for (r, l) in pairs:
+            lay = call["layers"][l]
+            hist[(r, l)]["tok"].append({n: lay[n][r].cpu() for n in ("k", "v", "alpha", "beta")})
+            if t > 0:
+                hist[(r, l)]["par"].append(parents_all[r][t])
+            if t in check_calls:
+                beams = rng.integers(0, wl.W, n_units)
+                beams[:4] = [0, wl.W - 1, wl.W // 2, min(wl.W - 1, 47)]        # tile edges
+                heads = rng.integers(0, wl.H, n_units)
+                ref = oracle.decode(S0[(r, l)], hist[(r, l)]["tok"], hist[(r, l)]["par"], lay["q"][r].cpu(),
+                                    sel=(beams, heads))
+                got = outs[l][r].float().cpu().numpy()[beams, heads]
+                e = rel_l2(got, ref)
+                worst = max(worst, float(e.max()))
+                assert e.max() <= REL_L2_BAR, f"pair {(r, l)} call {t}: rel-L2 {e.max():.3e}"
+        if keep_all_outputs:
+            kept[t] = [o.clone() for o in outs]
+        assert torch.isfinite(outs[0].float()).all()
+    assert run.ctx.onela_poll_device_status() == (0, 0)
+    return worst, kept, run
+
+
+def test_config2_beam512_zipf_every_call():
+    """32 heads, beam 512, depth 4, Zipf(1.2) parents, 16384-token prompt; sampled units at every call, and
+    the two kernels against each other on every unit."""
+    wl = inputs.WORKLOADS[2]
+    worst, fused, run = _run_and_check(wl, [(0, 0)], range(wl.D), keep_all_outputs=True)
+    assert run.ctx.onela_uses_tensor_core_path()
+    _, generic, run2 = _run_and_check(wl, [(0, 0)], [wl.D - 1], flags=P.FLAG_FORCE_GENERIC, keep_all_outputs=True)
+    assert not run2.ctx.onela_uses_tensor_core_path()
+    for t in range(wl.D):
+        a, b = fused[t][0].float().cpu().numpy(), generic[t][0].float().cpu().numpy()
+        assert rel_l2(a, b).max() <= REL_L2_BAR
+
+
+def test_config3_batch8_beam1024():
+    """8 requests in one shared arena, beam 1024, depth 6, uniform parents."""
+    wl = inputs.WORKLOADS[3]
+    _run_and_check(wl, [(0, 0), (7, 0)], [0, 2, wl.D - 1])
+
+
+def test_config4_stack16_beam512():
+    """16 layers x 4 requests, beam 512, depth 8, Zipf(1.5) parents with heavy duplication."""
+    wl = inputs.WORKLOADS[4]
+    _run_and_check(wl, [(0, 0), (3, 15), (1, 7)], [0, 1, 4, wl.D - 1])
