@@ -405,6 +405,19 @@ __global__ void __launch_bounds__(PT* NP, 1) decode_sm100_kernel(const DecodeArg
             }
             if (RND > 1) asm volatile("cp.async.commit_group;" ::: "memory");
 
+            // Ask L2 for the heads of this pipeline's NEXT tile now, a whole tile ahead of their loads: seven
+            // 128-byte lines per unit (record 4, query 2, gates 1), one per lane.
+            if (tile + NP < seg_end && g < 7) {
+#pragma unroll
+                for (int rnd = 0; rnd < RND; ++rnd) {
+                    const int bb = min(beam_of(tile + NP, rnd), a.W - 1);
+                    const char* rec = kv + (own_row0 + bb) * REC_BYTES;
+                    const char* qrow = reinterpret_cast<const char*>(qbase + (((long long)req * a.W + bb) * a.H + h) * DK);
+                    const char* line = g < 4 ? rec + g * 128
+                                             : (g < 6 ? qrow + (g - 4) * 128 : reinterpret_cast<const char*>(a.gates + own_row0 + bb));
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(line));
+                }
+            }
             int failed = 0;
 #pragma unroll
             for (int rnd = 0; rnd < RND; ++rnd) {
@@ -412,14 +425,25 @@ __global__ void __launch_bounds__(PT* NP, 1) decode_sm100_kernel(const DecodeArg
                 const int u = rnd * TU + grp;                      // row of this unit in the tile's operand buffers
 
                 // ---- 1. fold ----------------------------------------------------------------------
-                // lane g keeps the index of level g: the position in the staged list for staged levels, the
-                // arena slot otherwise; chains deeper than LPU read the rest on demand
-                int32_t my_idx = 0;
-                if (g < old) my_idx = __ldg((g < staged_levels ? sidx_r : table_r) + (long long)g * a.max_beam + bb);
+                // the unit's lanes keep the indices of its first levels (position in the staged list for staged
+                // levels, arena slot otherwise); deeper chains read the rest on demand
+                constexpr int NIDX = LPU >= 8 ? 1 : 8 / LPU;   // lanes of a unit hold the first max(LPU, 8) levels
+                int32_t my_idx[NIDX];
+#pragma unroll
+                for (int j = 0; j < NIDX; ++j) {
+                    const int lv = j * LPU + g;
+                    my_idx[j] = lv < old ? __ldg((lv < staged_levels ? sidx_r : table_r) + (long long)lv * a.max_beam + bb) : 0;
+                }
                 auto idx_of = [&](int level) -> int32_t {
-                    const int32_t s = __shfl_sync(0xffffffffu, my_idx, level & (LPU - 1), LPU);
-                    return level < LPU ? s
-                                       : __ldg((level < staged_levels ? sidx_r : table_r) + (long long)level * a.max_beam + bb);
+                    int32_t s = 0;
+#pragma unroll
+                    for (int j = 0; j < NIDX; ++j) {
+                        const int32_t t = __shfl_sync(0xffffffffu, my_idx[j], level & (LPU - 1), LPU);
+                        if (j == (level / LPU)) s = t;
+                    }
+                    return level < NIDX * LPU
+                               ? s
+                               : __ldg((level < staged_levels ? sidx_r : table_r) + (long long)level * a.max_beam + bb);
                 };
                 UnitHead uh;
                 if (rnd == 0) {
@@ -441,6 +465,11 @@ __global__ void __launch_bounds__(PT* NP, 1) decode_sm100_kernel(const DecodeArg
                 }
 
                 float2 r[NP2], corr[NP2];
+#ifdef ONELA_TIMING
+                // make the head's arrival visible to the phase clock: touch one word of each load
+                if ((uh.q[0].x ^ uh.own.k[0].x ^ uh.own.v[NCH - 1].w ^ __float_as_uint(uh.own.gate.x)) == 0x12345678u) tph[7]++;
+                if (rnd == 0) ONELA_TICK(2) else ONELA_TICK(4)   // head arrival of round 0 / later rounds
+#endif
 #pragma unroll
                 for (int c = 0; c < NCH; ++c) unpack8(uh.q[c], r + 4 * c);
 #pragma unroll
@@ -463,6 +492,7 @@ __global__ void __launch_bounds__(PT* NP, 1) decode_sm100_kernel(const DecodeArg
                                   [&](int level) { return L::load_shared(stage, gates_s, idx_of(level), g); }, r, corr, decay);
                 }
 
+                ONELA_TICK(0)   // fold arithmetic
                 // ---- 2. operands: folded query -> K-major swizzled row u; corr -> row u of the output tile
                 {
                     const int sw = u & 7;
@@ -487,7 +517,7 @@ __global__ void __launch_bounds__(PT* NP, 1) decode_sm100_kernel(const DecodeArg
                     }
                 }
             }
-            ONELA_TICK(0)   // folds + operand writes
+            ONELA_TICK(7)   // operand writes
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             failed |= *abort_flag;
@@ -505,7 +535,6 @@ __global__ void __launch_bounds__(PT* NP, 1) decode_sm100_kernel(const DecodeArg
             if (ptid == 0) {
                 bool ok = mbar_wait(bar_s0, seg_phase);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                ONELA_TICK(2)   // S0 wait
                 if (ok) {
                     constexpr uint32_t idesc = idesc_tf32(N);
                     const uint64_t ad = umma_desc(s0_addr), bd = umma_desc(r_addr);
@@ -526,7 +555,7 @@ __global__ void __launch_bounds__(PT* NP, 1) decode_sm100_kernel(const DecodeArg
             if (!mbar_wait(bar_mma, mma_phase)) failed = 1;
             mma_phase ^= 1;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            ONELA_TICK(4)   // MMA wait
+            ONELA_TICK(3)   // MMA wait (added to the issue column)
             if (pwarp < 4) {
                 // the pipeline's first four warps sit on the four lane quadrants of tensor memory: each adds
                 // accumulator rows (dv) 32*(warp&3) + lane of every beam of the tile onto the stored corr
@@ -580,10 +609,17 @@ __global__ void __launch_bounds__(PT* NP, 1) decode_sm100_kernel(const DecodeArg
         printf("span cta %d sm %u start %llu end %llu\n", (int)blockIdx.x, smid, gt0 % 100000000ull, gt1 % 100000000ull);
     }
     if ((ptid == 0 || ptid == PT - 1) && pipe == NP - 1 && (blockIdx.x == 0 || blockIdx.x == gridDim.x / 2 || blockIdx.x == gridDim.x - 1))
-        printf("cta %d tid %d depth %d tiles %d total %lld | folds %lld barA %lld s0wait %lld mmaissue %lld mmawait %lld ld+barB %lld store %lld\n",
-               (int)blockIdx.x, tid, a.depth, t_end - t_begin, clock64() - tstart, tph[0], tph[1], tph[2], tph[3], tph[4], tph[5], tph[6]);
+        printf("cta %d tid %d depth %d tiles %d total %lld | head0 %lld headN %lld foldmath %lld opwrite %lld barA %lld mma %lld ld+barB %lld store %lld\n",
+               (int)blockIdx.x, tid, a.depth, t_end - t_begin, clock64() - tstart, tph[2], tph[4], tph[0], tph[7], tph[1], tph[3], tph[5], tph[6]);
 #endif
 
+    // A CTA must not exit with bulk copies still landing in its shared memory.  In normal operation every
+    // segment's copies were waited for by the threads that consumed them; after a timeout (pipelines gave
+    // up early) wait for the last segment's copies here, again with a limit.
+    if (tid == 0 && *abort_flag && t_begin < t_end) {
+        mbar_wait(bar_s0, seg_phase ^ 1);
+        mbar_wait(bar_stage, seg_phase ^ 1);
+    }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 0) {

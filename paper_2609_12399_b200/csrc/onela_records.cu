@@ -11,22 +11,20 @@ namespace onela {
 
 namespace {
 
-// One warp per (request, beam, head) row.  The arena is head-major ([head][slot][k | v]) so that the
-// records one decode tile reads - consecutive beams of one head - are contiguous.
+// One warp per (beam, head) row of one request (blockIdx.y).  The arena is head-major ([head][slot][k | v])
+// so that the records one decode tile reads - consecutive beams of one head - are contiguous.
 __global__ void __launch_bounds__(256) append_kernel(const char* __restrict__ k, const char* __restrict__ v,
                                                      const float* __restrict__ alpha, const float* __restrict__ beta,
                                                      char* __restrict__ kv_plane, float2* __restrict__ gate_plane,
-                                                     long long arena_slots, int32_t req_count, int32_t W, int32_t H,
-                                                     int32_t k_bytes, int32_t v_bytes, BatchBases bases) {
-    const long long row = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+                                                     long long arena_slots, int32_t W, int32_t H, int32_t k_bytes,
+                                                     int32_t v_bytes, BatchBases bases) {
+    const int r = blockIdx.y;
+    const int row_in_req = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);   // b * H + h
     const int lane = threadIdx.x & 31;
-    const long long rows = (long long)req_count * W * H;
-    if (row >= rows) return;
-    const int h = (int)(row % H);
-    const long long rb = row / H;
-    const int b = (int)(rb % W), r = (int)(rb / W);
-    const long long slot = (long long)bases.base[r] + b;
-    const long long dst_row = (long long)h * arena_slots + slot;
+    if (row_in_req >= W * H) return;
+    const int b = row_in_req / H, h = row_in_req - b * H;
+    const long long row = (long long)r * (W * H) + row_in_req;
+    const long long dst_row = (long long)h * arena_slots + (bases.base[r] + b);
     const uint4* ksrc = reinterpret_cast<const uint4*>(k + row * k_bytes);
     const uint4* vsrc = reinterpret_cast<const uint4*>(v + row * v_bytes);
     uint4* dst = reinterpret_cast<uint4*>(kv_plane + dst_row * (k_bytes + v_bytes));
@@ -145,12 +143,11 @@ cudaError_t launch_append(const void* k, const void* v, const float* alpha, cons
                           float2* gate_plane, long long arena_slots, int32_t req_count, int32_t W, int32_t H,
                           int32_t dk, int32_t dv, int32_t elem_bytes, const BatchBases& bases,
                           cudaStream_t stream) {
-    const long long rows = (long long)req_count * W * H;
     const int warps_per_block = 8;
-    const long long blocks = (rows + warps_per_block - 1) / warps_per_block;
-    append_kernel<<<(unsigned)blocks, warps_per_block * 32, 0, stream>>>(
-        static_cast<const char*>(k), static_cast<const char*>(v), alpha, beta, kv_plane, gate_plane, arena_slots,
-        req_count, W, H, dk * elem_bytes, dv * elem_bytes, bases);
+    dim3 grid((unsigned)((W * H + warps_per_block - 1) / warps_per_block), (unsigned)req_count);
+    append_kernel<<<grid, warps_per_block * 32, 0, stream>>>(static_cast<const char*>(k), static_cast<const char*>(v),
+                                                             alpha, beta, kv_plane, gate_plane, arena_slots, W, H,
+                                                             dk * elem_bytes, dv * elem_bytes, bases);
     return cudaGetLastError();
 }
 
