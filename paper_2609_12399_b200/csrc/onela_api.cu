@@ -360,7 +360,11 @@ onela_status onela_decode_step(onela_ctx* ctx, int32_t req_begin, int32_t req_co
     a.s0_swizzled = ctx->tensor_core;
     for (int i = 0; i < req_count; ++i) a.bases.base[i] = ctx->req[req_begin + i].step_base.back();
     bool supported = true;
+#ifdef ONELA_PIPELINED
     const cudaError_t e = ctx->tensor_core ? launch_decode_sm100(a, c.out_dtype, s)
+#else
+    const cudaError_t e = ctx->tensor_core ? launch_decode_sm100_ws(a, c.out_dtype, s)
+#endif
                                            : launch_decode_generic(a, c.dk, c.dv, c.rec_dtype, c.out_dtype, &supported, s);
     if (!supported) return ONELA_E_UNSUPPORTED;
     if (e != cudaSuccess) return ONELA_E_CUDA;

@@ -26,14 +26,14 @@
 
 #include "onela_internal.h"
 #include "onela_layout.cuh"
+#include "onela_sm100.cuh"
 
 namespace onela {
 
 namespace {
 
-constexpr int DK = 128, DV = 128;
-constexpr int REC_BYTES = (DK + DV) * 2;       // 512: k | v in bf16
-constexpr int S0_BYTES = DV * DK * 4;          // 65536
+using namespace sm100;
+
 constexpr int OP = DV + 4;                     // pitch (floats) of the transposed accumulator
 constexpr int R_TOTAL = 96 * 128 * 4;          // all pipelines' folded-query operands: up to 96 beams x 512 B
 constexpr int O_TOTAL = 96 * OP * 4;           // all pipelines' output tiles (corr, then corr + accumulator)
@@ -42,205 +42,6 @@ constexpr int STAGE_BYTES = STAGE_CAP * REC_BYTES;
 constexpr int GATE_BYTES = STAGE_CAP * 8;
 constexpr int SMEM_BYTES = S0_BYTES + R_TOTAL + O_TOTAL + STAGE_BYTES + GATE_BYTES + 128 + 1024;
 constexpr uint32_t TMEM_COLS = 128;            // accumulator columns: one per beam in flight
-constexpr int WAIT_LIMIT = 1 << 20;
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait: false when the phase did not complete within WAIT_LIMIT probes.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (int i = 0; i < WAIT_LIMIT; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                 "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
-
-// Named barrier over `count` threads that also ORs a predicate across them.
-__device__ __forceinline__ int bar_or(int id, int count, int pred) {
-    uint32_t out;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 q, %1, 0;\n\t"
-        "barrier.cta.red.or.pred p, %2, %3, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(out)
-        : "r"(pred), "r"(id), "r"(count)
-        : "memory");
-    return (int)out;
-}
-
-// Shared-memory matrix descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);       // start address, 16-byte units
-    d |= (uint64_t)1 << 16;                            // leading byte offset (unused for swizzled K-major)
-    d |= (uint64_t)(1024 >> 4) << 32;                  // stride byte offset between 8-row groups
-    d |= (uint64_t)1 << 46;                            // descriptor version (sm_100)
-    d |= (uint64_t)2 << 61;                            // SWIZZLE_128B
-    return d;
-}
-// Instruction descriptor: D fp32, A and B TF32, both K-major, M = 128, N = n.
-__host__ __device__ constexpr uint32_t idesc_tf32(int n) {
-    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-}
-
-__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                          uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
-        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-        : "r"(taddr)
-        : "memory");
-}
-
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-    const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<const uint32_t*>(&t);
-}
-template <typename OutT>
-__device__ __forceinline__ void store8(OutT* p, const float* x);
-template <>
-__device__ __forceinline__ void store8<float>(float* p, const float* x) {
-    reinterpret_cast<float4*>(p)[0] = make_float4(x[0], x[1], x[2], x[3]);
-    reinterpret_cast<float4*>(p)[1] = make_float4(x[4], x[5], x[6], x[7]);
-}
-template <>
-__device__ __forceinline__ void store8<__nv_bfloat16>(__nv_bfloat16* p, const float* x) {
-    *reinterpret_cast<uint4*>(p) = make_uint4(pack_bf16x2(x[0], x[1]), pack_bf16x2(x[2], x[3]), pack_bf16x2(x[4], x[5]),
-                                              pack_bf16x2(x[6], x[7]));
-}
-
-// One lane's share of a record: NCH x 8 elements of k, NCH x 8 of v (packed bf16), and the gates.
-template <int NCH>
-struct Rec {
-    uint4 k[NCH], v[NCH];
-    float2 gate;
-};
-
-// two packed bf16 -> float2 {element 0, element 1}, exactly
-__device__ __forceinline__ float2 up2(uint32_t w) {
-    return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
-}
-__device__ __forceinline__ void unpack8(const uint4& x, float2* o) {
-    o[0] = up2(x.x); o[1] = up2(x.y); o[2] = up2(x.z); o[3] = up2(x.w);
-}
-
-// LPU lanes share one (beam, head) unit; lane g owns the 16-byte chunks c*LPU + g (c < NCH) of every
-// 256-byte vector, i.e. elements [(c*LPU + g)*8, +8): LPU consecutive lanes cover contiguous memory.
-template <int LPU>
-struct Lanes {
-    static constexpr int NCH = 16 / LPU;     // 16-byte chunks per lane per 128-element bf16 vector
-    static constexpr int NP2 = 4 * NCH;      // float2 pairs per lane
-    using R = Rec<NCH>;
-
-    static __device__ __forceinline__ R load_global(const char* kv, const float2* gates, long long row, int g) {
-        const uint4* p = reinterpret_cast<const uint4*>(kv + row * REC_BYTES) + g;
-        R r;
-#pragma unroll
-        for (int c = 0; c < NCH; ++c) {
-            r.k[c] = __ldg(p + c * LPU);
-            r.v[c] = __ldg(p + 16 + c * LPU);
-        }
-        r.gate = __ldg(gates + row);
-        return r;
-    }
-    static __device__ __forceinline__ R load_shared(const uint8_t* stage, const float2* gates_s, int idx, int g) {
-        const uint4* p = reinterpret_cast<const uint4*>(stage + idx * REC_BYTES) + g;
-        R r;
-#pragma unroll
-        for (int c = 0; c < NCH; ++c) {
-            r.k[c] = p[c * LPU];
-            r.v[c] = p[16 + c * LPU];
-        }
-        r.gate = gates_s[idx];
-        return r;
-    }
-    // One fold step on this lane's elements (packed fp32x2 FMAs), with the LPU-lane dot reduction:
-    //   c~ = k . r~ ;  corr += (decay beta c~) v ;  r~ -= (beta c~) k ;  decay *= alpha
-    static __device__ __forceinline__ void fold_step(const R& rec, float2* r, float2* corr, float& decay) {
-        float2 kx[NP2];
-#pragma unroll
-        for (int c = 0; c < NCH; ++c) unpack8(rec.k[c], kx + 4 * c);
-        float2 d0 = make_float2(0.f, 0.f), d1 = make_float2(0.f, 0.f);
-#pragma unroll
-        for (int e = 0; e < NP2; e += 2) {
-            d0 = __ffma2_rn(kx[e], r[e], d0);
-            d1 = __ffma2_rn(kx[e + 1], r[e + 1], d1);
-        }
-        float dot = (d0.x + d0.y) + (d1.x + d1.y);
-#pragma unroll
-        for (int o = LPU / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-        const float bc = rec.gate.y * dot;
-        const float wv = decay * bc;
-        const float2 nbc2 = make_float2(-bc, -bc), wv2 = make_float2(wv, wv);
-#pragma unroll
-        for (int e = 0; e < NP2; ++e) r[e] = __ffma2_rn(kx[e], nbc2, r[e]);
-#pragma unroll
-        for (int c = 0; c < NCH; ++c) {
-            float2 vx[4];
-            unpack8(rec.v[c], vx);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) corr[4 * c + e] = __ffma2_rn(vx[e], wv2, corr[4 * c + e]);
-        }
-        decay *= rec.gate.x;
-    }
-    // Fold `first` (already in registers) and then levels hi .. lo (newest first) fetched by `load`, keeping
-    // one record in flight while the previous one is folded.  Two buffers alternate so no record is moved.
-    template <class LoadFn>
-    static __device__ __forceinline__ void fold_chain(const R& first, int hi, int lo, LoadFn load, float2* r,
-                                                      float2* corr, float& decay) {
-        R A = first, B;
-        int level = hi + 1;   // level of the record held in A
-        while (true) {
-            if (level - 1 >= lo) B = load(level - 1);
-            fold_step(A, r, corr, decay);
-            if (--level < lo) break;
-            if (level - 1 >= lo) A = load(level - 1);
-            fold_step(B, r, corr, decay);
-            if (--level < lo) break;
-        }
-    }
-};
-
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async8(uint32_t dst, const void* src) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
-}
-
 // LPU lanes per unit, PT threads per pipeline (TU = PT/LPU units folded at a time), RND rounds of units per
 // tile (one MMA group per tile over N = RND * TU beams: issuing a tcgen05.mma costs ~90 cycles whatever its N,
 // so tiles are wide), NP pipelines per CTA.

@@ -1,0 +1,433 @@
+// Warp-specialised fused decode kernel for B200 (sm_100a): dk = dv = 128, bf16 records.
+//
+// One persistent CTA per SM, 12 warps in two roles that never wait for one another synchronously:
+//   * 8 FOLD warps.  8 lanes own one (beam, head) unit; a warp folds 4 units at a time ("quad"): query
+//     folded through the unit's records newest -> oldest (c = k.r; corr += beta c v; r -= beta c k; decay a
+//     scalar; packed fp32x2 FMAs).  The next quad's query and own record are loaded while the current
+//     quad is folded.  Results go into a ring slot in shared memory: the folded query as a row of the
+//     K-major 128-byte-swizzled MMA operand (rounded to TF32), corr as a row of the slot's corr tile.
+//     The warp whose quad completes a slot (all 64 rows written) issues the group's 16 tcgen05.mma
+//     (kind::tf32, M = dv = 128, N = 64 beams, K = 8) against the head's S_0 image, accumulating fp32 in
+//     tensor memory, and commits; the other fold warps are already folding the next group.
+//   * 4 EPILOGUE warps (one per tensor-memory lane quadrant).  When the MMA group has completed they read
+//     the accumulator, add corr and store the outputs (lane = dv index: 32 consecutive elements per store),
+//     then hand the slot back.
+// Two ring slots (operand rows, corr tile, 64 accumulator columns each) keep the MMA and the epilogue of one
+// group under the folds of the next.  Work = groups of 64 consecutive beams of one (request, head), a
+// contiguous range per CTA; consecutive groups of one head form a segment, per which ONE 64 KiB bulk async
+// copy brings the head's S_0 image (pre-swizzled TF32, kept in the store) and one 512-byte bulk copy per
+// DISTINCT ancestor record stages the oldest chain levels (as many whole levels as fit) in shared memory.
+// Every wait is bounded and also gives up when another role has raised the abort flag; a role that gives up
+// records ONELA_E_TIMEOUT, stops working but keeps joining the per-segment CTA barriers; before returning
+// the CTA waits (bounded) for bulk copies still in flight and frees its tensor memory.
+#include <cstdio>
+
+#include "onela_internal.h"
+#include "onela_layout.cuh"
+#include "onela_sm100.cuh"
+
+namespace onela {
+
+namespace {
+
+using namespace sm100;
+
+constexpr int FOLD_WARPS = 8;
+constexpr int THREADS = (FOLD_WARPS + 4) * 32;      // + 4 epilogue warps (12 warps: three per SM sub-partition)
+constexpr int GN = 64;                              // beams per group = MMA N
+constexpr int R_KB_STRIDE = GN * 128;               // bytes between the four 32-float K blocks of the operand
+constexpr int R_BYTES = 4 * R_KB_STRIDE;            // 32768
+constexpr int C_BYTES = GN * DV * 4;                // 32768: corr tile, row = beam
+constexpr int SLOT_BYTES = R_BYTES + C_BYTES;
+constexpr int SLOTS = 2;
+constexpr int STAGE_CAP = 64;                       // distinct ancestor records staged per segment
+constexpr int STAGE_BYTES = STAGE_CAP * REC_BYTES;
+constexpr int GATE_BYTES = STAGE_CAP * 8;
+constexpr int SMEM_BYTES = S0_BYTES + SLOTS * SLOT_BYTES + STAGE_BYTES + GATE_BYTES + 128 + 1024;
+constexpr uint32_t TMEM_COLS = SLOTS * GN;
+using L = Lanes<8>;
+using RecT = L::R;
+
+// Bounded wait that also gives up as soon as the CTA's abort flag is raised.
+__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    for (int i = 0; i < WAIT_LIMIT; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 63) == 63 && *abort_flag) return false;
+    }
+    return false;
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+struct Head {           // what a unit's fold needs first
+    uint4 q[2];
+    RecT own;
+};
+
+template <typename OutT>
+__global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs a, int total_groups, int groups_per_pair) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;            // swizzle atoms need 1024-byte alignment
+    uint8_t* smem = smem_raw + (base - raw);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t s0_addr = base;
+    uint8_t* ring = smem + S0_BYTES;
+    uint8_t* stage = ring + SLOTS * SLOT_BYTES;
+    float2* gates_s = reinterpret_cast<float2*>(stage + STAGE_BYTES);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(stage + STAGE_BYTES + GATE_BYTES);
+    // bars: 0 S_0 image, 1 staged records, 2+s slot s full, 4+s slot s MMA done, 6+s slot s free
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    int* quad_count = reinterpret_cast<int*>(tmem_slot + 2);   // [SLOTS] quads written into the slot in its current use
+    const uint32_t bar_s0 = smem_u32(bars), bar_stage = smem_u32(bars + 1);
+    auto bar_full = [&](int s) { return smem_u32(bars + 2 + s); };
+    auto bar_done = [&](int s) { return smem_u32(bars + 4 + s); };
+    auto bar_free = [&](int s) { return smem_u32(bars + 6 + s); };
+
+    if (tid == 0) {
+        mbar_init(bar_s0, 1);
+        mbar_init(bar_stage, 32);
+        for (int s = 0; s < SLOTS; ++s) {
+            mbar_init(bar_full(s), 2 * FOLD_WARPS);   // one arrival per quad: 16 quads of 4 beams per group
+            mbar_init(bar_done(s), 1);                // tcgen05.commit
+            mbar_init(bar_free(s), 4);                // the four epilogue warps
+        }
+        *abort_flag = 0;
+        quad_count[0] = quad_count[1] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int g_begin = (int)(((long long)blockIdx.x * total_groups) / gridDim.x);
+    const int g_end = (int)(((long long)(blockIdx.x + 1) * total_groups) / gridDim.x);
+    const int old = a.depth - 1;          // records older than a beam's own: levels old-1 .. 0
+    const char* kv = a.kv;
+    const __nv_bfloat16* qbase = static_cast<const __nv_bfloat16*>(a.q);
+
+#ifdef ONELA_TIMING
+    long long tph[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    long long tk = clock64();
+    const long long tstart = tk;
+#define ONELA_TICK(i) { const long long now = clock64(); tph[i] += now - tk; tk = now; }
+#else
+#define ONELA_TICK(i)
+#endif
+    bool dead = false;                    // this warp gave up (timeout or abort raised elsewhere)
+    int seg_idx = 0;
+    for (int sg_begin = g_begin, sg_end; sg_begin < g_end; sg_begin = sg_end, ++seg_idx) {
+        const int pair = sg_begin / groups_per_pair;
+        sg_end = min(g_end, (pair + 1) * groups_per_pair);
+        const int req = pair / a.H, h = pair - req * a.H;
+        const long long plane_row0 = (long long)h * a.arena_slots;
+        const long long own_row0 = plane_row0 + a.bases.base[req];
+        const uint32_t seg_parity = seg_idx & 1;
+
+        // How many of the oldest levels fit in the staging buffer (whole levels only; uniform over the CTA).
+        int staged_levels = 0, n_staged = 0;
+        {
+            const int32_t* uoff = a.uoff + req * a.uoff_req_stride;
+            for (int l = 0; l < old; ++l) {
+                const int e = __ldg(uoff + l + 1);
+                if (e > STAGE_CAP) break;
+                staged_levels = l + 1;
+                n_staged = e;
+            }
+        }
+
+        // The previous segment is fully consumed: the MMA warp and the epilogue warps pass this barrier only
+        // after the last group's MMA completed and was read back; the fold warps after their last staged read.
+        __syncthreads();
+        if (warp == 0 && !dead) {
+            if (lane == 0) {
+                mbar_expect_tx(bar_s0, S0_BYTES);
+                bulk_load(s0_addr, a.s0 + req * a.s0_req_stride + (long long)h * (DV * DK), S0_BYTES, bar_s0);
+            }
+            const int32_t* ulist = a.ulist + req * a.ulist_req_stride;
+            const int mine = (n_staged > lane) ? (n_staged - lane + 31) / 32 : 0;
+            mbar_expect_tx(bar_stage, mine * REC_BYTES);   // one arrival per lane, with the bytes it is about to request
+            for (int i = lane; i < n_staged; i += 32) {
+                const long long row = plane_row0 + __ldg(ulist + i);
+                bulk_load(smem_u32(stage + i * REC_BYTES), kv + row * REC_BYTES, REC_BYTES, bar_stage);
+            }
+        }
+        const int gcount0 = sg_begin - g_begin;   // groups this CTA finished before this segment
+
+        if (warp < FOLD_WARPS) {
+            // =============================== FOLD ===============================
+            const int grp = lane >> 3, g = lane & 7;
+            const int32_t* table_r = a.table + req * a.table_req_stride;
+            const int32_t* sidx_r = a.sidx + req * a.sidx_req_stride;
+            // the gates of the staged records: every fold warp writes all of them (same values), then syncs itself
+            if (!dead) {
+                const int32_t* ulist = a.ulist + req * a.ulist_req_stride;
+                for (int i = lane; i < n_staged; i += 32) gates_s[i] = __ldg(a.gates + plane_row0 + __ldg(ulist + i));
+                __syncwarp();
+            }
+            // quad k of the segment: group sg_begin + k/2, rows (k&1)*32 + 4*warp + grp
+            const int n_quads = 2 * (sg_end - sg_begin);
+            auto beam_of = [&](int k) { return ((sg_begin + (k >> 1)) - pair * groups_per_pair) * GN + (k & 1) * 32 + 4 * warp + grp; };
+            // The head of quad k (query, own record, gates of its four units) is copied asynchronously into the
+            // quad's own rows of its ring slot - free until the quad's results are written there - one quad ahead.
+            auto slot_of = [&](int k) { return (gcount0 + (k >> 1)) & 1; };
+            auto use_of = [&](int k) { return (gcount0 + (k >> 1)) >> 1; };
+            auto row_of = [&](int k) { return (k & 1) * 32 + 4 * warp + grp; };
+            auto stage_head = [&](int k) -> bool {     // false: gave up waiting for the slot
+                const int s = slot_of(k), use = use_of(k), u = row_of(k);
+                if ((k & 1) == 0 && use > 0 && !wait_or_abort(bar_free(s), (use - 1) & 1, abort_flag)) return false;
+                const int bb = min(beam_of(k), a.W - 1);   // idle groups shadow a live beam: uniform control flow
+                uint8_t* R_s = ring + s * SLOT_BYTES;
+                const uint32_t c_row = smem_u32(R_s + R_BYTES + u * (DV * 4));
+                const char* rec = kv + (own_row0 + bb) * REC_BYTES;
+                const char* qrow = reinterpret_cast<const char*>(qbase + (((long long)req * a.W + bb) * a.H + h) * DK);
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const int ci = c * 8 + g;   // 16-byte chunk of a 256-byte vector
+                    cp_async16(smem_u32(R_s + (ci >> 3) * R_KB_STRIDE + u * 128 + (ci & 7) * 16), rec + ci * 16);
+                    cp_async16(smem_u32(R_s + (2 + (ci >> 3)) * R_KB_STRIDE + u * 128 + (ci & 7) * 16), rec + 256 + ci * 16);
+                    cp_async16(c_row + ci * 16, qrow + ci * 16);
+                }
+                if (g == 0) cp_async8(c_row + 256, a.gates + own_row0 + bb);
+                asm volatile("cp.async.commit_group;" ::: "memory");
+                return true;
+            };
+            auto take_head = [&](int k) {
+                Head u;
+                const int s = slot_of(k), row = row_of(k);
+                const uint8_t* R_s = ring + s * SLOT_BYTES;
+                const uint4* c_row = reinterpret_cast<const uint4*>(R_s + R_BYTES + row * (DV * 4));
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const int ci = c * 8 + g;
+                    u.own.k[c] = *reinterpret_cast<const uint4*>(R_s + (ci >> 3) * R_KB_STRIDE + row * 128 + (ci & 7) * 16);
+                    u.own.v[c] = *reinterpret_cast<const uint4*>(R_s + (2 + (ci >> 3)) * R_KB_STRIDE + row * 128 + (ci & 7) * 16);
+                    u.q[c] = c_row[ci];
+                }
+                u.own.gate = *reinterpret_cast<const float2*>(c_row + 16);
+                return u;
+            };
+            auto l2_prefetch = [&](int k) {   // seven 128-byte lines per unit (record 4, query 2, gates 1), one per lane
+                if (g < 7) {
+                    const int bb = min(beam_of(k), a.W - 1);
+                    const char* rec = kv + (own_row0 + bb) * REC_BYTES;
+                    const char* qrow = reinterpret_cast<const char*>(qbase + (((long long)req * a.W + bb) * a.H + h) * DK);
+                    const char* line = g < 4 ? rec + g * 128
+                                             : (g < 6 ? qrow + (g - 4) * 128 : reinterpret_cast<const char*>(a.gates + own_row0 + bb));
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(line));
+                }
+            };
+            if (!dead && n_quads > 0) {
+                if (!stage_head(0)) dead = true;
+                if (1 < n_quads) l2_prefetch(1);
+                if (2 < n_quads) l2_prefetch(2);
+            }
+            bool staged_ready = false;
+            for (int k = 0; k < n_quads && !dead; ++k) {
+                const int s = slot_of(k), use = use_of(k);
+                const int u = row_of(k);                         // row of this unit in the slot
+                const int bb = min(beam_of(k), a.W - 1);
+                asm volatile("cp.async.wait_all;" ::: "memory");
+                __syncwarp();
+                const Head cur = take_head(k);
+                __syncwarp();                                    // every lane has read the scratch rows
+                // the next quad's head starts its trip now and lands while this quad is folded
+                if (k + 1 < n_quads && !stage_head(k + 1)) { dead = true; break; }
+                if (k + 3 < n_quads) l2_prefetch(k + 3);
+
+                // lane g keeps the index of level g: position in the staged list for staged levels, arena slot otherwise
+                int32_t my_idx = 0;
+                if (g < old) my_idx = __ldg((g < staged_levels ? sidx_r : table_r) + (long long)g * a.max_beam + bb);
+                auto idx_of = [&](int level) -> int32_t {
+                    const int32_t t = __shfl_sync(0xffffffffu, my_idx, level & 7, 8);
+                    return level < 8 ? t : __ldg((level < staged_levels ? sidx_r : table_r) + (long long)level * a.max_beam + bb);
+                };
+
+#ifdef ONELA_TIMING
+                if ((cur.q[0].x ^ cur.own.k[0].x ^ cur.own.v[1].w ^ __float_as_uint(cur.own.gate.x)) == 0x12345678u) tph[7]++;
+                ONELA_TICK(0)   // head arrival (+ issue of next head)
+#endif
+                float2 r[8], corr[8];
+                unpack8(cur.q[0], r);
+                unpack8(cur.q[1], r + 4);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) corr[e] = make_float2(0.f, 0.f);
+                float decay = 1.f;
+                L::fold_chain(cur.own, old - 1, staged_levels,
+                              [&](int level) { return L::load_global(kv, a.gates, plane_row0 + idx_of(level), g); }, r, corr, decay);
+                if (staged_levels > 0) {
+                    if (!staged_ready) {
+                        if (!wait_or_abort(bar_stage, seg_parity, abort_flag)) { dead = true; break; }
+                        staged_ready = true;
+                    }
+                    const RecT newest = L::load_shared(stage, gates_s, idx_of(staged_levels - 1), g);
+                    L::fold_chain(newest, staged_levels - 2, 0,
+                                  [&](int level) { return L::load_shared(stage, gates_s, idx_of(level), g); }, r, corr, decay);
+                }
+
+                ONELA_TICK(1)   // fold
+                uint8_t* R_s = ring + s * SLOT_BYTES;
+                float* C_s = reinterpret_cast<float*>(R_s + R_BYTES);
+                {
+                    const int sw = u & 7;
+                    const float2 dc = make_float2(decay, decay);
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        const int ci = c * 8 + g;                   // elements [8 ci, 8 ci + 8)
+                        const int kb = ci >> 2, ch = 2 * (ci & 3);  // K block of 32 floats; first of two 16-byte chunks
+                        uint8_t* row = R_s + kb * R_KB_STRIDE + u * 128;
+                        float2 x[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) x[e] = __fmul2_rn(r[4 * c + e], dc);
+                        *reinterpret_cast<float4*>(row + (((ch) ^ sw) << 4)) =
+                            make_float4(round_tf32(x[0].x), round_tf32(x[0].y), round_tf32(x[1].x), round_tf32(x[1].y));
+                        *reinterpret_cast<float4*>(row + (((ch + 1) ^ sw) << 4)) =
+                            make_float4(round_tf32(x[2].x), round_tf32(x[2].y), round_tf32(x[3].x), round_tf32(x[3].y));
+                        float* crow = C_s + u * DV + ci * 8;
+                        *reinterpret_cast<float4*>(crow) = make_float4(corr[4 * c].x, corr[4 * c].y, corr[4 * c + 1].x, corr[4 * c + 1].y);
+                        *reinterpret_cast<float4*>(crow + 4) =
+                            make_float4(corr[4 * c + 2].x, corr[4 * c + 2].y, corr[4 * c + 3].x, corr[4 * c + 3].y);
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
+                __syncwarp();
+                ONELA_TICK(3)   // operand write + proxy fence
+                // ---- the warp whose quad completes the group issues the group's MMAs -------------------
+                int mma_failed = 0;
+                if (lane == 0) {
+                    mbar_arrive(bar_full(s));
+                    if (atomicAdd(&quad_count[s], 1) == 2 * FOLD_WARPS - 1) {
+                        quad_count[s] = 0;   // the slot's next use cannot begin before this group's MMAs are read back
+                        bool ok = wait_or_abort(bar_full(s), use & 1, abort_flag);      // all 16 arrivals are in: acquire
+                        ok = ok && wait_or_abort(bar_s0, seg_parity, abort_flag);
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        if (ok) {
+                            constexpr uint32_t idesc = idesc_tf32(GN);
+                            const uint64_t ad = umma_desc(s0_addr), bd = umma_desc(smem_u32(R_s));
+#pragma unroll
+                            for (int kb = 0; kb < 4; ++kb)
+#pragma unroll
+                                for (int ks = 0; ks < 4; ++ks)
+                                    umma_tf32(tmem_base + s * GN, ad + (uint64_t)((kb * (DV * 128) + ks * 32) >> 4),
+                                              bd + (uint64_t)((kb * R_KB_STRIDE + ks * 32) >> 4), idesc, (kb | ks) ? 1u : 0u);
+                        } else {
+                            mma_failed = 1;
+                        }
+                        umma_commit(bar_done(s));   // arrives when the MMAs above (if any) have completed
+                    }
+                }
+                if (__shfl_sync(0xffffffffu, mma_failed, 0)) { dead = true; break; }
+                ONELA_TICK(4)   // arrive (+ MMA issue when last)
+            }
+        } else {
+            // =============================== EPILOGUE ===============================
+            const int quad = warp & 3;                    // tensor-memory lane quadrant of this warp
+            const int i = quad * 32 + lane;               // output element (dv index) of this thread
+            for (int gi = sg_begin; gi < sg_end && !dead; ++gi) {
+                const int gcount = gcount0 + (gi - sg_begin);
+                const int s = gcount & 1, use = gcount >> 1;
+                if (!wait_or_abort(bar_done(s), use & 1, abort_flag)) { dead = true; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                ONELA_TICK(5)   // epilogue: wait for the MMA group
+                float* C_s = reinterpret_cast<float*>(ring + s * SLOT_BYTES + R_BYTES);
+                const int b0 = (gi - pair * groups_per_pair) * GN;
+                const uint32_t taddr = tmem_base + s * GN + ((uint32_t)(quad * 32) << 16);
+                {
+                    // accumulator rows (dv) of this thread, all 64 beams, added onto the corr tile in place
+                    uint32_t v[GN];
+                    tmem_ld64(taddr, v);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int j = 0; j < GN; ++j) C_s[j * DV + i] += __uint_as_float(v[j]);
+                }
+                ONELA_TICK(2)   // tmem ld + add
+                if (bar_or(1, 128, 0)) { dead = true; break; }     // the four epilogue warps: tile complete
+                {
+                    // coalesced stores: 16 lanes cover one beam's 128 outputs, 8 elements each
+                    const int et = (warp - FOLD_WARPS) * 32 + lane;
+#pragma unroll
+                    for (int it = 0; it < GN * 16 / 128; ++it) {
+                        const int idx = it * 128 + et, j = idx >> 4, ch = idx & 15;
+                        if (b0 + j < a.W) {
+                            const float4 x0 = *reinterpret_cast<const float4*>(C_s + j * DV + ch * 8);
+                            const float4 x1 = *reinterpret_cast<const float4*>(C_s + j * DV + ch * 8 + 4);
+                            const float o[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+                            store8<OutT>(static_cast<OutT*>(a.out) + (((long long)req * a.W + b0 + j) * a.H + h) * DV + ch * 8, o);
+                        }
+                    }
+                }
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_free(s));
+                ONELA_TICK(6)   // epilogue: read back, add, store
+            }
+        }
+        if (dead) {
+            if (lane == 0) {
+                *abort_flag = 1;
+                if (atomicCAS(a.status, ONELA_OK, ONELA_E_TIMEOUT) == ONELA_OK) a.status[1] = (int32_t)blockIdx.x;
+            }
+        }
+    }
+
+#ifdef ONELA_TIMING
+    if (lane == 0 && (warp == 0 || warp == 7 || warp == 8) && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1) && (a.depth == 1 || a.depth == 8))
+        printf("cta %d warp %d depth %d groups %d total %lld | head %lld fold %lld slotwait %lld write %lld arrive+mma %lld | epi: wait %lld tmemld %lld rest %lld\n",
+               (int)blockIdx.x, warp, a.depth, g_end - g_begin, clock64() - tstart, tph[0], tph[1], tph[2], tph[3], tph[4], tph[5], tph[2], tph[6]);
+#endif
+    // A CTA must not exit with bulk copies still landing in its shared memory: after an abort nobody may
+    // have waited for the last segment's copies.
+    __syncthreads();
+    if (tid == 0 && *abort_flag && g_begin < g_end) {
+        mbar_wait(bar_s0, (seg_idx - 1) & 1);
+        mbar_wait(bar_stage, (seg_idx - 1) & 1);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+int sm_count_ws() {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+    return n;
+}
+
+template <typename OutT>
+cudaError_t launch_ws_t(const DecodeArgs& a, cudaStream_t stream) {
+    auto kern = decode_ws_kernel<OutT>;
+    static bool configured = false;
+    static int sms = 148;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        sms = sm_count_ws();
+        configured = true;
+    }
+    const int groups_per_pair = (a.W + GN - 1) / GN;
+    const int total_groups = a.req_count * a.H * groups_per_pair;
+    const int grid = total_groups < sms ? total_groups : sms;
+    kern<<<grid, THREADS, SMEM_BYTES, stream>>>(a, total_groups, groups_per_pair);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_decode_sm100_ws(const DecodeArgs& a, int32_t out_dtype, cudaStream_t stream) {
+    return out_dtype == ONELA_DTYPE_BF16 ? launch_ws_t<__nv_bfloat16>(a, stream) : launch_ws_t<float>(a, stream);
+}
+
+}  // namespace onela

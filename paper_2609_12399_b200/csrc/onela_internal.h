@@ -81,6 +81,7 @@ cudaError_t launch_decode_generic(const DecodeArgs& a, int32_t dk, int32_t dv, i
 bool decode_generic_supported(int32_t dk, int32_t dv, int32_t rec_dtype);
 // tcgen05 tensor-core kernel (sm_100a): dk = dv = 128, bf16 records, S_0 stored as the swizzled TF32 image
 bool decode_sm100_supported(int32_t dk, int32_t dv, int32_t rec_dtype);
-cudaError_t launch_decode_sm100(const DecodeArgs& a, int32_t out_dtype, cudaStream_t stream);
+cudaError_t launch_decode_sm100(const DecodeArgs& a, int32_t out_dtype, cudaStream_t stream);     // barrier-pipelined variant
+cudaError_t launch_decode_sm100_ws(const DecodeArgs& a, int32_t out_dtype, cudaStream_t stream);  // warp-specialised variant
 
 }  // namespace onela
