@@ -43,8 +43,12 @@ constexpr int SLOTS = 2;
 constexpr int STAGE_CAP = 64;                       // distinct ancestor records staged per segment
 constexpr int STAGE_BYTES = STAGE_CAP * REC_BYTES;
 constexpr int GATE_BYTES = STAGE_CAP * 8;
-constexpr int SMEM_BYTES = S0_BYTES + SLOTS * SLOT_BYTES + STAGE_BYTES + GATE_BYTES + 128 + 1024;
-constexpr uint32_t TMEM_COLS = SLOTS * GN;
+constexpr int HEAD_BYTES = 4 * (REC_BYTES + DK * 2);     // one quad's heads: 4 own records + 4 queries = 3072
+constexpr int HEAD_STAGES = 2;                         // heads in flight per fold warp
+constexpr int HEADS_TOTAL = FOLD_WARPS * HEAD_STAGES * HEAD_BYTES;
+constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + STAGE_BYTES + GATE_BYTES + HEADS_TOTAL + 256 + 1024;
+constexpr uint32_t TMEM_COLS = 256;              // accumulators of the two slots in [0, 128), the head's S_0 in [128, 256)
+constexpr uint32_t S0_COL = 128;
 using L = Lanes<8>;
 using RecT = L::R;
 
@@ -73,13 +77,14 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
     uint8_t* smem = smem_raw + (base - raw);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t s0_addr = base;
-    uint8_t* ring = smem + S0_BYTES;
+    uint8_t* ring = smem;
     uint8_t* stage = ring + SLOTS * SLOT_BYTES;
     float2* gates_s = reinterpret_cast<float2*>(stage + STAGE_BYTES);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(stage + STAGE_BYTES + GATE_BYTES);
-    // bars: 0 S_0 image, 1 staged records, 2+s slot s full, 4+s slot s MMA done, 6+s slot s free
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+    uint8_t* heads = stage + STAGE_BYTES + GATE_BYTES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(heads + HEADS_TOTAL);
+    // bars: 0 S_0 in tensor memory, 1 staged records, 2+s slot s full, 4+s slot s MMA done, 6+s slot s free,
+    //       8 + 2*w + st: head stage st of fold warp w
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8 + FOLD_WARPS * HEAD_STAGES);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int* quad_count = reinterpret_cast<int*>(tmem_slot + 2);   // [SLOTS] quads written into the slot in its current use
     const uint32_t bar_s0 = smem_u32(bars), bar_stage = smem_u32(bars + 1);
@@ -88,13 +93,14 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
     auto bar_free = [&](int s) { return smem_u32(bars + 6 + s); };
 
     if (tid == 0) {
-        mbar_init(bar_s0, 1);
+        mbar_init(bar_s0, 4);                         // the four epilogue warps, once S_0 sits in tensor memory
         mbar_init(bar_stage, 32);
         for (int s = 0; s < SLOTS; ++s) {
             mbar_init(bar_full(s), 2 * FOLD_WARPS);   // one arrival per quad: 16 quads of 4 beams per group
             mbar_init(bar_done(s), 1);                // tcgen05.commit
             mbar_init(bar_free(s), 4);                // the four epilogue warps
         }
+        for (int i = 0; i < FOLD_WARPS * HEAD_STAGES; ++i) mbar_init(smem_u32(bars + 8 + i), 1);
         *abort_flag = 0;
         quad_count[0] = quad_count[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -125,6 +131,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
 #define ONELA_TICK(i)
 #endif
     bool dead = false;                    // this warp gave up (timeout or abort raised elsewhere)
+    int heads_issued = 0, heads_taken = 0;   // fold warps: quads whose heads were requested / consumed so far
     int seg_idx = 0;
     for (int sg_begin = g_begin, sg_end; sg_begin < g_end; sg_begin = sg_end, ++seg_idx) {
         const int pair = sg_begin / groups_per_pair;
@@ -150,10 +157,6 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
         // after the last group's MMA completed and was read back; the fold warps after their last staged read.
         __syncthreads();
         if (warp == 0 && !dead) {
-            if (lane == 0) {
-                mbar_expect_tx(bar_s0, S0_BYTES);
-                bulk_load(s0_addr, a.s0 + req * a.s0_req_stride + (long long)h * (DV * DK), S0_BYTES, bar_s0);
-            }
             const int32_t* ulist = a.ulist + req * a.ulist_req_stride;
             const int mine = (n_staged > lane) ? (n_staged - lane + 31) / 32 : 0;
             mbar_expect_tx(bar_stage, mine * REC_BYTES);   // one arrival per lane, with the bytes it is about to request
@@ -178,72 +181,62 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
             // quad k of the segment: group sg_begin + k/2, rows (k&1)*32 + 4*warp + grp
             const int n_quads = 2 * (sg_end - sg_begin);
             auto beam_of = [&](int k) { return ((sg_begin + (k >> 1)) - pair * groups_per_pair) * GN + (k & 1) * 32 + 4 * warp + grp; };
-            // The head of quad k (query, own record, gates of its four units) is copied asynchronously into the
-            // quad's own rows of its ring slot - free until the quad's results are written there - one quad ahead.
+            // The heads of a quad (own record and query of its four units) arrive by 16-byte async copies into a
+            // two-stage ring private to the warp, two quads ahead of their use (each lane copies exactly the
+            // chunks it reads back); the gates ride in registers.
             auto slot_of = [&](int k) { return (gcount0 + (k >> 1)) & 1; };
             auto use_of = [&](int k) { return (gcount0 + (k >> 1)) >> 1; };
             auto row_of = [&](int k) { return (k & 1) * 32 + 4 * warp + grp; };
-            auto stage_head = [&](int k) -> bool {     // false: gave up waiting for the slot
-                const int s = slot_of(k), use = use_of(k), u = row_of(k);
-                if ((k & 1) == 0 && use > 0 && !wait_or_abort(bar_free(s), (use - 1) & 1, abort_flag)) return false;
-                const int bb = min(beam_of(k), a.W - 1);   // idle groups shadow a live beam: uniform control flow
-                uint8_t* R_s = ring + s * SLOT_BYTES;
-                const uint32_t c_row = smem_u32(R_s + R_BYTES + u * (DV * 4));
-                const char* rec = kv + (own_row0 + bb) * REC_BYTES;
-                const char* qrow = reinterpret_cast<const char*>(qbase + (((long long)req * a.W + bb) * a.H + h) * DK);
+            uint8_t* my_heads = heads + warp * (HEAD_STAGES * HEAD_BYTES);
+            auto head_bar = [&](int st) { return smem_u32(bars + 8 + warp * HEAD_STAGES + st); };
+            auto q_row = [&](int bb) { return reinterpret_cast<const char*>(qbase + (((long long)req * a.W + bb) * a.H + h) * DK); };
+            auto issue_head = [&](int k) {   // every lane copies the chunks it will read back itself
+                const int st = heads_issued & 1;
+                const int bb = min(beam_of(k), a.W - 1);             // idle units shadow a live beam
+                const uint32_t dst = smem_u32(my_heads + st * HEAD_BYTES);
+                const char* rec = kv + (own_row0 + bb) * REC_BYTES + g * 16;
+                const char* qr = q_row(bb) + g * 16;
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    const int ci = c * 8 + g;   // 16-byte chunk of a 256-byte vector
-                    cp_async16(smem_u32(R_s + (ci >> 3) * R_KB_STRIDE + u * 128 + (ci & 7) * 16), rec + ci * 16);
-                    cp_async16(smem_u32(R_s + (2 + (ci >> 3)) * R_KB_STRIDE + u * 128 + (ci & 7) * 16), rec + 256 + ci * 16);
-                    cp_async16(c_row + ci * 16, qrow + ci * 16);
-                }
-                if (g == 0) cp_async8(c_row + 256, a.gates + own_row0 + bb);
+                for (int c = 0; c < 4; ++c) cp_async16(dst + grp * REC_BYTES + (c * 8 + g) * 16, rec + c * 128);
+#pragma unroll
+                for (int c = 0; c < 2; ++c) cp_async16(dst + 4 * REC_BYTES + grp * (DK * 2) + (c * 8 + g) * 16, qr + c * 128);
                 asm volatile("cp.async.commit_group;" ::: "memory");
-                return true;
+                ++heads_issued;
             };
-            auto take_head = [&](int k) {
-                Head u;
-                const int s = slot_of(k), row = row_of(k);
-                const uint8_t* R_s = ring + s * SLOT_BYTES;
-                const uint4* c_row = reinterpret_cast<const uint4*>(R_s + R_BYTES + row * (DV * 4));
-#pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    const int ci = c * 8 + g;
-                    u.own.k[c] = *reinterpret_cast<const uint4*>(R_s + (ci >> 3) * R_KB_STRIDE + row * 128 + (ci & 7) * 16);
-                    u.own.v[c] = *reinterpret_cast<const uint4*>(R_s + (2 + (ci >> 3)) * R_KB_STRIDE + row * 128 + (ci & 7) * 16);
-                    u.q[c] = c_row[ci];
-                }
-                u.own.gate = *reinterpret_cast<const float2*>(c_row + 16);
-                return u;
-            };
-            auto l2_prefetch = [&](int k) {   // seven 128-byte lines per unit (record 4, query 2, gates 1), one per lane
-                if (g < 7) {
-                    const int bb = min(beam_of(k), a.W - 1);
-                    const char* rec = kv + (own_row0 + bb) * REC_BYTES;
-                    const char* qrow = reinterpret_cast<const char*>(qbase + (((long long)req * a.W + bb) * a.H + h) * DK);
-                    const char* line = g < 4 ? rec + g * 128
-                                             : (g < 6 ? qrow + (g - 4) * 128 : reinterpret_cast<const char*>(a.gates + own_row0 + bb));
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(line));
-                }
-            };
+            auto load_gate = [&](int k) { return __ldg(a.gates + own_row0 + min(beam_of(k), a.W - 1)); };
+            float2 gate0 = make_float2(1.f, 0.f), gate1 = gate0;
             if (!dead && n_quads > 0) {
-                if (!stage_head(0)) dead = true;
-                if (1 < n_quads) l2_prefetch(1);
-                if (2 < n_quads) l2_prefetch(2);
+                issue_head(0);
+                gate0 = load_gate(0);
+                if (1 < n_quads) { issue_head(1); gate1 = load_gate(1); }
             }
             bool staged_ready = false;
             for (int k = 0; k < n_quads && !dead; ++k) {
                 const int s = slot_of(k), use = use_of(k);
                 const int u = row_of(k);                         // row of this unit in the slot
                 const int bb = min(beam_of(k), a.W - 1);
-                asm volatile("cp.async.wait_all;" ::: "memory");
-                __syncwarp();
-                const Head cur = take_head(k);
-                __syncwarp();                                    // every lane has read the scratch rows
-                // the next quad's head starts its trip now and lands while this quad is folded
-                if (k + 1 < n_quads && !stage_head(k + 1)) { dead = true; break; }
-                if (k + 3 < n_quads) l2_prefetch(k + 3);
+                Head cur;
+                {
+                    const int st = heads_taken & 1;
+                    // the oldest copy group in flight is this quad's; a newer one (the next quad's) may stay pending
+                    if (heads_issued - heads_taken > 1) asm volatile("cp.async.wait_group 1;" ::: "memory");
+                    else asm volatile("cp.async.wait_group 0;" ::: "memory");
+                    ONELA_TICK(5)   // (fold warps) wait for the head
+                    const uint4* rec = reinterpret_cast<const uint4*>(my_heads + st * HEAD_BYTES + grp * REC_BYTES) + g;
+                    const uint4* qv = reinterpret_cast<const uint4*>(my_heads + st * HEAD_BYTES + 4 * REC_BYTES + grp * (DK * 2)) + g;
+                    cur.own.k[0] = rec[0]; cur.own.k[1] = rec[8];
+                    cur.own.v[0] = rec[16]; cur.own.v[1] = rec[24];
+                    cur.q[0] = qv[0]; cur.q[1] = qv[8];
+                    cur.own.gate = gate0;
+                    ++heads_taken;
+                }
+                gate0 = gate1;
+#ifdef ONELA_TIMING
+                if ((cur.q[0].x ^ cur.own.k[0].x ^ cur.own.v[1].w) == 0x12345678u) tph[7]++;
+                ONELA_TICK(6)   // (fold warps) read the head from the stage
+#endif
+                if (k + 2 < n_quads) { issue_head(k + 2); gate1 = load_gate(k + 2); }
+                ONELA_TICK(2)   // (fold warps) issue the head after next
 
                 // lane g keeps the index of level g: position in the staged list for staged levels, arena slot otherwise
                 int32_t my_idx = 0;
@@ -276,6 +269,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
                 }
 
                 ONELA_TICK(1)   // fold
+                // the slot must have been handed back by the epilogue of its previous use
+                if (use > 0 && !wait_or_abort(bar_free(s), (use - 1) & 1, abort_flag)) { dead = true; break; }
+                ONELA_TICK(7)   // wait for the slot
                 uint8_t* R_s = ring + s * SLOT_BYTES;
                 float* C_s = reinterpret_cast<float*>(R_s + R_BYTES);
                 {
@@ -313,13 +309,13 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                         if (ok) {
                             constexpr uint32_t idesc = idesc_tf32(GN);
-                            const uint64_t ad = umma_desc(s0_addr), bd = umma_desc(smem_u32(R_s));
+                            const uint64_t bd = umma_desc(smem_u32(R_s));
 #pragma unroll
                             for (int kb = 0; kb < 4; ++kb)
 #pragma unroll
                                 for (int ks = 0; ks < 4; ++ks)
-                                    umma_tf32(tmem_base + s * GN, ad + (uint64_t)((kb * (DV * 128) + ks * 32) >> 4),
-                                              bd + (uint64_t)((kb * R_KB_STRIDE + ks * 32) >> 4), idesc, (kb | ks) ? 1u : 0u);
+                                    umma_tf32_ts(tmem_base + s * GN, tmem_base + S0_COL + (kb * 4 + ks) * 8,
+                                                 bd + (uint64_t)((kb * R_KB_STRIDE + ks * 32) >> 4), idesc, (kb | ks) ? 1u : 0u);
                         } else {
                             mma_failed = 1;
                         }
@@ -333,6 +329,28 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
             // =============================== EPILOGUE ===============================
             const int quad = warp & 3;                    // tensor-memory lane quadrant of this warp
             const int i = quad * 32 + lane;               // output element (dv index) of this thread
+            if (!dead) {
+                // Row i of the head's S_0 goes to lane i of tensor memory (the MMA's A operand lives there: no
+                // shared-memory copy of S_0, no S_0 bandwidth per MMA).  The store keeps the rows as four
+                // 128-byte pieces with their 16-byte chunks permuted; all values are already TF32.
+                const float* img = a.s0 + req * a.s0_req_stride + (long long)h * (DV * DK);
+#pragma unroll 1
+                for (int kb = 0; kb < 4; ++kb) {
+                    uint32_t v[32];
+                    const float4* piece = reinterpret_cast<const float4*>(img + kb * (DV * 32) + i * 32);
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const float4 x = __ldg(piece + (c ^ (i & 7)));
+                        v[4 * c] = __float_as_uint(x.x); v[4 * c + 1] = __float_as_uint(x.y);
+                        v[4 * c + 2] = __float_as_uint(x.z); v[4 * c + 3] = __float_as_uint(x.w);
+                    }
+                    tmem_st32(tmem_base + S0_COL + kb * 32 + ((uint32_t)(quad * 32) << 16), v);
+                }
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_s0);
+            }
             for (int gi = sg_begin; gi < sg_end && !dead; ++gi) {
                 const int gcount = gcount0 + (gi - sg_begin);
                 const int s = gcount & 1, use = gcount >> 1;
@@ -382,16 +400,14 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
 
 #ifdef ONELA_TIMING
     if (lane == 0 && (warp == 0 || warp == 7 || warp == 8) && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1) && (a.depth == 1 || a.depth == 8))
-        printf("cta %d warp %d depth %d groups %d total %lld | head %lld fold %lld slotwait %lld write %lld arrive+mma %lld | epi: wait %lld tmemld %lld rest %lld\n",
-               (int)blockIdx.x, warp, a.depth, g_end - g_begin, clock64() - tstart, tph[0], tph[1], tph[2], tph[3], tph[4], tph[5], tph[2], tph[6]);
+        printf("cta %d warp %d depth %d groups %d total %lld | head %lld fold %lld slotwait %lld write %lld arrive+mma %lld | t5 %lld t2 %lld t6 %lld\n",
+               (int)blockIdx.x, warp, a.depth, g_end - g_begin, clock64() - tstart, tph[0], tph[1], tph[7], tph[3], tph[4], tph[5], tph[2], tph[6]);
 #endif
     // A CTA must not exit with bulk copies still landing in its shared memory: after an abort nobody may
-    // have waited for the last segment's copies.
+    // have waited for the last segment's copies, nor a fold warp for the heads it had requested.
+    asm volatile("cp.async.wait_all;" ::: "memory");
     __syncthreads();
-    if (tid == 0 && *abort_flag && g_begin < g_end) {
-        mbar_wait(bar_s0, (seg_idx - 1) & 1);
-        mbar_wait(bar_stage, (seg_idx - 1) & 1);
-    }
+    if (tid == 0 && *abort_flag && g_begin < g_end) mbar_wait(bar_stage, (seg_idx - 1) & 1);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 0) {
