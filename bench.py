@@ -5,7 +5,7 @@
 
 One STEP is one whole generation of the workload through the C ABI: reset, store every shared state
 (a1), then for every decode call: reorder_beams (a2) and, per layer, append_records (a3) and the fused
-decode_step (a4-a6).  The default workload is the 16-layer beam-512 decode stack (benchmark config 4:
+decode_step (a4-a6); by default the last two are the one-launch append_decode_step.  The default workload is the 16-layer beam-512 decode stack (benchmark config 4:
 4 requests x 16 layers x 32 heads, dk = dv = 128, depth 8, Zipf(1.5) parents, bf16 records, fp32 S_0),
 whose per-step inputs (4.6 GiB) are far larger than L2.
 
@@ -113,15 +113,21 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------------
 # our arm
 # ------------------------------------------------------------------------------------------------
-def launch_bytes(wl: inputs.Workload, out_bytes: int) -> list:
-    """Algorithmic / un-deduplicated bytes of one decode launch (all requests, one layer) per call depth."""
+def launch_bytes(wl: inputs.Workload, out_bytes: int, fused: bool) -> list:
+    """Algorithmic / un-deduplicated bytes of one decode launch (all requests, one layer) per call depth.
+    A fused append + decode launch also writes the call's records to the arena (it reads them from the
+    caller's tensors instead of the arena: same read bytes)."""
     res = []
     par = {r: [None] + [inputs.parents(wl, r, t).numpy() for t in range(1, wl.D)] for r in range(wl.R)}
     for t in range(wl.D):
         distinct = [sum(accounting.distinct_records(par[r][:t + 1], [wl.W] * (t + 1))) for r in range(wl.R)]
-        res.append(accounting.decode_bytes(R=wl.R, H=wl.H, dk=wl.dk, dv=wl.dv, W=wl.W, depth=t + 1,
-                                           elem_bytes=wl.elem_bytes, out_bytes=out_bytes,
-                                           distinct_per_request=distinct))
+        d = accounting.decode_bytes(R=wl.R, H=wl.H, dk=wl.dk, dv=wl.dv, W=wl.W, depth=t + 1,
+                                    elem_bytes=wl.elem_bytes, out_bytes=out_bytes, distinct_per_request=distinct)
+        if fused:
+            extra = wl.R * wl.W * wl.H * wl.record_bytes
+            d["algorithmic"] += extra
+            d["undeduplicated"] += extra
+        res.append(d)
     return res
 
 
@@ -143,14 +149,15 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     outs = run.alloc_outputs()
     torch.cuda.synchronize()
     units_per_step = wl.R * wl.W * wl.H * wl.L * wl.D
-    per_depth = launch_bytes(wl, out_bytes)
+    fused = not args.unfused
+    per_depth = launch_bytes(wl, out_bytes, fused)
 
     def generation(decode_events=None, stream=None):
         ctx.onela_reset(stream)
         for (r, l), S in S0.items():
             ctx.onela_init_shared_state(r, l, S, stream)
         for call in calls:
-            run.run_call(call, outs, stream, decode_events)
+            run.run_call(call, outs, stream, decode_events, fused=fused)
 
     def barrier():
         torch.cuda.synchronize()
@@ -240,11 +247,12 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
         "config": {"workload": describe(wl), "step": "one whole generation: reset, store S_0, then per decode call "
-                   "reorder + per layer append + decode", "units_per_step": units_per_step,
+                   "reorder + per layer append + decode (one fused launch per layer unless --unfused)", "units_per_step": units_per_step,
                    "l2": "inputs larger than L2 (%.1f GiB of records, queries and states per step)" %
                          ((wl.R * wl.W * wl.H * wl.L * wl.D * (wl.record_bytes + wl.dk * wl.elem_bytes)
                            + wl.R * wl.L * wl.H * wl.dk * wl.dv * 4) / 2 ** 30),
-                   "out_dtype": out_dtype, "launch": mode, "parallelism": f"replicas x{world} (requests are independent)",
+                   "out_dtype": out_dtype, "launch": mode,
+                   "per_layer_calls": "append_records + decode_step" if args.unfused else "append_decode_step (one launch)", "parallelism": f"replicas x{world} (requests are independent)",
                    "tensor_core_path": bool(ctx.onela_uses_tensor_core_path())},
         "clocks": {**clocks.summary(), "window": "sampled from the warm-up to the end of the timed legs"},
         "e2e": {"value": e2e["value"], "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
@@ -255,8 +263,9 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
                      "traffic_note": "ncu DRAM read+write bytes of one launch at the deepest call (depth %d), whose "
                                      "algorithmic bytes are %.1f MB; see profiles/" % (wl.D, per_depth[-1]["algorithmic"] / 1e6),
                      "peak_source": peak_src,
-                     "kernel": "decode_step (all requests of one layer per launch)",
-                     "bytes": "algorithmic: S_0 once + each distinct record once + q + o + ancestry rows",
+                     "kernel": ("decode_step" if args.unfused else "append_decode_step") + " (all requests of one layer per launch)",
+                     "bytes": "algorithmic: S_0 once + each distinct record once + q + o + ancestry rows"
+                              + ("" if args.unfused else " + the call's records written to the arena"),
                      "undeduplicated_gbs": und_total / (dur_ms.sum() * 1e-3) / 1e9,
                      "per_depth": [{"depth": t + 1, "us": float(ms_depth[t] * 1e3),
                                     "algorithmic_MB": per_depth[t]["algorithmic"] / 1e6,
@@ -298,7 +307,7 @@ def run_e2e(args, run, S0, calls, outs, units_per_step, barrier) -> dict:
             for dl, hl in zip(dcall["layers"], hc["layers"]):
                 for n in dl:
                     dl[n].copy_(hl[n], non_blocking=True)
-            run.run_call(stage, outs)
+            run.run_call(stage, outs, fused=not args.unfused)
             for ho, o in zip(houts, outs):
                 ho.copy_(o, non_blocking=True)
 
@@ -389,6 +398,7 @@ def main():
     ap.add_argument("--workload", default="cfg4")
     ap.add_argument("--out-dtype", default=None, choices=[None, "fp32", "bf16"])
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--unfused", action="store_true", help="separate append_records and decode_step launches per layer")
     ap.add_argument("--settle-seconds", type=float, default=1.0, help="extra untimed warm-up after the W steps")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling)")
     ap.add_argument("--force-generic", action="store_true", help="run the CUDA-core decode kernel")

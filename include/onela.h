@@ -139,6 +139,15 @@ onela_status onela_append_records(onela_ctx* ctx, int32_t req_begin, int32_t req
 onela_status onela_decode_step(onela_ctx* ctx, int32_t req_begin, int32_t req_count, int32_t layer,
                                const void* q_dev, void* out_dev, void* stream);
 
+/* append_records and decode_step of one layer in ONE launch (the paper's kernel also appends the new
+ * record inside the decode kernel, Section 3.4): the call's records are read from the caller's tensors,
+ * folded as each beam's newest record, and written to the arena by the same kernel, so they cross HBM
+ * once instead of three times.  Same arguments, checks and call-order rules as the two calls it replaces
+ * (it counts as the layer's one append of this decode call; decode_step may still be called afterwards). */
+onela_status onela_append_decode_step(onela_ctx* ctx, int32_t req_begin, int32_t req_count, int32_t layer,
+                                      const void* k_dev, const void* v_dev, const float* alpha_dev,
+                                      const float* beta_dev, const void* q_dev, void* out_dev, void* stream);
+
 /* Copy the ancestry rows of one request to slots_dev [W][depth] int32 (global slot ids, oldest first;
  * the last column is the beam's own record).  depth_host / width_host (host pointers, may be NULL)
  * receive the shape immediately. */

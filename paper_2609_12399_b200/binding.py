@@ -51,6 +51,8 @@ PROTOTYPES = {
     "onela_reorder_beams": (c_int32, [c_void_p, c_int32, c_int32, c_void_p, c_int32, c_void_p]),
     "onela_append_records": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
                                        c_void_p]),
+    "onela_append_decode_step": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
+                                           c_void_p, c_void_p, c_void_p]),
     "onela_decode_step": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p]),
     "onela_export_chains": (c_int32, [c_void_p, c_int32, c_void_p, POINTER(c_int32), POINTER(c_int32), c_void_p]),
     "onela_poll_device_status": (c_int32, [c_void_p, POINTER(c_int32), POINTER(c_int32)]),
@@ -207,6 +209,19 @@ class Onela:
             self.handle, req_begin, req_count, layer,
             self._ptr(q, self.rec_dtype, (req_count, W, c.num_heads, c.dk), "q"),
             self._ptr(out, self.out_dtype, (req_count, W, c.num_heads, c.dv), "out"), self._s(stream)), "onela_decode_step")
+
+    def onela_append_decode_step(self, req_begin, req_count, layer, k, v, alpha, beta, q, out, stream=None):
+        c = self.cfg
+        _, W = self._width(req_begin)
+        _check(self.lib.onela_append_decode_step(
+            self.handle, req_begin, req_count, layer,
+            self._ptr(k, self.rec_dtype, (req_count, W, c.num_heads, c.dk), "k"),
+            self._ptr(v, self.rec_dtype, (req_count, W, c.num_heads, c.dv), "v"),
+            self._ptr(alpha, torch.float32, (req_count, W, c.num_heads), "alpha"),
+            self._ptr(beta, torch.float32, (req_count, W, c.num_heads), "beta"),
+            self._ptr(q, self.rec_dtype, (req_count, W, c.num_heads, c.dk), "q"),
+            self._ptr(out, self.out_dtype, (req_count, W, c.num_heads, c.dv), "out"), self._s(stream)),
+            "onela_append_decode_step")
 
     def onela_export_chains(self, request, stream=None) -> torch.Tensor:
         """Returns int32 [W, depth] global slot ids (oldest first) on the device."""

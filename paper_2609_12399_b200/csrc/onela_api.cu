@@ -319,25 +319,25 @@ onela_status onela_append_records(onela_ctx* ctx, int32_t req_begin, int32_t req
     return ONELA_OK;
 }
 
-onela_status onela_decode_step(onela_ctx* ctx, int32_t req_begin, int32_t req_count, int32_t layer,
-                               const void* q_dev, void* out_dev, void* stream) {
-    onela_status st = check_batch(ctx, req_begin, req_count);
-    if (st != ONELA_OK) return st;
+}  // extern "C"
+
+namespace {
+
+// Shared by decode_step and append_decode_step: fill the kernel arguments and launch.
+onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count, int32_t layer, const void* q_dev,
+                           void* out_dev, const void* k_dev, const void* v_dev, const float* alpha_dev,
+                           const float* beta_dev, cudaStream_t s) {
     const onela_config& c = ctx->cfg;
-    if (layer < 0 || layer >= c.num_layers) return ONELA_E_INVAL;
-    if (!q_dev || !out_dev || !aligned16(q_dev) || !aligned16(out_dev)) return ONELA_E_INVAL;
     const int32_t depth = ctx->req[req_begin].depth, W = ctx->req[req_begin].W;
-    if (depth < 1) return ONELA_E_ORDER;
-    for (int i = 0; i < req_count; ++i) {
-        const ReqState& r = ctx->req[req_begin + i];
-        if (!r.has_state[layer] || r.appended_depth[layer] != depth) return ONELA_E_ORDER;
-    }
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if ((st = ctx->prepare(s)) != ONELA_OK) return st;
-    if (ctx->dry()) return ONELA_OK;
     DecodeArgs a{};
     a.q = q_dev;
     a.out = out_dev;
+    a.k_in = k_dev;
+    a.v_in = v_dev;
+    a.alpha_in = alpha_dev;
+    a.beta_in = beta_dev;
+    a.kv_out = ctx->kv_plane(layer);
+    a.gates_out = ctx->gate_plane(layer);
     a.s0 = ctx->s0_slot(req_begin, layer);
     a.kv = ctx->kv_plane(layer);
     a.gates = ctx->gate_plane(layer);
@@ -369,6 +369,70 @@ onela_status onela_decode_step(onela_ctx* ctx, int32_t req_begin, int32_t req_co
     if (!supported) return ONELA_E_UNSUPPORTED;
     if (e != cudaSuccess) return ONELA_E_CUDA;
     ctx->launches++;
+    return ONELA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+onela_status onela_decode_step(onela_ctx* ctx, int32_t req_begin, int32_t req_count, int32_t layer,
+                               const void* q_dev, void* out_dev, void* stream) {
+    onela_status st = check_batch(ctx, req_begin, req_count);
+    if (st != ONELA_OK) return st;
+    const onela_config& c = ctx->cfg;
+    if (layer < 0 || layer >= c.num_layers) return ONELA_E_INVAL;
+    if (!q_dev || !out_dev || !aligned16(q_dev) || !aligned16(out_dev)) return ONELA_E_INVAL;
+    const int32_t depth = ctx->req[req_begin].depth;
+    if (depth < 1) return ONELA_E_ORDER;
+    for (int i = 0; i < req_count; ++i) {
+        const ReqState& r = ctx->req[req_begin + i];
+        if (!r.has_state[layer] || r.appended_depth[layer] != depth) return ONELA_E_ORDER;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if ((st = ctx->prepare(s)) != ONELA_OK) return st;
+    if (ctx->dry()) return ONELA_OK;
+    return launch_decode(ctx, req_begin, req_count, layer, q_dev, out_dev, nullptr, nullptr, nullptr, nullptr, s);
+}
+
+onela_status onela_append_decode_step(onela_ctx* ctx, int32_t req_begin, int32_t req_count, int32_t layer,
+                                      const void* k_dev, const void* v_dev, const float* alpha_dev,
+                                      const float* beta_dev, const void* q_dev, void* out_dev, void* stream) {
+    onela_status st = check_batch(ctx, req_begin, req_count);
+    if (st != ONELA_OK) return st;
+    const onela_config& c = ctx->cfg;
+    if (layer < 0 || layer >= c.num_layers) return ONELA_E_INVAL;
+    if (!k_dev || !v_dev || !alpha_dev || !beta_dev || !aligned16(k_dev) || !aligned16(v_dev)) return ONELA_E_INVAL;
+    if (!q_dev || !out_dev || !aligned16(q_dev) || !aligned16(out_dev)) return ONELA_E_INVAL;
+    const int32_t depth = ctx->req[req_begin].depth, W = ctx->req[req_begin].W;
+    if (depth < 1) return ONELA_E_ORDER;
+    for (int i = 0; i < req_count; ++i) {
+        const ReqState& r = ctx->req[req_begin + i];
+        if (!r.has_state[layer] || r.appended_depth[layer] == depth) return ONELA_E_ORDER;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if ((st = ctx->prepare(s)) != ONELA_OK) return st;
+    if (!ctx->dry()) {
+        if (ctx->tensor_core) {
+#ifdef ONELA_PIPELINED
+            return ONELA_E_UNSUPPORTED;
+#else
+            st = launch_decode(ctx, req_begin, req_count, layer, q_dev, out_dev, k_dev, v_dev, alpha_dev, beta_dev, s);
+            if (st != ONELA_OK) return st;
+#endif
+        } else {   // shapes without the fused kernel: the copy kernel, then the decode kernel
+            BatchBases bases{};
+            for (int i = 0; i < req_count; ++i) bases.base[i] = ctx->req[req_begin + i].step_base.back();
+            if (launch_append(k_dev, v_dev, alpha_dev, beta_dev, ctx->kv_plane(layer), ctx->gate_plane(layer),
+                              c.arena_slots, req_count, W, c.num_heads, c.dk, c.dv, ctx->elem_bytes, bases,
+                              s) != cudaSuccess)
+                return ONELA_E_CUDA;
+            ctx->launches++;
+            st = launch_decode(ctx, req_begin, req_count, layer, q_dev, out_dev, nullptr, nullptr, nullptr, nullptr, s);
+            if (st != ONELA_OK) return st;
+        }
+    }
+    for (int i = 0; i < req_count; ++i) ctx->req[req_begin + i].appended_depth[layer] = depth;
     return ONELA_OK;
 }
 

@@ -32,23 +32,28 @@ namespace {
 
 using namespace sm100;
 
-constexpr int FOLD_WARPS = 8;
+#ifndef ONELA_FOLD_WARPS
+#define ONELA_FOLD_WARPS 12
+#endif
+constexpr int FOLD_WARPS = ONELA_FOLD_WARPS;
+constexpr int QPG = FOLD_WARPS == 8 ? 2 : 1;        // quads each fold warp contributes to a group
 constexpr int THREADS = (FOLD_WARPS + 4) * 32;      // + 4 epilogue warps (12 warps: three per SM sub-partition)
-constexpr int GN = 64;                              // beams per group = MMA N
+constexpr int GN = FOLD_WARPS * 4 * QPG;            // beams per group = MMA N (64 or 48)
 constexpr int R_KB_STRIDE = GN * 128;               // bytes between the four 32-float K blocks of the operand
 constexpr int R_BYTES = 4 * R_KB_STRIDE;            // 32768
 constexpr int C_BYTES = GN * DV * 4;                // 32768: corr tile, row = beam
 constexpr int SLOT_BYTES = R_BYTES + C_BYTES;
 constexpr int SLOTS = 2;
-constexpr int STAGE_CAP = 64;                       // distinct ancestor records staged per segment
+constexpr int STAGE_CAP = FOLD_WARPS == 8 ? 88 : 104;                       // distinct ancestor records staged per segment
 constexpr int STAGE_BYTES = STAGE_CAP * REC_BYTES;
 constexpr int GATE_BYTES = STAGE_CAP * 8;
 constexpr int HEAD_BYTES = 4 * (REC_BYTES + DK * 2);     // one quad's heads: 4 own records + 4 queries = 3072
 constexpr int HEAD_STAGES = 2;                         // heads in flight per fold warp
 constexpr int HEADS_TOTAL = FOLD_WARPS * HEAD_STAGES * HEAD_BYTES;
 constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + STAGE_BYTES + GATE_BYTES + HEADS_TOTAL + 256 + 1024;
-constexpr uint32_t TMEM_COLS = 256;              // accumulators of the two slots in [0, 128), the head's S_0 in [128, 256)
+constexpr uint32_t TMEM_COLS = 256;              // accumulators of the two slots in [0, 2 GN), the head's S_0 in [128, 256)
 constexpr uint32_t S0_COL = 128;
+static_assert(SMEM_BYTES <= 232448, "shared memory per CTA");
 using L = Lanes<8>;
 using RecT = L::R;
 
@@ -96,7 +101,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
         mbar_init(bar_s0, 4);                         // the four epilogue warps, once S_0 sits in tensor memory
         mbar_init(bar_stage, 32);
         for (int s = 0; s < SLOTS; ++s) {
-            mbar_init(bar_full(s), 2 * FOLD_WARPS);   // one arrival per quad: 16 quads of 4 beams per group
+            mbar_init(bar_full(s), QPG * FOLD_WARPS); // one arrival per quad of 4 beams
             mbar_init(bar_done(s), 1);                // tcgen05.commit
             mbar_init(bar_free(s), 4);                // the four epilogue warps
         }
@@ -119,6 +124,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
     const int g_begin = (int)(((long long)blockIdx.x * total_groups) / gridDim.x);
     const int g_end = (int)(((long long)(blockIdx.x + 1) * total_groups) / gridDim.x);
     const int old = a.depth - 1;          // records older than a beam's own: levels old-1 .. 0
+    const bool fused = a.k_in != nullptr;  // append fused in: the newest record comes from the caller's tensors
     const char* kv = a.kv;
     const __nv_bfloat16* qbase = static_cast<const __nv_bfloat16*>(a.q);
 
@@ -142,15 +148,14 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
         const uint32_t seg_parity = seg_idx & 1;
 
         // How many of the oldest levels fit in the staging buffer (whole levels only; uniform over the CTA).
+        // Lane l looks at level l (one load latency for the whole chain); offsets grow with the level.
         int staged_levels = 0, n_staged = 0;
         {
             const int32_t* uoff = a.uoff + req * a.uoff_req_stride;
-            for (int l = 0; l < old; ++l) {
-                const int e = __ldg(uoff + l + 1);
-                if (e > STAGE_CAP) break;
-                staged_levels = l + 1;
-                n_staged = e;
-            }
+            const int e = (lane < old) ? __ldg(uoff + lane + 1) : 0x7fffffff;
+            staged_levels = __popc(__ballot_sync(0xffffffffu, e <= STAGE_CAP));
+            n_staged = __shfl_sync(0xffffffffu, e, staged_levels > 0 ? staged_levels - 1 : 0);
+            if (staged_levels == 0) n_staged = 0;
         }
 
         // The previous segment is fully consumed: the MMA warp and the epilogue warps pass this barrier only
@@ -179,14 +184,16 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
                 __syncwarp();
             }
             // quad k of the segment: group sg_begin + k/2, rows (k&1)*32 + 4*warp + grp
-            const int n_quads = 2 * (sg_end - sg_begin);
-            auto beam_of = [&](int k) { return ((sg_begin + (k >> 1)) - pair * groups_per_pair) * GN + (k & 1) * 32 + 4 * warp + grp; };
+            const int n_quads = QPG * (sg_end - sg_begin);
+            auto group_of = [&](int k) { return QPG == 2 ? (k >> 1) : k; };
+            auto half_of = [&](int k) { return QPG == 2 ? (k & 1) : 0; };
+            auto beam_of = [&](int k) { return ((sg_begin + group_of(k)) - pair * groups_per_pair) * GN + half_of(k) * 32 + 4 * warp + grp; };
             // The heads of a quad (own record and query of its four units) arrive by 16-byte async copies into a
             // two-stage ring private to the warp, two quads ahead of their use (each lane copies exactly the
             // chunks it reads back); the gates ride in registers.
-            auto slot_of = [&](int k) { return (gcount0 + (k >> 1)) & 1; };
-            auto use_of = [&](int k) { return (gcount0 + (k >> 1)) >> 1; };
-            auto row_of = [&](int k) { return (k & 1) * 32 + 4 * warp + grp; };
+            auto slot_of = [&](int k) { return (gcount0 + group_of(k)) & 1; };
+            auto use_of = [&](int k) { return (gcount0 + group_of(k)) >> 1; };
+            auto row_of = [&](int k) { return half_of(k) * 32 + 4 * warp + grp; };
             uint8_t* my_heads = heads + warp * (HEAD_STAGES * HEAD_BYTES);
             auto head_bar = [&](int st) { return smem_u32(bars + 8 + warp * HEAD_STAGES + st); };
             auto q_row = [&](int bb) { return reinterpret_cast<const char*>(qbase + (((long long)req * a.W + bb) * a.H + h) * DK); };
@@ -194,16 +201,32 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
                 const int st = heads_issued & 1;
                 const int bb = min(beam_of(k), a.W - 1);             // idle units shadow a live beam
                 const uint32_t dst = smem_u32(my_heads + st * HEAD_BYTES);
-                const char* rec = kv + (own_row0 + bb) * REC_BYTES + g * 16;
                 const char* qr = q_row(bb) + g * 16;
+                if (fused) {   // the call's records come straight from the caller's k and v tensors
+                    const long long in_row = ((long long)req * a.W + bb) * a.H + h;
+                    const char* kr = static_cast<const char*>(a.k_in) + in_row * (DK * 2) + g * 16;
+                    const char* vr = static_cast<const char*>(a.v_in) + in_row * (DV * 2) + g * 16;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) cp_async16(dst + grp * REC_BYTES + (c * 8 + g) * 16, rec + c * 128);
+                    for (int c = 0; c < 2; ++c) {
+                        cp_async16(dst + grp * REC_BYTES + (c * 8 + g) * 16, kr + c * 128);
+                        cp_async16(dst + grp * REC_BYTES + (16 + c * 8 + g) * 16, vr + c * 128);
+                    }
+                } else {
+                    const char* rec = kv + (own_row0 + bb) * REC_BYTES + g * 16;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) cp_async16(dst + grp * REC_BYTES + (c * 8 + g) * 16, rec + c * 128);
+                }
 #pragma unroll
                 for (int c = 0; c < 2; ++c) cp_async16(dst + 4 * REC_BYTES + grp * (DK * 2) + (c * 8 + g) * 16, qr + c * 128);
                 asm volatile("cp.async.commit_group;" ::: "memory");
                 ++heads_issued;
             };
-            auto load_gate = [&](int k) { return __ldg(a.gates + own_row0 + min(beam_of(k), a.W - 1)); };
+            auto load_gate = [&](int k) {
+                const int bb = min(beam_of(k), a.W - 1);
+                if (!fused) return __ldg(a.gates + own_row0 + bb);
+                const long long in_row = ((long long)req * a.W + bb) * a.H + h;
+                return make_float2(__ldg(a.alpha_in + in_row), __ldg(a.beta_in + in_row));
+            };
             float2 gate0 = make_float2(1.f, 0.f), gate1 = gate0;
             if (!dead && n_quads > 0) {
                 issue_head(0);
@@ -229,6 +252,12 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
                     cur.q[0] = qv[0]; cur.q[1] = qv[8];
                     cur.own.gate = gate0;
                     ++heads_taken;
+                    if (fused && beam_of(k) < a.W) {   // the append: this beam's record goes to its arena slot, bit for bit
+                        uint4* dst = reinterpret_cast<uint4*>(a.kv_out + (own_row0 + bb) * REC_BYTES) + g;
+                        dst[0] = cur.own.k[0]; dst[8] = cur.own.k[1];
+                        dst[16] = cur.own.v[0]; dst[24] = cur.own.v[1];
+                        if (g == 0) a.gates_out[own_row0 + bb] = gate0;
+                    }
                 }
                 gate0 = gate1;
 #ifdef ONELA_TIMING
@@ -256,7 +285,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
 #pragma unroll
                 for (int e = 0; e < 8; ++e) corr[e] = make_float2(0.f, 0.f);
                 float decay = 1.f;
-                L::fold_chain(cur.own, old - 1, staged_levels,
+                L::fold_chain_simple(cur.own, old - 1, staged_levels,
                               [&](int level) { return L::load_global(kv, a.gates, plane_row0 + idx_of(level), g); }, r, corr, decay);
                 if (staged_levels > 0) {
                     if (!staged_ready) {
@@ -264,7 +293,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
                         staged_ready = true;
                     }
                     const RecT newest = L::load_shared(stage, gates_s, idx_of(staged_levels - 1), g);
-                    L::fold_chain(newest, staged_levels - 2, 0,
+                    L::fold_chain_simple(newest, staged_levels - 2, 0,
                                   [&](int level) { return L::load_shared(stage, gates_s, idx_of(level), g); }, r, corr, decay);
                 }
 
@@ -302,7 +331,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
                 int mma_failed = 0;
                 if (lane == 0) {
                     mbar_arrive(bar_full(s));
-                    if (atomicAdd(&quad_count[s], 1) == 2 * FOLD_WARPS - 1) {
+                    if (atomicAdd(&quad_count[s], 1) == QPG * FOLD_WARPS - 1) {
                         quad_count[s] = 0;   // the slot's next use cannot begin before this group's MMAs are read back
                         bool ok = wait_or_abort(bar_full(s), use & 1, abort_flag);      // all 16 arrivals are in: acquire
                         ok = ok && wait_or_abort(bar_s0, seg_parity, abort_flag);
@@ -363,7 +392,12 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
                 {
                     // accumulator rows (dv) of this thread, all 64 beams, added onto the corr tile in place
                     uint32_t v[GN];
-                    tmem_ld64(taddr, v);
+                    if (GN == 64) {
+                        tmem_ld64(taddr, v);
+                    } else {
+#pragma unroll
+                        for (int c0 = 0; c0 < GN; c0 += 16) tmem_ld16(taddr + c0, v + c0);
+                    }
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
                     for (int j = 0; j < GN; ++j) C_s[j * DV + i] += __uint_as_float(v[j]);
@@ -374,7 +408,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
                     // coalesced stores: 16 lanes cover one beam's 128 outputs, 8 elements each
                     const int et = (warp - FOLD_WARPS) * 32 + lane;
 #pragma unroll
-                    for (int it = 0; it < GN * 16 / 128; ++it) {
+                    for (int it = 0; it < GN * 16 / 128; ++it) {   // GN * 16 chunks of 16 bytes over 128 threads
                         const int idx = it * 128 + et, j = idx >> 4, ch = idx & 15;
                         if (b0 + j < a.W) {
                             const float4 x0 = *reinterpret_cast<const float4*>(C_s + j * DV + ch * 8);

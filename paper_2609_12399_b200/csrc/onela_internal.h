@@ -30,6 +30,12 @@ struct BatchBases {
 struct DecodeArgs {
     const void* q;          // [req_count][W][H][dk]
     void* out;              // [req_count][W][H][dv]
+    const void* k_in;       // fused append: this call's records [req_count][W][H][dk], [..][dv], gates [..][H];
+    const void* v_in;       //   null for a plain decode (the newest record is then read from the arena)
+    const float* alpha_in;
+    const float* beta_in;
+    char* kv_out;           // fused append: arena plane to write (same plane as kv)
+    float2* gates_out;
     const float* s0;        // store slot of (req_begin, layer)
     const char* kv;         // arena plane of this layer
     const float2* gates;    // gate plane of this layer

@@ -214,6 +214,16 @@ struct Lanes {
         }
         decay *= rec.gate.x;
     }
+    // Single-buffered chain: fetch a record, fold it (for sources whose latency is short, or to save registers).
+    template <class LoadFn>
+    static __device__ __forceinline__ void fold_chain_simple(const R& first, int hi, int lo, LoadFn load, float2* r,
+                                                             float2* corr, float& decay) {
+        fold_step(first, r, corr, decay);
+        for (int level = hi; level >= lo; --level) {
+            const R rec = load(level);
+            fold_step(rec, r, corr, decay);
+        }
+    }
     // Fold `first` (already in registers) and then levels hi .. lo (newest first) fetched by `load`, keeping
     // one record in flight while the previous one is folded.  Two buffers alternate so no record is moved.
     template <class LoadFn>

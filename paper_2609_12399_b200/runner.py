@@ -65,10 +65,11 @@ class WorkloadRun:
                 for _ in range(wl.L)]
 
     # ---- one decode call through the library ------------------------------------------------------
-    def run_call(self, call: dict, outs: list, stream=None, decode_events=None):
+    def run_call(self, call: dict, outs: list, stream=None, decode_events=None, fused: bool = False):
         """reorder_beams once, then append_records + decode_step per layer, batched over all requests
-        (in chunks of at most ONELA_MAX_BATCH).  ``decode_events``: optional list that receives a
-        (start, end) CUDA event pair around every decode launch."""
+        (in chunks of at most ONELA_MAX_BATCH); with ``fused`` the two per-layer calls are the one-launch
+        append_decode_step.  ``decode_events``: optional list that receives a (start, end) CUDA event pair
+        around every decode launch."""
         wl, ctx = self.wl, self.ctx
         for r0 in range(0, wl.R, MAX_BATCH):
             n = min(MAX_BATCH, wl.R - r0)
@@ -76,11 +77,16 @@ class WorkloadRun:
             ctx.onela_reorder_beams(r0, n, par, wl.W, stream)
             for l, lay in enumerate(call["layers"]):
                 sl = slice(r0, r0 + n)
-                ctx.onela_append_records(r0, n, l, lay["k"][sl], lay["v"][sl], lay["alpha"][sl], lay["beta"][sl], stream)
+                if not fused:
+                    ctx.onela_append_records(r0, n, l, lay["k"][sl], lay["v"][sl], lay["alpha"][sl], lay["beta"][sl], stream)
                 if decode_events is not None:
                     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                     e0.record(stream)
-                ctx.onela_decode_step(r0, n, l, lay["q"][sl], outs[l][sl], stream)
+                if fused:
+                    ctx.onela_append_decode_step(r0, n, l, lay["k"][sl], lay["v"][sl], lay["alpha"][sl], lay["beta"][sl],
+                                                 lay["q"][sl], outs[l][sl], stream)
+                else:
+                    ctx.onela_decode_step(r0, n, l, lay["q"][sl], outs[l][sl], stream)
                 if decode_events is not None:
                     e1.record(stream)
                     decode_events.append((e0, e1))

@@ -56,7 +56,7 @@ def run_oracle(case, upto=None, sel=None) -> tuple[dict, dict]:
     return outs, chains
 
 
-def run_library(case, out_dtype="fp32", flags=0, batched=True, device="cuda") -> tuple[dict, dict, P.Onela]:
+def run_library(case, out_dtype="fp32", flags=0, batched=True, device="cuda", fused=False) -> tuple[dict, dict, P.Onela]:
     """The same case through the C ABI.  Returns outs[(r,l,t)] (torch, CPU), slots[(r,t)] int32 [W_t, t+1]
     (global slot ids from onela_export_chains) and the context (kept alive for further queries)."""
     wl, widths = case["wl"], case["widths"]
@@ -76,10 +76,13 @@ def run_library(case, out_dtype="fp32", flags=0, batched=True, device="cuda") ->
             ctx.onela_reorder_beams(r0, n, par, W)
             for l in range(wl.L):
                 tk = {nm: torch.stack([case["tok"][(r, l, t)][nm] for r in g]).to(dev) for nm in ("k", "v", "alpha", "beta")}
-                ctx.onela_append_records(r0, n, l, tk["k"], tk["v"], tk["alpha"], tk["beta"])
                 q = torch.stack([case["q"][(r, l, t)] for r in g]).to(dev)
                 out = torch.empty((n, W, wl.H, wl.dv), dtype=ctx.out_dtype, device=dev)
-                ctx.onela_decode_step(r0, n, l, q, out)
+                if fused:     # one launch: append + decode
+                    ctx.onela_append_decode_step(r0, n, l, tk["k"], tk["v"], tk["alpha"], tk["beta"], q, out)
+                else:
+                    ctx.onela_append_records(r0, n, l, tk["k"], tk["v"], tk["alpha"], tk["beta"])
+                    ctx.onela_decode_step(r0, n, l, q, out)
                 for i, r in enumerate(g):
                     outs[(r, l, t)] = out[i].float().cpu()
             for r in g:

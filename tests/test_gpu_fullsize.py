@@ -1,5 +1,5 @@
 """Parity at the benchmark configs' FULL sizes, in the launch configuration bench.py times (all requests
-of a layer in one batched call, bf16 outputs, the tensor-core kernel).
+of a layer in one batched call, the one-launch append_decode_step, bf16 outputs, the tensor-core kernel).
 
 The oracle cannot replay every unit of these sizes in seconds, so it computes a seeded sample of
 (beam, head) units one by one for a few (request, layer) pairs at several call depths; for those pairs
@@ -30,7 +30,7 @@ def _oracle_state(wl, r, l):
     return torch.from_numpy(oracle.prefill(p["k"], p["v"], p["alpha"], p["beta"]).astype(np.float32))
 
 
-def _run_and_check(wl, pairs, check_calls, n_units=384, flags=0, keep_all_outputs=False):
+def _run_and_check(wl, pairs, check_calls, n_units=384, flags=0, keep_all_outputs=False, fused=True):
     run = WorkloadRun(wl, "cuda", "bf16", flags=flags)
     S0 = {pr: _oracle_state(wl, *pr) for pr in pairs}
     run.prefill_states(overrides=S0)
@@ -41,7 +41,7 @@ def _run_and_check(wl, pairs, check_calls, n_units=384, flags=0, keep_all_output
     worst, kept = 0.0, {}
     for t in range(wl.D):
         call = run.generate_call(t)
-        run.run_call(call, outs)
+        run.run_call(call, outs, fused=fused)     # fused: the launch configuration bench.py times
         torch.cuda.synchronize()
         if t > 0:
             par = call["parents"].cpu().numpy()
@@ -81,7 +81,8 @@ def test_config2_beam512_zipf_every_call():
     wl = inputs.WORKLOADS[2]
     worst, fused, run = _run_and_check(wl, [(0, 0)], range(wl.D), keep_all_outputs=True)
     assert run.ctx.onela_uses_tensor_core_path()
-    _, generic, run2 = _run_and_check(wl, [(0, 0)], [wl.D - 1], flags=P.FLAG_FORCE_GENERIC, keep_all_outputs=True)
+    _, generic, run2 = _run_and_check(wl, [(0, 0)], [wl.D - 1], flags=P.FLAG_FORCE_GENERIC, keep_all_outputs=True,
+                                      fused=False)
     assert not run2.ctx.onela_uses_tensor_core_path()
     for t in range(wl.D):
         a, b = fused[t][0].float().cpu().numpy(), generic[t][0].float().cpu().numpy()
@@ -89,9 +90,10 @@ def test_config2_beam512_zipf_every_call():
 
 
 def test_config3_batch8_beam1024():
-    """8 requests in one shared arena, beam 1024, depth 6, uniform parents."""
+    """8 requests in one shared arena, beam 1024, depth 6, uniform parents; fused and separate launches."""
     wl = inputs.WORKLOADS[3]
     _run_and_check(wl, [(0, 0), (7, 0)], [0, 2, wl.D - 1])
+    _run_and_check(wl, [(3, 0)], [1, wl.D - 1], fused=False)
 
 
 def test_config4_stack16_beam512():

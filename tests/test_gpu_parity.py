@@ -23,9 +23,9 @@ def _small(base, **kw):
     return base.scaled(**kw)
 
 
-def _full_check(case, out_dtype, flags=0, batched=True, tight=None):
+def _full_check(case, out_dtype, flags=0, batched=True, tight=None, fused=False):
     ref, chains = run_oracle(case)
-    outs, slots, ctx = run_library(case, out_dtype=out_dtype, flags=flags, batched=batched)
+    outs, slots, ctx = run_library(case, out_dtype=out_dtype, flags=flags, batched=batched, fused=fused)
     want = expected_slots(case, chains)
     for key in want:
         assert np.array_equal(slots[key], want[key]), f"ancestry rows of {key} differ"
@@ -44,6 +44,19 @@ def test_config0_tiny_reference():
 def test_config1_beam128(out_dtype, tight):
     """16 heads, dk = dv = 128, bf16 records, beam 128, depth 4, uniform parents; every call, every unit."""
     _full_check(make_case(CFG1), out_dtype, tight=tight)
+
+
+@pytest.mark.parametrize("out_dtype", ["fp32", "bf16"])
+def test_config1_fused_append_decode(out_dtype):
+    """The one-launch append + decode entry point on config 1: same outputs, same chains."""
+    _full_check(make_case(CFG1), out_dtype, fused=True)
+
+
+def test_fused_append_decode_other_paths():
+    _full_check(make_case(CFG0), "fp32", fused=True, tight=2e-6)                       # CUDA-core shapes: two launches inside
+    wl = CFG1.scaled(R=3, L=2, H=4, W=77, D=4, prompt_len=96, parents="zipf", zipf_s=1.3, seed=78)
+    _full_check(make_case(wl), "bf16", fused=True)                                      # ragged width, shared ancestors
+    _full_check(make_case(wl, widths=[77, 5, 130, 48]), "fp32", fused=True, batched=False)
 
 
 def test_config1_cuda_core_kernel_is_fp32_accurate():
@@ -107,12 +120,14 @@ def test_shared_chains_give_identical_outputs_on_gpu():
     assert torch.equal(o, o[0:1].expand_as(o))
 
 
-def test_records_are_stored_bit_exactly_and_never_rewritten():
+@pytest.mark.parametrize("fused", [False, True])
+def test_records_are_stored_bit_exactly_and_never_rewritten(fused):
     """The arena planes hold exactly the appended bytes at slot base(req, t) + beam, head-major, and a
-    later reorder/append leaves earlier records untouched (read straight out of the workspace)."""
+    later reorder/append leaves earlier records untouched (read straight out of the workspace); the same
+    through the fused append + decode launch."""
     wl = CFG1.scaled(R=2, H=3, W=20, D=3, prompt_len=32, seed=5)
     case = make_case(wl)
-    outs, slots, ctx = run_library(case, out_dtype="fp32")
+    outs, slots, ctx = run_library(case, out_dtype="fp32", fused=fused)
     c = ctx.cfg
     al = lambda n: (n + 1023) // 1024 * 1024
     off_tables = al(16)

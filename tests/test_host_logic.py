@@ -99,6 +99,23 @@ def test_call_order_is_enforced():
     assert o.depth_and_width(0) == (2, 5)
 
 
+def test_fused_append_decode_counts_as_the_append():
+    o = ctx()
+    o.onela_init_shared_state(0, 0, FAKE)
+    with raises(binding.E_ORDER):
+        o.onela_append_decode_step(0, 1, 0, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE)    # no decode call opened
+    o.onela_reorder_beams(0, 1, None, 8)
+    o.onela_append_decode_step(0, 1, 0, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE)
+    with raises(binding.E_ORDER):
+        o.onela_append_decode_step(0, 1, 0, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE)    # exactly one append per call
+    with raises(binding.E_ORDER):
+        o.onela_append_records(0, 1, 0, FAKE, FAKE, FAKE, FAKE)
+    o.onela_decode_step(0, 1, 0, FAKE, FAKE)                                       # decoding again is fine
+    o.onela_reorder_beams(0, 1, FAKE, 8)                                           # and the next call may open
+    with raises(binding.E_INVAL):
+        o.onela_append_decode_step(0, 1, 0, FAKE, FAKE, FAKE, FAKE, None, FAKE)
+
+
 def test_every_layer_with_state_must_append_before_next_call():
     o = ctx()
     o.onela_init_shared_state(0, 0, FAKE)
