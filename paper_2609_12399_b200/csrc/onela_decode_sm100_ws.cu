@@ -6,9 +6,7 @@
 //     scalar; packed fp32x2 FMAs).  The next quad's query and own record are loaded while the current
 //     quad is folded.  Results go into a ring slot in shared memory: the folded query as a row of the
 //     K-major 128-byte-swizzled MMA operand (rounded to TF32), corr as a row of the slot's corr tile.
-//     The warp whose quad completes a slot (all 64 rows written) issues the group's 16 tcgen05.mma
-//     (kind::tf32, M = dv = 128, N = 64 beams, K = 8) against the head's S_0 image, accumulating fp32 in
-//     tensor memory, and commits; the other fold warps are already folding the next group.
+
 //   * 4 EPILOGUE warps (one per tensor-memory lane quadrant).  When the MMA group has completed they read
 //     the accumulator, add corr and store the outputs (lane = dv index: 32 consecutive elements per store),
 //     then hand the slot back.
@@ -74,6 +72,19 @@ struct Head {           // what a unit's fold needs first
     RecT own;
 };
 
+#ifdef ONELA_TIMELINE
+__device__ __forceinline__ unsigned long long gtime() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ unsigned long long g_marks[64];
+__device__ int g_nmarks;
+#define ONELA_MARK(name) if (blockIdx.x == 0 && lane == 0) { const int mi = atomicAdd(&g_nmarks, 1); if (mi < 32) { g_marks[2 * mi] = gtime(); g_marks[2 * mi + 1] = (unsigned long long)(name[0]) | ((unsigned long long)(name[1]) << 8) | ((unsigned long long)(name[2]) << 16) | ((unsigned long long)(name[3]) << 24) | ((unsigned long long)warp << 32); } }
+#else
+#define ONELA_MARK(name)
+#endif
+
 template <typename OutT>
 __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs a, int total_groups, int groups_per_pair) {
     extern __shared__ uint8_t smem_raw[];
@@ -82,6 +93,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
     uint8_t* smem = smem_raw + (base - raw);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (warp == 0 || warp == FOLD_WARPS) { ONELA_MARK("start") }
     uint8_t* ring = smem;
     uint8_t* stage = ring + SLOTS * SLOT_BYTES;
     float2* gates_s = reinterpret_cast<float2*>(stage + STAGE_BYTES);
@@ -91,7 +103,6 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
     //       8 + 2*w + st: head stage st of fold warp w
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8 + FOLD_WARPS * HEAD_STAGES);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    int* quad_count = reinterpret_cast<int*>(tmem_slot + 2);   // [SLOTS] quads written into the slot in its current use
     const uint32_t bar_s0 = smem_u32(bars), bar_stage = smem_u32(bars + 1);
     auto bar_full = [&](int s) { return smem_u32(bars + 2 + s); };
     auto bar_done = [&](int s) { return smem_u32(bars + 4 + s); };
@@ -107,7 +118,6 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
         }
         for (int i = 0; i < FOLD_WARPS * HEAD_STAGES; ++i) mbar_init(smem_u32(bars + 8 + i), 1);
         *abort_flag = 0;
-        quad_count[0] = quad_count[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
@@ -120,6 +130,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
+    if (warp == 0) { ONELA_MARK("prologue done") }
 
     const int g_begin = (int)(((long long)blockIdx.x * total_groups) / gridDim.x);
     const int g_end = (int)(((long long)(blockIdx.x + 1) * total_groups) / gridDim.x);
@@ -245,6 +256,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
                     if (heads_issued - heads_taken > 1) asm volatile("cp.async.wait_group 1;" ::: "memory");
                     else asm volatile("cp.async.wait_group 0;" ::: "memory");
                     ONELA_TICK(5)   // (fold warps) wait for the head
+                    if (warp == 0) { ONELA_MARK("head arrived") }
                     const uint4* rec = reinterpret_cast<const uint4*>(my_heads + st * HEAD_BYTES + grp * REC_BYTES) + g;
                     const uint4* qv = reinterpret_cast<const uint4*>(my_heads + st * HEAD_BYTES + 4 * REC_BYTES + grp * (DK * 2)) + g;
                     cur.own.k[0] = rec[0]; cur.own.k[1] = rec[8];
@@ -327,32 +339,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
                 __syncwarp();
                 ONELA_TICK(3)   // operand write + proxy fence
-                // ---- the warp whose quad completes the group issues the group's MMAs -------------------
-                int mma_failed = 0;
-                if (lane == 0) {
-                    mbar_arrive(bar_full(s));
-                    if (atomicAdd(&quad_count[s], 1) == QPG * FOLD_WARPS - 1) {
-                        quad_count[s] = 0;   // the slot's next use cannot begin before this group's MMAs are read back
-                        bool ok = wait_or_abort(bar_full(s), use & 1, abort_flag);      // all 16 arrivals are in: acquire
-                        ok = ok && wait_or_abort(bar_s0, seg_parity, abort_flag);
-                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                        if (ok) {
-                            constexpr uint32_t idesc = idesc_tf32(GN);
-                            const uint64_t bd = umma_desc(smem_u32(R_s));
-#pragma unroll
-                            for (int kb = 0; kb < 4; ++kb)
-#pragma unroll
-                                for (int ks = 0; ks < 4; ++ks)
-                                    umma_tf32_ts(tmem_base + s * GN, tmem_base + S0_COL + (kb * 4 + ks) * 8,
-                                                 bd + (uint64_t)((kb * R_KB_STRIDE + ks * 32) >> 4), idesc, (kb | ks) ? 1u : 0u);
-                        } else {
-                            mma_failed = 1;
-                        }
-                        umma_commit(bar_done(s));   // arrives when the MMAs above (if any) have completed
-                    }
-                }
-                if (__shfl_sync(0xffffffffu, mma_failed, 0)) { dead = true; break; }
-                ONELA_TICK(4)   // arrive (+ MMA issue when last)
+                if (warp == 0) { ONELA_MARK("quad written") }
+                if (lane == 0) mbar_arrive(bar_full(s));
+                ONELA_TICK(4)   // arrive
             }
         } else {
             // =============================== EPILOGUE ===============================
@@ -379,13 +368,40 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_s0);
+                if (warp == FOLD_WARPS) { ONELA_MARK("S0 in tmem") }
             }
             for (int gi = sg_begin; gi < sg_end && !dead; ++gi) {
                 const int gcount = gcount0 + (gi - sg_begin);
                 const int s = gcount & 1, use = gcount >> 1;
+                if (warp == FOLD_WARPS) {
+                    // One thread issues the group's 16 MMAs as soon as all its rows are written (the fold warps
+                    // never stop for it: whichever fold warp issued would be the last to finish its next quad).
+                    int mma_failed = 0;
+                    if (lane == 0) {
+                        bool ok = wait_or_abort(bar_full(s), use & 1, abort_flag);
+                        ok = ok && wait_or_abort(bar_s0, seg_parity, abort_flag);
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        if (ok) {
+                            constexpr uint32_t idesc = idesc_tf32(GN);
+                            const uint64_t bd = umma_desc(smem_u32(ring + s * SLOT_BYTES));
+#pragma unroll
+                            for (int kb = 0; kb < 4; ++kb)
+#pragma unroll
+                                for (int ks = 0; ks < 4; ++ks)
+                                    umma_tf32_ts(tmem_base + s * GN, tmem_base + S0_COL + (kb * 4 + ks) * 8,
+                                                 bd + (uint64_t)((kb * R_KB_STRIDE + ks * 32) >> 4), idesc, (kb | ks) ? 1u : 0u);
+                        } else {
+                            mma_failed = 1;
+                        }
+                        umma_commit(bar_done(s));   // arrives when the MMAs above (if any) have completed
+                        ONELA_MARK("mma issued")
+                    }
+                    if (__shfl_sync(0xffffffffu, mma_failed, 0)) { dead = true; break; }
+                }
                 if (!wait_or_abort(bar_done(s), use & 1, abort_flag)) { dead = true; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 ONELA_TICK(5)   // epilogue: wait for the MMA group
+                if (warp == FOLD_WARPS) { ONELA_MARK("mma done") }
                 float* C_s = reinterpret_cast<float*>(ring + s * SLOT_BYTES + R_BYTES);
                 const int b0 = (gi - pair * groups_per_pair) * GN;
                 const uint32_t taddr = tmem_base + s * GN + ((uint32_t)(quad * 32) << 16);
@@ -422,6 +438,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_free(s));
                 ONELA_TICK(6)   // epilogue: read back, add, store
+                if (warp == FOLD_WARPS) { ONELA_MARK("epilogue done") }
             }
         }
         if (dead) {
@@ -444,6 +461,18 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
     if (tid == 0 && *abort_flag && g_begin < g_end) mbar_wait(bar_stage, (seg_idx - 1) & 1);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if (warp == 0) { ONELA_MARK("exit") }
+#ifdef ONELA_TIMELINE
+    if (blockIdx.x == 0 && tid == 0) {
+        const int n = min(g_nmarks, 32);
+        for (int i = 0; i < n; ++i) {
+            const unsigned long long tag = g_marks[2 * i + 1];
+            printf("mark %c%c%c%c warp %2d t=%llu ns\n", (char)(tag & 255), (char)((tag >> 8) & 255), (char)((tag >> 16) & 255),
+                   (char)((tag >> 24) & 255), (int)(tag >> 32), g_marks[2 * i] - g_marks[0]);
+        }
+        g_nmarks = 0;
+    }
+#endif
     if (warp == 0) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
