@@ -157,7 +157,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
         for (r, l), S in S0.items():
             ctx.onela_init_shared_state(r, l, S, stream)
         for call in calls:
-            run.run_call(call, outs, stream, decode_events, fused=fused)
+            run.run_call(call, outs, stream, decode_events, fused=fused, group_events=True)
 
     def barrier():
         torch.cuda.synchronize()
@@ -218,9 +218,12 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
         for _ in range(n_b):
             generation(decode_events=pairs)
         torch.cuda.synchronize()
-    dur_ms = np.array([a.elapsed_time(b) for a, b in pairs]).reshape(n_b, wl.D, -1)   # [step, call, launches]
-    ms_depth = dur_ms.mean(axis=(0, 2))                                                     # mean per launch at each depth
-    n_per_depth = dur_ms.shape[2]
+    # event pairs: one per decode launch, or (fused launches: nothing else runs between the layers of a call)
+    # one around the L back-to-back launches of a call; either way [step, call, pairs] with `per` launches each
+    per = pairs[0][2]
+    dur_ms = np.array([a.elapsed_time(b) for a, b, _ in pairs]).reshape(n_b, wl.D, -1)
+    ms_depth = dur_ms.mean(axis=(0, 2)) / per                                               # mean per launch at each depth
+    n_per_depth = dur_ms.shape[2] * per
     alg_total = sum(per_depth[t]["algorithmic"] for t in range(wl.D)) * n_per_depth * n_b
     und_total = sum(per_depth[t]["undeduplicated"] for t in range(wl.D)) * n_per_depth * n_b
     achieved_gbs = alg_total / (dur_ms.sum() * 1e-3) / 1e9
@@ -263,6 +266,8 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
                      "traffic_note": "ncu DRAM read+write bytes of one launch at the deepest call (depth %d), whose "
                                      "algorithmic bytes are %.1f MB; see profiles/" % (wl.D, per_depth[-1]["algorithmic"] / 1e6),
                      "peak_source": peak_src,
+                     "timing": "CUDA events around every decode launch" if per == 1 else
+                               "CUDA events around the %d back-to-back decode launches (one per layer) of each decode call" % per,
                      "kernel": ("decode_step" if args.unfused else "append_decode_step") + " (all requests of one layer per launch)",
                      "bytes": "algorithmic: S_0 once + each distinct record once + q + o + ancestry rows"
                               + ("" if args.unfused else " + the call's records written to the arena"),

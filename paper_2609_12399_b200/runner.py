@@ -65,21 +65,27 @@ class WorkloadRun:
                 for _ in range(wl.L)]
 
     # ---- one decode call through the library ------------------------------------------------------
-    def run_call(self, call: dict, outs: list, stream=None, decode_events=None, fused: bool = False):
+    def run_call(self, call: dict, outs: list, stream=None, decode_events=None, fused: bool = False,
+                 group_events: bool = False):
         """reorder_beams once, then append_records + decode_step per layer, batched over all requests
         (in chunks of at most ONELA_MAX_BATCH); with ``fused`` the two per-layer calls are the one-launch
-        append_decode_step.  ``decode_events``: optional list that receives a (start, end) CUDA event pair
-        around every decode launch."""
+        append_decode_step.  ``decode_events``: optional list that receives (start, end, launches) CUDA event
+        pairs: around every decode launch, or - with ``group_events`` and fused launches, where nothing else
+        runs between the layers - one pair around all the layers' launches of the call."""
         wl, ctx = self.wl, self.ctx
         for r0 in range(0, wl.R, MAX_BATCH):
             n = min(MAX_BATCH, wl.R - r0)
             par = None if call["parents"] is None else call["parents"][r0:r0 + n]
             ctx.onela_reorder_beams(r0, n, par, wl.W, stream)
+            per_group = decode_events is not None and group_events and fused
+            if per_group:
+                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                g0.record(stream)
             for l, lay in enumerate(call["layers"]):
                 sl = slice(r0, r0 + n)
                 if not fused:
                     ctx.onela_append_records(r0, n, l, lay["k"][sl], lay["v"][sl], lay["alpha"][sl], lay["beta"][sl], stream)
-                if decode_events is not None:
+                if decode_events is not None and not per_group:
                     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                     e0.record(stream)
                 if fused:
@@ -87,6 +93,9 @@ class WorkloadRun:
                                                  lay["q"][sl], outs[l][sl], stream)
                 else:
                     ctx.onela_decode_step(r0, n, l, lay["q"][sl], outs[l][sl], stream)
-                if decode_events is not None:
+                if decode_events is not None and not per_group:
                     e1.record(stream)
-                    decode_events.append((e0, e1))
+                    decode_events.append((e0, e1, 1))
+            if per_group:
+                g1.record(stream)
+                decode_events.append((g0, g1, len(call["layers"])))
