@@ -111,9 +111,8 @@ onela_status onela_prefill_shared_state(onela_ctx* ctx, int32_t request, int32_t
                                         const void* v_dev, const float* alpha_dev, const float* beta_dev,
                                         int32_t n_tokens, void* stream);
 
-/* Read the store slot of (request, layer) back as S0_out_dev [num_heads][dv][dk] fp32 row-major (the
- * values the decode kernels consume: identical to what was stored, except that the tensor-core path
- * keeps S_0 rounded to TF32, 10 mantissa bits). */
+/* Read the store slot of (request, layer) back as S0_out_dev [num_heads][dv][dk] fp32 row-major, bit for
+ * bit what was stored (the tensor-core kernel rounds S_0 to TF32 only on its way into tensor memory). */
 onela_status onela_export_shared_state(onela_ctx* ctx, int32_t request, int32_t layer, float* S0_out_dev,
                                        void* stream);
 

@@ -66,7 +66,7 @@ struct onela_ctx {
     int64_t cursor = 0;        // next free arena slot
     int64_t launches = 0;
     bool status_cleared = false;
-    bool tensor_core = false;  // decode_step runs the tcgen05 kernel; S_0 is stored as its operand image
+    bool tensor_core = false;  // decode_step runs the tcgen05 kernel
     int32_t elem_bytes = 4;
 
     bool dry() const { return cfg.flags & ONELA_FLAG_DRY_RUN; }
@@ -188,7 +188,7 @@ onela_status onela_init_shared_state(onela_ctx* ctx, int32_t request, int32_t la
     if ((st = ctx->prepare(s)) != ONELA_OK) return st;
     if (!ctx->dry()) {
         if (launch_store_state(S0_dev, ctx->s0_slot(request, layer), ctx->cfg.num_heads, ctx->cfg.dk, ctx->cfg.dv,
-                               ctx->tensor_core, s) != cudaSuccess)
+                               s) != cudaSuccess)
             return ONELA_E_CUDA;
         ctx->launches++;
     }
@@ -210,7 +210,7 @@ onela_status onela_prefill_shared_state(onela_ctx* ctx, int32_t request, int32_t
         bool supported = true;
         const cudaError_t e = launch_prefill(k_dev, v_dev, alpha_dev, beta_dev, ctx->s0_slot(request, layer), n_tokens,
                                              ctx->cfg.num_heads, ctx->cfg.dk, ctx->cfg.dv, ctx->cfg.rec_dtype,
-                                             ctx->tensor_core, &supported, s);
+                                             &supported, s);
         if (!supported) return ONELA_E_UNSUPPORTED;
         if (e != cudaSuccess) return ONELA_E_CUDA;
         ctx->launches++;
@@ -229,7 +229,7 @@ onela_status onela_export_shared_state(onela_ctx* ctx, int32_t request, int32_t 
     if ((st = ctx->prepare(s)) != ONELA_OK) return st;
     if (ctx->dry()) return ONELA_OK;
     if (launch_export_state(ctx->s0_slot(request, layer), S0_out_dev, ctx->cfg.num_heads, ctx->cfg.dk, ctx->cfg.dv,
-                            ctx->tensor_core, s) != cudaSuccess)
+                            s) != cudaSuccess)
         return ONELA_E_CUDA;
     ctx->launches++;
     return ONELA_OK;
@@ -357,14 +357,9 @@ onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count,
     a.H = c.num_heads;
     a.depth = depth;
     a.max_beam = c.max_beam;
-    a.s0_swizzled = ctx->tensor_core;
     for (int i = 0; i < req_count; ++i) a.bases.base[i] = ctx->req[req_begin + i].step_base.back();
     bool supported = true;
-#ifdef ONELA_PIPELINED
-    const cudaError_t e = ctx->tensor_core ? launch_decode_sm100(a, c.out_dtype, s)
-#else
     const cudaError_t e = ctx->tensor_core ? launch_decode_sm100_ws(a, c.out_dtype, s)
-#endif
                                            : launch_decode_generic(a, c.dk, c.dv, c.rec_dtype, c.out_dtype, &supported, s);
     if (!supported) return ONELA_E_UNSUPPORTED;
     if (e != cudaSuccess) return ONELA_E_CUDA;
@@ -414,12 +409,8 @@ onela_status onela_append_decode_step(onela_ctx* ctx, int32_t req_begin, int32_t
     if ((st = ctx->prepare(s)) != ONELA_OK) return st;
     if (!ctx->dry()) {
         if (ctx->tensor_core) {
-#ifdef ONELA_PIPELINED
-            return ONELA_E_UNSUPPORTED;
-#else
             st = launch_decode(ctx, req_begin, req_count, layer, q_dev, out_dev, k_dev, v_dev, alpha_dev, beta_dev, s);
             if (st != ONELA_OK) return st;
-#endif
         } else {   // shapes without the fused kernel: the copy kernel, then the decode kernel
             BatchBases bases{};
             for (int i = 0; i < req_count; ++i) bases.base[i] = ctx->req[req_begin + i].step_base.back();

@@ -48,7 +48,7 @@ struct DecodeArgs {
     const int32_t* ulist;
     const int32_t* uoff;
     long long sidx_req_stride, ulist_req_stride, uoff_req_stride;
-    int32_t req_count, W, H, depth, max_beam, s0_swizzled;
+    int32_t req_count, W, H, depth, max_beam;
     BatchBases bases;
 };
 
@@ -72,22 +72,19 @@ cudaError_t launch_append(const void* k, const void* v, const float* alpha, cons
                           float2* gate_plane, long long arena_slots, int32_t req_count, int32_t W, int32_t H,
                           int32_t dk, int32_t dv, int32_t elem_bytes, const BatchBases& bases,
                           cudaStream_t stream);
-cudaError_t launch_store_state(const float* S0_in, float* slot, int32_t H, int32_t dk, int32_t dv,
-                               int32_t swizzled, cudaStream_t stream);
-cudaError_t launch_export_state(const float* slot, float* S0_out, int32_t H, int32_t dk, int32_t dv,
-                                int32_t swizzled, cudaStream_t stream);
+cudaError_t launch_store_state(const float* S0_in, float* slot, int32_t H, int32_t dk, int32_t dv, cudaStream_t stream);
+cudaError_t launch_export_state(const float* slot, float* S0_out, int32_t H, int32_t dk, int32_t dv, cudaStream_t stream);
 // returns cudaErrorInvalidValue with *supported = false when (dk, dv, dtype) has no instantiation
 cudaError_t launch_prefill(const void* k, const void* v, const float* alpha, const float* beta, float* slot,
-                           int32_t n_tokens, int32_t H, int32_t dk, int32_t dv, int32_t rec_dtype,
-                           int32_t swizzled, bool* supported, cudaStream_t stream);
+                           int32_t n_tokens, int32_t H, int32_t dk, int32_t dv, int32_t rec_dtype, bool* supported,
+                           cudaStream_t stream);
 
 // decode kernels
 cudaError_t launch_decode_generic(const DecodeArgs& a, int32_t dk, int32_t dv, int32_t rec_dtype,
                                   int32_t out_dtype, bool* supported, cudaStream_t stream);
 bool decode_generic_supported(int32_t dk, int32_t dv, int32_t rec_dtype);
-// tcgen05 tensor-core kernel (sm_100a): dk = dv = 128, bf16 records, S_0 stored as the swizzled TF32 image
+// tcgen05 tensor-core kernel (sm_100a): dk = dv = 128, bf16 records
 bool decode_sm100_supported(int32_t dk, int32_t dv, int32_t rec_dtype);
-cudaError_t launch_decode_sm100(const DecodeArgs& a, int32_t out_dtype, cudaStream_t stream);     // barrier-pipelined variant
-cudaError_t launch_decode_sm100_ws(const DecodeArgs& a, int32_t out_dtype, cudaStream_t stream);  // warp-specialised variant
+cudaError_t launch_decode_sm100_ws(const DecodeArgs& a, int32_t out_dtype, cudaStream_t stream);
 
 }  // namespace onela

@@ -1,4 +1,4 @@
-// Device helpers shared by the kernel files: the shared-state image layout and bf16 unpacking.
+// Device helpers shared by the kernel files: TF32 rounding and bf16 unpacking.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -6,18 +6,8 @@
 
 namespace onela {
 
-// Shared-state image for the tensor-core kernel (dk = dv = 128): the [dv][dk] fp32 matrix of one head
-// stored as the K-major, 128-byte-swizzled shared-memory operand the tcgen05 MMA reads, so that the
-// decode kernel brings a head in with ONE contiguous 64 KiB bulk copy.  K is split into 4 blocks of
-// 32 floats (128 bytes); inside a block row i holds its 32 floats as eight 16-byte chunks, chunk c
-// stored at position c ^ (i & 7).  Returns the float offset of element (i, k) inside the head image.
-__host__ __device__ __forceinline__ int s0_image_index(int i, int k) {
-    const int kb = k >> 5, kk = k & 31;
-    return kb * (128 * 32) + i * 32 + ((((kk >> 2) ^ (i & 7)) << 2) | (kk & 3));
-}
-
 // Round to the nearest TF32 value (10 explicit mantissa bits), ties away from zero.  The tensor core
-// reads only the upper 19 bits of an fp32 operand; rounding once when the state is stored makes that
+// reads only the upper 19 bits of an fp32 operand; rounding an operand before it is handed over makes that
 // read unbiased instead of a truncation.
 __device__ __forceinline__ float round_tf32(float x) {
     uint32_t u;

@@ -33,22 +33,6 @@ __global__ void __launch_bounds__(256) append_kernel(const char* __restrict__ k,
     if (lane == 0) gate_plane[dst_row] = make_float2(__ldg(alpha + row), __ldg(beta + row));
 }
 
-__global__ void __launch_bounds__(256) store_state_swizzled_kernel(const float* __restrict__ in, float* __restrict__ slot,
-                                                                   int32_t n) {
-    const int e = blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= n) return;
-    const int h = e >> 14, i = (e >> 7) & 127, k = e & 127;
-    slot[(h << 14) + s0_image_index(i, k)] = round_tf32(__ldg(in + e));
-}
-
-__global__ void __launch_bounds__(256) export_state_swizzled_kernel(const float* __restrict__ slot, float* __restrict__ out,
-                                                                    int32_t n) {
-    const int e = blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= n) return;
-    const int h = e >> 14, i = (e >> 7) & 127, k = e & 127;
-    out[e] = __ldg(slot + (h << 14) + s0_image_index(i, k));
-}
-
 template <typename T>
 __device__ __forceinline__ float to_float(T x);
 template <>
@@ -60,8 +44,7 @@ __device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat16 x) { retu
 template <int DK, int DV, typename T>
 __global__ void __launch_bounds__(DV) prefill_kernel(const T* __restrict__ k, const T* __restrict__ v,
                                                      const float* __restrict__ alpha, const float* __restrict__ beta,
-                                                     float* __restrict__ slot, int32_t n_tokens, int32_t H,
-                                                     int32_t swizzled) {
+                                                     float* __restrict__ slot, int32_t n_tokens, int32_t H) {
     __shared__ __align__(16) float k_s[2][DK];
     const int h = blockIdx.x, i = threadIdx.x;
     float S[DK];
@@ -116,24 +99,19 @@ __global__ void __launch_bounds__(DV) prefill_kernel(const T* __restrict__ k, co
         __syncthreads();
     }
     float* dst = slot + (long long)h * DV * DK;
-    if (swizzled) {
 #pragma unroll
-        for (int j = 0; j < DK; ++j) dst[s0_image_index(i, j)] = round_tf32(S[j]);
-    } else {
-#pragma unroll
-        for (int j = 0; j < DK; ++j) dst[(long long)i * DK + j] = S[j];
-    }
+    for (int j = 0; j < DK; ++j) dst[(long long)i * DK + j] = S[j];
 }
 
 template <int DK, int DV>
 cudaError_t prefill_dispatch(const void* k, const void* v, const float* alpha, const float* beta, float* slot,
-                             int32_t n_tokens, int32_t H, int32_t rec_dtype, int32_t swizzled, cudaStream_t stream) {
+                             int32_t n_tokens, int32_t H, int32_t rec_dtype, cudaStream_t stream) {
     if (rec_dtype == ONELA_DTYPE_BF16)
         prefill_kernel<DK, DV, __nv_bfloat16><<<H, DV, 0, stream>>>(
-            static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(v), alpha, beta, slot, n_tokens, H, swizzled);
+            static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(v), alpha, beta, slot, n_tokens, H);
     else
         prefill_kernel<DK, DV, float><<<H, DV, 0, stream>>>(static_cast<const float*>(k), static_cast<const float*>(v),
-                                                           alpha, beta, slot, n_tokens, H, swizzled);
+                                                           alpha, beta, slot, n_tokens, H);
     return cudaGetLastError();
 }
 
@@ -151,31 +129,21 @@ cudaError_t launch_append(const void* k, const void* v, const float* alpha, cons
     return cudaGetLastError();
 }
 
-cudaError_t launch_store_state(const float* S0_in, float* slot, int32_t H, int32_t dk, int32_t dv,
-                               int32_t swizzled, cudaStream_t stream) {
-    const long long n = (long long)H * dk * dv;
-    if (!swizzled)
-        return cudaMemcpyAsync(slot, S0_in, n * sizeof(float), cudaMemcpyDeviceToDevice, stream);
-    store_state_swizzled_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(S0_in, slot, (int32_t)n);
-    return cudaGetLastError();
+cudaError_t launch_store_state(const float* S0_in, float* slot, int32_t H, int32_t dk, int32_t dv, cudaStream_t stream) {
+    return cudaMemcpyAsync(slot, S0_in, (size_t)H * dk * dv * sizeof(float), cudaMemcpyDeviceToDevice, stream);
 }
 
-cudaError_t launch_export_state(const float* slot, float* S0_out, int32_t H, int32_t dk, int32_t dv,
-                                int32_t swizzled, cudaStream_t stream) {
-    const long long n = (long long)H * dk * dv;
-    if (!swizzled)
-        return cudaMemcpyAsync(S0_out, slot, n * sizeof(float), cudaMemcpyDeviceToDevice, stream);
-    export_state_swizzled_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(slot, S0_out, (int32_t)n);
-    return cudaGetLastError();
+cudaError_t launch_export_state(const float* slot, float* S0_out, int32_t H, int32_t dk, int32_t dv, cudaStream_t stream) {
+    return cudaMemcpyAsync(S0_out, slot, (size_t)H * dk * dv * sizeof(float), cudaMemcpyDeviceToDevice, stream);
 }
 
 cudaError_t launch_prefill(const void* k, const void* v, const float* alpha, const float* beta, float* slot,
-                           int32_t n_tokens, int32_t H, int32_t dk, int32_t dv, int32_t rec_dtype,
-                           int32_t swizzled, bool* supported, cudaStream_t stream) {
+                           int32_t n_tokens, int32_t H, int32_t dk, int32_t dv, int32_t rec_dtype, bool* supported,
+                           cudaStream_t stream) {
     *supported = true;
-    if (dk == 32 && dv == 32) return prefill_dispatch<32, 32>(k, v, alpha, beta, slot, n_tokens, H, rec_dtype, swizzled, stream);
-    if (dk == 64 && dv == 64) return prefill_dispatch<64, 64>(k, v, alpha, beta, slot, n_tokens, H, rec_dtype, swizzled, stream);
-    if (dk == 128 && dv == 128) return prefill_dispatch<128, 128>(k, v, alpha, beta, slot, n_tokens, H, rec_dtype, swizzled, stream);
+    if (dk == 32 && dv == 32) return prefill_dispatch<32, 32>(k, v, alpha, beta, slot, n_tokens, H, rec_dtype, stream);
+    if (dk == 64 && dv == 64) return prefill_dispatch<64, 64>(k, v, alpha, beta, slot, n_tokens, H, rec_dtype, stream);
+    if (dk == 128 && dv == 128) return prefill_dispatch<128, 128>(k, v, alpha, beta, slot, n_tokens, H, rec_dtype, stream);
     *supported = false;
     return cudaErrorInvalidValue;
 }
