@@ -34,26 +34,33 @@ using namespace sm100;
 #ifndef ONELA_FOLD_WARPS
 #define ONELA_FOLD_WARPS 12
 #endif
+#ifndef ONELA_LPU
+#define ONELA_LPU 8
+#endif
 constexpr int FOLD_WARPS = ONELA_FOLD_WARPS;
-constexpr int QPG = FOLD_WARPS == 8 ? 2 : 1;        // quads each fold warp contributes to a group
+constexpr int LPU = ONELA_LPU;                      // lanes per (beam, head) unit
+constexpr int UPW = 32 / LPU;                       // units a fold warp folds at a time (a "quad" when LPU = 8)
+constexpr int NCH = 16 / LPU;                       // 16-byte chunks per lane per 256-byte vector
+constexpr int QPG = (FOLD_WARPS * UPW == 32) ? 2 : 1;   // quads each fold warp contributes to a group
 constexpr int THREADS = (FOLD_WARPS + 4) * 32;      // + 4 epilogue warps (12 warps: three per SM sub-partition)
-constexpr int GN = FOLD_WARPS * 4 * QPG;            // beams per group = MMA N (64 or 48)
+constexpr int GN = FOLD_WARPS * UPW * QPG;          // beams per group = MMA N (64 or 48)
 constexpr int R_KB_STRIDE = GN * 128;               // bytes between the four 32-float K blocks of the operand
 constexpr int R_BYTES = 4 * R_KB_STRIDE;            // 32768
 constexpr int C_BYTES = GN * DV * 4;                // 32768: corr tile, row = beam
 constexpr int SLOT_BYTES = R_BYTES + C_BYTES;
 constexpr int SLOTS = 2;
-constexpr int STAGE_CAP = FOLD_WARPS == 8 ? 88 : 104;                       // distinct ancestor records staged per segment
+constexpr int HEAD_BYTES = UPW * (REC_BYTES + DK * 2);   // one quad's heads: own records + queries of its units
+constexpr int HEAD_STAGES = LPU == 8 ? 2 : 1;          // heads in flight per fold warp
+constexpr int HEADS_TOTAL = FOLD_WARPS * HEAD_STAGES * HEAD_BYTES;
+constexpr int STAGE_CAP = (232448 - 1024 - 256 - SLOTS * SLOT_BYTES - HEADS_TOTAL) / (REC_BYTES + 8) / 4 * 4 > 104
+                              ? 104 : (232448 - 1024 - 256 - SLOTS * SLOT_BYTES - HEADS_TOTAL) / (REC_BYTES + 8) / 4 * 4;                       // distinct ancestor records staged per segment
 constexpr int STAGE_BYTES = STAGE_CAP * REC_BYTES;
 constexpr int GATE_BYTES = STAGE_CAP * 8;
-constexpr int HEAD_BYTES = 4 * (REC_BYTES + DK * 2);     // one quad's heads: 4 own records + 4 queries = 3072
-constexpr int HEAD_STAGES = 2;                         // heads in flight per fold warp
-constexpr int HEADS_TOTAL = FOLD_WARPS * HEAD_STAGES * HEAD_BYTES;
 constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + STAGE_BYTES + GATE_BYTES + HEADS_TOTAL + 256 + 1024;
 constexpr uint32_t TMEM_COLS = 256;              // accumulators of the two slots in [0, 2 GN), the head's S_0 in [128, 256)
 constexpr uint32_t S0_COL = 128;
 static_assert(SMEM_BYTES <= 232448, "shared memory per CTA");
-using L = Lanes<8>;
+using L = Lanes<LPU>;
 using RecT = L::R;
 
 // Bounded wait that also gives up as soon as the CTA's abort flag is raised.
@@ -69,7 +76,7 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 }
 
 struct Head {           // what a unit's fold needs first
-    uint4 q[2];
+    uint4 q[NCH];
     RecT own;
 };
 
@@ -186,7 +193,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
 
         if (warp < FOLD_WARPS) {
             // =============================== FOLD ===============================
-            const int grp = lane >> 3, g = lane & 7;
+            const int grp = lane / LPU, g = lane % LPU;
             const int32_t* table_r = a.table + req * a.table_req_stride;
             const int32_t* sidx_r = a.sidx + req * a.sidx_req_stride;
             // the gates of the staged records: every fold warp writes all of them (same values), then syncs itself
@@ -199,18 +206,18 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
             const int n_quads = QPG * (sg_end - sg_begin);
             auto group_of = [&](int k) { return QPG == 2 ? (k >> 1) : k; };
             auto half_of = [&](int k) { return QPG == 2 ? (k & 1) : 0; };
-            auto beam_of = [&](int k) { return ((sg_begin + group_of(k)) - pair * groups_per_pair) * GN + half_of(k) * 32 + 4 * warp + grp; };
+            auto beam_of = [&](int k) { return ((sg_begin + group_of(k)) - pair * groups_per_pair) * GN + half_of(k) * (FOLD_WARPS * UPW) + UPW * warp + grp; };
             // The heads of a quad (own record and query of its four units) arrive by 16-byte async copies into a
             // two-stage ring private to the warp, two quads ahead of their use (each lane copies exactly the
             // chunks it reads back); the gates ride in registers.
             auto slot_of = [&](int k) { return (gcount0 + group_of(k)) & 1; };
             auto use_of = [&](int k) { return (gcount0 + group_of(k)) >> 1; };
-            auto row_of = [&](int k) { return half_of(k) * 32 + 4 * warp + grp; };
+            auto row_of = [&](int k) { return half_of(k) * (FOLD_WARPS * UPW) + UPW * warp + grp; };
             uint8_t* my_heads = heads + warp * (HEAD_STAGES * HEAD_BYTES);
             auto head_bar = [&](int st) { return smem_u32(bars + 8 + warp * HEAD_STAGES + st); };
             auto q_row = [&](int bb) { return reinterpret_cast<const char*>(qbase + (((long long)req * a.W + bb) * a.H + h) * DK); };
             auto issue_head = [&](int k) {   // every lane copies the chunks it will read back itself
-                const int st = heads_issued & 1;
+                const int st = heads_issued % HEAD_STAGES;
                 const int bb = min(beam_of(k), a.W - 1);             // idle units shadow a live beam
                 const uint32_t dst = smem_u32(my_heads + st * HEAD_BYTES);
                 const char* qr = q_row(bb) + g * 16;
@@ -219,17 +226,17 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
                     const char* kr = static_cast<const char*>(a.k_in) + in_row * (DK * 2) + g * 16;
                     const char* vr = static_cast<const char*>(a.v_in) + in_row * (DV * 2) + g * 16;
 #pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        cp_async16(dst + grp * REC_BYTES + (c * 8 + g) * 16, kr + c * 128);
-                        cp_async16(dst + grp * REC_BYTES + (16 + c * 8 + g) * 16, vr + c * 128);
+                    for (int c = 0; c < NCH; ++c) {
+                        cp_async16(dst + grp * REC_BYTES + (c * LPU + g) * 16, kr + c * LPU * 16);
+                        cp_async16(dst + grp * REC_BYTES + (16 + c * LPU + g) * 16, vr + c * LPU * 16);
                     }
                 } else {
                     const char* rec = kv + (own_row0 + bb) * REC_BYTES + g * 16;
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) cp_async16(dst + grp * REC_BYTES + (c * 8 + g) * 16, rec + c * 128);
+                    for (int c = 0; c < 2 * NCH; ++c) cp_async16(dst + grp * REC_BYTES + (c * LPU + g) * 16, rec + c * LPU * 16);
                 }
 #pragma unroll
-                for (int c = 0; c < 2; ++c) cp_async16(dst + 4 * REC_BYTES + grp * (DK * 2) + (c * 8 + g) * 16, qr + c * 128);
+                for (int c = 0; c < NCH; ++c) cp_async16(dst + UPW * REC_BYTES + grp * (DK * 2) + (c * LPU + g) * 16, qr + c * LPU * 16);
                 asm volatile("cp.async.commit_group;" ::: "memory");
                 ++heads_issued;
             };
@@ -239,17 +246,28 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
                 const long long in_row = ((long long)req * a.W + bb) * a.H + h;
                 return make_float2(__ldg(a.alpha_in + in_row), __ldg(a.beta_in + in_row));
             };
-            auto load_idx = [&](int k) -> int32_t {
+            constexpr int NIDX = LPU >= 8 ? 1 : 8 / LPU;     // the unit's lanes hold the indices of its first 8 levels
+            struct Idx { int32_t v[NIDX]; };
+            auto load_idx = [&](int k) -> Idx {
                 const int bb = min(beam_of(k), a.W - 1);
-                return g < old ? __ldg((g < staged_levels ? sidx_r : table_r) + (long long)g * a.max_beam + bb) : 0;
+                Idx x;
+#pragma unroll
+                for (int j = 0; j < NIDX; ++j) {
+                    const int lv = j * LPU + g;
+                    x.v[j] = lv < old ? __ldg((lv < staged_levels ? sidx_r : table_r) + (long long)lv * a.max_beam + bb) : 0;
+                }
+                return x;
             };
             float2 gate0 = make_float2(1.f, 0.f), gate1 = gate0;
-            int32_t idx_next = 0;
+            Idx idx_next{};
             if (!dead && n_quads > 0) {
                 idx_next = load_idx(0);
                 issue_head(0);
                 gate0 = load_gate(0);
-                if (1 < n_quads) { issue_head(1); gate1 = load_gate(1); }
+                if (1 < n_quads) {
+                    if (HEAD_STAGES > 1) issue_head(1);
+                    gate1 = load_gate(1);
+                }
             }
             bool staged_ready = false;
             for (int k = 0; k < n_quads && !dead; ++k) {
@@ -258,52 +276,65 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
                 const int bb = min(beam_of(k), a.W - 1);
                 Head cur;
                 {
-                    const int st = heads_taken & 1;
+                    const int st = heads_taken % HEAD_STAGES;
                     // the oldest copy group in flight is this quad's; a newer one (the next quad's) may stay pending
                     if (heads_issued - heads_taken > 1) asm volatile("cp.async.wait_group 1;" ::: "memory");
                     else asm volatile("cp.async.wait_group 0;" ::: "memory");
                     ONELA_TICK(5)   // (fold warps) wait for the head
                     if (warp == 0) { ONELA_MARK("head arrived") }
                     const uint4* rec = reinterpret_cast<const uint4*>(my_heads + st * HEAD_BYTES + grp * REC_BYTES) + g;
-                    const uint4* qv = reinterpret_cast<const uint4*>(my_heads + st * HEAD_BYTES + 4 * REC_BYTES + grp * (DK * 2)) + g;
-                    cur.own.k[0] = rec[0]; cur.own.k[1] = rec[8];
-                    cur.own.v[0] = rec[16]; cur.own.v[1] = rec[24];
-                    cur.q[0] = qv[0]; cur.q[1] = qv[8];
+                    const uint4* qv = reinterpret_cast<const uint4*>(my_heads + st * HEAD_BYTES + UPW * REC_BYTES + grp * (DK * 2)) + g;
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) {
+                        cur.own.k[c] = rec[c * LPU];
+                        cur.own.v[c] = rec[16 + c * LPU];
+                        cur.q[c] = qv[c * LPU];
+                    }
                     cur.own.gate = gate0;
                     ++heads_taken;
                     if (fused && beam_of(k) < a.W) {   // the append: this beam's record goes to its arena slot, bit for bit
                         uint4* dst = reinterpret_cast<uint4*>(a.kv_out + (own_row0 + bb) * REC_BYTES) + g;
-                        dst[0] = cur.own.k[0]; dst[8] = cur.own.k[1];
-                        dst[16] = cur.own.v[0]; dst[24] = cur.own.v[1];
+#pragma unroll
+                        for (int c = 0; c < NCH; ++c) {
+                            dst[c * LPU] = cur.own.k[c];
+                            dst[16 + c * LPU] = cur.own.v[c];
+                        }
                         if (g == 0) a.gates_out[own_row0 + bb] = gate0;
                     }
                 }
                 gate0 = gate1;
 #ifdef ONELA_TIMING
-                if ((cur.q[0].x ^ cur.own.k[0].x ^ cur.own.v[1].w) == 0x12345678u) tph[7]++;
+                if ((cur.q[0].x ^ cur.own.k[0].x ^ cur.own.v[NCH - 1].w) == 0x12345678u) tph[7]++;
                 ONELA_TICK(6)   // (fold warps) read the head from the stage
 #endif
-                if (k + 2 < n_quads) { issue_head(k + 2); gate1 = load_gate(k + 2); }
+                if (k + HEAD_STAGES < n_quads) issue_head(k + HEAD_STAGES);
+                if (k + 2 < n_quads) gate1 = load_gate(k + 2);
                 ONELA_TICK(2)   // (fold warps) issue the head after next
 
                 // lane g keeps the index of level g (position in the staged list for staged levels, arena slot
                 // otherwise); it was fetched while the previous quad was folded, the next quad's is fetched now
-                const int32_t my_idx = idx_next;
+                const Idx my_idx = idx_next;
                 if (k + 1 < n_quads) idx_next = load_idx(k + 1);
                 auto idx_of = [&](int level) -> int32_t {
-                    const int32_t t = __shfl_sync(0xffffffffu, my_idx, level & 7, 8);
-                    return level < 8 ? t : __ldg((level < staged_levels ? sidx_r : table_r) + (long long)level * a.max_beam + bb);
+                    int32_t t = 0;
+#pragma unroll
+                    for (int j = 0; j < NIDX; ++j) {
+                        const int32_t x = __shfl_sync(0xffffffffu, my_idx.v[j], level & (LPU - 1), LPU);
+                        if (j == level / LPU) t = x;
+                    }
+                    return level < NIDX * LPU ? t
+                                              : __ldg((level < staged_levels ? sidx_r : table_r) + (long long)level * a.max_beam + bb);
                 };
 
 #ifdef ONELA_TIMING
-                if ((cur.q[0].x ^ cur.own.k[0].x ^ cur.own.v[1].w ^ __float_as_uint(cur.own.gate.x)) == 0x12345678u) tph[7]++;
+                if ((cur.q[0].x ^ cur.own.k[0].x ^ cur.own.v[NCH - 1].w ^ __float_as_uint(cur.own.gate.x)) == 0x12345678u) tph[7]++;
                 ONELA_TICK(0)   // head arrival (+ issue of next head)
 #endif
-                float2 r[8], corr[8];
-                unpack8(cur.q[0], r);
-                unpack8(cur.q[1], r + 4);
+                float2 r[4 * NCH], corr[4 * NCH];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) corr[e] = make_float2(0.f, 0.f);
+                for (int c = 0; c < NCH; ++c) unpack8(cur.q[c], r + 4 * c);
+#pragma unroll
+                for (int e = 0; e < 4 * NCH; ++e) corr[e] = make_float2(0.f, 0.f);
                 float decay = 1.f;
                 L::fold_chain_simple(cur.own, old - 1, staged_levels,
                               [&](int level) { return L::load_global(kv, a.gates, plane_row0 + idx_of(level), g); }, r, corr, decay);
@@ -327,8 +358,8 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
                     const int sw = u & 7;
                     const float2 dc = make_float2(decay, decay);
 #pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        const int ci = c * 8 + g;                   // elements [8 ci, 8 ci + 8)
+                    for (int c = 0; c < NCH; ++c) {
+                        const int ci = c * LPU + g;                 // elements [8 ci, 8 ci + 8)
                         const int kb = ci >> 2, ch = 2 * (ci & 3);  // K block of 32 floats; first of two 16-byte chunks
                         uint8_t* row = R_s + kb * R_KB_STRIDE + u * 128;
                         float2 x[4];
