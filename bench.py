@@ -40,11 +40,11 @@ from paper_2609_12399_b200 import accounting, inputs, replicas  # noqa: E402
 METRIC = "beam-head GDN decodes/s per layer at beam 512"
 UNIT = "decodes/s"
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of ONE decode launch of the default workload at its deepest
-# call (depth 8, all 4 requests of one layer), from the ncu capture summarised in
-# profiles/decode_sm100_cfg4_ncu.md; the algorithmic bytes of that same launch are 84.6 MB (the 16.8 MB of
-# outputs were still in L2 when the kernel ended, so DRAM saw the 67.8 MB of reads and little else).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 72.66e6
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE fused append + decode launch of the default workload at
+# its deepest call (depth 8, all 4 requests of one layer), from the ncu capture summarised in
+# profiles/decode_ws_kernel_cfg4_ncu.md (72.7 MB read + 14.5 MB written).  The algorithmic bytes of that launch
+# are 118.7 MB; of the 50.9 MB it writes, 36 MB were still in L2 when the kernel ended.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 87.2e6
 
 
 def workload_by_name(name: str) -> inputs.Workload:
@@ -262,7 +262,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
                 "ms_per_step": e2e["ms_per_step"]},
         "gpu_launches": int(launches_per_step * args.steps),
         "roofline": {"bound": "hbm", "achieved": achieved_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": achieved_gbs / peak, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                     "frac": achieved_gbs / peak, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if not args.unfused else None,
                      "traffic_note": "ncu DRAM read+write bytes of one launch at the deepest call (depth %d), whose "
                                      "algorithmic bytes are %.1f MB; see profiles/" % (wl.D, per_depth[-1]["algorithmic"] / 1e6),
                      "peak_source": peak_src,
