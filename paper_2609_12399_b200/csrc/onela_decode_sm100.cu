@@ -1,24 +1,27 @@
 // Warp-specialised fused decode kernel for B200 (sm_100a): dk = dv = 128, bf16 records.
 //
-// One persistent CTA per SM, 12 warps in two roles that never wait for one another synchronously:
-//   * 8 FOLD warps.  8 lanes own one (beam, head) unit; a warp folds 4 units at a time ("quad"): query
+// One persistent CTA per SM, 16 warps in two roles coupled only by mbarriers:
+//   * 12 FOLD warps.  8 lanes own one (beam, head) unit; a warp folds 4 units at a time ("quad"): query
 //     folded through the unit's records newest -> oldest (c = k.r; corr += beta c v; r -= beta c k; decay a
-//     scalar; packed fp32x2 FMAs).  The next quad's query and own record are loaded while the current
-//     quad is folded.  Results go into a ring slot in shared memory: the folded query as a row of the
-//     K-major 128-byte-swizzled MMA operand (rounded to TF32), corr as a row of the slot's corr tile.
-
-//   * 4 EPILOGUE warps (one per tensor-memory lane quadrant).  When the MMA group has completed they read
-//     the accumulator, add corr and store the outputs (lane = dv index: 32 consecutive elements per store),
-//     then hand the slot back.
-// Two ring slots (operand rows, corr tile, 64 accumulator columns each) keep the MMA and the epilogue of one
-// group under the folds of the next.  Work = groups of 64 consecutive beams of one (request, head), a
-// contiguous range per CTA; consecutive groups of one head form a segment, per which the epilogue warps
-// load the head's S_0 into tensor memory (rounded to TF32; it is the MMA's A operand there) and one 512-byte
-// bulk copy per DISTINCT ancestor record stages the oldest chain levels (as many whole levels as fit) in
-// shared memory.
+//     scalar; packed fp32x2 FMAs).  A quad's query and own record arrive through a per-warp ring of 16-byte
+//     async copies, two quads ahead; with the append fused in they come from the caller's token tensors and
+//     the warp also writes them to the arena.  Results go into a ring slot in shared memory: the folded query
+//     as a row of the K-major 128-byte-swizzled MMA operand (rounded to TF32), corr as a row of the slot's
+//     corr tile.
+//   * 4 EPILOGUE warps (one per tensor-memory lane quadrant).  One lane issues the group's 16 MMAs once all
+//     its rows are written; when they have completed the four warps read the accumulator, add it onto the
+//     corr tile, store the outputs as coalesced 16-byte rows and hand the slot back.
+// Two ring slots (operand rows, corr tile, 48 accumulator columns each) keep the MMA and the epilogue of one
+// group under the folds of the next.  Work = groups of 48 consecutive beams of one (request, head), a
+// contiguous range per CTA chosen on the host; consecutive groups of one head form a segment, per which all
+// warps load the head's S_0 into tensor memory (rounded to TF32; it is the MMA's A operand there) and the
+// epilogue warps stage the oldest chain levels in shared memory, one 512-byte bulk copy per DISTINCT
+// ancestor record (as many whole levels as fit).
+// The kernel is launched as a programmatic dependent launch: it sets itself up and reads the first S_0 while
+// the previous kernel of the stream drains, and waits for that kernel before it touches anything else.
 // Every wait is bounded and also gives up when another role has raised the abort flag; a role that gives up
 // records ONELA_E_TIMEOUT, stops working but keeps joining the per-segment CTA barriers; before returning
-// the CTA waits (bounded) for bulk copies still in flight and frees its tensor memory.
+// the CTA waits (bounded) for copies still in flight and frees its tensor memory.
 #include <cstdio>
 
 #include "onela_internal.h"
@@ -50,7 +53,7 @@ constexpr int C_BYTES = GN * DV * 4;                // 32768: corr tile, row = b
 constexpr int SLOT_BYTES = R_BYTES + C_BYTES;
 constexpr int SLOTS = 2;
 constexpr int HEAD_BYTES = UPW * (REC_BYTES + DK * 2);   // one quad's heads: own records + queries of its units
-constexpr int HEAD_STAGES = LPU == 8 ? 2 : 1;          // heads in flight per fold warp
+constexpr int HEAD_STAGES = LPU >= 8 ? 2 : 1;         // heads in flight per fold warp
 constexpr int HEADS_TOTAL = FOLD_WARPS * HEAD_STAGES * HEAD_BYTES;
 constexpr int STAGE_CAP = (232448 - 1024 - 256 - SLOTS * SLOT_BYTES - HEADS_TOTAL) / (REC_BYTES + 8) / 4 * 4 > 104
                               ? 104 : (232448 - 1024 - 256 - SLOTS * SLOT_BYTES - HEADS_TOTAL) / (REC_BYTES + 8) / 4 * 4;                       // distinct ancestor records staged per segment
@@ -93,9 +96,28 @@ __device__ int g_nmarks;
 #define ONELA_MARK(name)
 #endif
 
+#ifdef ONELA_SPAN
+__device__ unsigned long long g_span[64][160][4];
+__device__ __forceinline__ unsigned long long gtime2() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#endif
+
+// Contiguous ranges of groups, one per CTA, balanced on the host with the cost of starting a segment counted in.
+constexpr int MAX_CTAS = 160;
+struct Partition {
+    int32_t begin[MAX_CTAS + 1];
+};
+
 template <typename OutT>
-__global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs a, int total_groups, int groups_per_pair) {
+__global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ Partition part,
+                                                               int groups_per_pair, int launch_id) {
     extern __shared__ uint8_t smem_raw[];
+#ifdef ONELA_SPAN
+    if (threadIdx.x == 0) g_span[launch_id & 63][blockIdx.x][0] = gtime2();
+#endif
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;            // swizzle atoms need 1024-byte alignment
     uint8_t* smem = smem_raw + (base - raw);
@@ -117,8 +139,8 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
     auto bar_free = [&](int s) { return smem_u32(bars + 6 + s); };
 
     if (tid == 0) {
-        mbar_init(bar_s0, 4);                         // the four epilogue warps, once S_0 sits in tensor memory
-        mbar_init(bar_stage, 32);
+        mbar_init(bar_s0, THREADS / 32);              // every warp, once its share of S_0 sits in tensor memory
+        mbar_init(bar_stage, 128);                    // every lane of the four epilogue warps
         for (int s = 0; s < SLOTS; ++s) {
             mbar_init(bar_full(s), QPG * FOLD_WARPS); // one arrival per quad of 4 beams
             mbar_init(bar_done(s), 1);                // tcgen05.commit
@@ -139,9 +161,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
     if (warp == 0) { ONELA_MARK("prologue done") }
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next launch may set itself up under this one
 
-    const int g_begin = (int)(((long long)blockIdx.x * total_groups) / gridDim.x);
-    const int g_end = (int)(((long long)(blockIdx.x + 1) * total_groups) / gridDim.x);
+    const int g_begin = part.begin[blockIdx.x], g_end = part.begin[blockIdx.x + 1];
     const int old = a.depth - 1;          // records older than a beam's own: levels old-1 .. 0
     const bool fused = a.k_in != nullptr;  // append fused in: the newest record comes from the caller's tensors
     const char* kv = a.kv;
@@ -157,6 +179,49 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
 #endif
     bool dead = false;                    // this warp gave up (timeout or abort raised elsewhere)
     int heads_issued = 0, heads_taken = 0;   // fold warps: quads whose heads were requested / consumed so far
+    const int grp = lane / LPU, g = lane % LPU;
+
+    // S_0 of a (request, head) goes to tensor memory, rounded to TF32 on the way: it is the MMA's A operand there, so
+    // there is no shared-memory copy of S_0 and no S_0 traffic per MMA.  Row-major fp32 in the store; lane i of
+    // tensor memory holds row i.  Every warp takes the 32 rows of its lane quadrant and one block of 32 columns,
+    // so the whole 64 KiB costs one load latency; the next segment's S_0 is requested into L2 on the way.
+    auto load_s0 = [&](int pair_now, bool has_next) {
+        const int quad = warp & 3, i = quad * 32 + lane;
+        const int req = pair_now / a.H, h = pair_now - req * a.H;
+        const float* row = a.s0 + req * a.s0_req_stride + (long long)h * (DV * DK) + (long long)i * DK;
+#pragma unroll 1
+        for (int kb = warp >> 2; kb < 4; kb += THREADS / 128) {
+            uint32_t v[32];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const float4 x = __ldg(reinterpret_cast<const float4*>(row + kb * 32) + c);
+                v[4 * c] = __float_as_uint(round_tf32(x.x)); v[4 * c + 1] = __float_as_uint(round_tf32(x.y));
+                v[4 * c + 2] = __float_as_uint(round_tf32(x.z)); v[4 * c + 3] = __float_as_uint(round_tf32(x.w));
+            }
+            tmem_st32(tmem_base + S0_COL + kb * 32 + ((uint32_t)(quad * 32) << 16), v);
+            if (has_next) {
+                const int nreq = (pair_now + 1) / a.H, nh = (pair_now + 1) - nreq * a.H;
+                const float* nrow = a.s0 + nreq * a.s0_req_stride + (long long)nh * (DV * DK) + (long long)i * DK + kb * 32;
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(nrow));
+            }
+        }
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_s0);
+    };
+    // The first segment's S_0 is read before the launch's dependencies are waited for: the store is written only
+    // by the state calls (a copy or a prefill kernel), and a reorder launch always separates those from a decode.
+    if (g_begin < g_end) {
+        const int pair0 = g_begin / groups_per_pair;
+        load_s0(pair0, (pair0 + 1) * groups_per_pair < g_end);
+    }
+    // Everything below reads what earlier launches of the stream wrote (tokens, queries, ancestry rows).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+#ifdef ONELA_SPAN
+    if (threadIdx.x == 0) g_span[launch_id & 63][blockIdx.x][2] = gtime2();
+#endif
+
     int seg_idx = 0;
     for (int sg_begin = g_begin, sg_end; sg_begin < g_end; sg_begin = sg_end, ++seg_idx) {
         const int pair = sg_begin / groups_per_pair;
@@ -165,6 +230,61 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
         const long long plane_row0 = (long long)h * a.arena_slots;
         const long long own_row0 = plane_row0 + a.bases.base[req];
         const uint32_t seg_parity = seg_idx & 1;
+        const int gcount0 = sg_begin - g_begin;   // groups this CTA finished before this segment
+
+        // ---- fold warps: head prefetch machinery.  Quad k of the segment: group sg_begin + k / QPG.
+        const int n_quads = QPG * (sg_end - sg_begin);
+        auto group_of = [&](int k) { return QPG == 2 ? (k >> 1) : k; };
+        auto half_of = [&](int k) { return QPG == 2 ? (k & 1) : 0; };
+        auto beam_of = [&](int k) { return ((sg_begin + group_of(k)) - pair * groups_per_pair) * GN + half_of(k) * (FOLD_WARPS * UPW) + UPW * warp + grp; };
+        // The heads of a quad (own record and query of its four units) arrive by 16-byte async copies into a
+        // two-stage ring private to the warp, two quads ahead of their use (each lane copies exactly the
+        // chunks it reads back); the gates ride in registers.
+        auto slot_of = [&](int k) { return (gcount0 + group_of(k)) & 1; };
+        auto use_of = [&](int k) { return (gcount0 + group_of(k)) >> 1; };
+        auto row_of = [&](int k) { return half_of(k) * (FOLD_WARPS * UPW) + UPW * warp + grp; };
+        uint8_t* my_heads = heads + (warp < FOLD_WARPS ? warp : 0) * (HEAD_STAGES * HEAD_BYTES);
+        auto q_row = [&](int bb) { return reinterpret_cast<const char*>(qbase + (((long long)req * a.W + bb) * a.H + h) * DK); };
+        auto issue_head = [&](int k) {   // every lane copies the chunks it will read back itself
+            const int st = heads_issued % HEAD_STAGES;
+            const int bb = min(beam_of(k), a.W - 1);             // idle units shadow a live beam
+            const uint32_t dst = smem_u32(my_heads + st * HEAD_BYTES);
+            const char* qr = q_row(bb) + g * 16;
+            if (fused) {   // the call's records come straight from the caller's k and v tensors
+                const long long in_row = ((long long)req * a.W + bb) * a.H + h;
+                const char* kr = static_cast<const char*>(a.k_in) + in_row * (DK * 2) + g * 16;
+                const char* vr = static_cast<const char*>(a.v_in) + in_row * (DV * 2) + g * 16;
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    cp_async16(dst + grp * REC_BYTES + (c * LPU + g) * 16, kr + c * LPU * 16);
+                    cp_async16(dst + grp * REC_BYTES + (16 + c * LPU + g) * 16, vr + c * LPU * 16);
+                }
+            } else {
+                const char* rec = kv + (own_row0 + bb) * REC_BYTES + g * 16;
+#pragma unroll
+                for (int c = 0; c < 2 * NCH; ++c) cp_async16(dst + grp * REC_BYTES + (c * LPU + g) * 16, rec + c * LPU * 16);
+            }
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) cp_async16(dst + UPW * REC_BYTES + grp * (DK * 2) + (c * LPU + g) * 16, qr + c * LPU * 16);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            ++heads_issued;
+        };
+        auto load_gate = [&](int k) {
+            const int bb = min(beam_of(k), a.W - 1);
+            if (!fused) return __ldg(a.gates + own_row0 + bb);
+            const long long in_row = ((long long)req * a.W + bb) * a.H + h;
+            return make_float2(__ldg(a.alpha_in + in_row), __ldg(a.beta_in + in_row));
+        };
+        // The segment's first heads go out before anything else: they depend on nothing the segment sets up.
+        float2 gate0 = make_float2(1.f, 0.f), gate1 = gate0;
+        if (warp < FOLD_WARPS && !dead && n_quads > 0) {
+            issue_head(0);
+            gate0 = load_gate(0);
+            if (1 < n_quads) {
+                if (HEAD_STAGES > 1) issue_head(1);
+                gate1 = load_gate(1);
+            }
+        }
 
         // How many of the oldest levels fit in the staging buffer (whole levels only; uniform over the CTA).
         // Lane l looks at level l (one load latency for the whole chain); offsets grow with the level.
@@ -177,75 +297,28 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
             if (staged_levels == 0) n_staged = 0;
         }
 
-        // The previous segment is fully consumed: the MMA warp and the epilogue warps pass this barrier only
-        // after the last group's MMA completed and was read back; the fold warps after their last staged read.
+        // The previous segment is fully consumed: the epilogue warps pass this barrier only after the last
+        // group's MMA completed and was read back; the fold warps after their last staged read.
         __syncthreads();
-        if (warp == 0 && !dead) {
-            const int32_t* ulist = a.ulist + req * a.ulist_req_stride;
-            const int mine = (n_staged > lane) ? (n_staged - lane + 31) / 32 : 0;
-            mbar_expect_tx(bar_stage, mine * REC_BYTES);   // one arrival per lane, with the bytes it is about to request
-            for (int i = lane; i < n_staged; i += 32) {
-                const long long row = plane_row0 + __ldg(ulist + i);
+        if (warp >= FOLD_WARPS && !dead) {
+            // The epilogue warps (idle until the first group is folded) stage the distinct records: one 512-byte bulk
+            // copy per record, its gates by a plain load, one record per lane.  Every lane arrives once, announcing
+            // the bytes it requested; its gate store is ordered before the arrival.
+            static_assert(STAGE_CAP <= 128, "one staged record per epilogue lane");
+            const int i = (warp - FOLD_WARPS) * 32 + lane;
+            if (i < n_staged) {
+                const long long row = plane_row0 + __ldg(a.ulist + req * a.ulist_req_stride + i);
                 bulk_load(smem_u32(stage + i * REC_BYTES), kv + row * REC_BYTES, REC_BYTES, bar_stage);
+                gates_s[i] = __ldg(a.gates + row);
             }
+            mbar_expect_tx(bar_stage, i < n_staged ? REC_BYTES : 0);
         }
-        const int gcount0 = sg_begin - g_begin;   // groups this CTA finished before this segment
+        if (seg_idx > 0 && !dead) load_s0(pair, sg_end < g_end);
 
         if (warp < FOLD_WARPS) {
             // =============================== FOLD ===============================
-            const int grp = lane / LPU, g = lane % LPU;
             const int32_t* table_r = a.table + req * a.table_req_stride;
             const int32_t* sidx_r = a.sidx + req * a.sidx_req_stride;
-            // the gates of the staged records: every fold warp writes all of them (same values), then syncs itself
-            if (!dead) {
-                const int32_t* ulist = a.ulist + req * a.ulist_req_stride;
-                for (int i = lane; i < n_staged; i += 32) gates_s[i] = __ldg(a.gates + plane_row0 + __ldg(ulist + i));
-                __syncwarp();
-            }
-            // quad k of the segment: group sg_begin + k/2, rows (k&1)*32 + 4*warp + grp
-            const int n_quads = QPG * (sg_end - sg_begin);
-            auto group_of = [&](int k) { return QPG == 2 ? (k >> 1) : k; };
-            auto half_of = [&](int k) { return QPG == 2 ? (k & 1) : 0; };
-            auto beam_of = [&](int k) { return ((sg_begin + group_of(k)) - pair * groups_per_pair) * GN + half_of(k) * (FOLD_WARPS * UPW) + UPW * warp + grp; };
-            // The heads of a quad (own record and query of its four units) arrive by 16-byte async copies into a
-            // two-stage ring private to the warp, two quads ahead of their use (each lane copies exactly the
-            // chunks it reads back); the gates ride in registers.
-            auto slot_of = [&](int k) { return (gcount0 + group_of(k)) & 1; };
-            auto use_of = [&](int k) { return (gcount0 + group_of(k)) >> 1; };
-            auto row_of = [&](int k) { return half_of(k) * (FOLD_WARPS * UPW) + UPW * warp + grp; };
-            uint8_t* my_heads = heads + warp * (HEAD_STAGES * HEAD_BYTES);
-            auto head_bar = [&](int st) { return smem_u32(bars + 8 + warp * HEAD_STAGES + st); };
-            auto q_row = [&](int bb) { return reinterpret_cast<const char*>(qbase + (((long long)req * a.W + bb) * a.H + h) * DK); };
-            auto issue_head = [&](int k) {   // every lane copies the chunks it will read back itself
-                const int st = heads_issued % HEAD_STAGES;
-                const int bb = min(beam_of(k), a.W - 1);             // idle units shadow a live beam
-                const uint32_t dst = smem_u32(my_heads + st * HEAD_BYTES);
-                const char* qr = q_row(bb) + g * 16;
-                if (fused) {   // the call's records come straight from the caller's k and v tensors
-                    const long long in_row = ((long long)req * a.W + bb) * a.H + h;
-                    const char* kr = static_cast<const char*>(a.k_in) + in_row * (DK * 2) + g * 16;
-                    const char* vr = static_cast<const char*>(a.v_in) + in_row * (DV * 2) + g * 16;
-#pragma unroll
-                    for (int c = 0; c < NCH; ++c) {
-                        cp_async16(dst + grp * REC_BYTES + (c * LPU + g) * 16, kr + c * LPU * 16);
-                        cp_async16(dst + grp * REC_BYTES + (16 + c * LPU + g) * 16, vr + c * LPU * 16);
-                    }
-                } else {
-                    const char* rec = kv + (own_row0 + bb) * REC_BYTES + g * 16;
-#pragma unroll
-                    for (int c = 0; c < 2 * NCH; ++c) cp_async16(dst + grp * REC_BYTES + (c * LPU + g) * 16, rec + c * LPU * 16);
-                }
-#pragma unroll
-                for (int c = 0; c < NCH; ++c) cp_async16(dst + UPW * REC_BYTES + grp * (DK * 2) + (c * LPU + g) * 16, qr + c * LPU * 16);
-                asm volatile("cp.async.commit_group;" ::: "memory");
-                ++heads_issued;
-            };
-            auto load_gate = [&](int k) {
-                const int bb = min(beam_of(k), a.W - 1);
-                if (!fused) return __ldg(a.gates + own_row0 + bb);
-                const long long in_row = ((long long)req * a.W + bb) * a.H + h;
-                return make_float2(__ldg(a.alpha_in + in_row), __ldg(a.beta_in + in_row));
-            };
             constexpr int NIDX = LPU >= 8 ? 1 : 8 / LPU;     // the unit's lanes hold the indices of its first 8 levels
             struct Idx { int32_t v[NIDX]; };
             auto load_idx = [&](int k) -> Idx {
@@ -258,17 +331,8 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
                 }
                 return x;
             };
-            float2 gate0 = make_float2(1.f, 0.f), gate1 = gate0;
             Idx idx_next{};
-            if (!dead && n_quads > 0) {
-                idx_next = load_idx(0);
-                issue_head(0);
-                gate0 = load_gate(0);
-                if (1 < n_quads) {
-                    if (HEAD_STAGES > 1) issue_head(1);
-                    gate1 = load_gate(1);
-                }
-            }
+            if (!dead && n_quads > 0) idx_next = load_idx(0);
             bool staged_ready = false;
             for (int k = 0; k < n_quads && !dead; ++k) {
                 const int s = slot_of(k), use = use_of(k);
@@ -386,28 +450,6 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
             // =============================== EPILOGUE ===============================
             const int quad = warp & 3;                    // tensor-memory lane quadrant of this warp
             const int i = quad * 32 + lane;               // output element (dv index) of this thread
-            if (!dead) {
-                // Row i of the head's S_0 (row-major fp32 in the store) goes to lane i of tensor memory, rounded to
-                // TF32 on the way: the MMA's A operand lives there, so there is no shared-memory copy of S_0 and
-                // no S_0 traffic per MMA.
-                const float* row = a.s0 + req * a.s0_req_stride + (long long)h * (DV * DK) + (long long)i * DK;
-#pragma unroll 1
-                for (int kb = 0; kb < 4; ++kb) {
-                    uint32_t v[32];
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        const float4 x = __ldg(reinterpret_cast<const float4*>(row + kb * 32) + c);
-                        v[4 * c] = __float_as_uint(round_tf32(x.x)); v[4 * c + 1] = __float_as_uint(round_tf32(x.y));
-                        v[4 * c + 2] = __float_as_uint(round_tf32(x.z)); v[4 * c + 3] = __float_as_uint(round_tf32(x.w));
-                    }
-                    tmem_st32(tmem_base + S0_COL + kb * 32 + ((uint32_t)(quad * 32) << 16), v);
-                }
-                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_s0);
-                if (warp == FOLD_WARPS) { ONELA_MARK("S0 in tmem") }
-            }
             for (int gi = sg_begin; gi < sg_end && !dead; ++gi) {
                 const int gcount = gcount0 + (gi - sg_begin);
                 const int s = gcount & 1, use = gcount >> 1;
@@ -488,7 +530,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
     }
 
 #ifdef ONELA_TIMING
-    if (lane == 0 && (warp == 0 || warp == 7 || warp == 8) && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1) && (a.depth == 1 || a.depth == 8))
+    if (lane == 0 && (warp == 0 || warp == 5 || warp == FOLD_WARPS || warp == FOLD_WARPS + 1) && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1) && (a.depth == 1 || a.depth == 8))
         printf("cta %d warp %d depth %d groups %d total %lld | head %lld fold %lld slotwait %lld write %lld arrive+mma %lld | t5 %lld t2 %lld t6 %lld\n",
                (int)blockIdx.x, warp, a.depth, g_end - g_begin, clock64() - tstart, tph[0], tph[1], tph[7], tph[3], tph[4], tph[5], tph[2], tph[6]);
 #endif
@@ -514,6 +556,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const DecodeArgs 
     if (warp == 0) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
+#ifdef ONELA_SPAN
+    if (threadIdx.x == 0) g_span[launch_id & 63][blockIdx.x][1] = gtime2();
+#endif
 }
 
 int sm_count_ws() {
@@ -521,6 +566,44 @@ int sm_count_ws() {
     if (cudaGetDevice(&dev) != cudaSuccess) return 148;
     if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
     return n;
+}
+
+// Contiguous group ranges for the CTAs.  Starting a segment (a new (request, head): pipeline drained, S_0 reloaded,
+// staging refilled) costs about as much as SEG_COST / GROUP_COST groups, so a CTA's cost is counted as
+// GROUP_COST * groups + SEG_COST * segments and the smallest bound T is searched for which a greedy fill needs no
+// more CTAs than there are SMs.  Returns the number of CTAs used.
+constexpr int GROUP_COST = 4, SEG_COST = 7;
+int greedy_fill(int total_groups, int gpp, int limit, int max_ctas, int32_t* begin) {
+    int n = 0, gi = 0;
+    while (gi < total_groups) {
+        if (n == max_ctas) return max_ctas + 1;
+        if (begin) begin[n] = gi;
+        int cost = 0;
+        bool any = false;
+        while (gi < total_groups) {
+            const int pair_end = (gi / gpp + 1) * gpp;
+            const int room = (limit - cost - SEG_COST) / GROUP_COST;     // groups of this segment that still fit
+            if (room <= 0) break;
+            const int take = room < pair_end - gi ? room : pair_end - gi;
+            gi += take;
+            cost += SEG_COST + take * GROUP_COST;
+            any = true;
+            if (gi < pair_end) break;
+        }
+        if (!any) return max_ctas + 1;   // the bound does not admit a single group
+        ++n;
+    }
+    if (begin) begin[n] = total_groups;
+    return n;
+}
+int make_partition(int total_groups, int gpp, int sms, Partition* part) {
+    int lo = SEG_COST + GROUP_COST, hi = SEG_COST * (total_groups / gpp + 2) + GROUP_COST * total_groups;
+    while (lo < hi) {
+        const int mid = (lo + hi) / 2;
+        if (greedy_fill(total_groups, gpp, mid, sms, nullptr) <= sms) hi = mid;
+        else lo = mid + 1;
+    }
+    return greedy_fill(total_groups, gpp, lo, sms, part->begin);
 }
 
 template <typename OutT>
@@ -532,16 +615,40 @@ cudaError_t launch_ws_t(const DecodeArgs& a, cudaStream_t stream) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) return e;
         sms = sm_count_ws();
+        if (sms > MAX_CTAS) sms = MAX_CTAS;
         configured = true;
     }
     const int groups_per_pair = (a.W + GN - 1) / GN;
     const int total_groups = a.req_count * a.H * groups_per_pair;
-    const int grid = total_groups < sms ? total_groups : sms;
-    kern<<<grid, THREADS, SMEM_BYTES, stream>>>(a, total_groups, groups_per_pair);
-    return cudaGetLastError();
+    static thread_local Partition part;          // the last launch's partition, reused while the shape stays
+    static thread_local int part_total = -1, part_gpp = -1, part_sms = -1, part_ctas = 0;
+    if (part_total != total_groups || part_gpp != groups_per_pair || part_sms != sms) {
+        part_ctas = make_partition(total_groups, groups_per_pair, sms, &part);
+        part_total = total_groups; part_gpp = groups_per_pair; part_sms = sms;
+    }
+    static int launch_id = 0;
+    // Programmatic dependent launch: this launch's CTAs may start, allocate and read S_0 while the previous
+    // kernel of the stream drains; the kernel waits for that kernel's completion before it reads anything else.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(part_ctas);
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, a, part, groups_per_pair, launch_id++);
 }
 
 }  // namespace
+
+#ifdef ONELA_SPAN
+extern "C" int onela_debug_spans(unsigned long long* host_out) {   // instrumented builds only
+    return (int)cudaMemcpyFromSymbol(host_out, g_span, sizeof(g_span));
+}
+#endif
 
 bool decode_sm100_supported(int32_t dk, int32_t dv, int32_t rec_dtype) {
     return dk == 128 && dv == 128 && rec_dtype == ONELA_DTYPE_BF16;
