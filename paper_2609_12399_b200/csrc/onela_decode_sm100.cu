@@ -45,7 +45,15 @@ constexpr int LPU = ONELA_LPU;                      // lanes per (beam, head) un
 constexpr int UPW = 32 / LPU;                       // units a fold warp folds at a time (a "quad" when LPU = 8)
 constexpr int NCH = 16 / LPU;                       // 16-byte chunks per lane per 256-byte vector
 constexpr int QPG = (FOLD_WARPS * UPW == 32) ? 2 : 1;   // quads each fold warp contributes to a group
-constexpr int THREADS = (FOLD_WARPS + 4) * 32;      // + 4 epilogue warps (12 warps: three per SM sub-partition)
+#ifndef ONELA_ISSUER_WARP
+#define ONELA_ISSUER_WARP 0
+#endif
+#ifndef ONELA_NISSUE
+#define ONELA_NISSUE 1
+#endif
+constexpr int ISSUER_WARPS = ONELA_ISSUER_WARP;    // 1: a warp of its own issues the MMAs; 0: the first epilogue warp does
+constexpr int ISSUER = ISSUER_WARPS ? FOLD_WARPS + 4 : FOLD_WARPS;
+constexpr int THREADS = (FOLD_WARPS + 4 + ISSUER_WARPS) * 32;      // + 4 epilogue warps (12 warps: three per SM sub-partition)
 constexpr int GN = FOLD_WARPS * UPW * QPG;          // beams per group = MMA N (64 or 48)
 constexpr int R_KB_STRIDE = GN * 128;               // bytes between the four 32-float K blocks of the operand
 constexpr int R_BYTES = 4 * R_KB_STRIDE;            // 32768
@@ -60,8 +68,16 @@ constexpr int STAGE_CAP = (232448 - 1024 - 256 - SLOTS * SLOT_BYTES - HEADS_TOTA
 constexpr int STAGE_BYTES = STAGE_CAP * REC_BYTES;
 constexpr int GATE_BYTES = STAGE_CAP * 8;
 constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + STAGE_BYTES + GATE_BYTES + HEADS_TOTAL + 256 + 1024;
-constexpr uint32_t TMEM_COLS = 256;              // accumulators of the two slots in [0, 2 GN), the head's S_0 in [128, 256)
-constexpr uint32_t S0_COL = 128;
+#ifndef ONELA_NACC
+#define ONELA_NACC 1
+#endif
+// A group's 16 MMAs accumulate along K; MMAs into one accumulator are issued a full pipeline latency apart, so
+// the K blocks go round-robin to NACC independent accumulators that the epilogue sums.
+constexpr int NACC = ONELA_NACC;
+constexpr uint32_t S0_COL = SLOTS * NACC * GN <= 128 ? 128 : SLOTS * NACC * GN;   // accumulators first, then the head's S_0
+constexpr uint32_t TMEM_COLS = S0_COL + 128 <= 256 ? 256 : 512;
+static_assert(S0_COL + 128 <= 512, "tensor memory columns");
+static_assert(ONELA_NISSUE <= NACC && NACC % ONELA_NISSUE == 0, "each issuing thread owns whole accumulators");
 static_assert(SMEM_BYTES <= 232448, "shared memory per CTA");
 using L = Lanes<LPU>;
 using RecT = L::R;
@@ -77,6 +93,10 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+
+// Position of 16-byte chunk q (4 floats) of a corr-tile row: chunks swap in pairs in every other 128-byte stretch,
+// which keeps the fold warps' 32-byte-strided writes and the epilogue's 32-byte-strided reads off shared banks.
+__device__ __forceinline__ int corr_chunk(int q) { return q ^ ((q >> 3) & 1); }
 
 struct Head {           // what a unit's fold needs first
     uint4 q[NCH];
@@ -143,7 +163,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         mbar_init(bar_stage, 128);                    // every lane of the four epilogue warps
         for (int s = 0; s < SLOTS; ++s) {
             mbar_init(bar_full(s), QPG * FOLD_WARPS); // one arrival per quad of 4 beams
-            mbar_init(bar_done(s), 1);                // tcgen05.commit
+            mbar_init(bar_done(s), ONELA_NISSUE);     // tcgen05.commit of every issuing thread
             mbar_init(bar_free(s), 4);                // the four epilogue warps
         }
         for (int i = 0; i < FOLD_WARPS * HEAD_STAGES; ++i) mbar_init(smem_u32(bars + 8 + i), 1);
@@ -250,6 +270,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             const int bb = min(beam_of(k), a.W - 1);             // idle units shadow a live beam
             const uint32_t dst = smem_u32(my_heads + st * HEAD_BYTES);
             const char* qr = q_row(bb) + g * 16;
+#ifdef ONELA_EXP_NOHEADS   // timing experiment only: results are wrong
+            if (heads_issued >= ONELA_EXP_NOHEADS) { asm volatile("cp.async.commit_group;" ::: "memory"); ++heads_issued; return; }
+#endif
             if (fused) {   // the call's records come straight from the caller's k and v tensors
                 const long long in_row = ((long long)req * a.W + bb) * a.H + h;
                 const char* kr = static_cast<const char*>(a.k_in) + in_row * (DK * 2) + g * 16;
@@ -300,7 +323,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         // The previous segment is fully consumed: the epilogue warps pass this barrier only after the last
         // group's MMA completed and was read back; the fold warps after their last staged read.
         __syncthreads();
-        if (warp >= FOLD_WARPS && !dead) {
+        if (warp >= FOLD_WARPS && warp < FOLD_WARPS + 4 && !dead) {
             // The epilogue warps (idle until the first group is folded) stage the distinct records: one 512-byte bulk
             // copy per record, its gates by a plain load, one record per lane.  Every lane arrives once, announcing
             // the bytes it requested; its gate store is ordered before the arrival.
@@ -314,6 +337,36 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             mbar_expect_tx(bar_stage, i < n_staged ? REC_BYTES : 0);
         }
         if (seg_idx > 0 && !dead) load_s0(pair, sg_end < g_end);
+
+        // One thread issues a group's 16 MMAs as soon as all its rows are written (never a fold warp: whichever fold
+        // warp issued would be the last to finish its next quad).  Returns true when it had to give up.
+        auto issue_group = [&](int s, int use, int part = 0) -> bool {
+            int mma_failed = 0;
+            if (lane == 0) {
+                bool ok = wait_or_abort(bar_full(s), use & 1, abort_flag);
+                ok = ok && wait_or_abort(bar_s0, seg_parity, abort_flag);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                ONELA_TICK(0)   // (issuer) wait for the group's rows
+                if (ok) {
+                    constexpr uint32_t idesc = idesc_tf32(GN);
+                    const uint64_t bd = umma_desc(smem_u32(ring + s * SLOT_BYTES));
+#pragma unroll
+                    for (int kb = 0; kb < 4; ++kb)
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks)
+                            if ((kb * 4 + ks) % ONELA_NISSUE == part)
+                            umma_tf32_ts(tmem_base + (s * NACC + (kb * 4 + ks) % NACC) * GN, tmem_base + S0_COL + (kb * 4 + ks) * 8,
+                                         bd + (uint64_t)((kb * R_KB_STRIDE + ks * 32) >> 4), idesc,
+                                         (kb * 4 + ks) >= NACC ? 1u : 0u);
+                } else {
+                    mma_failed = 1;
+                }
+                umma_commit(bar_done(s));   // arrives when the MMAs above (if any) have completed
+                ONELA_TICK(1)   // (issuer) issue
+                ONELA_MARK("mma issued")
+            }
+            return __shfl_sync(0xffffffffu, mma_failed, 0) != 0;
+        };
 
         if (warp < FOLD_WARPS) {
             // =============================== FOLD ===============================
@@ -356,7 +409,12 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                     }
                     cur.own.gate = gate0;
                     ++heads_taken;
-                    if (fused && beam_of(k) < a.W) {   // the append: this beam's record goes to its arena slot, bit for bit
+#ifdef ONELA_EXP_NOAPPEND
+                    if (false) {
+#else
+                    if (fused && beam_of(k) < a.W) {   // the append
+#endif
+                    // (the append): this beam's record goes to its arena slot, bit for bit
                         uint4* dst = reinterpret_cast<uint4*>(a.kv_out + (own_row0 + bb) * REC_BYTES) + g;
 #pragma unroll
                         for (int c = 0; c < NCH; ++c) {
@@ -419,7 +477,12 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 uint8_t* R_s = ring + s * SLOT_BYTES;
                 float* C_s = reinterpret_cast<float*>(R_s + R_BYTES);
                 {
+                    // Bank conflicts: the lanes g and g + 4 of a unit own the same chunk positions of two operand rows
+                    // 48 * 128 bytes apart, so the upper four lanes write their two chunks in the opposite order;
+                    // the corr tile (a layout of our own) swaps each pair of 16-byte chunks in every other 128-byte
+                    // stretch of a row instead (corr_chunk below; the epilogue reads it the same way).
                     const int sw = u & 7;
+                    const bool hi = (g >> 2) & 1;
                     const float2 dc = make_float2(decay, decay);
 #pragma unroll
                     for (int c = 0; c < NCH; ++c) {
@@ -429,13 +492,14 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                         float2 x[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) x[e] = __fmul2_rn(r[4 * c + e], dc);
-                        *reinterpret_cast<float4*>(row + (((ch) ^ sw) << 4)) =
-                            make_float4(round_tf32(x[0].x), round_tf32(x[0].y), round_tf32(x[1].x), round_tf32(x[1].y));
-                        *reinterpret_cast<float4*>(row + (((ch + 1) ^ sw) << 4)) =
-                            make_float4(round_tf32(x[2].x), round_tf32(x[2].y), round_tf32(x[3].x), round_tf32(x[3].y));
-                        float* crow = C_s + u * DV + ci * 8;
-                        *reinterpret_cast<float4*>(crow) = make_float4(corr[4 * c].x, corr[4 * c].y, corr[4 * c + 1].x, corr[4 * c + 1].y);
-                        *reinterpret_cast<float4*>(crow + 4) =
+                        const float4 lo4 = make_float4(round_tf32(x[0].x), round_tf32(x[0].y), round_tf32(x[1].x), round_tf32(x[1].y));
+                        const float4 hi4 = make_float4(round_tf32(x[2].x), round_tf32(x[2].y), round_tf32(x[3].x), round_tf32(x[3].y));
+                        *reinterpret_cast<float4*>(row + (((ch + (hi ? 1 : 0)) ^ sw) << 4)) = hi ? hi4 : lo4;
+                        *reinterpret_cast<float4*>(row + (((ch + (hi ? 0 : 1)) ^ sw) << 4)) = hi ? lo4 : hi4;
+                        float* crow = C_s + u * DV;
+                        *reinterpret_cast<float4*>(crow + corr_chunk(2 * ci) * 4) =
+                            make_float4(corr[4 * c].x, corr[4 * c].y, corr[4 * c + 1].x, corr[4 * c + 1].y);
+                        *reinterpret_cast<float4*>(crow + corr_chunk(2 * ci + 1) * 4) =
                             make_float4(corr[4 * c + 2].x, corr[4 * c + 2].y, corr[4 * c + 3].x, corr[4 * c + 3].y);
                     }
                 }
@@ -446,6 +510,12 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 if (lane == 0) mbar_arrive(bar_full(s));
                 ONELA_TICK(4)   // arrive
             }
+        } else if (ISSUER_WARPS && warp == ISSUER) {
+            // =============================== MMA ISSUE ===============================
+            for (int gi = sg_begin; gi < sg_end && !dead; ++gi) {
+                const int gcount = gcount0 + (gi - sg_begin);
+                if (issue_group(gcount & 1, gcount >> 1)) dead = true;
+            }
         } else {
             // =============================== EPILOGUE ===============================
             const int quad = warp & 3;                    // tensor-memory lane quadrant of this warp
@@ -453,38 +523,14 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             for (int gi = sg_begin; gi < sg_end && !dead; ++gi) {
                 const int gcount = gcount0 + (gi - sg_begin);
                 const int s = gcount & 1, use = gcount >> 1;
-                if (warp == FOLD_WARPS) {
-                    // One thread issues the group's 16 MMAs as soon as all its rows are written (the fold warps
-                    // never stop for it: whichever fold warp issued would be the last to finish its next quad).
-                    int mma_failed = 0;
-                    if (lane == 0) {
-                        bool ok = wait_or_abort(bar_full(s), use & 1, abort_flag);
-                        ok = ok && wait_or_abort(bar_s0, seg_parity, abort_flag);
-                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                        if (ok) {
-                            constexpr uint32_t idesc = idesc_tf32(GN);
-                            const uint64_t bd = umma_desc(smem_u32(ring + s * SLOT_BYTES));
-#pragma unroll
-                            for (int kb = 0; kb < 4; ++kb)
-#pragma unroll
-                                for (int ks = 0; ks < 4; ++ks)
-                                    umma_tf32_ts(tmem_base + s * GN, tmem_base + S0_COL + (kb * 4 + ks) * 8,
-                                                 bd + (uint64_t)((kb * R_KB_STRIDE + ks * 32) >> 4), idesc, (kb | ks) ? 1u : 0u);
-                        } else {
-                            mma_failed = 1;
-                        }
-                        umma_commit(bar_done(s));   // arrives when the MMAs above (if any) have completed
-                        ONELA_MARK("mma issued")
-                    }
-                    if (__shfl_sync(0xffffffffu, mma_failed, 0)) { dead = true; break; }
-                }
+                if (!ISSUER_WARPS && warp >= ISSUER && warp < ISSUER + ONELA_NISSUE && issue_group(s, use, warp - ISSUER)) { dead = true; break; }
                 if (!wait_or_abort(bar_done(s), use & 1, abort_flag)) { dead = true; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 ONELA_TICK(5)   // epilogue: wait for the MMA group
                 if (warp == FOLD_WARPS) { ONELA_MARK("mma done") }
                 float* C_s = reinterpret_cast<float*>(ring + s * SLOT_BYTES + R_BYTES);
                 const int b0 = (gi - pair * groups_per_pair) * GN;
-                const uint32_t taddr = tmem_base + s * GN + ((uint32_t)(quad * 32) << 16);
+                const uint32_t taddr = tmem_base + s * NACC * GN + ((uint32_t)(quad * 32) << 16);
                 {
                     // accumulator rows (dv) of this thread, all 64 beams, added onto the corr tile in place
                     uint32_t v[GN];
@@ -496,7 +542,19 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                     }
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-                    for (int j = 0; j < GN; ++j) C_s[j * DV + i] += __uint_as_float(v[j]);
+                    for (int acc = 1; acc < NACC; ++acc) {     // the other partial accumulators
+#pragma unroll
+                        for (int c0 = 0; c0 < GN; c0 += 16) {
+                            uint32_t w[16];
+                            tmem_ld16(taddr + acc * GN + c0, w);
+                            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) v[c0 + j] = __float_as_uint(__uint_as_float(v[c0 + j]) + __uint_as_float(w[j]));
+                        }
+                    }
+                    const int ip = corr_chunk(i >> 2) * 4 + (i & 3);   // where the corr tile keeps element i of a row
+#pragma unroll
+                    for (int j = 0; j < GN; ++j) C_s[j * DV + ip] += __uint_as_float(v[j]);
                 }
                 ONELA_TICK(2)   // tmem ld + add
                 if (bar_or(1, 128, 0)) { dead = true; break; }     // the four epilogue warps: tile complete
@@ -506,9 +564,13 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
 #pragma unroll
                     for (int it = 0; it < GN * 16 / 128; ++it) {   // GN * 16 chunks of 16 bytes over 128 threads
                         const int idx = it * 128 + et, j = idx >> 4, ch = idx & 15;
+#ifdef ONELA_EXP_NOSTORE
+                        if (b0 + j < a.W && a.depth < 0) {
+#else
                         if (b0 + j < a.W) {
-                            const float4 x0 = *reinterpret_cast<const float4*>(C_s + j * DV + ch * 8);
-                            const float4 x1 = *reinterpret_cast<const float4*>(C_s + j * DV + ch * 8 + 4);
+#endif
+                            const float4 x0 = *reinterpret_cast<const float4*>(C_s + j * DV + corr_chunk(2 * ch) * 4);
+                            const float4 x1 = *reinterpret_cast<const float4*>(C_s + j * DV + corr_chunk(2 * ch + 1) * 4);
                             const float o[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
                             store8<OutT>(static_cast<OutT*>(a.out) + (((long long)req * a.W + b0 + j) * a.H + h) * DV + ch * 8, o);
                         }
@@ -530,7 +592,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     }
 
 #ifdef ONELA_TIMING
-    if (lane == 0 && (warp == 0 || warp == 5 || warp == FOLD_WARPS || warp == FOLD_WARPS + 1) && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1) && (a.depth == 1 || a.depth == 8))
+    if (lane == 0 && (warp == 0 || warp == 5 || warp == FOLD_WARPS || warp == FOLD_WARPS + 1 || warp == ISSUER) && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1) && (a.depth == 1 || a.depth == 8))
         printf("cta %d warp %d depth %d groups %d total %lld | head %lld fold %lld slotwait %lld write %lld arrive+mma %lld | t5 %lld t2 %lld t6 %lld\n",
                (int)blockIdx.x, warp, a.depth, g_end - g_begin, clock64() - tstart, tph[0], tph[1], tph[7], tph[3], tph[4], tph[5], tph[2], tph[6]);
 #endif
