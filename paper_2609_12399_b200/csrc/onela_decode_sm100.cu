@@ -45,40 +45,35 @@ constexpr int LPU = ONELA_LPU;                      // lanes per (beam, head) un
 constexpr int UPW = 32 / LPU;                       // units a fold warp folds at a time (a "quad" when LPU = 8)
 constexpr int NCH = 16 / LPU;                       // 16-byte chunks per lane per 256-byte vector
 constexpr int QPG = (FOLD_WARPS * UPW == 32) ? 2 : 1;   // quads each fold warp contributes to a group
-#ifndef ONELA_ISSUER_WARP
-#define ONELA_ISSUER_WARP 0
-#endif
-#ifndef ONELA_NISSUE
-#define ONELA_NISSUE 1
-#endif
-constexpr int ISSUER_WARPS = ONELA_ISSUER_WARP;    // 1: a warp of its own issues the MMAs; 0: the first epilogue warp does
-constexpr int ISSUER = ISSUER_WARPS ? FOLD_WARPS + 4 : FOLD_WARPS;
-constexpr int THREADS = (FOLD_WARPS + 4 + ISSUER_WARPS) * 32;      // + 4 epilogue warps (12 warps: three per SM sub-partition)
+constexpr int THREADS = (FOLD_WARPS + 4) * 32;      // + 4 epilogue warps (16 warps: four per SM sub-partition)
 constexpr int GN = FOLD_WARPS * UPW * QPG;          // beams per group = MMA N (64 or 48)
 constexpr int R_KB_STRIDE = GN * 128;               // bytes between the four 32-float K blocks of the operand
 constexpr int R_BYTES = 4 * R_KB_STRIDE;            // 32768
 constexpr int C_BYTES = GN * DV * 4;                // 32768: corr tile, row = beam
 constexpr int SLOT_BYTES = R_BYTES + C_BYTES;
-constexpr int SLOTS = 2;
+#ifndef ONELA_SLOTS
+#define ONELA_SLOTS 2
+#endif
+constexpr int SLOTS = ONELA_SLOTS;
 constexpr int HEAD_BYTES = UPW * (REC_BYTES + DK * 2);   // one quad's heads: own records + queries of its units
-constexpr int HEAD_STAGES = LPU >= 8 ? 2 : 1;         // heads in flight per fold warp
+#ifndef ONELA_HEAD_STAGES
+#define ONELA_HEAD_STAGES 1
+#endif
+constexpr int HEAD_STAGES = ONELA_HEAD_STAGES;          // heads in flight per fold warp
 constexpr int HEADS_TOTAL = FOLD_WARPS * HEAD_STAGES * HEAD_BYTES;
-constexpr int STAGE_CAP = (232448 - 1024 - 256 - SLOTS * SLOT_BYTES - HEADS_TOTAL) / (REC_BYTES + 8) / 4 * 4 > 104
-                              ? 104 : (232448 - 1024 - 256 - SLOTS * SLOT_BYTES - HEADS_TOTAL) / (REC_BYTES + 8) / 4 * 4;                       // distinct ancestor records staged per segment
+#ifndef ONELA_STAGE_MAX
+#define ONELA_STAGE_MAX 104
+#endif
+constexpr int STAGE_ROOM = (232448 - 1024 - 256 - SLOTS * SLOT_BYTES - HEADS_TOTAL) / (REC_BYTES + 8) / 4 * 4;
+constexpr int STAGE_CAP = STAGE_ROOM > ONELA_STAGE_MAX ? ONELA_STAGE_MAX : STAGE_ROOM;   // distinct ancestor records staged per segment
 constexpr int STAGE_BYTES = STAGE_CAP * REC_BYTES;
 constexpr int GATE_BYTES = STAGE_CAP * 8;
 constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + STAGE_BYTES + GATE_BYTES + HEADS_TOTAL + 256 + 1024;
-#ifndef ONELA_NACC
-#define ONELA_NACC 1
-#endif
-// A group's 16 MMAs accumulate along K; MMAs into one accumulator are issued a full pipeline latency apart, so
-// the K blocks go round-robin to NACC independent accumulators that the epilogue sums.
-constexpr int NACC = ONELA_NACC;
-constexpr uint32_t S0_COL = SLOTS * NACC * GN <= 128 ? 128 : SLOTS * NACC * GN;   // accumulators first, then the head's S_0
+constexpr uint32_t S0_COL = SLOTS * GN <= 128 ? 128 : SLOTS * GN;   // accumulators of the ring slots first, then the head's S_0
 constexpr uint32_t TMEM_COLS = S0_COL + 128 <= 256 ? 256 : 512;
 static_assert(S0_COL + 128 <= 512, "tensor memory columns");
-static_assert(ONELA_NISSUE <= NACC && NACC % ONELA_NISSUE == 0, "each issuing thread owns whole accumulators");
 static_assert(SMEM_BYTES <= 232448, "shared memory per CTA");
+static_assert(HEAD_STAGES >= 1 && HEAD_STAGES <= 3, "head ring depth");
 using L = Lanes<LPU>;
 using RecT = L::R;
 
@@ -149,24 +144,22 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     float2* gates_s = reinterpret_cast<float2*>(stage + STAGE_BYTES);
     uint8_t* heads = stage + STAGE_BYTES + GATE_BYTES;
     uint64_t* bars = reinterpret_cast<uint64_t*>(heads + HEADS_TOTAL);
-    // bars: 0 S_0 in tensor memory, 1 staged records, 2+s slot s full, 4+s slot s MMA done, 6+s slot s free,
-    //       8 + 2*w + st: head stage st of fold warp w
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8 + FOLD_WARPS * HEAD_STAGES);
+    // bars: 0 S_0 in tensor memory, 1 staged records, then per ring slot s: full, MMA done, free
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 + 3 * SLOTS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     const uint32_t bar_s0 = smem_u32(bars), bar_stage = smem_u32(bars + 1);
     auto bar_full = [&](int s) { return smem_u32(bars + 2 + s); };
-    auto bar_done = [&](int s) { return smem_u32(bars + 4 + s); };
-    auto bar_free = [&](int s) { return smem_u32(bars + 6 + s); };
+    auto bar_done = [&](int s) { return smem_u32(bars + 2 + SLOTS + s); };
+    auto bar_free = [&](int s) { return smem_u32(bars + 2 + 2 * SLOTS + s); };
 
     if (tid == 0) {
         mbar_init(bar_s0, THREADS / 32);              // every warp, once its share of S_0 sits in tensor memory
         mbar_init(bar_stage, 128);                    // every lane of the four epilogue warps
         for (int s = 0; s < SLOTS; ++s) {
             mbar_init(bar_full(s), QPG * FOLD_WARPS); // one arrival per quad of 4 beams
-            mbar_init(bar_done(s), ONELA_NISSUE);     // tcgen05.commit of every issuing thread
+            mbar_init(bar_done(s), 1);                // tcgen05.commit
             mbar_init(bar_free(s), 4);                // the four epilogue warps
         }
-        for (int i = 0; i < FOLD_WARPS * HEAD_STAGES; ++i) mbar_init(smem_u32(bars + 8 + i), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -260,8 +253,8 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         // The heads of a quad (own record and query of its four units) arrive by 16-byte async copies into a
         // two-stage ring private to the warp, two quads ahead of their use (each lane copies exactly the
         // chunks it reads back); the gates ride in registers.
-        auto slot_of = [&](int k) { return (gcount0 + group_of(k)) & 1; };
-        auto use_of = [&](int k) { return (gcount0 + group_of(k)) >> 1; };
+        auto slot_of = [&](int k) { return (gcount0 + group_of(k)) % SLOTS; };
+        auto use_of = [&](int k) { return (gcount0 + group_of(k)) / SLOTS; };
         auto row_of = [&](int k) { return half_of(k) * (FOLD_WARPS * UPW) + UPW * warp + grp; };
         uint8_t* my_heads = heads + (warp < FOLD_WARPS ? warp : 0) * (HEAD_STAGES * HEAD_BYTES);
         auto q_row = [&](int bb) { return reinterpret_cast<const char*>(qbase + (((long long)req * a.W + bb) * a.H + h) * DK); };
@@ -270,9 +263,6 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             const int bb = min(beam_of(k), a.W - 1);             // idle units shadow a live beam
             const uint32_t dst = smem_u32(my_heads + st * HEAD_BYTES);
             const char* qr = q_row(bb) + g * 16;
-#ifdef ONELA_EXP_NOHEADS   // timing experiment only: results are wrong
-            if (heads_issued >= ONELA_EXP_NOHEADS) { asm volatile("cp.async.commit_group;" ::: "memory"); ++heads_issued; return; }
-#endif
             if (fused) {   // the call's records come straight from the caller's k and v tensors
                 const long long in_row = ((long long)req * a.W + bb) * a.H + h;
                 const char* kr = static_cast<const char*>(a.k_in) + in_row * (DK * 2) + g * 16;
@@ -303,10 +293,10 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         if (warp < FOLD_WARPS && !dead && n_quads > 0) {
             issue_head(0);
             gate0 = load_gate(0);
-            if (1 < n_quads) {
-                if (HEAD_STAGES > 1) issue_head(1);
-                gate1 = load_gate(1);
-            }
+            if (1 < n_quads) gate1 = load_gate(1);
+#pragma unroll
+            for (int st = 1; st < HEAD_STAGES; ++st)
+                if (st < n_quads) issue_head(st);
         }
 
         // How many of the oldest levels fit in the staging buffer (whole levels only; uniform over the CTA).
@@ -340,7 +330,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
 
         // One thread issues a group's 16 MMAs as soon as all its rows are written (never a fold warp: whichever fold
         // warp issued would be the last to finish its next quad).  Returns true when it had to give up.
-        auto issue_group = [&](int s, int use, int part = 0) -> bool {
+        auto issue_group = [&](int s, int use) -> bool {
             int mma_failed = 0;
             if (lane == 0) {
                 bool ok = wait_or_abort(bar_full(s), use & 1, abort_flag);
@@ -354,10 +344,8 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                     for (int kb = 0; kb < 4; ++kb)
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks)
-                            if ((kb * 4 + ks) % ONELA_NISSUE == part)
-                            umma_tf32_ts(tmem_base + (s * NACC + (kb * 4 + ks) % NACC) * GN, tmem_base + S0_COL + (kb * 4 + ks) * 8,
-                                         bd + (uint64_t)((kb * R_KB_STRIDE + ks * 32) >> 4), idesc,
-                                         (kb * 4 + ks) >= NACC ? 1u : 0u);
+                            umma_tf32_ts(tmem_base + s * GN, tmem_base + S0_COL + (kb * 4 + ks) * 8,
+                                         bd + (uint64_t)((kb * R_KB_STRIDE + ks * 32) >> 4), idesc, (kb | ks) ? 1u : 0u);
                 } else {
                     mma_failed = 1;
                 }
@@ -395,7 +383,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 {
                     const int st = heads_taken % HEAD_STAGES;
                     // the oldest copy group in flight is this quad's; a newer one (the next quad's) may stay pending
-                    if (heads_issued - heads_taken > 1) asm volatile("cp.async.wait_group 1;" ::: "memory");
+                    const int newer = heads_issued - heads_taken - 1;
+                    if (newer >= 2) asm volatile("cp.async.wait_group 2;" ::: "memory");
+                    else if (newer == 1) asm volatile("cp.async.wait_group 1;" ::: "memory");
                     else asm volatile("cp.async.wait_group 0;" ::: "memory");
                     ONELA_TICK(5)   // (fold warps) wait for the head
                     if (warp == 0) { ONELA_MARK("head arrived") }
@@ -409,12 +399,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                     }
                     cur.own.gate = gate0;
                     ++heads_taken;
-#ifdef ONELA_EXP_NOAPPEND
-                    if (false) {
-#else
-                    if (fused && beam_of(k) < a.W) {   // the append
-#endif
-                    // (the append): this beam's record goes to its arena slot, bit for bit
+                    if (fused && beam_of(k) < a.W) {   // the append: this beam's record goes to its arena slot, bit for bit
                         uint4* dst = reinterpret_cast<uint4*>(a.kv_out + (own_row0 + bb) * REC_BYTES) + g;
 #pragma unroll
                         for (int c = 0; c < NCH; ++c) {
@@ -510,27 +495,21 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 if (lane == 0) mbar_arrive(bar_full(s));
                 ONELA_TICK(4)   // arrive
             }
-        } else if (ISSUER_WARPS && warp == ISSUER) {
-            // =============================== MMA ISSUE ===============================
-            for (int gi = sg_begin; gi < sg_end && !dead; ++gi) {
-                const int gcount = gcount0 + (gi - sg_begin);
-                if (issue_group(gcount & 1, gcount >> 1)) dead = true;
-            }
         } else {
             // =============================== EPILOGUE ===============================
             const int quad = warp & 3;                    // tensor-memory lane quadrant of this warp
             const int i = quad * 32 + lane;               // output element (dv index) of this thread
             for (int gi = sg_begin; gi < sg_end && !dead; ++gi) {
                 const int gcount = gcount0 + (gi - sg_begin);
-                const int s = gcount & 1, use = gcount >> 1;
-                if (!ISSUER_WARPS && warp >= ISSUER && warp < ISSUER + ONELA_NISSUE && issue_group(s, use, warp - ISSUER)) { dead = true; break; }
+                const int s = gcount % SLOTS, use = gcount / SLOTS;
+                if (warp == FOLD_WARPS && issue_group(s, use)) { dead = true; break; }
                 if (!wait_or_abort(bar_done(s), use & 1, abort_flag)) { dead = true; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 ONELA_TICK(5)   // epilogue: wait for the MMA group
                 if (warp == FOLD_WARPS) { ONELA_MARK("mma done") }
                 float* C_s = reinterpret_cast<float*>(ring + s * SLOT_BYTES + R_BYTES);
                 const int b0 = (gi - pair * groups_per_pair) * GN;
-                const uint32_t taddr = tmem_base + s * NACC * GN + ((uint32_t)(quad * 32) << 16);
+                const uint32_t taddr = tmem_base + s * GN + ((uint32_t)(quad * 32) << 16);
                 {
                     // accumulator rows (dv) of this thread, all 64 beams, added onto the corr tile in place
                     uint32_t v[GN];
@@ -541,17 +520,6 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                         for (int c0 = 0; c0 < GN; c0 += 16) tmem_ld16(taddr + c0, v + c0);
                     }
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-                    for (int acc = 1; acc < NACC; ++acc) {     // the other partial accumulators
-#pragma unroll
-                        for (int c0 = 0; c0 < GN; c0 += 16) {
-                            uint32_t w[16];
-                            tmem_ld16(taddr + acc * GN + c0, w);
-                            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) v[c0 + j] = __float_as_uint(__uint_as_float(v[c0 + j]) + __uint_as_float(w[j]));
-                        }
-                    }
                     const int ip = corr_chunk(i >> 2) * 4 + (i & 3);   // where the corr tile keeps element i of a row
 #pragma unroll
                     for (int j = 0; j < GN; ++j) C_s[j * DV + ip] += __uint_as_float(v[j]);
@@ -564,11 +532,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
 #pragma unroll
                     for (int it = 0; it < GN * 16 / 128; ++it) {   // GN * 16 chunks of 16 bytes over 128 threads
                         const int idx = it * 128 + et, j = idx >> 4, ch = idx & 15;
-#ifdef ONELA_EXP_NOSTORE
-                        if (b0 + j < a.W && a.depth < 0) {
-#else
                         if (b0 + j < a.W) {
-#endif
                             const float4 x0 = *reinterpret_cast<const float4*>(C_s + j * DV + corr_chunk(2 * ch) * 4);
                             const float4 x1 = *reinterpret_cast<const float4*>(C_s + j * DV + corr_chunk(2 * ch + 1) * 4);
                             const float o[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
@@ -592,7 +556,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     }
 
 #ifdef ONELA_TIMING
-    if (lane == 0 && (warp == 0 || warp == 5 || warp == FOLD_WARPS || warp == FOLD_WARPS + 1 || warp == ISSUER) && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1) && (a.depth == 1 || a.depth == 8))
+    if (lane == 0 && (warp == 0 || warp == 5 || warp == FOLD_WARPS || warp == FOLD_WARPS + 1) && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1) && (a.depth == 1 || a.depth == 8))
         printf("cta %d warp %d depth %d groups %d total %lld | head %lld fold %lld slotwait %lld write %lld arrive+mma %lld | t5 %lld t2 %lld t6 %lld\n",
                (int)blockIdx.x, warp, a.depth, g_end - g_begin, clock64() - tstart, tph[0], tph[1], tph[7], tph[3], tph[4], tph[5], tph[2], tph[6]);
 #endif
@@ -634,7 +598,10 @@ int sm_count_ws() {
 // staging refilled) costs about as much as SEG_COST / GROUP_COST groups, so a CTA's cost is counted as
 // GROUP_COST * groups + SEG_COST * segments and the smallest bound T is searched for which a greedy fill needs no
 // more CTAs than there are SMs.  Returns the number of CTAs used.
-constexpr int GROUP_COST = 4, SEG_COST = 7;
+#ifndef ONELA_SEG_COST
+#define ONELA_SEG_COST 7
+#endif
+constexpr int GROUP_COST = 4, SEG_COST = ONELA_SEG_COST;
 int greedy_fill(int total_groups, int gpp, int limit, int max_ctas, int32_t* begin) {
     int n = 0, gi = 0;
     while (gi < total_groups) {
