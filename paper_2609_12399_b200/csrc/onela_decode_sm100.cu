@@ -68,7 +68,10 @@ constexpr int STAGE_ROOM = (232448 - 1024 - 256 - SLOTS * SLOT_BYTES - HEADS_TOT
 constexpr int STAGE_CAP = STAGE_ROOM > ONELA_STAGE_MAX ? ONELA_STAGE_MAX : STAGE_ROOM;   // distinct ancestor records staged per segment
 constexpr int STAGE_BYTES = STAGE_CAP * REC_BYTES;
 constexpr int GATE_BYTES = STAGE_CAP * 8;
-constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + STAGE_BYTES + GATE_BYTES + HEADS_TOTAL + 256 + 1024;
+#ifndef ONELA_SMEM_PAD
+#define ONELA_SMEM_PAD 0
+#endif
+constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + STAGE_BYTES + GATE_BYTES + HEADS_TOTAL + 256 + 1024 + ONELA_SMEM_PAD;
 constexpr uint32_t S0_COL = SLOTS * GN <= 128 ? 128 : SLOTS * GN;   // accumulators of the ring slots first, then the head's S_0
 constexpr uint32_t TMEM_COLS = S0_COL + 128 <= 256 ? 256 : 512;
 static_assert(S0_COL + 128 <= 512, "tensor memory columns");
@@ -184,6 +187,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
 
 #ifdef ONELA_TIMING
     long long tph[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    long long t_issue = 0;
     long long tk = clock64();
     const long long tstart = tk;
 #define ONELA_TICK(i) { const long long now = clock64(); tph[i] += now - tk; tk = now; }
@@ -280,7 +284,26 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
 #pragma unroll
             for (int c = 0; c < NCH; ++c) cp_async16(dst + UPW * REC_BYTES + grp * (DK * 2) + (c * LPU + g) * 16, qr + c * LPU * 16);
             asm volatile("cp.async.commit_group;" ::: "memory");
+#ifdef ONELA_TIMING
+            t_issue = clock64();
+#endif
             ++heads_issued;
+#ifndef ONELA_L2_AHEAD
+#define ONELA_L2_AHEAD 1
+#endif
+#if ONELA_L2_AHEAD > 0
+            // the quad after this one: its 128-byte lines are requested into L2 (no shared memory needed for them yet)
+            if (k + ONELA_L2_AHEAD < n_quads && lane < UPW * 6) {
+                const int un = lane / 6, item = lane % 6;
+                const int b2 = min(beam_of(k + ONELA_L2_AHEAD) - grp + un, a.W - 1);
+                const long long in_row = ((long long)req * a.W + b2) * a.H + h;
+                const char* base_p = item < 2 ? reinterpret_cast<const char*>(qbase) + in_row * (DK * 2)
+                                   : fused ? (item < 4 ? static_cast<const char*>(a.k_in) + in_row * (DK * 2)
+                                                       : static_cast<const char*>(a.v_in) + in_row * (DV * 2))
+                                           : kv + (own_row0 + b2) * REC_BYTES + (item < 4 ? 0 : 256);
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(base_p + (item & 1) * 128));
+            }
+#endif
         };
         auto load_gate = [&](int k) {
             const int bb = min(beam_of(k), a.W - 1);
@@ -388,6 +411,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                     else if (newer == 1) asm volatile("cp.async.wait_group 1;" ::: "memory");
                     else asm volatile("cp.async.wait_group 0;" ::: "memory");
                     ONELA_TICK(5)   // (fold warps) wait for the head
+#ifdef ONELA_TIMING
+                    tph[4] += clock64() - t_issue;   // issue -> arrival observed (one stage in flight)
+#endif
                     if (warp == 0) { ONELA_MARK("head arrived") }
                     const uint4* rec = reinterpret_cast<const uint4*>(my_heads + st * HEAD_BYTES + grp * REC_BYTES) + g;
                     const uint4* qv = reinterpret_cast<const uint4*>(my_heads + st * HEAD_BYTES + UPW * REC_BYTES + grp * (DK * 2)) + g;
