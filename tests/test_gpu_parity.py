@@ -78,6 +78,17 @@ def test_multi_request_multi_layer_batched_and_unbatched():
     _full_check(case, "fp32", batched=False)
 
 
+@pytest.mark.parametrize("fused", [False, True])
+def test_many_short_segments_per_cta(fused):
+    """More (request, head) pairs than three per SM, each a single group or two: every CTA of the tensor-core
+    kernel walks through several segments, alternating its two S_0 / staging buffers, with staged ancestors
+    (Zipf parents, depth 4) and a ragged last group."""
+    wl = CFG1.scaled(R=20, L=1, H=32, W=40, D=4, prompt_len=16, parents="zipf", zipf_s=1.4, seed=4242)
+    _full_check(make_case(wl), "bf16", fused=fused)
+    wl = CFG1.scaled(R=12, L=1, H=32, W=70, D=3, prompt_len=16, parents="uniform", seed=4243)
+    _full_check(make_case(wl), "fp32", fused=fused)
+
+
 def test_varying_beam_width_between_calls():
     wl = CFG1.scaled(H=2, W=96, D=4, prompt_len=64, seed=91)
     _full_check(make_case(wl, widths=[96, 17, 64, 5]), "fp32")
