@@ -129,7 +129,8 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     uint64_t* bars = reinterpret_cast<uint64_t*>(heads + HEADS_TOTAL);
     // bars: per S_0 / staging buffer b: S_0 in tensor memory, records staged, staging buffer read out;
     //       per ring slot s: full, MMA done, free
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 6 + 3 * SLOTS);
+    const uint32_t bar_s0_first = smem_u32(bars + 6 + 3 * SLOTS);   // the first segment's S_0, put there by all warps
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 7 + 3 * SLOTS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     auto bar_s0 = [&](int b) { return smem_u32(bars + b); };
     auto bar_stage = [&](int b) { return smem_u32(bars + 2 + b); };
@@ -149,6 +150,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             mbar_init(bar_done(s), 1);                // tcgen05.commit
             mbar_init(bar_free(s), 4);                // the four epilogue warps
         }
+        mbar_init(bar_s0_first, THREADS / 32);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -204,12 +206,36 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     };
-    // The first segment's S_0 is read by all warps before the launch's dependencies are waited for: the store is
-    // written only by the state calls (a copy or a prefill kernel), and a reorder launch always separates those
-    // from a decode.
-    if (n_segs > 0) load_s0(pair_begin, 0, warp >> 2, THREADS / 128, n_segs > 1);
-    __syncthreads();
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    // The first segment's S_0 is requested by all warps (one 32-column block each) before the launch's dependencies are
+    // waited for, and put into tensor memory after the first heads have been requested: the store is written only by
+    // the state calls (a copy or a prefill kernel), and a reorder launch always separates those from a decode.
+    static_assert(THREADS == 512, "one 32-column block of the first S_0 per warp");
+    float4 s0_first[8];
+    if (n_segs > 0) {
+        const int req = pair_begin / a.H, h = pair_begin - req * a.H;
+        const float* row = a.s0 + req * a.s0_req_stride + (long long)h * (DV * DK) + (long long)((warp & 3) * 32 + lane) * DK + (warp >> 2) * 32;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) s0_first[c] = __ldg(reinterpret_cast<const float4*>(row) + c);
+        if (n_segs > 1) {
+            const int nreq = (pair_begin + 1) / a.H, nh = (pair_begin + 1) - nreq * a.H;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(a.s0 + nreq * a.s0_req_stride + (long long)nh * (DV * DK) +
+                                                          (long long)((warp & 3) * 32 + lane) * DK + (warp >> 2) * 32));
+        }
+    }
+    auto put_first_s0 = [&]() {
+        if (n_segs == 0) return;
+        uint32_t v[32];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            v[4 * c] = __float_as_uint(round_tf32(s0_first[c].x)); v[4 * c + 1] = __float_as_uint(round_tf32(s0_first[c].y));
+            v[4 * c + 2] = __float_as_uint(round_tf32(s0_first[c].z)); v[4 * c + 3] = __float_as_uint(round_tf32(s0_first[c].w));
+        }
+        tmem_st32(tmem_base + S0_COL + (warp >> 2) * 32 + ((uint32_t)((warp & 3) * 32) << 16), v);
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_s0_first);
+    };
     // Everything below reads what earlier launches of the stream wrote (tokens, queries, ancestry rows).
     asm volatile("griddepcontrol.wait;" ::: "memory");
 #ifdef ONELA_SPAN
@@ -322,6 +348,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             if (1 < n_quads) gate1 = load_gate(u1);
             idx_next = load_idx(u0);
         }
+        put_first_s0();
         int cur_seg = -1, buf = 0, staged_levels = 0;
         bool staged_ready = false;
         long long plane_row0 = 0, own_row0 = 0;
@@ -473,6 +500,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             if (lane == 0) mbar_arrive(bar_s0(seg & 1));
         };
         if (n_segs > 0) stage_segment(0);
+        put_first_s0();
         if (n_segs > 1) {          // (doing this part later, or before the dependency wait with all warps, measured slower)
             stage_segment(1);
             prepare_s0(1);
@@ -490,9 +518,10 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 int mma_failed = 0;
                 if (lane == 0) {
                     bool ok = wait_or_abort(bar_full(s), use & 1, abort_flag);
-                    // segment 0's S_0 was complete before the main loop; segment seg >= 1 is use ((seg + 1) >> 1) - 1 of its
+                    // segment 0's S_0 has a barrier of its own; segment seg >= 1 is use ((seg + 1) >> 1) - 1 of its
                     // buffer's barrier
                     if (ok && seg_first && seg >= 1) ok = wait_or_abort(bar_s0(seg & 1), (((seg + 1) >> 1) - 1) & 1, abort_flag);
+                    if (ok && gi == g_begin) ok = wait_or_abort(bar_s0_first, 0, abort_flag);
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     if (ok) {
                         constexpr uint32_t idesc = idesc_tf32(GN);
