@@ -164,6 +164,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
+#ifdef ONELA_SPAN
+    if (threadIdx.x == 0) g_span[launch_id & 63][blockIdx.x][3] = gtime2();
+#endif
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next launch may set itself up under this one
 
     const int g_begin = part.begin[blockIdx.x], g_end = part.begin[blockIdx.x + 1];
@@ -236,11 +239,15 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_s0_first);
     };
-    // Everything below reads what earlier launches of the stream wrote (tokens, queries, ancestry rows).
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Each role waits for the launch's dependencies below (`dependency_wait`), before it reads anything earlier
+    // launches of the stream wrote (tokens, queries, ancestry rows).  Requests of lines into L2 are not reads in that
+    // sense - L2 is the point of coherence - and are made before it.
+    auto dependency_wait = [&]() {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
 #ifdef ONELA_SPAN
-    if (threadIdx.x == 0) g_span[launch_id & 63][blockIdx.x][2] = gtime2();
+        if (threadIdx.x == 0) g_span[launch_id & 63][blockIdx.x][2] = gtime2();
 #endif
+    };
 
     // How many of the oldest levels of a request's chains fit in `stage_cap` staged records (whole levels only), and
     // how many records that is.  Lane l looks at level l (one load latency for the whole chain); warp-uniform.
@@ -279,6 +286,18 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         // The heads of a quad (own record and query of its units) arrive by 16-byte async copies into the warp's
         // stage, one quad ahead of their use (each lane copies exactly the chunks it reads back); the lines of the
         // quad after that are requested into L2; the gates ride in registers.
+        auto request_heads = [&](const Unit& n) {        // the 128-byte lines of a quad's heads, into L2
+            if (lane < UPW * 6) {
+                const int un = lane / 6, item = lane % 6;
+                const int b2 = min(n.gip * GN + UPW * warp + un, a.W - 1);
+                const long long row2 = ((long long)n.req * a.W + b2) * a.H + n.h;
+                const char* p2 = item < 2 ? reinterpret_cast<const char*>(qbase) + row2 * (DK * 2)
+                                 : fused  ? (item < 4 ? static_cast<const char*>(a.k_in) + row2 * (DK * 2)
+                                                      : static_cast<const char*>(a.v_in) + row2 * (DV * 2))
+                                          : kv + ((long long)n.h * a.arena_slots + a.bases.base[n.req] + b2) * REC_BYTES + (item < 4 ? 0 : 256);
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(p2 + (item & 1) * 128));
+            }
+        };
         auto issue_head = [&](const Unit& u, const Unit& n, bool has_next) {
             const uint32_t dst = smem_u32(my_heads);
             const int bb = live_beam(u);
@@ -300,16 +319,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
 #pragma unroll
             for (int c = 0; c < NCH; ++c) cp_async16(dst + UPW * REC_BYTES + grp * (DK * 2) + (c * LPU + g) * 16, qr + c * LPU * 16);
             asm volatile("cp.async.commit_group;" ::: "memory");
-            if (has_next && lane < UPW * 6) {
-                const int un = lane / 6, item = lane % 6;
-                const int b2 = min(n.gip * GN + UPW * warp + un, a.W - 1);
-                const long long row2 = ((long long)n.req * a.W + b2) * a.H + n.h;
-                const char* p2 = item < 2 ? reinterpret_cast<const char*>(qbase) + row2 * (DK * 2)
-                                 : fused  ? (item < 4 ? static_cast<const char*>(a.k_in) + row2 * (DK * 2)
-                                                      : static_cast<const char*>(a.v_in) + row2 * (DV * 2))
-                                          : kv + ((long long)n.h * a.arena_slots + a.bases.base[n.req] + b2) * REC_BYTES + (item < 4 ? 0 : 256);
-                asm volatile("prefetch.global.L2 [%0];" ::"l"(p2 + (item & 1) * 128));
-            }
+            if (has_next) request_heads(n);
         };
         auto load_gate = [&](const Unit& u) {
             const int bb = live_beam(u);
@@ -342,6 +352,8 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         float2 gate0 = make_float2(1.f, 0.f), gate1 = gate0;
         Idx idx_next{};
         Unit u1 = next_unit(u0), u2 = next_unit(u1);
+        if (n_quads > 0) request_heads(u0);
+        dependency_wait();
         if (n_quads > 0) {
             issue_head(u0, u1, 1 < n_quads);
             gate0 = load_gate(u0);
@@ -472,6 +484,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         }
     } else {
         // =============================== EPILOGUE (+ MMA issue, + preparation of the next segments) ===============================
+        dependency_wait();
         const int quad = warp & 3;                    // tensor-memory lane quadrant of this warp
         const int i = quad * 32 + lane;               // output element (dv index) of this thread
         int staged_issued[2] = {0, 0};                // stagings requested per buffer (what teardown must wait for)
