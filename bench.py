@@ -141,7 +141,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
         wl = wl.scaled(L=args.layers)
     out_dtype = args.out_dtype or wl.dtype
     out_bytes = 4 if out_dtype == "fp32" else 2
-    run = WorkloadRun(wl, dev, out_dtype, flags=2 if args.force_generic else 0)
+    run = WorkloadRun(wl, dev, out_dtype, flags=(2 if args.force_generic else 0) | (4 if args.delta_records else 0))
     ctx = run.ctx
     run.prefill_states()
     S0 = {(r, l): ctx.onela_export_shared_state(r, l) for r in range(wl.R) for l in range(wl.L)}
@@ -256,13 +256,15 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
                            + wl.R * wl.L * wl.H * wl.dk * wl.dv * 4) / 2 ** 30),
                    "out_dtype": out_dtype, "launch": mode,
                    "per_layer_calls": "append_records + decode_step" if args.unfused else "append_decode_step (one launch)", "parallelism": f"replicas x{world} (requests are independent)",
-                   "tensor_core_path": bool(ctx.onela_uses_tensor_core_path())},
+                   "tensor_core_path": bool(ctx.onela_uses_tensor_core_path()),
+                   "record_format": "(alpha, delta, k), forward projection replay" if args.delta_records
+                                    else "(k, v, alpha, beta), backward query fold"},
         "clocks": {**clocks.summary(), "window": "sampled from the warm-up to the end of the timed legs"},
         "e2e": {"value": e2e["value"], "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                 "ms_per_step": e2e["ms_per_step"]},
         "gpu_launches": int(launches_per_step * args.steps),
         "roofline": {"bound": "hbm", "achieved": achieved_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": achieved_gbs / peak, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if not args.unfused else None,
+                     "frac": achieved_gbs / peak, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if not (args.unfused or args.delta_records or args.force_generic) else None,
                      "traffic_note": "ncu DRAM read+write bytes of one launch at the deepest call (depth %d), whose "
                                      "algorithmic bytes are %.1f MB; see profiles/" % (wl.D, per_depth[-1]["algorithmic"] / 1e6),
                      "peak_source": peak_src,
@@ -407,6 +409,9 @@ def main():
     ap.add_argument("--settle-seconds", type=float, default=1.0, help="extra untimed warm-up after the W steps")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling)")
     ap.add_argument("--force-generic", action="store_true", help="run the CUDA-core decode kernel")
+    ap.add_argument("--delta-records", action="store_true",
+                    help="(alpha, delta, k) records with forward projection replay (Section 3.2) instead of raw records "
+                         "with the backward fold: the CUDA-core comparison kernel")
     ap.add_argument("--profile", action="store_true", help="eager generations only, for ncu")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (kernel experiments)")

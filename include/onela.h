@@ -72,6 +72,15 @@ typedef int32_t onela_status;
 /* flags */
 #define ONELA_FLAG_DRY_RUN 1u       /* validate and advance host bookkeeping, launch nothing (host-logic tests) */
 #define ONELA_FLAG_FORCE_GENERIC 2u /* use the CUDA-core decode kernel even where the tensor-core kernel applies */
+/* Record format and replay order of Section 3.2 (Eq. 2-4): the arena keeps (alpha_t, delta_t, k_t) with
+ * delta_t = beta_t (v_t - alpha_t S_{t-1} k_t) in rec_dtype in place of v_t, and a decode call replays the two
+ * projection accumulators S q_t and S k_t forward from S_0 through the beam's records (oldest first).  delta_t
+ * depends on the parent state, so records can only be produced where the replay runs: in this mode
+ * onela_append_decode_step is the one call per layer and decode call; onela_append_records and onela_decode_step
+ * return ONELA_E_UNSUPPORTED.  dk == dv in {32, 64, 128}; CUDA cores only.  Later calls replay the ROUNDED
+ * delta, so with bf16 records the result drifts from the exact recurrence by about one bf16 rounding per record
+ * (the default raw-record format has no such term). */
+#define ONELA_FLAG_GTR_DELTA 4u
 
 typedef struct onela_config {
     int32_t num_requests; /* request slots */

@@ -70,6 +70,7 @@ struct onela_ctx {
     int32_t elem_bytes = 4;
 
     bool dry() const { return cfg.flags & ONELA_FLAG_DRY_RUN; }
+    bool gtr() const { return cfg.flags & ONELA_FLAG_GTR_DELTA; }   // (alpha, delta, k) records, forward replay
     long long table_req_stride() const { return 2LL * cfg.max_steps * cfg.max_beam; }
     long long s0_layer_floats() const { return (long long)cfg.num_heads * cfg.dv * cfg.dk; }
     float* s0_slot(int r, int l) const { return lay.s0 + ((long long)r * cfg.num_layers + l) * s0_layer_floats(); }
@@ -146,6 +147,8 @@ onela_status onela_create(const onela_config* cfg, void* workspace_dev, size_t w
     if (!config_sane(cfg) || !workspace_dev) return ONELA_E_INVAL;
     if (reinterpret_cast<uintptr_t>(workspace_dev) % kAlign != 0) return ONELA_E_INVAL;
     if (!decode_generic_supported(cfg->dk, cfg->dv, cfg->rec_dtype)) return ONELA_E_UNSUPPORTED;
+    if ((cfg->flags & ONELA_FLAG_GTR_DELTA) && !(cfg->dk == cfg->dv && (cfg->dk == 32 || cfg->dk == 64 || cfg->dk == 128)))
+        return ONELA_E_UNSUPPORTED;
     const Layout lay = carve(*cfg, static_cast<char*>(workspace_dev));
     if (workspace_bytes < lay.total_bytes) return ONELA_E_CAPACITY;
     onela_ctx* ctx = new (std::nothrow) onela_ctx();
@@ -158,7 +161,8 @@ onela_status onela_create(const onela_config* cfg, void* workspace_dev, size_t w
         r.has_state.assign(cfg->num_layers, 0);
         r.appended_depth.assign(cfg->num_layers, -1);
     }
-    ctx->tensor_core = decode_sm100_supported(cfg->dk, cfg->dv, cfg->rec_dtype) && !(cfg->flags & ONELA_FLAG_FORCE_GENERIC);
+    ctx->tensor_core = decode_sm100_supported(cfg->dk, cfg->dv, cfg->rec_dtype) &&
+                       !(cfg->flags & (ONELA_FLAG_FORCE_GENERIC | ONELA_FLAG_GTR_DELTA));
     *out = ctx;
     return ONELA_OK;
 }
@@ -295,6 +299,7 @@ onela_status onela_append_records(onela_ctx* ctx, int32_t req_begin, int32_t req
                                   const float* beta_dev, void* stream) {
     onela_status st = check_batch(ctx, req_begin, req_count);
     if (st != ONELA_OK) return st;
+    if (ctx->gtr()) return ONELA_E_UNSUPPORTED;   // delta records are produced by append_decode_step only
     const onela_config& c = ctx->cfg;
     if (layer < 0 || layer >= c.num_layers) return ONELA_E_INVAL;
     if (!k_dev || !v_dev || !alpha_dev || !beta_dev || !aligned16(k_dev) || !aligned16(v_dev)) return ONELA_E_INVAL;
@@ -359,8 +364,9 @@ onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count,
     a.max_beam = c.max_beam;
     for (int i = 0; i < req_count; ++i) a.bases.base[i] = ctx->req[req_begin + i].step_base.back();
     bool supported = true;
-    const cudaError_t e = ctx->tensor_core ? launch_decode_sm100_ws(a, c.out_dtype, s)
-                                           : launch_decode_generic(a, c.dk, c.dv, c.rec_dtype, c.out_dtype, &supported, s);
+    const cudaError_t e = ctx->gtr()         ? launch_decode_gtr(a, c.dk, c.dv, c.rec_dtype, c.out_dtype, &supported, s)
+                          : ctx->tensor_core ? launch_decode_sm100_ws(a, c.out_dtype, s)
+                                             : launch_decode_generic(a, c.dk, c.dv, c.rec_dtype, c.out_dtype, &supported, s);
     if (!supported) return ONELA_E_UNSUPPORTED;
     if (e != cudaSuccess) return ONELA_E_CUDA;
     ctx->launches++;
@@ -375,6 +381,7 @@ onela_status onela_decode_step(onela_ctx* ctx, int32_t req_begin, int32_t req_co
                                const void* q_dev, void* out_dev, void* stream) {
     onela_status st = check_batch(ctx, req_begin, req_count);
     if (st != ONELA_OK) return st;
+    if (ctx->gtr()) return ONELA_E_UNSUPPORTED;   // the forward replay needs the call's token: append_decode_step
     const onela_config& c = ctx->cfg;
     if (layer < 0 || layer >= c.num_layers) return ONELA_E_INVAL;
     if (!q_dev || !out_dev || !aligned16(q_dev) || !aligned16(out_dev)) return ONELA_E_INVAL;
@@ -408,7 +415,7 @@ onela_status onela_append_decode_step(onela_ctx* ctx, int32_t req_begin, int32_t
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if ((st = ctx->prepare(s)) != ONELA_OK) return st;
     if (!ctx->dry()) {
-        if (ctx->tensor_core) {
+        if (ctx->tensor_core || ctx->gtr()) {
             st = launch_decode(ctx, req_begin, req_count, layer, q_dev, out_dev, k_dev, v_dev, alpha_dev, beta_dev, s);
             if (st != ONELA_OK) return st;
         } else {   // shapes without the fused kernel: the copy kernel, then the decode kernel

@@ -84,6 +84,9 @@ cudaError_t launch_decode_generic(const DecodeArgs& a, int32_t dk, int32_t dv, i
                                   int32_t out_dtype, bool* supported, cudaStream_t stream);
 bool decode_generic_supported(int32_t dk, int32_t dv, int32_t rec_dtype);
 // tcgen05 tensor-core kernel (sm_100a): dk = dv = 128, bf16 records
+// forward projection replay over (alpha, delta, k) records (ONELA_FLAG_GTR_DELTA): append + decode of one layer
+cudaError_t launch_decode_gtr(const DecodeArgs& a, int32_t dk, int32_t dv, int32_t rec_dtype, int32_t out_dtype,
+                              bool* supported, cudaStream_t stream);
 bool decode_sm100_supported(int32_t dk, int32_t dv, int32_t rec_dtype);
 cudaError_t launch_decode_sm100_ws(const DecodeArgs& a, int32_t out_dtype, cudaStream_t stream);
 

@@ -1,0 +1,114 @@
+"""Parity of the (alpha, delta, k) record format with forward projection replay (Section 3.2, Eq. 2-4;
+ONELA_FLAG_GTR_DELTA) against the same fp64 full-state oracle as the default path, through the C ABI.
+
+With fp32 records the stored update vectors are exact to fp32 rounding and the outputs must match the oracle
+tightly; with bf16 records every stored delta carries one bf16 rounding, which later calls replay, so the bar
+is the path's stated 5e-3 (observed: a few 1e-3 with bf16 outputs).  Ancestry rows are bit-exact as always;
+the stored keys are the caller's bytes and the stored deltas match delta_t = beta_t (v_t - alpha_t S_{t-1} k_t)
+computed from the oracle's states."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2609_12399_b200 as P
+from paper_2609_12399_b200 import inputs
+
+from _cases import REL_L2_BAR, check_parity, expected_slots, make_case, rel_l2, run_library, run_oracle
+
+pytestmark = pytest.mark.gpu
+
+CFG0, CFG1 = inputs.WORKLOADS[0], inputs.WORKLOADS[1]
+
+
+def _check(case, out_dtype, tight=None, batched=True):
+    ref, chains = run_oracle(case)
+    outs, slots, ctx = run_library(case, out_dtype=out_dtype, flags=P.FLAG_GTR_DELTA, batched=batched, fused=True)
+    assert not ctx.onela_uses_tensor_core_path()
+    want = expected_slots(case, chains)
+    for key in want:
+        assert np.array_equal(slots[key], want[key]), f"ancestry rows of {key} differ"
+    worst = check_parity(case, outs, ref, tight=tight)
+    assert ctx.onela_poll_device_status() == (0, 0)
+    return worst, ctx
+
+
+def test_config0_fp32_records_are_tight():
+    worst, _ = _check(make_case(CFG0), "fp32", tight=5e-6)
+    assert worst > 0.0
+
+
+@pytest.mark.parametrize("out_dtype", ["fp32", "bf16"])
+def test_config1_bf16_records(out_dtype):
+    _check(make_case(CFG1), out_dtype)
+
+
+def test_fp32_records_other_shapes_and_ragged_widths():
+    wl = CFG1.scaled(R=2, L=2, H=3, dk=64, dv=64, dtype="fp32", W=37, D=4, prompt_len=48, parents="zipf", zipf_s=1.3, seed=61)
+    _check(make_case(wl), "fp32", tight=5e-6)
+    wl = CFG1.scaled(R=1, L=1, H=2, dtype="fp32", W=50, D=5, prompt_len=64, seed=62)
+    _check(make_case(wl, widths=[50, 7, 33, 64, 20]), "fp32", tight=5e-6, batched=False)
+
+
+def test_bf16_records_deep_chain_with_shared_ancestors():
+    wl = CFG1.scaled(R=2, H=4, W=96, D=8, prompt_len=128, parents="zipf", zipf_s=1.5, seed=63)
+    worst, _ = _check(make_case(wl), "fp32")
+    assert worst <= REL_L2_BAR
+
+
+def test_stored_records_are_key_bytes_and_update_vectors():
+    """The arena holds (k_t bit for bit | delta_t), gates (alpha_t, beta_t); delta_t is checked against
+    beta_t (v_t - alpha_t S_{t-1} k_t) with S_{t-1} the parent beam's state from the fp64 full-state recurrence."""
+    wl = CFG1.scaled(R=1, H=2, dtype="fp32", W=12, D=3, prompt_len=32, seed=64)
+    case = make_case(wl)
+    outs, slots, ctx = run_library(case, out_dtype="fp32", flags=P.FLAG_GTR_DELTA, fused=True)
+    c = ctx.cfg
+    al = lambda n: (n + 1023) // 1024 * 1024
+    n_idx = c.num_requests * c.max_steps * c.max_beam * 4
+    off_s0 = al(16) + al(2 * n_idx) + al(n_idx) + al(n_idx) + al(c.num_requests * (c.max_steps + 1) * 4)
+    off_gates = off_s0 + al(c.num_requests * c.num_layers * c.num_heads * c.dv * c.dk * 4)
+    off_kv = off_gates + al(c.num_layers * c.num_heads * c.arena_slots * 8)
+    ws = ctx.workspace[ctx.workspace_ptr - ctx.workspace.data_ptr():]
+    gates = ws[off_gates:off_gates + c.num_heads * c.arena_slots * 8].view(torch.float32).view(c.num_heads, c.arena_slots, 2).cpu()
+    kv = ws[off_kv:off_kv + c.num_heads * c.arena_slots * 1024].view(torch.float32).view(c.num_heads, c.arena_slots, 256).cpu()
+    S0 = case["S0"][(0, 0)].double().numpy()                      # [H, dv, dk]
+    states = {b: S0.copy() for b in range(1)}                      # per beam: [H, dv, dk]; call 0: all from S_0
+    prev = None
+    for t in range(wl.D):
+        tk = case["tok"][(0, 0, t)]
+        par = case["parents"][(0, t)]
+        base = ctx.onela_get_step_base(0, t)
+        new = {}
+        for b in range(wl.W):
+            S_par = S0 if t == 0 else prev[int(par[b])]
+            S_new = np.empty_like(S_par)
+            for h in range(wl.H):
+                k = tk["k"][b, h].double().numpy(); v = tk["v"][b, h].double().numpy()
+                a_, b_ = float(tk["alpha"][b, h]), float(tk["beta"][b, h])
+                delta = b_ * (v - a_ * (S_par[h] @ k))
+                S_new[h] = a_ * S_par[h] + np.outer(delta, k)     # Eq. 1 in the paper's record form
+                got = kv[h, base + b, 128:].double().numpy()
+                assert np.linalg.norm(got - delta) <= 2e-5 * max(np.linalg.norm(delta), 1e-3), (t, b, h)
+                assert torch.equal(kv[h, base + b, :128], tk["k"][b, h])
+                assert float(gates[h, base + b, 0]) == a_
+            new[b] = S_new
+        prev = new
+
+
+def test_separate_append_and_decode_are_refused_in_this_mode():
+    wl = CFG1.scaled(H=2, W=16, D=2, prompt_len=32)
+    case = make_case(wl)
+    cfg = P.make_config(wl.R, wl.L, wl.H, wl.dk, wl.dv, wl.W, wl.D, wl.dtype, "fp32", wl.R * wl.W * wl.D, P.FLAG_GTR_DELTA)
+    ctx = P.Onela(cfg, device="cuda")
+    ctx.onela_init_shared_state(0, 0, case["S0"][(0, 0)].cuda())
+    ctx.onela_reorder_beams(0, 1, None, wl.W)
+    tk = {n: x.cuda()[None] for n, x in case["tok"][(0, 0, 0)].items()}
+    q = case["q"][(0, 0, 0)].cuda()[None]
+    out = torch.empty((1, wl.W, wl.H, wl.dv), dtype=torch.float32, device="cuda")
+    with pytest.raises(P.OnelaError):
+        ctx.onela_append_records(0, 1, 0, tk["k"], tk["v"], tk["alpha"], tk["beta"])
+    with pytest.raises(P.OnelaError):
+        ctx.onela_decode_step(0, 1, 0, q, out)
+    ctx.onela_append_decode_step(0, 1, 0, tk["k"], tk["v"], tk["alpha"], tk["beta"], q, out)
+    ref = oracle.decode(case["S0"][(0, 0)], [case["tok"][(0, 0, 0)]], [None], case["q"][(0, 0, 0)])
+    assert rel_l2(out[0].cpu().numpy(), ref).max() <= REL_L2_BAR

@@ -116,6 +116,35 @@ def test_fused_append_decode_counts_as_the_append():
         o.onela_append_decode_step(0, 1, 0, FAKE, FAKE, FAKE, FAKE, None, FAKE)
 
 
+def test_delta_record_mode_takes_only_the_fused_call():
+    """(alpha, delta, k) records (Section 3.2) are produced where the replay runs: the separate append and decode
+    calls are refused, the fused call drives the same state machine; the format needs dk == dv in {32, 64, 128}."""
+    cfg = P.make_config(1, 2, 4, 32, 32, 8, 3, "fp32", "fp32", 64, P.FLAG_DRY_RUN | P.FLAG_GTR_DELTA)
+    o = P.Onela(cfg, device="cpu")
+    assert not o.onela_uses_tensor_core_path()
+    o.onela_init_shared_state(0, 0, FAKE)
+    o.onela_init_shared_state(0, 1, FAKE)
+    o.onela_reorder_beams(0, 1, None, 8)
+    with raises(binding.E_UNSUPPORTED):
+        o.onela_append_records(0, 1, 0, FAKE, FAKE, FAKE, FAKE)
+    with raises(binding.E_UNSUPPORTED):
+        o.onela_decode_step(0, 1, 0, FAKE, FAKE)
+    o.onela_append_decode_step(0, 1, 0, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE)
+    with raises(binding.E_ORDER):
+        o.onela_append_decode_step(0, 1, 0, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE)    # one append per layer and call
+    with raises(binding.E_ORDER):
+        o.onela_reorder_beams(0, 1, FAKE, 8)                                       # layer 1 has not appended yet
+    o.onela_append_decode_step(0, 1, 1, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE)
+    o.onela_reorder_beams(0, 1, FAKE, 8)
+    assert o.onela_get_step_base(0, 1) == 8
+    for (dk, dv) in [(128, 256), (256, 256)]:
+        bad = P.make_config(1, 1, 2, dk, dv, 8, 3, "bf16", "bf16", 64, P.FLAG_DRY_RUN | P.FLAG_GTR_DELTA)
+        with raises(binding.E_UNSUPPORTED):
+            P.Onela(bad, device="cpu")
+    tc = P.make_config(1, 1, 2, 128, 128, 8, 3, "bf16", "bf16", 64, P.FLAG_DRY_RUN | P.FLAG_GTR_DELTA)
+    assert not P.Onela(tc, device="cpu").onela_uses_tensor_core_path()
+
+
 def test_every_layer_with_state_must_append_before_next_call():
     o = ctx()
     o.onela_init_shared_state(0, 0, FAKE)
