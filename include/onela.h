@@ -25,7 +25,12 @@
  *    host object released by onela_destroy(), which never touches the workspace.
  *  - `stream` is a cudaStream_t passed as void*.  Every call is asynchronous and ordered on that
  *    stream; inputs may be reused as soon as the stream has passed the call.  Only
- *    onela_poll_device_status() synchronises.
+ *    onela_poll_device_status() synchronises.  The tensor-core decode kernel is launched with programmatic
+ *    stream serialisation: it may start while the previous kernel of the stream drains, but it reads only its
+ *    own shared-state store before it has waited for that kernel's completion, so stream order holds for every
+ *    tensor the caller passes.  A caller kernel that follows it AND is itself launched with programmatic stream
+ *    serialisation must wait for its grid dependency before it reads the decode outputs, as that launch mode
+ *    requires of any kernel.
  *  - Tensors are dense, row-major, last index contiguous.  q, k, v use cfg.rec_dtype, outputs
  *    cfg.out_dtype, gates and S_0 are fp32.  All tensor pointers must be 16-byte aligned.
  *  - Errors the host can see return a negative status and launch nothing.  Errors only the device can
