@@ -292,31 +292,68 @@ def run_e2e(args, run, S0, calls, outs, units_per_step, barrier) -> dict:
     hcalls = [{"parents": None if c["parents"] is None else pin(c["parents"]),
                "layers": [{n: pin(x) for n, x in lay.items()} for lay in c["layers"]]} for c in calls]
     houts = [torch.empty(o.shape, dtype=o.dtype).pin_memory() for o in outs]
-    dS0 = next(iter(S0.values())).clone()
-    dcall = {"parents": torch.empty_like(calls[-1]["parents"]) if wl.D > 1 else None,
-             "layers": [{n: torch.empty_like(x) for n, x in lay.items()} for lay in calls[0]["layers"]]}
+    # Double-buffered device staging and three streams (copies in, library calls, copies out): the upload of call
+    # t+1 and the read-back of call t-1 run under the kernels of call t.  Everything stays inside the timed region.
+    dS0 = [next(iter(S0.values())).clone() for _ in range(2)]
+    dcalls = [{"parents": torch.empty_like(calls[-1]["parents"]) if wl.D > 1 else None,
+               "layers": [{n: torch.empty_like(x) for n, x in lay.items()} for lay in calls[0]["layers"]]} for _ in range(2)]
+    douts = [outs, [torch.empty_like(o) for o in outs]]
     h2d = sum(v.numel() * v.element_size() for v in hS0.values())
     for c in hcalls:
         h2d += 0 if c["parents"] is None else c["parents"].numel() * 4
         h2d += sum(x.numel() * x.element_size() for lay in c["layers"] for x in lay.values())
     d2h = sum(o.numel() * o.element_size() for o in houts) * wl.D
+    comp = torch.cuda.current_stream()
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
 
     def generation():
+        start = torch.cuda.Event()
+        start.record(comp)
+        s_in.wait_event(start)
+        s_out.wait_event(start)
         ctx.onela_reset()
-        for key, hS in hS0.items():
-            dS0.copy_(hS, non_blocking=True)
-            ctx.onela_init_shared_state(key[0], key[1], dS0)
-        for hc in hcalls:
-            stage = {"parents": None, "layers": dcall["layers"]}
-            if hc["parents"] is not None:
-                dcall["parents"].copy_(hc["parents"], non_blocking=True)
-                stage["parents"] = dcall["parents"]
-            for dl, hl in zip(dcall["layers"], hc["layers"]):
-                for n in dl:
-                    dl[n].copy_(hl[n], non_blocking=True)
-            run.run_call(stage, outs, fused=not args.unfused)
-            for ho, o in zip(houts, outs):
-                ho.copy_(o, non_blocking=True)
+        state_used = [None, None]
+        for i, (key, hS) in enumerate(hS0.items()):
+            with torch.cuda.stream(s_in):
+                if state_used[i % 2] is not None:
+                    s_in.wait_event(state_used[i % 2])          # the store call has read this staging buffer
+                dS0[i % 2].copy_(hS, non_blocking=True)
+                up = torch.cuda.Event()
+                up.record(s_in)
+            comp.wait_event(up)
+            ctx.onela_init_shared_state(key[0], key[1], dS0[i % 2])
+            state_used[i % 2] = torch.cuda.Event()
+            state_used[i % 2].record(comp)
+        computed, read_back = [None, None], [None, None]
+        for t, hc in enumerate(hcalls):
+            b = t % 2
+            dc = dcalls[b]
+            with torch.cuda.stream(s_in):
+                if computed[b] is not None:
+                    s_in.wait_event(computed[b])                # call t-2 has consumed this staging buffer
+                stage = {"parents": None, "layers": dc["layers"]}
+                if hc["parents"] is not None:
+                    dc["parents"].copy_(hc["parents"], non_blocking=True)
+                    stage["parents"] = dc["parents"]
+                for dl, hl in zip(dc["layers"], hc["layers"]):
+                    for n in dl:
+                        dl[n].copy_(hl[n], non_blocking=True)
+                up = torch.cuda.Event()
+                up.record(s_in)
+            comp.wait_event(up)
+            if read_back[b] is not None:
+                comp.wait_event(read_back[b])                   # call t-2's outputs have left this buffer
+            run.run_call(stage, douts[b], fused=not args.unfused)
+            computed[b] = torch.cuda.Event()
+            computed[b].record(comp)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(computed[b])
+                for ho, o in zip(houts, douts[b]):
+                    ho.copy_(o, non_blocking=True)
+                read_back[b] = torch.cuda.Event()
+                read_back[b].record(s_out)
+        comp.wait_stream(s_in)
+        comp.wait_stream(s_out)
 
     for _ in range(max(1, min(args.warmup, 2))):
         generation()
