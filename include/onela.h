@@ -138,6 +138,20 @@ onela_status onela_export_shared_state(onela_ctx* ctx, int32_t request, int32_t 
 onela_status onela_reorder_beams(onela_ctx* ctx, int32_t req_begin, int32_t req_count, const int32_t* parents_dev,
                                  int32_t W_new, void* stream);
 
+/* Global beam selection feeding onela_reorder_beams ("all active beams are expanded over the codebook and the
+ * global top-k candidates are retained", Section 2.2): for each request of [req_begin, req_begin+req_count),
+ * candidate (p, c) scores beam_scores_dev[req][p] + cand_logp_dev[req][p][c], added in fp32, with p over the
+ * W_prev beams of the request's current decode call (W_prev = 1, the root, before the first call) and c over the C
+ * codes.  The W_new best are written best first: parents_out_dev [req_count][W_new] int32 (the parent map pi_t in
+ * the form reorder_beams takes), codes_out_dev [req_count][W_new] int32, scores_out_dev [req_count][W_new] fp32.
+ * Equal scores go to the smaller flat index p * C + c; NaN ranks below every number; -0 equals +0.  Reads and
+ * writes only the caller's buffers and changes no state of the context, so selection, reorder and the layers'
+ * decode launches of a step can be captured in one CUDA graph.  1 <= W_new <= min(1024, W_prev * C), else
+ * ONELA_E_CAPACITY. */
+onela_status onela_select_beams(onela_ctx* ctx, int32_t req_begin, int32_t req_count, const float* beam_scores_dev,
+                                const float* cand_logp_dev, int32_t C, int32_t W_new, int32_t* parents_out_dev,
+                                int32_t* codes_out_dev, float* scores_out_dev, void* stream);
+
 /* Append this call's transition records for one layer ("appends only the compact record ... rather
  * than writing back a full recurrent state", Section 3.4): k_dev [req_count][W][H][dk],
  * v_dev [req_count][W][H][dv] in rec_dtype, alpha_dev, beta_dev [req_count][W][H] fp32.  Values are

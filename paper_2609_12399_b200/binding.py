@@ -49,6 +49,8 @@ PROTOTYPES = {
                                              c_int32, c_void_p]),
     "onela_export_shared_state": (c_int32, [c_void_p, c_int32, c_int32, c_void_p, c_void_p]),
     "onela_reorder_beams": (c_int32, [c_void_p, c_int32, c_int32, c_void_p, c_int32, c_void_p]),
+    "onela_select_beams": (c_int32, [c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p,
+                                     c_void_p, c_void_p]),
     "onela_append_records": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
                                        c_void_p]),
     "onela_append_decode_step": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -191,6 +193,18 @@ class Onela:
         p = None if parents is None else self._ptr(parents, torch.int32, (req_count, W_new), "parents")
         _check(self.lib.onela_reorder_beams(self.handle, req_begin, req_count, p, W_new, self._s(stream)),
                "onela_reorder_beams")
+
+    def onela_select_beams(self, req_begin, req_count, beam_scores, cand_logp, C, W_new, parents_out, codes_out, scores_out,
+                           stream=None):
+        depth, W = self._width(req_begin)
+        W_prev = W if depth >= 1 else 1
+        _check(self.lib.onela_select_beams(
+            self.handle, req_begin, req_count,
+            self._ptr(beam_scores, torch.float32, (req_count, W_prev), "beam_scores"),
+            self._ptr(cand_logp, torch.float32, (req_count, W_prev, C), "cand_logp"), C, W_new,
+            self._ptr(parents_out, torch.int32, (req_count, W_new), "parents_out"),
+            self._ptr(codes_out, torch.int32, (req_count, W_new), "codes_out"),
+            self._ptr(scores_out, torch.float32, (req_count, W_new), "scores_out"), self._s(stream)), "onela_select_beams")
 
     def onela_append_records(self, req_begin, req_count, layer, k, v, alpha, beta, stream=None):
         c = self.cfg

@@ -1,6 +1,7 @@
 // Host side of the C ABI: context, workspace carve-up, per-request state machine, slot allocation and
 // kernel dispatch.  No device memory is allocated here; every launch goes to the caller's stream.
 #include <algorithm>
+#include <cstdint>
 #include <new>
 #include <vector>
 
@@ -53,6 +54,8 @@ Layout carve(const onela_config& c, char* base) {
     l.s0 = reinterpret_cast<float*>(take((size_t)c.num_requests * c.num_layers * c.num_heads * c.dv * c.dk * sizeof(float)));
     l.gates = reinterpret_cast<float2*>(take((size_t)c.num_layers * c.num_heads * (size_t)c.arena_slots * sizeof(float2)));
     l.kv = take((size_t)c.num_layers * c.num_heads * (size_t)c.arena_slots * (c.dk + c.dv) * es);
+    l.select_scratch = reinterpret_cast<unsigned long long*>(
+        take((size_t)c.num_requests * ONELA_SELECT_PARTS * ONELA_SELECT_CAP * sizeof(unsigned long long)));
     l.total_bytes = off;
     return l;
 }
@@ -291,6 +294,28 @@ onela_status onela_reorder_beams(onela_ctx* ctx, int32_t req_begin, int32_t req_
         r.step_width.push_back(W_new);
     }
     ctx->cursor += (int64_t)req_count * W_new;
+    return ONELA_OK;
+}
+
+onela_status onela_select_beams(onela_ctx* ctx, int32_t req_begin, int32_t req_count, const float* beam_scores_dev,
+                                const float* cand_logp_dev, int32_t C, int32_t W_new, int32_t* parents_out_dev,
+                                int32_t* codes_out_dev, float* scores_out_dev, void* stream) {
+    onela_status st = check_batch(ctx, req_begin, req_count);
+    if (st != ONELA_OK) return st;
+    if (!beam_scores_dev || !cand_logp_dev || !parents_out_dev || !codes_out_dev || !scores_out_dev || C < 1 || W_new < 1)
+        return ONELA_E_INVAL;
+    const ReqState& r0 = ctx->req[req_begin];
+    const int64_t W_prev = r0.depth >= 1 ? r0.W : 1;
+    if (W_prev * C > (int64_t)ONELA_SELECT_PARTS * 4096) return ONELA_E_CAPACITY;
+    if (W_new > ONELA_SELECT_CAP || W_new > W_prev * C) return ONELA_E_CAPACITY;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if ((st = ctx->prepare(s)) != ONELA_OK) return st;
+    if (ctx->dry()) return ONELA_OK;
+    if (launch_select(beam_scores_dev, cand_logp_dev, req_count, (int32_t)W_prev, C, W_new,
+                      ctx->lay.select_scratch + (size_t)req_begin * ONELA_SELECT_PARTS * ONELA_SELECT_CAP, parents_out_dev,
+                      codes_out_dev, scores_out_dev, s) != cudaSuccess)
+        return ONELA_E_CUDA;
+    ctx->launches += (W_prev * C > 4096) ? 2 : 1;
     return ONELA_OK;
 }
 

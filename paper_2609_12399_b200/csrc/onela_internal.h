@@ -19,6 +19,7 @@ struct Layout {
     float* s0;         // [request][layer][head][dv*dk] fp32
     float2* gates;     // [layer][head][arena_slots] (alpha, beta)
     char* kv;          // [layer][head][arena_slots][dk + dv] in rec_dtype: one row = k | v of one record
+    unsigned long long* select_scratch;   // [request][ONELA_SELECT_PARTS][ONELA_SELECT_CAP]: partial results of beam selection
     size_t total_bytes;
 };
 
@@ -66,6 +67,15 @@ cudaError_t launch_dedupe(const int32_t* tables_cur_req0, long long table_req_st
                           int32_t depth, int32_t max_beam, cudaStream_t stream);
 cudaError_t launch_export_chains(const int32_t* table_cur, int32_t W, int32_t depth, int32_t max_beam,
                                  int32_t* slots_out, cudaStream_t stream);
+
+// global beam selection: the W_new best (parent, code) pairs per request, best first (see onela_select.cu).
+// `scratch` ([request][ONELA_SELECT_PARTS][ONELA_SELECT_CAP] 64-bit words) is used when a request has more than
+// 4096 candidates; at most ONELA_SELECT_PARTS * 4096 candidates per request.
+#define ONELA_SELECT_CAP 1024
+#define ONELA_SELECT_PARTS 256
+cudaError_t launch_select(const float* beam_scores, const float* cand_logp, int32_t req_count, int32_t W_prev, int32_t C,
+                          int32_t W_new, unsigned long long* scratch, int32_t* parents, int32_t* codes, float* scores,
+                          cudaStream_t stream);
 
 // record / state kernels
 cudaError_t launch_append(const void* k, const void* v, const float* alpha, const float* beta, char* kv_plane,

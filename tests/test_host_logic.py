@@ -69,7 +69,8 @@ def test_workspace_carve_up_size():
     arena = 16 * 32 * (4 * 512 * 8) * 520
     tables = 4 * 2 * 8 * 512 * 4
     index = 2 * (4 * 8 * 512 * 4) + 4 * 9 * 4          # distinct-record index: positions, slot list, level offsets
-    assert s0 + arena + tables + index <= n <= s0 + arena + tables + index + 8 * 1024
+    select = 4 * 256 * 1024 * 8                        # beam selection: per request 256 partial lists of 1024 candidates
+    assert s0 + arena + tables + index + select <= n <= s0 + arena + tables + index + select + 9 * 1024
 
 
 def test_call_order_is_enforced():
@@ -143,6 +144,28 @@ def test_delta_record_mode_takes_only_the_fused_call():
             P.Onela(bad, device="cpu")
     tc = P.make_config(1, 1, 2, 128, 128, 8, 3, "bf16", "bf16", 64, P.FLAG_DRY_RUN | P.FLAG_GTR_DELTA)
     assert not P.Onela(tc, device="cpu").onela_uses_tensor_core_path()
+
+
+def test_select_beams_argument_checks():
+    """Selection reads the request's current beam width (1, the root, before the first call), changes no state,
+    and refuses widths it cannot deliver."""
+    o = ctx(W=8)
+    o.onela_init_shared_state(0, 0, FAKE)
+    o.onela_select_beams(0, 1, FAKE, FAKE, 16, 8, FAKE, FAKE, FAKE)               # root x 16 codes -> 8 beams
+    with raises(binding.E_CAPACITY):
+        o.onela_select_beams(0, 1, FAKE, FAKE, 4, 8, FAKE, FAKE, FAKE)            # only 1 x 4 candidates
+    with raises(binding.E_INVAL):
+        o.onela_select_beams(0, 1, FAKE, FAKE, 0, 8, FAKE, FAKE, FAKE)
+    with raises(binding.E_INVAL):
+        o.onela_select_beams(0, 1, FAKE, None, 16, 8, FAKE, FAKE, FAKE)
+    o.onela_reorder_beams(0, 1, None, 8)
+    o.onela_append_records(0, 1, 0, FAKE, FAKE, FAKE, FAKE)
+    o.onela_select_beams(0, 1, FAKE, FAKE, 4, 8, FAKE, FAKE, FAKE)                # now 8 x 4 candidates
+    with raises(binding.E_CAPACITY):
+        o.onela_select_beams(0, 1, FAKE, FAKE, 4, 33, FAKE, FAKE, FAKE)
+    with raises(binding.E_CAPACITY):
+        o.onela_select_beams(0, 1, FAKE, FAKE, 1024, 1025, FAKE, FAKE, FAKE)      # more survivors than the kernel keeps
+    o.onela_reorder_beams(0, 1, FAKE, 8)                                          # the call order is untouched
 
 
 def test_every_layer_with_state_must_append_before_next_call():
