@@ -152,6 +152,25 @@ onela_status onela_select_beams(onela_ctx* ctx, int32_t req_begin, int32_t req_c
                                 const float* cand_logp_dev, int32_t C, int32_t W_new, int32_t* parents_out_dev,
                                 int32_t* codes_out_dev, float* scores_out_dev, void* stream);
 
+/* onela_select_beams for callers that cannot hand the library a workspace.  (The paper has no counterpart: this
+ * is a packaging variant, not part of the method.)  Some hosts may not allocate device memory where selection
+ * runs: a serving process that gave every byte of the GPU to its own pool at start-up, a plug-in that is called
+ * on a stream it does not own and must not trigger cudaMalloc's device-wide synchronisation, a real-time loop
+ * with an allocation ban.  They have no onela context either, so the call takes the shapes directly
+ * (beam_scores_dev [req_count][W_prev], cand_logp_dev [req_count][W_prev][C], outputs [req_count][W_new], as in
+ * onela_select_beams) and keeps its partial results in an array built into the library: 4 MiB of every GPU that
+ * loads the library, held until the process exits.  Limits, fixed at build time: req_count <= 2,
+ * W_prev * C <= 1,048,576 candidates per request, W_new <= 1024; anything larger returns ONELA_E_CAPACITY and
+ * launches nothing (split the batch, or use onela_select_beams).  The call allocates nothing and frees nothing.
+ * The first call on a device looks the array's device address up; make that call before any stream capture
+ * begins on that device.  All calls share the one array: it keeps whatever the last call left (nothing in it has
+ * to start at zero), and two calls that overlap on the GPU - different streams, or a call inside a graph that is
+ * replayed while another call runs - race on it; keep them ordered on one stream or by events.  Results are those
+ * of onela_select_beams, bit for bit. */
+onela_status onela_select_beams_static(const float* beam_scores_dev, const float* cand_logp_dev, int32_t req_count,
+                                       int32_t W_prev, int32_t C, int32_t W_new, int32_t* parents_out_dev,
+                                       int32_t* codes_out_dev, float* scores_out_dev, void* stream);
+
 /* Append this call's transition records for one layer ("appends only the compact record ... rather
  * than writing back a full recurrent state", Section 3.4): k_dev [req_count][W][H][dk],
  * v_dev [req_count][W][H][dv] in rec_dtype, alpha_dev, beta_dev [req_count][W][H] fp32.  Values are

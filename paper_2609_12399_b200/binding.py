@@ -49,6 +49,8 @@ PROTOTYPES = {
                                              c_int32, c_void_p]),
     "onela_export_shared_state": (c_int32, [c_void_p, c_int32, c_int32, c_void_p, c_void_p]),
     "onela_reorder_beams": (c_int32, [c_void_p, c_int32, c_int32, c_void_p, c_int32, c_void_p]),
+    "onela_select_beams_static": (c_int32, [c_void_p, c_void_p, c_int32, c_int32, c_int32, c_int32, c_void_p, c_void_p,
+                                            c_void_p, c_void_p]),
     "onela_select_beams": (c_int32, [c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p,
                                      c_void_p, c_void_p]),
     "onela_append_records": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -100,6 +102,20 @@ def make_config(num_requests, num_layers, num_heads, dk, dv, max_beam, max_steps
                 arena_slots, flags=0) -> OnelaConfig:
     return OnelaConfig(num_requests, num_layers, num_heads, dk, dv, max_beam, max_steps,
                        _DTYPE_CODE[rec_dtype], _DTYPE_CODE[out_dtype], arena_slots, flags)
+
+
+def onela_select_beams_static(beam_scores, cand_logp, W_new, parents_out, codes_out, scores_out, stream=None) -> None:
+    """Beam selection for callers without a workspace or a context (see onela.h): shapes are read off the tensors
+    (beam_scores [R, W_prev] fp32, cand_logp [R, W_prev, C] fp32, outputs [R, W_new]); allocates nothing."""
+    R, W_prev, C = cand_logp.shape
+    for t, dt, shape, name in ((beam_scores, torch.float32, (R, W_prev), "beam_scores"), (cand_logp, torch.float32, (R, W_prev, C), "cand_logp"),
+                               (parents_out, torch.int32, (R, W_new), "parents_out"), (codes_out, torch.int32, (R, W_new), "codes_out"),
+                               (scores_out, torch.float32, (R, W_new), "scores_out")):
+        if t.device.type != "cuda" or t.dtype != dt or tuple(t.shape) != shape or not t.is_contiguous():
+            raise ValueError(f"{name}: expected a contiguous CUDA {dt} tensor of shape {shape}")
+    _check(load_library().onela_select_beams_static(
+        c_void_p(beam_scores.data_ptr()), c_void_p(cand_logp.data_ptr()), R, W_prev, C, W_new, c_void_p(parents_out.data_ptr()),
+        c_void_p(codes_out.data_ptr()), c_void_p(scores_out.data_ptr()), c_void_p(_stream_ptr(stream))), "onela_select_beams_static")
 
 
 def onela_workspace_bytes(cfg: OnelaConfig) -> int:

@@ -11,6 +11,8 @@
 // Two launches per call: `select_part_kernel` cuts a request's candidates into parts of 4096 and leaves each part's
 // own top-k (unordered) in a scratch area of the workspace; `select_merge_kernel` (one CTA per request) selects
 // among those and orders the survivors with a bitonic sort.  A request with a single part skips the scratch.
+#include <mutex>
+
 #include "onela_internal.h"
 
 namespace onela {
@@ -189,3 +191,57 @@ cudaError_t launch_select(const float* beam_scores, const float* cand_logp, int3
 }
 
 }  // namespace onela
+
+// ---------------------------------------------------------------------------------------------------------------
+// Beam selection without a workspace (declared in onela.h as onela_select_beams_static).
+//
+// The partial lists go to an array that is part of the library image instead of the caller's workspace.  Its size is
+// fixed when the library is built: room for STATIC_REQUESTS requests of the same candidate count the workspace
+// version takes (ONELA_SELECT_PARTS parts of 4096 candidates, ONELA_SELECT_CAP survivors each) = 4 MiB, which
+// every GPU that loads the library holds until the process ends.  In host code the array's name is only a handle;
+// the device address comes from cudaGetSymbolAddress, asked for once per device on that device's first call.
+namespace onela {
+namespace {
+
+constexpr int STATIC_REQUESTS = 2;
+static __device__ __align__(256) unsigned long long g_static_select_scratch[(size_t)STATIC_REQUESTS * ONELA_SELECT_PARTS * ONELA_SELECT_CAP];
+
+constexpr int MAX_DEVICES = 64;
+std::mutex g_static_mutex;
+unsigned long long* g_static_ptr[MAX_DEVICES] = {};
+
+// device address of the array on the current device; nullptr when the runtime refuses
+unsigned long long* static_scratch_of_current_device() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return nullptr;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_select_scratch) != cudaSuccess) return nullptr;
+        g_static_ptr[dev] = static_cast<unsigned long long*>(p);
+    }
+    return g_static_ptr[dev];
+}
+
+}  // namespace
+}  // namespace onela
+
+extern "C" onela_status onela_select_beams_static(const float* beam_scores_dev, const float* cand_logp_dev, int32_t req_count,
+                                                  int32_t W_prev, int32_t C, int32_t W_new, int32_t* parents_out_dev,
+                                                  int32_t* codes_out_dev, float* scores_out_dev, void* stream) {
+    using namespace onela;
+    if (!beam_scores_dev || !cand_logp_dev || !parents_out_dev || !codes_out_dev || !scores_out_dev) return ONELA_E_INVAL;
+    if (req_count < 1 || W_prev < 1 || C < 1 || W_new < 1) return ONELA_E_INVAL;
+    // beyond what the built-in array holds: the caller has to use onela_select_beams with a workspace, or split the batch
+    if (req_count > STATIC_REQUESTS) return ONELA_E_CAPACITY;
+    if ((int64_t)W_prev * C > (int64_t)ONELA_SELECT_PARTS * 4096) return ONELA_E_CAPACITY;
+    if (W_new > ONELA_SELECT_CAP || W_new > (int64_t)W_prev * C) return ONELA_E_CAPACITY;
+    unsigned long long* scratch = static_scratch_of_current_device();
+    if (!scratch) return ONELA_E_CUDA;
+    // nothing in the array has to start at zero: every word the merge step reads is written by the part step of
+    // the same call
+    if (launch_select(beam_scores_dev, cand_logp_dev, req_count, W_prev, C, W_new, scratch, parents_out_dev, codes_out_dev,
+                      scores_out_dev, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return ONELA_E_CUDA;
+    return ONELA_OK;
+}
