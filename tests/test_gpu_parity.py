@@ -89,6 +89,15 @@ def test_many_short_segments_per_cta(fused):
     _full_check(make_case(wl), "fp32", fused=fused)
 
 
+def test_degenerate_shapes():
+    """A single beam; the largest batch one call takes (64 requests) with one head and one beam each; one group
+    that is exactly full (48 beams) and one that has a single beam in its second group (49)."""
+    _full_check(make_case(CFG1.scaled(H=2, W=1, D=3, prompt_len=32, seed=701)), "fp32")
+    _full_check(make_case(CFG1.scaled(R=64, H=1, W=1, D=2, prompt_len=8, seed=702)), "bf16", fused=True)
+    _full_check(make_case(CFG1.scaled(H=2, W=48, D=2, prompt_len=32, seed=703)), "fp32", fused=True)
+    _full_check(make_case(CFG1.scaled(H=2, W=49, D=2, prompt_len=32, parents="zipf", zipf_s=2.0, seed=704)), "fp32", fused=True)
+
+
 def test_varying_beam_width_between_calls():
     wl = CFG1.scaled(H=2, W=96, D=4, prompt_len=64, seed=91)
     _full_check(make_case(wl, widths=[96, 17, 64, 5]), "fp32")
