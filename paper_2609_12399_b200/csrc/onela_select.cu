@@ -43,6 +43,8 @@ struct ScoreSource {     // composites computed from the caller's scores; item i
 };
 struct SelectShared {
     unsigned int hist[256];
+    unsigned int suffix[256];
+    unsigned int warp_total[8];
     unsigned long long sel[SEL_CAP];
     unsigned long long prefix;
     unsigned int k, count, equal;
@@ -61,6 +63,7 @@ __device__ void select_topk(const Src& src, uint32_t n, int k, SelectShared& sh)
         if (tid < 256) sh.hist[tid] = 0u;
         __syncthreads();
         const unsigned long long prefix = sh.prefix;
+        const unsigned want = sh.k;               // (read here: the bin search below rewrites it)
         const unsigned long long hi_mask = p == 7 ? 0ull : (~0ull << (8 * (p + 1)));
         for (uint32_t i = tid; i < n_padded; i += SEL_THREADS) {
             // whole warps stay in the loop (padding iterations carry no candidate) so the peer vote is complete
@@ -76,16 +79,28 @@ __device__ void select_topk(const Src& src, uint32_t n, int k, SelectShared& sh)
             }
         }
         __syncthreads();
-        if (tid == 0) {
-            unsigned want = sh.k, above = 0;
-            int b = 255;
-            for (; b > 0; --b) {
-                if (above + sh.hist[b] >= want) break;
-                above += sh.hist[b];
+        // the bin that holds the k-th largest: suffix counts over the 256 bins (bin >= b), by the first eight warps
+        if (tid < 256) {
+            unsigned v = sh.hist[tid];
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const unsigned up = __shfl_down_sync(0xffffffffu, v, off);
+                if ((tid & 31) + off < 32) v += up;
             }
-            sh.prefix = prefix | ((unsigned long long)b << (8 * p));
-            sh.k = want - above;
-            sh.equal = sh.hist[b];
+            if ((tid & 31) == 0) sh.warp_total[tid >> 5] = v;      // lane 0 holds its warp's whole count
+            sh.suffix[tid] = v;
+        }
+        __syncthreads();
+        if (tid < 256) {
+            unsigned higher = 0;
+            for (int w = (tid >> 5) + 1; w < 8; ++w) higher += sh.warp_total[w];
+            const unsigned here = sh.suffix[tid] + higher;                                   // candidates in bins >= tid
+            const unsigned next = here - sh.hist[tid];                                       // ... in bins > tid
+            if (here >= want && next < want) {                                               // exactly one bin qualifies
+                sh.prefix = prefix | ((unsigned long long)tid << (8 * p));
+                sh.k = want - next;
+                sh.equal = sh.hist[tid];
+            }
         }
         __syncthreads();
         // the score word is fixed and exactly the candidates that share it are still wanted: no tie straddles the cut
@@ -106,12 +121,14 @@ __device__ void select_topk(const Src& src, uint32_t n, int k, SelectShared& sh)
 __device__ void sort_and_emit(SelectShared& sh, int k, const float* bs, const float* lp, int C, int32_t* parents,
                               int32_t* codes, float* scores) {
     const int tid = threadIdx.x;
-    for (int i = tid; i < SEL_CAP; i += SEL_THREADS)
+    int n_sort = 2;
+    while (n_sort < k) n_sort <<= 1;                        // the sort runs over the next power of two
+    for (int i = tid; i < n_sort; i += SEL_THREADS)
         if (i >= k) sh.sel[i] = 0ull;
     __syncthreads();
-    for (int size = 2; size <= SEL_CAP; size <<= 1) {       // bitonic sort, descending
+    for (int size = 2; size <= n_sort; size <<= 1) {        // bitonic sort, descending
         for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            for (int i = tid; i < SEL_CAP / 2; i += SEL_THREADS) {
+            for (int i = tid; i < n_sort / 2; i += SEL_THREADS) {
                 const int lo = 2 * i - (i & (stride - 1)), hi = lo + stride;
                 const bool desc = (lo & size) == 0;
                 const unsigned long long x = sh.sel[lo], y = sh.sel[hi];
