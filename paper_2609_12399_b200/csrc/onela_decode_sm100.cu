@@ -150,7 +150,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             mbar_init(bar_done(s), 1);                // tcgen05.commit
             mbar_init(bar_free(s), 4);                // the four epilogue warps
         }
-        mbar_init(bar_s0_first, THREADS / 32);
+        mbar_init(bar_s0_first, 16);                  // the sixteen warps that bring the first S_0 in
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -212,9 +212,10 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     // The first segment's S_0 is requested by all warps (one 32-column block each) before the launch's dependencies are
     // waited for, and put into tensor memory after the first heads have been requested: the store is written only by
     // the state calls (a copy or a prefill kernel), and a reorder launch always separates those from a decode.
-    static_assert(THREADS == 512, "one 32-column block of the first S_0 per warp");
+    static_assert(THREADS >= 512, "the first sixteen warps take one 32-column block of the first S_0 each");
+    const bool s0_mine = warp < 16;
     float4 s0_first[8];
-    if (n_segs > 0) {
+    if (n_segs > 0 && s0_mine) {
         const int req = pair_begin / a.H, h = pair_begin - req * a.H;
         const float* row = a.s0 + req * a.s0_req_stride + (long long)h * (DV * DK) + (long long)((warp & 3) * 32 + lane) * DK + (warp >> 2) * 32;
 #pragma unroll
@@ -226,7 +227,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         }
     }
     auto put_first_s0 = [&]() {
-        if (n_segs == 0) return;
+        if (n_segs == 0 || !s0_mine) return;
         uint32_t v[32];
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
