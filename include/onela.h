@@ -138,6 +138,16 @@ onela_status onela_export_shared_state(onela_ctx* ctx, int32_t request, int32_t 
 onela_status onela_reorder_beams(onela_ctx* ctx, int32_t req_begin, int32_t req_count, const int32_t* parents_dev,
                                  int32_t W_new, void* stream);
 
+/* Give a finished request's record slots back (the paper is silent on reclamation; the reading taken: once a
+ * request's generation is over its records are dead).  Host bookkeeping only: every slot range the request was
+ * given by its reorder_beams calls returns to the context, the request drops its beams and its stored states (it
+ * needs init/prefill_shared_state again before it decodes).  Later reorder_beams calls place a request's W_new
+ * slots in the lowest released range that holds them and fall back on the bump cursor; ranges that touch are
+ * merged, and a range that reaches the cursor lowers it.  Kernels already enqueued that read the released records
+ * finish before later calls overwrite the slots as long as all calls go to one stream (or are ordered by events).
+ * A request slot that is re-initialised WITHOUT being released keeps its old slots occupied until onela_reset. */
+onela_status onela_release_request(onela_ctx* ctx, int32_t request);
+
 /* Global beam selection feeding onela_reorder_beams ("all active beams are expanded over the codebook and the
  * global top-k candidates are retained", Section 2.2): for each request of [req_begin, req_begin+req_count),
  * candidate (p, c) scores beam_scores_dev[req][p] + cand_logp_dev[req][p][c], added in fp32, with p over the

@@ -49,6 +49,7 @@ PROTOTYPES = {
                                              c_int32, c_void_p]),
     "onela_export_shared_state": (c_int32, [c_void_p, c_int32, c_int32, c_void_p, c_void_p]),
     "onela_reorder_beams": (c_int32, [c_void_p, c_int32, c_int32, c_void_p, c_int32, c_void_p]),
+    "onela_release_request": (c_int32, [c_void_p, c_int32]),
     "onela_select_beams_static": (c_int32, [c_void_p, c_void_p, c_int32, c_int32, c_int32, c_int32, c_void_p, c_void_p,
                                             c_void_p, c_void_p]),
     "onela_select_beams": (c_int32, [c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p,
@@ -209,6 +210,9 @@ class Onela:
         p = None if parents is None else self._ptr(parents, torch.int32, (req_count, W_new), "parents")
         _check(self.lib.onela_reorder_beams(self.handle, req_begin, req_count, p, W_new, self._s(stream)),
                "onela_reorder_beams")
+
+    def onela_release_request(self, request):
+        _check(self.lib.onela_release_request(self.handle, request), "onela_release_request")
 
     def onela_select_beams(self, req_begin, req_count, beam_scores, cand_logp, C, W_new, parents_out, codes_out, scores_out,
                            stream=None):

@@ -93,6 +93,47 @@ struct onela_ctx {
         status_cleared = true;
         return ONELA_OK;
     }
+    // Slots given back by onela_release_request: (first slot, count), ascending, neighbours merged; a range that
+    // ends at the cursor lowers the cursor instead.  Allocation takes the lowest range that fits, else the cursor.
+    std::vector<std::pair<int64_t, int64_t>> free_ranges;
+    int64_t free_slots() const {
+        int64_t n = 0;
+        for (const auto& f : free_ranges) n += f.second;
+        return n;
+    }
+    static int64_t take_slots(std::vector<std::pair<int64_t, int64_t>>& ranges, int64_t& cur, int64_t limit, int64_t n) {
+        for (size_t i = 0; i < ranges.size(); ++i) {
+            if (ranges[i].second >= n) {
+                const int64_t at = ranges[i].first;
+                ranges[i].first += n;
+                ranges[i].second -= n;
+                if (ranges[i].second == 0) ranges.erase(ranges.begin() + (long)i);
+                return at;
+            }
+        }
+        if (cur + n > limit) return -1;
+        const int64_t at = cur;
+        cur += n;
+        return at;
+    }
+    void give_back(int64_t first, int64_t n) {
+        if (n <= 0) return;
+        auto it = free_ranges.begin();
+        while (it != free_ranges.end() && it->first < first) ++it;
+        it = free_ranges.insert(it, {first, n});
+        if (it + 1 != free_ranges.end() && it->first + it->second == (it + 1)->first) {   // merge with the next range
+            it->second += (it + 1)->second;
+            free_ranges.erase(it + 1);
+        }
+        if (it != free_ranges.begin() && (it - 1)->first + (it - 1)->second == it->first) {   // and with the one before
+            (it - 1)->second += it->second;
+            it = free_ranges.erase(it) - 1;
+        }
+        if (!free_ranges.empty() && free_ranges.back().first + free_ranges.back().second == cursor) {
+            cursor = free_ranges.back().first;
+            free_ranges.pop_back();
+        }
+    }
     void restart(ReqState& r) {
         r.depth = 0;
         r.W = 0;
@@ -182,6 +223,7 @@ onela_status onela_reset(onela_ctx* ctx, void* stream) {
         std::fill(r.has_state.begin(), r.has_state.end(), 0);
     }
     ctx->cursor = 0;
+    ctx->free_ranges.clear();
     ctx->status_cleared = false;
     return ctx->prepare(static_cast<cudaStream_t>(stream));
 }
@@ -262,11 +304,18 @@ onela_status onela_reorder_beams(onela_ctx* ctx, int32_t req_begin, int32_t req_
                 if (r.has_state[l] && r.appended_depth[l] != depth_old) return ONELA_E_ORDER;
     }
     if (depth_old >= c.max_steps) return ONELA_E_CAPACITY;
-    if (ctx->cursor + (int64_t)req_count * W_new > c.arena_slots) return ONELA_E_CAPACITY;
+    // slots of this call's records, request by request: the lowest released range that fits, else the bump cursor
+    // (with nothing released this is base(req, t) = cursor, cursor += W_new in request order)
+    auto ranges = ctx->free_ranges;
+    int64_t cur = ctx->cursor;
+    BatchBases bases{};
+    for (int i = 0; i < req_count; ++i) {
+        const int64_t at = onela_ctx::take_slots(ranges, cur, c.arena_slots, W_new);
+        if (at < 0) return ONELA_E_CAPACITY;          // nothing has been changed yet
+        bases.base[i] = (int32_t)at;
+    }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if ((st = ctx->prepare(s)) != ONELA_OK) return st;
-    BatchBases bases{};
-    for (int i = 0; i < req_count; ++i) bases.base[i] = (int32_t)(ctx->cursor + (int64_t)i * W_new);
     if (!ctx->dry()) {
         if (launch_reorder(ctx->lay.tables + req_begin * ctx->table_req_stride(), ctx->table_req_stride(), req_count,
                            parents_dev, W_new, W_prev, depth_old, c.max_beam, c.max_steps, bases, ctx->lay.status,
@@ -293,7 +342,17 @@ onela_status onela_reorder_beams(onela_ctx* ctx, int32_t req_begin, int32_t req_
         r.step_base.push_back(bases.base[i]);
         r.step_width.push_back(W_new);
     }
-    ctx->cursor += (int64_t)req_count * W_new;
+    ctx->free_ranges.swap(ranges);
+    ctx->cursor = cur;
+    return ONELA_OK;
+}
+
+onela_status onela_release_request(onela_ctx* ctx, int32_t request) {
+    if (!ctx || request < 0 || request >= ctx->cfg.num_requests) return ONELA_E_INVAL;
+    ReqState& r = ctx->req[request];
+    for (size_t t = 0; t < r.step_base.size(); ++t) ctx->give_back(r.step_base[t], r.step_width[t]);
+    ctx->restart(r);
+    std::fill(r.has_state.begin(), r.has_state.end(), 0);
     return ONELA_OK;
 }
 
@@ -501,7 +560,8 @@ onela_status onela_get_stats(const onela_ctx* ctx, int64_t* s0_bytes_host, int64
     }
     const int64_t rec_bytes = (int64_t)(c.dk + c.dv) * ctx->elem_bytes + 2 * (int64_t)sizeof(float);
     if (s0_bytes_host) *s0_bytes_host = states * ctx->s0_layer_floats() * (int64_t)sizeof(float);
-    if (arena_bytes_used_host) *arena_bytes_used_host = ctx->cursor * c.num_heads * rec_bytes * c.num_layers;
+    if (arena_bytes_used_host)
+        *arena_bytes_used_host = (ctx->cursor - ctx->free_slots()) * c.num_heads * rec_bytes * c.num_layers;
     if (index_bytes_host) *index_bytes_host = index;
     return ONELA_OK;
 }

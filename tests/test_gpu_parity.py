@@ -98,6 +98,44 @@ def test_degenerate_shapes():
     _full_check(make_case(CFG1.scaled(H=2, W=49, D=2, prompt_len=32, parents="zipf", zipf_s=2.0, seed=704)), "fp32", fused=True)
 
 
+def test_released_slots_are_reused_while_another_request_goes_on():
+    """Continuous batching: request 0 finishes after two calls and is released; a new generation starts in its slot
+    and lands on the freed record slots while request 1 keeps decoding.  Both must match the oracle: the newcomer is
+    not disturbed by stale records, the survivor's records are not touched."""
+    wl = CFG1.scaled(R=2, L=1, H=4, W=40, D=4, prompt_len=64, parents="zipf", zipf_s=1.3, seed=911)
+    case = make_case(wl)
+    ref, _ = run_oracle(case)
+    W = wl.W
+    cfg = P.make_config(wl.R, wl.L, wl.H, wl.dk, wl.dv, W, wl.D, wl.dtype, "fp32", 6 * W, 0)
+    ctx = P.Onela(cfg, device="cuda")
+    dev = torch.device("cuda")
+
+    def step(r, t):
+        par = None if t == 0 else case["parents"][(r, t)][None].to(dev)
+        ctx.onela_reorder_beams(r, 1, par, W)
+        tk = {n: x[None].to(dev) for n, x in case["tok"][(r, 0, t)].items()}
+        out = torch.empty((1, W, wl.H, wl.dv), dtype=torch.float32, device=dev)
+        ctx.onela_append_decode_step(r, 1, 0, tk["k"], tk["v"], tk["alpha"], tk["beta"], case["q"][(r, 0, t)][None].to(dev), out)
+        e = rel_l2(out[0].cpu().numpy(), ref[(r, 0, t)])
+        assert e.max() <= REL_L2_BAR, f"request {r} call {t}: rel-L2 {e.max():.3e}"
+
+    for r in range(2):
+        ctx.onela_init_shared_state(r, 0, case["S0"][(r, 0)].to(dev))
+    for t in range(2):
+        for r in range(2):
+            step(r, t)
+    assert [ctx.onela_get_step_base(r, t) for r in range(2) for t in range(2)] == [0, 2 * W, W, 3 * W]
+    ctx.onela_release_request(0)
+    ctx.onela_init_shared_state(0, 0, case["S0"][(0, 0)].to(dev))      # the next prompt in slot 0
+    step(0, 0)                                                          # -> freed [0, W)
+    step(1, 2)                                                          # -> freed [2W, 3W)
+    step(0, 1)                                                          # -> the cursor
+    step(1, 3)
+    assert [ctx.onela_get_step_base(0, t) for t in range(2)] == [0, 4 * W]
+    assert [ctx.onela_get_step_base(1, t) for t in range(4)] == [W, 3 * W, 2 * W, 5 * W]
+    assert ctx.onela_poll_device_status() == (0, 0)
+
+
 def test_varying_beam_width_between_calls():
     wl = CFG1.scaled(H=2, W=96, D=4, prompt_len=64, seed=91)
     _full_check(make_case(wl, widths=[96, 17, 64, 5]), "fp32")

@@ -252,6 +252,51 @@ def test_new_prompt_restarts_a_request():
     assert o.onela_get_step_base(0, 0) == 16      # the arena is append-only: no slot is reused
 
 
+def test_released_slots_are_reused_lowest_first():
+    o = ctx(R=3, L=1, slots=64, W=8)
+    for r in range(3):
+        o.onela_init_shared_state(r, 0, FAKE)
+    for r in range(3):                                   # bases 0, 8, 16 and then 24, 32, 40
+        full_step(o, r, 1, 8, None, [0])
+    for r in range(3):
+        full_step(o, r, 1, 8, FAKE, [0])
+    assert [o.onela_get_step_base(r, t) for r in range(3) for t in range(2)] == [0, 24, 8, 32, 16, 40]
+    used = lambda: o.onela_get_stats()["arena_bytes_used"] // (4 * (64 * 4 + 8))   # slots, from the resident bytes
+    assert used() == 48
+    o.onela_release_request(1)                           # frees [8, 16) and [32, 40)
+    assert used() == 32 and o.depth_and_width(1) == (0, 0)
+    with raises(binding.E_ORDER):
+        o.onela_reorder_beams(1, 1, None, 8)             # its states went with it
+    o.onela_init_shared_state(1, 0, FAKE)
+    o.onela_reorder_beams(1, 1, None, 4)                 # 4 slots: the lowest hole, [8, 12)
+    assert o.onela_get_step_base(1, 0) == 8
+    o.onela_append_records(1, 1, 0, FAKE, FAKE, FAKE, FAKE)
+    o.onela_reorder_beams(1, 1, FAKE, 8)                 # 8 slots do not fit [12, 16): the next hole, [32, 40)
+    assert o.onela_get_step_base(1, 1) == 32
+    o.onela_append_records(1, 1, 0, FAKE, FAKE, FAKE, FAKE)
+    o.onela_reorder_beams(1, 1, FAKE, 8)                 # no hole left that fits: the cursor, [48, 56)
+    assert o.onela_get_step_base(1, 2) == 48
+    o.onela_release_request(2)                           # [16, 24) merges with [12, 16); [40, 48) stays apart
+    o.onela_release_request(1)                           # [8, 12) merges in front; [32, 40) + [40, 48) + [48, 56) reach the
+    o.onela_release_request(0)                           # cursor and lower it; request 0 then empties the arena
+    assert used() == 0
+    o.onela_init_shared_state(0, 0, FAKE)
+    o.onela_reorder_beams(0, 1, None, 8)
+    assert o.onela_get_step_base(0, 0) == 0              # back to a clean bump allocator
+
+
+def test_batched_reorder_that_does_not_fit_changes_nothing():
+    o = ctx(R=2, L=1, slots=20, W=8)
+    for r in range(2):
+        o.onela_init_shared_state(r, 0, FAKE)
+    full_step(o, 0, 2, 8, None, [0])                     # 16 of 20 slots
+    with raises(binding.E_CAPACITY):
+        o.onela_reorder_beams(0, 2, FAKE, 8)             # the first request would fit nowhere either: nothing moves
+    assert o.depth_and_width(0) == (1, 8) and o.depth_and_width(1) == (1, 8)
+    o.onela_reorder_beams(0, 2, FAKE, 2)                 # 4 more slots do
+    assert [o.onela_get_step_base(r, 1) for r in range(2)] == [16, 18]
+
+
 def test_storage_arithmetic_matches_section_4_4():
     """The resident-byte arithmetic reproduces the capacities and write volumes the paper prints, with
     the paper's 516-byte record; the raw (k, v, alpha, beta) record kept here is 520 bytes."""
