@@ -38,10 +38,13 @@
  *    clamped to 0, and nothing traps.
  *  - Call order per request:  init/prefill_shared_state for each layer used (restarts the request at
  *    depth 0)  ->  repeat {  reorder_beams (once per decode call; shared by all layers and heads)  ->
- *    per layer { append_records exactly once  ->  decode_step any number of times } }.
+ *    per layer { append_records exactly once  ->  decode_step any number of times } }, where
+ *    append_decode_step stands for the layer's append and its first decode in one launch.  select_beams
+ *    may run before a reorder_beams to produce its parents; release_request ends a request.
  *    Violations return ONELA_E_ORDER.
  *  - Slot numbering: one bump cursor per context.  reorder_beams over requests [b, b+n) assigns, in
- *    request order, base(req, t) = cursor, cursor += W_new.  The record of beam i at decode call t lives
+ *    request order, base(req, t) = cursor, cursor += W_new (after a release_request: the lowest released
+ *    range that fits, first).  The record of beam i at decode call t lives
  *    at global slot base(req, t) + i in every layer ("written once to the physical slots of the current
  *    decoding step and never relocated", Section 3.3).
  *  - Batched calls (req_count > 1) need the same beam width and depth on every request of the batch,
