@@ -140,3 +140,27 @@ def prefill(k, v, alpha, beta, nthreads: int = 0) -> np.ndarray:
     lib.oracle_gdn_prefill(H, dk, dv, N, k.ctypes.data, v.ctypes.data, alpha.ctypes.data,
                            beta.ctypes.data, S.ctypes.data, nthreads)
     return S
+
+
+def decode_grouped(S0, steps, parents, q, sel=None, nthreads: int = 0, return_chains: bool = False):
+    """Grouped value heads: Hv value heads share Hk = Hv / g key heads (value head j reads the query and keys of
+    key head j // g; states, values and gates are per value head).  By definition this is the ungrouped recurrence
+    with every key head's q and k repeated g times, which is how it is evaluated.
+
+    S0 [Hv, dv, dk]; steps: k [W_t, Hk, dk], v [W_t, Hv, dv], alpha, beta [W_t, Hv]; q [W, Hk, dk]."""
+    S0 = _f32(S0)
+    Hv = S0.shape[0]
+    q = _f32(q)
+    Hk = q.shape[1]
+    assert Hv % Hk == 0
+    g = Hv // Hk
+    wide = [dict(s, k=np.repeat(_f32(s["k"]), g, axis=1)) for s in steps]
+    return decode(S0, wide, parents, np.repeat(q, g, axis=1), sel=sel, nthreads=nthreads, return_chains=return_chains)
+
+
+def prefill_grouped(k, v, alpha, beta, nthreads: int = 0) -> np.ndarray:
+    """Eq. 1 from the zero state with grouped value heads: k [N, Hk, dk], v [N, Hv, dv], gates [N, Hv]."""
+    k, v = _f32(k), _f32(v)
+    g = v.shape[1] // k.shape[1]
+    assert g * k.shape[1] == v.shape[1]
+    return prefill(np.repeat(k, g, axis=1), v, alpha, beta, nthreads)

@@ -348,3 +348,26 @@ def test_prefill_then_decode_equals_one_long_chain():
     # S0 is handed over in fp32 (as the store holds it), so compare at fp32 resolution
     short = oracle.decode(S0.astype(np.float32), tok[N:], ident(T), q)
     np.testing.assert_allclose(short, long, rtol=0, atol=5e-6)
+
+
+def test_grouped_value_heads_equal_one_single_head_run_per_value_head():
+    """Value head j of a grouped layer is an ordinary single-head layer with key head j // g's queries and keys:
+    the grouped evaluation must equal Hv separate one-head runs (each through the pinned ungrouped routine)."""
+    rng = np.random.default_rng(21)
+    Hk, g, dk, dv, W, T = 2, 3, 8, 6, 5, 3
+    Hv = Hk * g
+    S0 = rng.normal(size=(Hv, dv, dk))
+    steps = [{"k": rng.normal(size=(W, Hk, dk)), "v": rng.normal(size=(W, Hv, dv)),
+              "alpha": rng.uniform(0.9, 1.0, size=(W, Hv)), "beta": rng.uniform(0.1, 0.9, size=(W, Hv))} for _ in range(T)]
+    parents = [None] + [rng.integers(0, W, W) for _ in range(T - 1)]
+    q = rng.normal(size=(W, Hk, dk))
+    got = oracle.decode_grouped(S0, steps, parents, q)
+    for j in range(Hv):
+        one = [{"k": s["k"][:, j // g:j // g + 1], "v": s["v"][:, j:j + 1], "alpha": s["alpha"][:, j:j + 1],
+                "beta": s["beta"][:, j:j + 1]} for s in steps]
+        want = oracle.decode(S0[j:j + 1], one, parents, q[:, j // g:j // g + 1])
+        # inputs pass through fp32 on the way in, identically on both sides
+        assert np.allclose(got[:, j], want[:, 0], rtol=1e-12, atol=1e-12)
+    # g = 1 is the ungrouped routine itself
+    steps1 = [dict(s, v=s["v"][:, :Hk], alpha=s["alpha"][:, :Hk], beta=s["beta"][:, :Hk]) for s in steps]
+    assert np.array_equal(oracle.decode_grouped(S0[:Hk], steps1, parents, q), oracle.decode(S0[:Hk], steps1, parents, q))
