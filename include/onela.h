@@ -93,7 +93,7 @@ typedef int32_t onela_status;
 typedef struct onela_config {
     int32_t num_requests; /* request slots */
     int32_t num_layers;   /* GDN layers sharing the ancestry index */
-    int32_t num_heads;    /* key heads == value heads */
+    int32_t num_heads;    /* key heads (and value heads, unless num_v_heads says otherwise) */
     int32_t dk, dv;       /* head dimensions of k/q and of v/o */
     int32_t max_beam;     /* largest beam width W_t */
     int32_t max_steps;    /* largest number of decode calls per request (chain depth) */
@@ -101,6 +101,14 @@ typedef struct onela_config {
     int32_t out_dtype;    /* dtype of o */
     int64_t arena_slots;  /* record slots per layer, shared by all requests (< 2^31) */
     uint32_t flags;
+    /* Grouped value heads (shapes of the operator suite of Section 4.1): 0 or num_heads = one value head per key
+     * head; otherwise a multiple g * num_heads: value head j reads the queries and keys of key head j / g, while
+     * states, values, gates and outputs are per value head.  Then q, k are [..][num_heads][dk]; v, alpha, beta, out
+     * and S_0 are [..][num_v_heads][..]; a record keeps k once per key head and (v, alpha, beta) per value head
+     * (num_heads * dk + num_v_heads * (dv + 8 bytes of gates) per slot instead of num_v_heads * (dk + dv + ..)).
+     * CUDA-core kernels; (dk, dv) in {(64, 64), (128, 128), (128, 256)}; onela_prefill_shared_state and
+     * ONELA_FLAG_GTR_DELTA are not available (ONELA_E_UNSUPPORTED). */
+    int32_t num_v_heads;
 } onela_config;
 
 /* Bytes of device workspace the configuration needs; 0 if the configuration is invalid. */

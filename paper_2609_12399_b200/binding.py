@@ -27,7 +27,12 @@ _DTYPE_CODE = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16, "fp32": DTY
 class OnelaConfig(ctypes.Structure):
     _fields_ = [("num_requests", c_int32), ("num_layers", c_int32), ("num_heads", c_int32), ("dk", c_int32),
                 ("dv", c_int32), ("max_beam", c_int32), ("max_steps", c_int32), ("rec_dtype", c_int32),
-                ("out_dtype", c_int32), ("arena_slots", c_int64), ("flags", c_uint32)]
+                ("out_dtype", c_int32), ("arena_slots", c_int64), ("flags", c_uint32), ("num_v_heads", c_int32)]
+
+    @property
+    def value_heads(self) -> int:
+        """Value heads: num_v_heads, or num_heads when that is 0 (one value head per key head)."""
+        return self.num_v_heads or self.num_heads
 
 
 class OnelaError(RuntimeError):
@@ -100,9 +105,9 @@ def _stream_ptr(stream) -> int:
 
 
 def make_config(num_requests, num_layers, num_heads, dk, dv, max_beam, max_steps, rec_dtype, out_dtype,
-                arena_slots, flags=0) -> OnelaConfig:
+                arena_slots, flags=0, num_v_heads=0) -> OnelaConfig:
     return OnelaConfig(num_requests, num_layers, num_heads, dk, dv, max_beam, max_steps,
-                       _DTYPE_CODE[rec_dtype], _DTYPE_CODE[out_dtype], arena_slots, flags)
+                       _DTYPE_CODE[rec_dtype], _DTYPE_CODE[out_dtype], arena_slots, flags, num_v_heads)
 
 
 def onela_select_beams_static(beam_scores, cand_logp, W_new, parents_out, codes_out, scores_out, stream=None) -> None:
@@ -186,7 +191,7 @@ class Onela:
 
     def onela_init_shared_state(self, request, layer, S0, stream=None):
         c = self.cfg
-        p = self._ptr(S0, torch.float32, (c.num_heads, c.dv, c.dk), "S0")
+        p = self._ptr(S0, torch.float32, (c.value_heads, c.dv, c.dk), "S0")
         _check(self.lib.onela_init_shared_state(self.handle, request, layer, p, self._s(stream)), "onela_init_shared_state")
 
     def onela_prefill_shared_state(self, request, layer, k, v, alpha, beta, stream=None):
@@ -201,7 +206,7 @@ class Onela:
     def onela_export_shared_state(self, request, layer, stream=None) -> torch.Tensor:
         """Returns the stored S_0 of (request, layer) as fp32 [H, dv, dk] on the device."""
         c = self.cfg
-        out = torch.empty((c.num_heads, c.dv, c.dk), dtype=torch.float32, device=self.device)
+        out = torch.empty((c.value_heads, c.dv, c.dk), dtype=torch.float32, device=self.device)
         _check(self.lib.onela_export_shared_state(self.handle, request, layer, c_void_p(out.data_ptr()),
                                                   self._s(stream)), "onela_export_shared_state")
         return out
@@ -232,9 +237,9 @@ class Onela:
         _check(self.lib.onela_append_records(
             self.handle, req_begin, req_count, layer,
             self._ptr(k, self.rec_dtype, (req_count, W, c.num_heads, c.dk), "k"),
-            self._ptr(v, self.rec_dtype, (req_count, W, c.num_heads, c.dv), "v"),
-            self._ptr(alpha, torch.float32, (req_count, W, c.num_heads), "alpha"),
-            self._ptr(beta, torch.float32, (req_count, W, c.num_heads), "beta"), self._s(stream)), "onela_append_records")
+            self._ptr(v, self.rec_dtype, (req_count, W, c.value_heads, c.dv), "v"),
+            self._ptr(alpha, torch.float32, (req_count, W, c.value_heads), "alpha"),
+            self._ptr(beta, torch.float32, (req_count, W, c.value_heads), "beta"), self._s(stream)), "onela_append_records")
 
     def onela_decode_step(self, req_begin, req_count, layer, q, out, stream=None):
         c = self.cfg
@@ -242,7 +247,7 @@ class Onela:
         _check(self.lib.onela_decode_step(
             self.handle, req_begin, req_count, layer,
             self._ptr(q, self.rec_dtype, (req_count, W, c.num_heads, c.dk), "q"),
-            self._ptr(out, self.out_dtype, (req_count, W, c.num_heads, c.dv), "out"), self._s(stream)), "onela_decode_step")
+            self._ptr(out, self.out_dtype, (req_count, W, c.value_heads, c.dv), "out"), self._s(stream)), "onela_decode_step")
 
     def onela_append_decode_step(self, req_begin, req_count, layer, k, v, alpha, beta, q, out, stream=None):
         c = self.cfg
@@ -250,11 +255,11 @@ class Onela:
         _check(self.lib.onela_append_decode_step(
             self.handle, req_begin, req_count, layer,
             self._ptr(k, self.rec_dtype, (req_count, W, c.num_heads, c.dk), "k"),
-            self._ptr(v, self.rec_dtype, (req_count, W, c.num_heads, c.dv), "v"),
-            self._ptr(alpha, torch.float32, (req_count, W, c.num_heads), "alpha"),
-            self._ptr(beta, torch.float32, (req_count, W, c.num_heads), "beta"),
+            self._ptr(v, self.rec_dtype, (req_count, W, c.value_heads, c.dv), "v"),
+            self._ptr(alpha, torch.float32, (req_count, W, c.value_heads), "alpha"),
+            self._ptr(beta, torch.float32, (req_count, W, c.value_heads), "beta"),
             self._ptr(q, self.rec_dtype, (req_count, W, c.num_heads, c.dk), "q"),
-            self._ptr(out, self.out_dtype, (req_count, W, c.num_heads, c.dv), "out"), self._s(stream)),
+            self._ptr(out, self.out_dtype, (req_count, W, c.value_heads, c.dv), "out"), self._s(stream)),
             "onela_append_decode_step")
 
     def onela_export_chains(self, request, stream=None) -> torch.Tensor:

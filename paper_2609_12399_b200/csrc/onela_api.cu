@@ -31,6 +31,7 @@ bool config_sane(const onela_config* c) {
         (c->out_dtype != ONELA_DTYPE_F32 && c->out_dtype != ONELA_DTYPE_BF16))
         return false;
     if (c->arena_slots < 1 || c->arena_slots > 0x7fffffffLL - c->max_beam) return false;
+    if (c->num_v_heads < 0 || (c->num_v_heads > 0 && c->num_v_heads % c->num_heads != 0)) return false;
     const int es = c->rec_dtype == ONELA_DTYPE_BF16 ? 2 : 4;
     if ((c->dk * es) % 16 != 0 || (c->dv * es) % 16 != 0) return false;  // 16-byte vector rows
     return true;
@@ -39,6 +40,7 @@ bool config_sane(const onela_config* c) {
 // Carve the workspace.  `base` may be null (size query only).
 Layout carve(const onela_config& c, char* base) {
     const size_t es = c.rec_dtype == ONELA_DTYPE_BF16 ? 2 : 4;
+    const size_t Hv = c.num_v_heads > 0 ? c.num_v_heads : c.num_heads;   // value heads
     size_t off = 0;
     Layout l{};
     auto take = [&](size_t bytes) {
@@ -51,9 +53,14 @@ Layout carve(const onela_config& c, char* base) {
     l.sidx = reinterpret_cast<int32_t*>(take((size_t)c.num_requests * c.max_steps * c.max_beam * sizeof(int32_t)));
     l.ulist = reinterpret_cast<int32_t*>(take((size_t)c.num_requests * c.max_steps * c.max_beam * sizeof(int32_t)));
     l.uoff = reinterpret_cast<int32_t*>(take((size_t)c.num_requests * (c.max_steps + 1) * sizeof(int32_t)));
-    l.s0 = reinterpret_cast<float*>(take((size_t)c.num_requests * c.num_layers * c.num_heads * c.dv * c.dk * sizeof(float)));
-    l.gates = reinterpret_cast<float2*>(take((size_t)c.num_layers * c.num_heads * (size_t)c.arena_slots * sizeof(float2)));
-    l.kv = take((size_t)c.num_layers * c.num_heads * (size_t)c.arena_slots * (c.dk + c.dv) * es);
+    l.s0 = reinterpret_cast<float*>(take((size_t)c.num_requests * c.num_layers * Hv * c.dv * c.dk * sizeof(float)));
+    l.gates = reinterpret_cast<float2*>(take((size_t)c.num_layers * Hv * (size_t)c.arena_slots * sizeof(float2)));
+    if (Hv == (size_t)c.num_heads) {
+        l.kv = take((size_t)c.num_layers * c.num_heads * (size_t)c.arena_slots * (c.dk + c.dv) * es);
+    } else {   // grouped value heads: keys per key head, values per value head
+        l.kv = take((size_t)c.num_layers * c.num_heads * (size_t)c.arena_slots * c.dk * es);
+        l.vv = take((size_t)c.num_layers * Hv * (size_t)c.arena_slots * c.dv * es);
+    }
     l.select_scratch = reinterpret_cast<unsigned long long*>(
         take((size_t)c.num_requests * ONELA_SELECT_PARTS * ONELA_SELECT_CAP * sizeof(unsigned long long)));
     l.total_bytes = off;
@@ -74,8 +81,12 @@ struct onela_ctx {
 
     bool dry() const { return cfg.flags & ONELA_FLAG_DRY_RUN; }
     bool gtr() const { return cfg.flags & ONELA_FLAG_GTR_DELTA; }   // (alpha, delta, k) records, forward replay
+    int32_t Hv() const { return cfg.num_v_heads > 0 ? cfg.num_v_heads : cfg.num_heads; }   // value heads
+    bool grouped() const { return Hv() != cfg.num_heads; }
+    char* k_plane(int l) const { return lay.kv + (size_t)l * cfg.num_heads * (size_t)cfg.arena_slots * cfg.dk * elem_bytes; }
+    char* v_plane(int l) const { return lay.vv + (size_t)l * Hv() * (size_t)cfg.arena_slots * cfg.dv * elem_bytes; }
     long long table_req_stride() const { return 2LL * cfg.max_steps * cfg.max_beam; }
-    long long s0_layer_floats() const { return (long long)cfg.num_heads * cfg.dv * cfg.dk; }
+    long long s0_layer_floats() const { return (long long)Hv() * cfg.dv * cfg.dk; }
     float* s0_slot(int r, int l) const { return lay.s0 + ((long long)r * cfg.num_layers + l) * s0_layer_floats(); }
     int32_t* table_cur(int r) const {
         const int d = req[r].depth;
@@ -85,7 +96,7 @@ struct onela_ctx {
     long long uoff_req_stride() const { return cfg.max_steps + 1; }
     size_t plane_rows() const { return (size_t)cfg.num_heads * (size_t)cfg.arena_slots; }
     char* kv_plane(int l) const { return lay.kv + (size_t)l * plane_rows() * (cfg.dk + cfg.dv) * elem_bytes; }
-    float2* gate_plane(int l) const { return lay.gates + (size_t)l * plane_rows(); }
+    float2* gate_plane(int l) const { return lay.gates + (size_t)l * Hv() * (size_t)cfg.arena_slots; }
 
     onela_status prepare(cudaStream_t s) {
         if (dry() || status_cleared) return ONELA_OK;
@@ -193,6 +204,9 @@ onela_status onela_create(const onela_config* cfg, void* workspace_dev, size_t w
     if (!decode_generic_supported(cfg->dk, cfg->dv, cfg->rec_dtype)) return ONELA_E_UNSUPPORTED;
     if ((cfg->flags & ONELA_FLAG_GTR_DELTA) && !(cfg->dk == cfg->dv && (cfg->dk == 32 || cfg->dk == 64 || cfg->dk == 128)))
         return ONELA_E_UNSUPPORTED;
+    const bool grouped_cfg = cfg->num_v_heads > 0 && cfg->num_v_heads != cfg->num_heads;
+    if (grouped_cfg && (!decode_grouped_supported(cfg->dk, cfg->dv) || (cfg->flags & ONELA_FLAG_GTR_DELTA)))
+        return ONELA_E_UNSUPPORTED;
     const Layout lay = carve(*cfg, static_cast<char*>(workspace_dev));
     if (workspace_bytes < lay.total_bytes) return ONELA_E_CAPACITY;
     onela_ctx* ctx = new (std::nothrow) onela_ctx();
@@ -205,7 +219,7 @@ onela_status onela_create(const onela_config* cfg, void* workspace_dev, size_t w
         r.has_state.assign(cfg->num_layers, 0);
         r.appended_depth.assign(cfg->num_layers, -1);
     }
-    ctx->tensor_core = decode_sm100_supported(cfg->dk, cfg->dv, cfg->rec_dtype) &&
+    ctx->tensor_core = decode_sm100_supported(cfg->dk, cfg->dv, cfg->rec_dtype) && !grouped_cfg &&
                        !(cfg->flags & (ONELA_FLAG_FORCE_GENERIC | ONELA_FLAG_GTR_DELTA));
     *out = ctx;
     return ONELA_OK;
@@ -236,7 +250,7 @@ onela_status onela_init_shared_state(onela_ctx* ctx, int32_t request, int32_t la
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if ((st = ctx->prepare(s)) != ONELA_OK) return st;
     if (!ctx->dry()) {
-        if (launch_store_state(S0_dev, ctx->s0_slot(request, layer), ctx->cfg.num_heads, ctx->cfg.dk, ctx->cfg.dv,
+        if (launch_store_state(S0_dev, ctx->s0_slot(request, layer), ctx->Hv(), ctx->cfg.dk, ctx->cfg.dv,
                                s) != cudaSuccess)
             return ONELA_E_CUDA;
         ctx->launches++;
@@ -250,6 +264,7 @@ onela_status onela_prefill_shared_state(onela_ctx* ctx, int32_t request, int32_t
                                         int32_t n_tokens, void* stream) {
     onela_status st = begin_state_write(ctx, request, layer);
     if (st != ONELA_OK) return st;
+    if (ctx->grouped()) return ONELA_E_UNSUPPORTED;   // grouped value heads: the state comes through init_shared_state
     if (n_tokens < 0) return ONELA_E_INVAL;
     if (n_tokens > 0 && (!k_dev || !v_dev || !alpha_dev || !beta_dev || !aligned16(k_dev) || !aligned16(v_dev)))
         return ONELA_E_INVAL;
@@ -277,7 +292,7 @@ onela_status onela_export_shared_state(onela_ctx* ctx, int32_t request, int32_t 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if ((st = ctx->prepare(s)) != ONELA_OK) return st;
     if (ctx->dry()) return ONELA_OK;
-    if (launch_export_state(ctx->s0_slot(request, layer), S0_out_dev, ctx->cfg.num_heads, ctx->cfg.dk, ctx->cfg.dv,
+    if (launch_export_state(ctx->s0_slot(request, layer), S0_out_dev, ctx->Hv(), ctx->cfg.dk, ctx->cfg.dv,
                             s) != cudaSuccess)
         return ONELA_E_CUDA;
     ctx->launches++;
@@ -398,10 +413,13 @@ onela_status onela_append_records(onela_ctx* ctx, int32_t req_begin, int32_t req
     BatchBases bases{};
     for (int i = 0; i < req_count; ++i) bases.base[i] = ctx->req[req_begin + i].step_base.back();
     if (!ctx->dry()) {
-        if (launch_append(k_dev, v_dev, alpha_dev, beta_dev, ctx->kv_plane(layer), ctx->gate_plane(layer),
-                          c.arena_slots, req_count, W, c.num_heads, c.dk, c.dv, ctx->elem_bytes, bases,
-                          s) != cudaSuccess)
-            return ONELA_E_CUDA;
+        const cudaError_t e =
+            ctx->grouped() ? launch_append_grouped(k_dev, v_dev, alpha_dev, beta_dev, ctx->k_plane(layer), ctx->v_plane(layer),
+                                                   ctx->gate_plane(layer), c.arena_slots, req_count, W, c.num_heads,
+                                                   ctx->Hv() / c.num_heads, c.dk, c.dv, ctx->elem_bytes, bases, s)
+                           : launch_append(k_dev, v_dev, alpha_dev, beta_dev, ctx->kv_plane(layer), ctx->gate_plane(layer),
+                                           c.arena_slots, req_count, W, c.num_heads, c.dk, c.dv, ctx->elem_bytes, bases, s);
+        if (e != cudaSuccess) return ONELA_E_CUDA;
         ctx->launches++;
     }
     for (int i = 0; i < req_count; ++i) ctx->req[req_begin + i].appended_depth[layer] = depth;
@@ -418,6 +436,29 @@ onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count,
                            const float* beta_dev, cudaStream_t s) {
     const onela_config& c = ctx->cfg;
     const int32_t depth = ctx->req[req_begin].depth, W = ctx->req[req_begin].W;
+    if (ctx->grouped()) {
+        GroupedArgs ga{};
+        ga.q = q_dev;
+        ga.out = out_dev;
+        ga.s0 = ctx->s0_slot(req_begin, layer);
+        ga.kplane = ctx->k_plane(layer);
+        ga.vplane = ctx->v_plane(layer);
+        ga.gates = ctx->gate_plane(layer);
+        ga.table = ctx->table_cur(req_begin);
+        ga.s0_req_stride = (long long)c.num_layers * ctx->s0_layer_floats();
+        ga.table_req_stride = ctx->table_req_stride();
+        ga.arena_slots = c.arena_slots;
+        ga.req_count = req_count;
+        ga.W = W;
+        ga.Hk = c.num_heads;
+        ga.g = ctx->Hv() / c.num_heads;
+        ga.depth = depth;
+        ga.max_beam = c.max_beam;
+        for (int i = 0; i < req_count; ++i) ga.bases.base[i] = ctx->req[req_begin + i].step_base.back();
+        if (launch_decode_grouped(ga, c.dk, c.dv, c.rec_dtype, c.out_dtype, s) != cudaSuccess) return ONELA_E_CUDA;
+        ctx->launches++;
+        return ONELA_OK;
+    }
     DecodeArgs a{};
     a.q = q_dev;
     a.out = out_dev;
@@ -505,10 +546,13 @@ onela_status onela_append_decode_step(onela_ctx* ctx, int32_t req_begin, int32_t
         } else {   // shapes without the fused kernel: the copy kernel, then the decode kernel
             BatchBases bases{};
             for (int i = 0; i < req_count; ++i) bases.base[i] = ctx->req[req_begin + i].step_base.back();
-            if (launch_append(k_dev, v_dev, alpha_dev, beta_dev, ctx->kv_plane(layer), ctx->gate_plane(layer),
-                              c.arena_slots, req_count, W, c.num_heads, c.dk, c.dv, ctx->elem_bytes, bases,
-                              s) != cudaSuccess)
-                return ONELA_E_CUDA;
+            const cudaError_t e =
+                ctx->grouped() ? launch_append_grouped(k_dev, v_dev, alpha_dev, beta_dev, ctx->k_plane(layer), ctx->v_plane(layer),
+                                                       ctx->gate_plane(layer), c.arena_slots, req_count, W, c.num_heads,
+                                                       ctx->Hv() / c.num_heads, c.dk, c.dv, ctx->elem_bytes, bases, s)
+                               : launch_append(k_dev, v_dev, alpha_dev, beta_dev, ctx->kv_plane(layer), ctx->gate_plane(layer),
+                                               c.arena_slots, req_count, W, c.num_heads, c.dk, c.dv, ctx->elem_bytes, bases, s);
+            if (e != cudaSuccess) return ONELA_E_CUDA;
             ctx->launches++;
             st = launch_decode(ctx, req_begin, req_count, layer, q_dev, out_dev, nullptr, nullptr, nullptr, nullptr, s);
             if (st != ONELA_OK) return st;
@@ -558,10 +602,12 @@ onela_status onela_get_stats(const onela_ctx* ctx, int64_t* s0_bytes_host, int64
         for (uint8_t hs : r.has_state) states += hs;
         index += (int64_t)r.W * r.depth * (int64_t)sizeof(int32_t);
     }
-    const int64_t rec_bytes = (int64_t)(c.dk + c.dv) * ctx->elem_bytes + 2 * (int64_t)sizeof(float);
+    // bytes one slot holds across the heads of a layer: k per key head, v and the two gates per value head
+    const int64_t slot_bytes = (int64_t)c.num_heads * c.dk * ctx->elem_bytes +
+                               (int64_t)ctx->Hv() * (c.dv * ctx->elem_bytes + 2 * (int64_t)sizeof(float));
     if (s0_bytes_host) *s0_bytes_host = states * ctx->s0_layer_floats() * (int64_t)sizeof(float);
     if (arena_bytes_used_host)
-        *arena_bytes_used_host = (ctx->cursor - ctx->free_slots()) * c.num_heads * rec_bytes * c.num_layers;
+        *arena_bytes_used_host = (ctx->cursor - ctx->free_slots()) * slot_bytes * c.num_layers;
     if (index_bytes_host) *index_bytes_host = index;
     return ONELA_OK;
 }

@@ -19,6 +19,8 @@ struct Layout {
     float* s0;         // [request][layer][head][dv*dk] fp32
     float2* gates;     // [layer][head][arena_slots] (alpha, beta)
     char* kv;          // [layer][head][arena_slots][dk + dv] in rec_dtype: one row = k | v of one record
+                       // (grouped value heads: keys only, [layer][key head][arena_slots][dk])
+    char* vv;          // grouped value heads only: values [layer][value head][arena_slots][dv]
     unsigned long long* select_scratch;   // [request][ONELA_SELECT_PARTS][ONELA_SELECT_CAP]: partial results of beam selection
     size_t total_bytes;
 };
@@ -52,6 +54,27 @@ struct DecodeArgs {
     int32_t req_count, W, H, depth, max_beam;
     BatchBases bases;
 };
+
+// Grouped value heads (Hv = g * Hk): what the grouped decode kernel needs.
+struct GroupedArgs {
+    const void* q;          // [req_count][W][Hk][dk]
+    void* out;              // [req_count][W][Hv][dv]
+    const float* s0;        // store slot of (req_begin, layer): [Hv][dv][dk]
+    const char* kplane;     // this layer's keys   [Hk][arena_slots][dk]
+    const char* vplane;     // this layer's values [Hv][arena_slots][dv]
+    const float2* gates;    // this layer's gates  [Hv][arena_slots]
+    const int32_t* table;   // current ancestry buffer of req_begin
+    long long s0_req_stride, table_req_stride, arena_slots;
+    int32_t req_count, W, Hk, g, depth, max_beam;
+    BatchBases bases;
+};
+bool decode_grouped_supported(int32_t dk, int32_t dv);
+cudaError_t launch_decode_grouped(const GroupedArgs& a, int32_t dk, int32_t dv, int32_t rec_dtype, int32_t out_dtype,
+                                  cudaStream_t stream);
+cudaError_t launch_append_grouped(const void* k, const void* v, const float* alpha, const float* beta, char* kplane,
+                                  char* vplane, float2* gates, long long arena_slots, int32_t req_count, int32_t W,
+                                  int32_t Hk, int32_t g, int32_t dk, int32_t dv, int32_t elem_bytes, const BatchBases& bases,
+                                  cudaStream_t stream);
 
 // index kernels
 cudaError_t launch_reorder(int32_t* tables_req0, long long table_req_stride, int32_t req_count,

@@ -168,6 +168,29 @@ def test_select_beams_argument_checks():
     o.onela_reorder_beams(0, 1, FAKE, 8)                                          # the call order is untouched
 
 
+def test_grouped_value_heads_configs():
+    """num_v_heads must be a multiple of num_heads; grouped contexts run on CUDA cores, take no prefill and no delta
+    records, and count k once per key head in the resident bytes."""
+    ok = P.make_config(1, 1, 2, 128, 128, 8, 3, "bf16", "bf16", 64, P.FLAG_DRY_RUN, num_v_heads=6)
+    o = P.Onela(ok, device="cpu")
+    assert not o.onela_uses_tensor_core_path()
+    o.onela_init_shared_state(0, 0, FAKE)
+    assert o.lib.onela_prefill_shared_state(o.handle, 0, 0, FAKE, FAKE, FAKE, FAKE, 4, None) == binding.E_UNSUPPORTED
+    o.onela_reorder_beams(0, 1, None, 8)
+    o.onela_append_decode_step(0, 1, 0, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE)
+    assert o.onela_get_stats()["arena_bytes_used"] == 8 * (2 * 128 * 2 + 6 * (128 * 2 + 8))
+    assert o.onela_get_stats()["s0_bytes"] == 6 * 128 * 128 * 4
+    same = P.make_config(1, 1, 2, 128, 128, 8, 3, "bf16", "bf16", 64, P.FLAG_DRY_RUN, num_v_heads=2)
+    assert P.Onela(same, device="cpu").onela_uses_tensor_core_path()           # 2 value heads on 2 key heads: not grouped
+    assert P.onela_workspace_bytes(P.make_config(1, 1, 2, 128, 128, 8, 3, "bf16", "bf16", 64, 0, num_v_heads=3)) == 0
+    for kw in (dict(flags=P.FLAG_DRY_RUN | P.FLAG_GTR_DELTA), dict(dk=32, dv=32)):
+        args = dict(dk=128, dv=128, flags=P.FLAG_DRY_RUN)
+        args.update(kw)
+        bad = P.make_config(1, 1, 2, args["dk"], args["dv"], 8, 3, "fp32", "fp32", 64, args["flags"], num_v_heads=4)
+        with raises(binding.E_UNSUPPORTED):
+            P.Onela(bad, device="cpu")
+
+
 def test_every_layer_with_state_must_append_before_next_call():
     o = ctx()
     o.onela_init_shared_state(0, 0, FAKE)
