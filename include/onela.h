@@ -106,8 +106,8 @@ typedef struct onela_config {
      * states, values, gates and outputs are per value head.  Then q, k are [..][num_heads][dk]; v, alpha, beta, out
      * and S_0 are [..][num_v_heads][..]; a record keeps k once per key head and (v, alpha, beta) per value head
      * (num_heads * dk + num_v_heads * (dv + 8 bytes of gates) per slot instead of num_v_heads * (dk + dv + ..)).
-     * CUDA-core kernels; (dk, dv) in {(64, 64), (128, 128), (128, 256)}; onela_prefill_shared_state and
-     * ONELA_FLAG_GTR_DELTA are not available (ONELA_E_UNSUPPORTED). */
+     * (dk, dv) in {(64, 64), (128, 128), (128, 256)}: 128 x 128 bf16 on the tensor-core kernel, the rest on CUDA
+     * cores; onela_prefill_shared_state and ONELA_FLAG_GTR_DELTA are not available (ONELA_E_UNSUPPORTED). */
     int32_t num_v_heads;
 } onela_config;
 

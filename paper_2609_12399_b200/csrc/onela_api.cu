@@ -219,7 +219,7 @@ onela_status onela_create(const onela_config* cfg, void* workspace_dev, size_t w
         r.has_state.assign(cfg->num_layers, 0);
         r.appended_depth.assign(cfg->num_layers, -1);
     }
-    ctx->tensor_core = decode_sm100_supported(cfg->dk, cfg->dv, cfg->rec_dtype) && !grouped_cfg &&
+    ctx->tensor_core = decode_sm100_supported(cfg->dk, cfg->dv, cfg->rec_dtype) &&
                        !(cfg->flags & (ONELA_FLAG_FORCE_GENERIC | ONELA_FLAG_GTR_DELTA));
     *out = ctx;
     return ONELA_OK;
@@ -436,7 +436,7 @@ onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count,
                            const float* beta_dev, cudaStream_t s) {
     const onela_config& c = ctx->cfg;
     const int32_t depth = ctx->req[req_begin].depth, W = ctx->req[req_begin].W;
-    if (ctx->grouped()) {
+    if (ctx->grouped() && !ctx->tensor_core) {
         GroupedArgs ga{};
         ga.q = q_dev;
         ga.out = out_dev;
@@ -466,10 +466,14 @@ onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count,
     a.v_in = v_dev;
     a.alpha_in = alpha_dev;
     a.beta_in = beta_dev;
-    a.kv_out = ctx->kv_plane(layer);
+    a.kv_out = ctx->grouped() ? ctx->k_plane(layer) : ctx->kv_plane(layer);
+    a.vv_out = ctx->grouped() ? ctx->v_plane(layer) : nullptr;
     a.gates_out = ctx->gate_plane(layer);
     a.s0 = ctx->s0_slot(req_begin, layer);
-    a.kv = ctx->kv_plane(layer);
+    a.kv = a.kv_out;
+    a.vv = a.vv_out;
+    a.Hk = c.num_heads;
+    a.g = ctx->Hv() / c.num_heads;
     a.gates = ctx->gate_plane(layer);
     a.table = ctx->table_cur(req_begin);
     a.status = ctx->lay.status;
@@ -484,13 +488,13 @@ onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count,
     a.uoff_req_stride = ctx->uoff_req_stride();
     a.req_count = req_count;
     a.W = W;
-    a.H = c.num_heads;
+    a.H = ctx->Hv();
     a.depth = depth;
     a.max_beam = c.max_beam;
     for (int i = 0; i < req_count; ++i) a.bases.base[i] = ctx->req[req_begin + i].step_base.back();
     bool supported = true;
     const cudaError_t e = ctx->gtr()         ? launch_decode_gtr(a, c.dk, c.dv, c.rec_dtype, c.out_dtype, &supported, s)
-                          : ctx->tensor_core ? launch_decode_sm100_ws(a, c.out_dtype, s)
+                          : ctx->tensor_core ? launch_decode_sm100_ws(a, c.out_dtype, ctx->grouped(), s)
                                              : launch_decode_generic(a, c.dk, c.dv, c.rec_dtype, c.out_dtype, &supported, s);
     if (!supported) return ONELA_E_UNSUPPORTED;
     if (e != cudaSuccess) return ONELA_E_CUDA;

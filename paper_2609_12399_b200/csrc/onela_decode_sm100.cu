@@ -110,7 +110,9 @@ struct Partition {
     int32_t begin[MAX_CTAS + 1];
 };
 
-template <typename OutT>
+// GROUPED: value head h reads the queries and keys of key head h / g; a.H counts VALUE heads, the record's k lives in
+// the key heads' plane (a.kv) and its v in the value heads' plane (a.vv), 256 bytes each.
+template <typename OutT, bool GROUPED>
 __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ Partition part,
                                                                int groups_per_pair, int launch_id) {
     extern __shared__ uint8_t smem_raw[];
@@ -178,6 +180,17 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     const bool fused = a.k_in != nullptr;  // append fused in: the newest record comes from the caller's tensors
     const char* kv = a.kv;
     const __nv_bfloat16* qbase = static_cast<const __nv_bfloat16*>(a.q);
+    // rows of the caller's tensors: q and k have one row per KEY head, v, the gates and the outputs per VALUE head
+    auto key_head = [&](int h) { return GROUPED ? h / a.g : h; };
+    auto krow_in = [&](int req, int bb, int h) { return ((long long)req * a.W + bb) * (GROUPED ? a.Hk : a.H) + key_head(h); };
+    auto vrow_in = [&](int req, int bb, int h) { return ((long long)req * a.W + bb) * a.H + h; };
+    // rows of the arena: ungrouped one 512-byte row (k | v) per (head, slot); grouped a 256-byte row in each plane
+    auto k_at = [&](int h, long long slot) {
+        return GROUPED ? kv + ((long long)key_head(h) * a.arena_slots + slot) * (DK * 2) : kv + ((long long)h * a.arena_slots + slot) * REC_BYTES;
+    };
+    auto v_at = [&](int h, long long slot) {
+        return GROUPED ? a.vv + ((long long)h * a.arena_slots + slot) * (DV * 2) : kv + ((long long)h * a.arena_slots + slot) * REC_BYTES + DK * 2;
+    };
     const int grp = lane / LPU, g = lane % LPU;
     bool dead = false;                    // this warp gave up (timeout or abort raised elsewhere)
 
@@ -291,31 +304,37 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             if (lane < UPW * 6) {
                 const int un = lane / 6, item = lane % 6;
                 const int b2 = min(n.gip * GN + UPW * warp + un, a.W - 1);
-                const long long row2 = ((long long)n.req * a.W + b2) * a.H + n.h;
-                const char* p2 = item < 2 ? reinterpret_cast<const char*>(qbase) + row2 * (DK * 2)
-                                 : fused  ? (item < 4 ? static_cast<const char*>(a.k_in) + row2 * (DK * 2)
-                                                      : static_cast<const char*>(a.v_in) + row2 * (DV * 2))
-                                          : kv + ((long long)n.h * a.arena_slots + a.bases.base[n.req] + b2) * REC_BYTES + (item < 4 ? 0 : 256);
+                const long long krow2 = krow_in(n.req, b2, n.h), vrow2 = vrow_in(n.req, b2, n.h);
+                const long long slot2 = a.bases.base[n.req] + b2;
+                const char* p2 = item < 2 ? reinterpret_cast<const char*>(qbase) + krow2 * (DK * 2)
+                                 : fused  ? (item < 4 ? static_cast<const char*>(a.k_in) + krow2 * (DK * 2)
+                                                      : static_cast<const char*>(a.v_in) + vrow2 * (DV * 2))
+                                          : (item < 4 ? k_at(n.h, slot2) : v_at(n.h, slot2));
                 asm volatile("prefetch.global.L2 [%0];" ::"l"(p2 + (item & 1) * 128));
             }
         };
         auto issue_head = [&](const Unit& u, const Unit& n, bool has_next) {
             const uint32_t dst = smem_u32(my_heads);
             const int bb = live_beam(u);
-            const long long in_row = ((long long)u.req * a.W + bb) * a.H + u.h;
-            const char* qr = reinterpret_cast<const char*>(qbase + in_row * DK) + g * 16;
+            const long long krow = krow_in(u.req, bb, u.h);
+            const char* qr = reinterpret_cast<const char*>(qbase + krow * DK) + g * 16;
             if (fused) {   // the call's records come straight from the caller's k and v tensors
-                const char* kr = static_cast<const char*>(a.k_in) + in_row * (DK * 2) + g * 16;
-                const char* vr = static_cast<const char*>(a.v_in) + in_row * (DV * 2) + g * 16;
+                const char* kr = static_cast<const char*>(a.k_in) + krow * (DK * 2) + g * 16;
+                const char* vr = static_cast<const char*>(a.v_in) + vrow_in(u.req, bb, u.h) * (DV * 2) + g * 16;
 #pragma unroll
                 for (int c = 0; c < NCH; ++c) {
                     cp_async16(dst + grp * REC_BYTES + (c * LPU + g) * 16, kr + c * LPU * 16);
                     cp_async16(dst + grp * REC_BYTES + (16 + c * LPU + g) * 16, vr + c * LPU * 16);
                 }
             } else {
-                const char* rec = kv + ((long long)u.h * a.arena_slots + a.bases.base[u.req] + bb) * REC_BYTES + g * 16;
+                const long long slot = a.bases.base[u.req] + bb;
+                const char* kr = k_at(u.h, slot) + g * 16;
+                const char* vr = v_at(u.h, slot) + g * 16;
 #pragma unroll
-                for (int c = 0; c < 2 * NCH; ++c) cp_async16(dst + grp * REC_BYTES + (c * LPU + g) * 16, rec + c * LPU * 16);
+                for (int c = 0; c < NCH; ++c) {
+                    cp_async16(dst + grp * REC_BYTES + (c * LPU + g) * 16, kr + c * LPU * 16);
+                    cp_async16(dst + grp * REC_BYTES + (16 + c * LPU + g) * 16, vr + c * LPU * 16);
+                }
             }
 #pragma unroll
             for (int c = 0; c < NCH; ++c) cp_async16(dst + UPW * REC_BYTES + grp * (DK * 2) + (c * LPU + g) * 16, qr + c * LPU * 16);
@@ -325,7 +344,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         auto load_gate = [&](const Unit& u) {
             const int bb = live_beam(u);
             if (!fused) return __ldg(a.gates + (long long)u.h * a.arena_slots + a.bases.base[u.req] + bb);
-            const long long in_row = ((long long)u.req * a.W + bb) * a.H + u.h;
+            const long long in_row = vrow_in(u.req, bb, u.h);
             return make_float2(__ldg(a.alpha_in + in_row), __ldg(a.beta_in + in_row));
         };
         // staging layout of the request whose quads are being looked at (the same for all heads of a request)
@@ -394,11 +413,23 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 }
                 cur.own.gate = gate0;
                 if (fused && beam_of(u0) < a.W) {   // the append: this beam's record goes to its arena slot, bit for bit
-                    uint4* dst = reinterpret_cast<uint4*>(a.kv_out + (own_row0 + bb) * REC_BYTES) + g;
+                    if constexpr (GROUPED) {
+                        const long long slot = a.bases.base[u0.req] + bb;
+                        uint4* vdst = reinterpret_cast<uint4*>(a.vv_out + ((long long)u0.h * a.arena_slots + slot) * (DV * 2)) + g;
 #pragma unroll
-                    for (int c = 0; c < NCH; ++c) {
-                        dst[c * LPU] = cur.own.k[c];
-                        dst[16 + c * LPU] = cur.own.v[c];
+                        for (int c = 0; c < NCH; ++c) vdst[c * LPU] = cur.own.v[c];
+                        if (u0.h % a.g == 0) {     // the key is stored once per key head: by its first value head
+                            uint4* kdst = reinterpret_cast<uint4*>(a.kv_out + ((long long)key_head(u0.h) * a.arena_slots + slot) * (DK * 2)) + g;
+#pragma unroll
+                            for (int c = 0; c < NCH; ++c) kdst[c * LPU] = cur.own.k[c];
+                        }
+                    } else {
+                        uint4* dst = reinterpret_cast<uint4*>(a.kv_out + (own_row0 + bb) * REC_BYTES) + g;
+#pragma unroll
+                        for (int c = 0; c < NCH; ++c) {
+                            dst[c * LPU] = cur.own.k[c];
+                            dst[16 + c * LPU] = cur.own.v[c];
+                        }
                     }
                     if (g == 0) a.gates_out[own_row0 + bb] = gate0;
                 }
@@ -429,7 +460,23 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             for (int e = 0; e < 4 * NCH; ++e) corr[e] = make_float2(0.f, 0.f);
             float decay = 1.f;
             L::fold_chain_simple(cur.own, old - 1, staged_levels,
-                          [&](int level) { return L::load_global(kv, a.gates, plane_row0 + idx_of(level), g); }, r, corr, decay);
+                          [&](int level) {
+                              const long long slot = idx_of(level);
+                              if constexpr (GROUPED) {
+                                  RecT rec;
+                                  const uint4* kp = reinterpret_cast<const uint4*>(k_at(u0.h, slot)) + g;
+                                  const uint4* vp = reinterpret_cast<const uint4*>(v_at(u0.h, slot)) + g;
+#pragma unroll
+                                  for (int c = 0; c < NCH; ++c) {
+                                      rec.k[c] = __ldg(kp + c * LPU);
+                                      rec.v[c] = __ldg(vp + c * LPU);
+                                  }
+                                  rec.gate = __ldg(a.gates + plane_row0 + slot);
+                                  return rec;
+                              } else {
+                                  return L::load_global(kv, a.gates, plane_row0 + slot, g);
+                              }
+                          }, r, corr, decay);
             // The segment's staging is waited for even when it holds nothing: it keeps this warp from running past
             // the epilogue warps' preparation of the segment after next (whose barriers share these phases).
             if (!staged_ready && (staged_levels > 0 || seg_last)) {
@@ -500,8 +547,14 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             const long long plane_row0 = (long long)h * a.arena_slots;
             const int li = (warp - FOLD_WARPS) * 32 + lane;
             if (li < count) {
-                const long long row = plane_row0 + __ldg(a.ulist + req * a.ulist_req_stride + li);
-                bulk_load(smem_u32(stage + (b * STAGE_BUF + li) * REC_BYTES), kv + row * REC_BYTES, REC_BYTES, bar_stage(b));
+                const long long slot = __ldg(a.ulist + req * a.ulist_req_stride + li), row = plane_row0 + slot;
+                const uint32_t dst = smem_u32(stage + (b * STAGE_BUF + li) * REC_BYTES);
+                if constexpr (GROUPED) {      // the two halves of the staged row come from the two planes
+                    bulk_load(dst, k_at(h, slot), DK * 2, bar_stage(b));
+                    bulk_load(dst + DK * 2, v_at(h, slot), DV * 2, bar_stage(b));
+                } else {
+                    bulk_load(dst, kv + row * REC_BYTES, REC_BYTES, bar_stage(b));
+                }
                 gates_s[b * STAGE_BUF + li] = __ldg(a.gates + row);
             }
             mbar_expect_tx(bar_stage(b), li < count ? REC_BYTES : 0);
@@ -669,9 +722,9 @@ int make_partition(int total_groups, int gpp, int sms, Partition* part) {
     return greedy_fill(total_groups, gpp, lo, sms, part->begin);
 }
 
-template <typename OutT>
+template <typename OutT, bool GROUPED>
 cudaError_t launch_ws_t(const DecodeArgs& a, cudaStream_t stream) {
-    auto kern = decode_ws_kernel<OutT>;
+    auto kern = decode_ws_kernel<OutT, GROUPED>;
     static bool configured = false;
     static int sms = 148;
     if (!configured) {
@@ -717,8 +770,9 @@ bool decode_sm100_supported(int32_t dk, int32_t dv, int32_t rec_dtype) {
     return dk == 128 && dv == 128 && rec_dtype == ONELA_DTYPE_BF16;
 }
 
-cudaError_t launch_decode_sm100_ws(const DecodeArgs& a, int32_t out_dtype, cudaStream_t stream) {
-    return out_dtype == ONELA_DTYPE_BF16 ? launch_ws_t<__nv_bfloat16>(a, stream) : launch_ws_t<float>(a, stream);
+cudaError_t launch_decode_sm100_ws(const DecodeArgs& a, int32_t out_dtype, bool grouped, cudaStream_t stream) {
+    if (grouped) return out_dtype == ONELA_DTYPE_BF16 ? launch_ws_t<__nv_bfloat16, true>(a, stream) : launch_ws_t<float, true>(a, stream);
+    return out_dtype == ONELA_DTYPE_BF16 ? launch_ws_t<__nv_bfloat16, false>(a, stream) : launch_ws_t<float, false>(a, stream);
 }
 
 }  // namespace onela

@@ -53,6 +53,11 @@ struct DecodeArgs {
     long long sidx_req_stride, ulist_req_stride, uoff_req_stride;
     int32_t req_count, W, H, depth, max_beam;
     BatchBases bases;
+    // grouped value heads (tensor-core kernel only; H above is then the number of VALUE heads): kv / kv_out are the
+    // layer's key plane [Hk][arena_slots][dk], vv / vv_out its value plane [H][arena_slots][dv]; q and k_in have Hk heads
+    const char* vv;
+    char* vv_out;
+    int32_t Hk, g;
 };
 
 // Grouped value heads (Hv = g * Hk): what the grouped decode kernel needs.
@@ -121,6 +126,6 @@ bool decode_generic_supported(int32_t dk, int32_t dv, int32_t rec_dtype);
 cudaError_t launch_decode_gtr(const DecodeArgs& a, int32_t dk, int32_t dv, int32_t rec_dtype, int32_t out_dtype,
                               bool* supported, cudaStream_t stream);
 bool decode_sm100_supported(int32_t dk, int32_t dv, int32_t rec_dtype);
-cudaError_t launch_decode_sm100_ws(const DecodeArgs& a, int32_t out_dtype, cudaStream_t stream);
+cudaError_t launch_decode_sm100_ws(const DecodeArgs& a, int32_t out_dtype, bool grouped, cudaStream_t stream);
 
 }  // namespace onela

@@ -35,12 +35,13 @@ def _grouped_case(wl, g):
     return case
 
 
-def _run(wl, g, out_dtype, fused, tight=None):
+def _run(wl, g, out_dtype, fused, tight=None, flags=0):
     Hk = wl.H // g
     case = _grouped_case(wl, g)
-    cfg = P.make_config(wl.R, wl.L, Hk, wl.dk, wl.dv, wl.W, wl.D, wl.dtype, out_dtype, wl.R * wl.W * wl.D, 0, num_v_heads=wl.H)
+    cfg = P.make_config(wl.R, wl.L, Hk, wl.dk, wl.dv, wl.W, wl.D, wl.dtype, out_dtype, wl.R * wl.W * wl.D, flags, num_v_heads=wl.H)
     ctx = P.Onela(cfg, device="cuda")
-    assert not ctx.onela_uses_tensor_core_path()
+    # the tensor-core kernel takes 128 x 128 bf16 records, grouped or not; everything else runs on CUDA cores
+    assert bool(ctx.onela_uses_tensor_core_path()) == ((wl.dk, wl.dv, wl.dtype) == (128, 128, "bf16") and not flags)
     dev = torch.device("cuda")
     for (r, l), S in case["S0"].items():
         ctx.onela_init_shared_state(r, l, S.to(dev))
@@ -68,10 +69,20 @@ def _run(wl, g, out_dtype, fused, tight=None):
     return case, ctx, worst
 
 
-@pytest.mark.parametrize("g,fused", [(2, False), (4, True)])
-def test_grouped_heads_bf16(g, fused):
+@pytest.mark.parametrize("g,fused,flags", [(2, False, 0), (4, True, 0), (2, True, P.FLAG_FORCE_GENERIC), (1, True, 0)])
+def test_grouped_heads_bf16(g, fused, flags):
+    """Tensor-core kernel (separate and fused append) and, forced, the CUDA-core kernels; g = 1 with num_v_heads set
+    is the ungrouped path."""
     wl = CFG1.scaled(R=2, L=2, H=8, W=70, D=3, prompt_len=64, parents="zipf", zipf_s=1.3, seed=1300 + g)
-    _run(wl, g, "bf16", fused)
+    _run(wl, g, "bf16", fused, flags=flags)
+
+
+def test_grouped_heads_on_the_tensor_core_kernel_many_segments_and_depth():
+    """More (request, value head) pairs than SMs, staged and gathered ancestors, ragged groups: the grouped
+    instantiation of the tensor-core kernel walks several segments per CTA."""
+    wl = CFG1.scaled(R=6, L=1, H=32, W=100, D=6, prompt_len=32, parents="zipf", zipf_s=1.4, seed=1330)
+    _, ctx, worst = _run(wl, 4, "fp32", True)
+    assert ctx.onela_uses_tensor_core_path() and worst <= REL_L2_BAR
 
 
 def test_grouped_heads_fp32_is_tight_and_other_shapes():
@@ -80,10 +91,11 @@ def test_grouped_heads_fp32_is_tight_and_other_shapes():
     _run(CFG1.scaled(H=4, dk=128, dv=256, W=40, D=3, prompt_len=32, seed=1312), 2, "fp32", True)
 
 
-def test_split_record_planes_hold_the_appended_bytes():
+@pytest.mark.parametrize("fused", [False, True])
+def test_split_record_planes_hold_the_appended_bytes(fused):
     wl = CFG1.scaled(R=1, L=1, H=4, W=10, D=2, prompt_len=16, seed=1320)
     g, Hk = 2, 2
-    case, ctx, _ = _run(wl, g, "fp32", False)
+    case, ctx, _ = _run(wl, g, "fp32", fused)
     c = ctx.cfg
     al = lambda n: (n + 1023) // 1024 * 1024
     n_idx = c.num_requests * c.max_steps * c.max_beam * 4

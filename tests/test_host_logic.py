@@ -169,11 +169,11 @@ def test_select_beams_argument_checks():
 
 
 def test_grouped_value_heads_configs():
-    """num_v_heads must be a multiple of num_heads; grouped contexts run on CUDA cores, take no prefill and no delta
-    records, and count k once per key head in the resident bytes."""
+    """num_v_heads must be a multiple of num_heads; grouped contexts take no prefill and no delta records, and count
+    k once per key head in the resident bytes."""
     ok = P.make_config(1, 1, 2, 128, 128, 8, 3, "bf16", "bf16", 64, P.FLAG_DRY_RUN, num_v_heads=6)
     o = P.Onela(ok, device="cpu")
-    assert not o.onela_uses_tensor_core_path()
+    assert o.onela_uses_tensor_core_path()                                      # 128 x 128 bf16: grouped or not
     o.onela_init_shared_state(0, 0, FAKE)
     assert o.lib.onela_prefill_shared_state(o.handle, 0, 0, FAKE, FAKE, FAKE, FAKE, 4, None) == binding.E_UNSUPPORTED
     o.onela_reorder_beams(0, 1, None, 8)
