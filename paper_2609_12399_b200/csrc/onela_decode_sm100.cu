@@ -19,6 +19,9 @@
 // levels are staged in shared memory, one 512-byte bulk copy per DISTINCT ancestor record (as many whole levels
 // as fit).  S_0 and the staging area are double-buffered, so a CTA moves from one segment to the next without
 // draining: nothing in the main loop is a CTA-wide barrier.
+// A second instantiation (GROUPED) serves grouped value heads: segments are (request, VALUE head), the query and the
+// keys are those of key head h / g, and a record's two halves live in two planes (keys per key head, values per value
+// head), so staging and gathers read both and the fused append writes a key once, by its first value head.
 // The kernel is launched as a programmatic dependent launch: it sets itself up and reads the first S_0 while
 // the previous kernel of the stream drains, and waits for that kernel before it touches anything else.
 // Every wait is bounded and also gives up when another role has raised the abort flag; a role that gives up
