@@ -98,14 +98,6 @@ struct Head {           // what a unit's fold needs first
     RecT own;
 };
 
-#ifdef ONELA_SPAN   // instrumented builds only: per-CTA start / dependency-wait return / end times
-__device__ unsigned long long g_span[64][160][4];
-__device__ __forceinline__ unsigned long long gtime2() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-#endif
 
 // Contiguous ranges of groups, one per CTA, balanced on the host with the cost of starting a segment counted in.
 constexpr int MAX_CTAS = 160;
@@ -117,11 +109,8 @@ struct Partition {
 // the key heads' plane (a.kv) and its v in the value heads' plane (a.vv), 256 bytes each.
 template <typename OutT, bool GROUPED>
 __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ Partition part,
-                                                               int groups_per_pair, int launch_id) {
+                                                               int groups_per_pair) {
     extern __shared__ uint8_t smem_raw[];
-#ifdef ONELA_SPAN
-    if (threadIdx.x == 0) g_span[launch_id & 63][blockIdx.x][0] = gtime2();
-#endif
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;            // swizzle atoms need 1024-byte alignment
     uint8_t* smem = smem_raw + (base - raw);
@@ -169,9 +158,6 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
-#ifdef ONELA_SPAN
-    if (threadIdx.x == 0) g_span[launch_id & 63][blockIdx.x][3] = gtime2();
-#endif
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next launch may set itself up under this one
 
     const int g_begin = part.begin[blockIdx.x], g_end = part.begin[blockIdx.x + 1];
@@ -261,9 +247,6 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     // sense - L2 is the point of coherence - and are made before it.
     auto dependency_wait = [&]() {
         asm volatile("griddepcontrol.wait;" ::: "memory");
-#ifdef ONELA_SPAN
-        if (threadIdx.x == 0) g_span[launch_id & 63][blockIdx.x][2] = gtime2();
-#endif
     };
 
     // How many of the oldest levels of a request's chains fit in `stage_cap` staged records (whole levels only), and
@@ -672,9 +655,6 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     if (warp == 0) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
-#ifdef ONELA_SPAN
-    if (threadIdx.x == 0) g_span[launch_id & 63][blockIdx.x][1] = gtime2();
-#endif
 }
 
 int sm_count_ws() {
@@ -745,7 +725,6 @@ cudaError_t launch_ws_t(const DecodeArgs& a, cudaStream_t stream) {
         part_ctas = make_partition(total_groups, groups_per_pair, sms, &part);
         part_total = total_groups; part_gpp = groups_per_pair; part_sms = sms;
     }
-    static int launch_id = 0;
     // Programmatic dependent launch: this launch's CTAs may start, allocate and read S_0 while the previous
     // kernel of the stream drains; the kernel waits for that kernel's completion before it reads anything else.
     cudaLaunchConfig_t cfg = {};
@@ -758,16 +737,11 @@ cudaError_t launch_ws_t(const DecodeArgs& a, cudaStream_t stream) {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, a, part, groups_per_pair, launch_id++);
+    return cudaLaunchKernelEx(&cfg, kern, a, part, groups_per_pair);
 }
 
 }  // namespace
 
-#ifdef ONELA_SPAN
-extern "C" int onela_debug_spans(unsigned long long* host_out) {   // instrumented builds only
-    return (int)cudaMemcpyFromSymbol(host_out, g_span, sizeof(g_span));
-}
-#endif
 
 bool decode_sm100_supported(int32_t dk, int32_t dv, int32_t rec_dtype) {
     return dk == 128 && dv == 128 && rec_dtype == ONELA_DTYPE_BF16;
