@@ -268,6 +268,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
                      "traffic_note": "ncu DRAM read+write bytes of one launch at the deepest call (depth %d), whose "
                                      "algorithmic bytes are %.1f MB; see profiles/" % (wl.D, per_depth[-1]["algorithmic"] / 1e6),
                      "peak_source": peak_src,
+                     "frac_of_nominal_8_tbs": achieved_gbs / 8000.0,   # context: the paper-independent nominal HBM3e figure
                      "timing": "CUDA events around every decode launch" if per == 1 else
                                "CUDA events around the %d back-to-back decode launches (one per layer) of each decode call" % per,
                      "kernel": ("decode_step" if args.unfused else "append_decode_step") + " (all requests of one layer per launch)",
