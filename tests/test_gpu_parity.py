@@ -235,6 +235,29 @@ def test_prefill_kernel_matches_oracle_prefill():
         assert err.max() < 1e-5, err      # fp32 recurrence against the fp64 one
 
 
+def test_empty_prompt_gives_the_zero_state():
+    """A prompt of no tokens: the prefill call stores S_0 = 0 and the decode outputs come from the records alone."""
+    wl = CFG1.scaled(H=2, W=24, D=2, prompt_len=0, seed=88)
+    cfg = P.make_config(1, 1, wl.H, wl.dk, wl.dv, wl.W, wl.D, wl.dtype, "fp32", wl.W * wl.D, 0)
+    ctx = P.Onela(cfg, device="cuda")
+    empty = lambda *shape: torch.empty(shape, device="cuda")
+    ctx.onela_prefill_shared_state(0, 0, empty(0, wl.H, wl.dk).to(wl.torch_dtype), empty(0, wl.H, wl.dv).to(wl.torch_dtype),
+                                   empty(0, wl.H), empty(0, wl.H))
+    assert torch.count_nonzero(ctx.onela_export_shared_state(0, 0)) == 0
+    S0 = np.zeros((wl.H, wl.dv, wl.dk), np.float32)
+    steps, pars = [], []
+    for t in range(wl.D):
+        par = None if t == 0 else inputs.parents(wl, 0, t)
+        tk = inputs.decode_token(wl, 0, 0, t)
+        q = inputs.decode_query(wl, 0, 0, t)
+        steps.append(tk); pars.append(par)
+        ctx.onela_reorder_beams(0, 1, None if par is None else par[None].cuda(), wl.W)
+        out = torch.empty((1, wl.W, wl.H, wl.dv), dtype=torch.float32, device="cuda")
+        ctx.onela_append_decode_step(0, 1, 0, *(tk[n][None].cuda() for n in ("k", "v", "alpha", "beta")), q[None].cuda(), out)
+        ref = oracle.decode(S0, steps, pars, q)
+        assert rel_l2(out[0].cpu().numpy(), ref).max() <= REL_L2_BAR
+
+
 def test_init_then_export_round_trip():
     wl = CFG1.scaled(H=2)
     ctx = P.Onela(P.make_config(1, 1, 2, 128, 128, 8, 2, "bf16", "fp32", 16))
