@@ -235,6 +235,37 @@ def test_prefill_kernel_matches_oracle_prefill():
         assert err.max() < 1e-5, err      # fp32 recurrence against the fp64 one
 
 
+def test_two_contexts_interleaved_on_one_stream():
+    """Two contexts of different shapes take turns on the same stream: per-launch set-up that depends on the shape
+    (group partition, head counts) must follow the call, not the previous context's."""
+    wa = CFG1.scaled(R=2, H=4, W=130, D=3, prompt_len=32, parents="zipf", zipf_s=1.3, seed=931)
+    wb = CFG1.scaled(R=1, H=7, W=49, D=3, prompt_len=32, seed=932)
+    cases = [make_case(wa), make_case(wb)]
+    refs = [run_oracle(c)[0] for c in cases]
+    dev = torch.device("cuda")
+    ctxs = []
+    for wl, case in zip((wa, wb), cases):
+        cfg = P.make_config(wl.R, 1, wl.H, wl.dk, wl.dv, wl.W, wl.D, wl.dtype, "fp32", wl.R * wl.W * wl.D, 0)
+        ctx = P.Onela(cfg, device="cuda")
+        for r in range(wl.R):
+            ctx.onela_init_shared_state(r, 0, case["S0"][(r, 0)].to(dev))
+        ctxs.append(ctx)
+    for t in range(3):
+        outs = []
+        for wl, case, ctx in zip((wa, wb), cases, ctxs):       # a, b, a, b, ... with no synchronisation in between
+            par = None if t == 0 else torch.stack([case["parents"][(r, t)] for r in range(wl.R)]).to(dev)
+            ctx.onela_reorder_beams(0, wl.R, par, wl.W)
+            tk = {n: torch.stack([case["tok"][(r, 0, t)][n] for r in range(wl.R)]).to(dev) for n in ("k", "v", "alpha", "beta")}
+            q = torch.stack([case["q"][(r, 0, t)] for r in range(wl.R)]).to(dev)
+            out = torch.empty((wl.R, wl.W, wl.H, wl.dv), dtype=torch.float32, device=dev)
+            ctx.onela_append_decode_step(0, wl.R, 0, tk["k"], tk["v"], tk["alpha"], tk["beta"], q, out)
+            outs.append(out)
+        for wl, ref, out in zip((wa, wb), refs, outs):
+            for r in range(wl.R):
+                assert rel_l2(out[r].cpu().numpy(), ref[(r, 0, t)]).max() <= REL_L2_BAR
+    assert all(c.onela_poll_device_status() == (0, 0) for c in ctxs)
+
+
 def test_empty_prompt_gives_the_zero_state():
     """A prompt of no tokens: the prefill call stores S_0 = 0 and the decode outputs come from the records alone."""
     wl = CFG1.scaled(H=2, W=24, D=2, prompt_len=0, seed=88)
