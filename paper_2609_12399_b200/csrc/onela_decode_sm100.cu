@@ -71,9 +71,11 @@ constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + STAGE_BYTES + GATE_BYTES + HEADS
 constexpr uint32_t S0_COL = 128;                 // accumulators of the ring slots in [0, SLOTS * GN); S_0 buffers at 128 and 256
 constexpr uint32_t TMEM_COLS = 512;
 static_assert(SLOTS * GN <= 128, "accumulator columns");
+static_assert(R_BYTES >= C_BYTES, "the accumulators are transposed over the operand rows");
 static_assert(2 * STAGE_BUF <= 128, "one staged record per epilogue lane");
 static_assert(SMEM_BYTES <= 232448, "shared memory per CTA");
 static_assert(GN % 16 == 0 && GN >= 16 && GN <= 256, "MMA N");
+static_assert((GN * 16) % 96 == 0, "three storing warps share a group's 16-byte chunks evenly");
 using L = Lanes<LPU>;
 using RecT = L::R;
 
@@ -559,73 +561,97 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             prepare_s0(1);
         }
 
-        for (int gi = g_begin; gi < g_end && !dead; ++gi) {
-            const int gcount = gi - g_begin;
+        // The first epilogue warp issues a group's 16 MMAs as soon as all its rows are written (never a fold warp:
+        // whichever fold warp issued would be the last to finish its next quad).  It does so one group AHEAD: once
+        // the tile of group k is complete (the named barrier below) it issues group k + 1 while the other three
+        // warps store group k, so neither the issuing nor the MMAs' latency lies between two epilogues.
+        auto issue_mma = [&](int gcount, int seg, bool seg_first) -> bool {     // warp FOLD_WARPS only; true: gave up
             const int s = gcount % SLOTS, use = gcount / SLOTS;
-            const int pair = gi / groups_per_pair, seg = pair - pair_begin;
-            const int req = pair / a.H, h = pair - req * a.H;
-            const bool seg_first = gi == g_begin || gi == pair * groups_per_pair;
-            if (warp == FOLD_WARPS) {
-                // One thread issues the group's 16 MMAs as soon as all its rows are written (never a fold warp:
-                // whichever fold warp issued would be the last to finish its next quad).
-                int mma_failed = 0;
-                if (lane == 0) {
-                    bool ok = wait_or_abort(bar_full(s), use & 1, abort_flag);
-                    // segment 0's S_0 has a barrier of its own; segment seg >= 1 is use ((seg + 1) >> 1) - 1 of its
-                    // buffer's barrier
-                    if (ok && seg_first && seg >= 1) ok = wait_or_abort(bar_s0(seg & 1), (((seg + 1) >> 1) - 1) & 1, abort_flag);
-                    if (ok && gi == g_begin) ok = wait_or_abort(bar_s0_first, 0, abort_flag);
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    if (ok) {
-                        constexpr uint32_t idesc = idesc_tf32(GN);
-                        const uint64_t bd = umma_desc(smem_u32(ring + s * SLOT_BYTES));
-                        const uint32_t s0_at = tmem_base + S0_COL + (seg & 1) * 128;
+            int mma_failed = 0;
+            if (lane == 0) {
+                bool ok = wait_or_abort(bar_full(s), use & 1, abort_flag);
+                // segment 0's S_0 has a barrier of its own; segment seg >= 1 is use ((seg + 1) >> 1) - 1 of its
+                // buffer's barrier
+                if (ok && seg_first && seg >= 1) ok = wait_or_abort(bar_s0(seg & 1), (((seg + 1) >> 1) - 1) & 1, abort_flag);
+                if (ok && gcount == 0) ok = wait_or_abort(bar_s0_first, 0, abort_flag);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                if (ok) {
+                    constexpr uint32_t idesc = idesc_tf32(GN);
+                    const uint64_t bd = umma_desc(smem_u32(ring + s * SLOT_BYTES));
+                    const uint32_t s0_at = tmem_base + S0_COL + (seg & 1) * 128;
 #pragma unroll
-                        for (int kb = 0; kb < 4; ++kb)
+                    for (int kb = 0; kb < 4; ++kb)
 #pragma unroll
-                            for (int ks = 0; ks < 4; ++ks)
-                                umma_tf32_ts(tmem_base + s * GN, s0_at + (kb * 4 + ks) * 8,
-                                             bd + (uint64_t)((kb * R_KB_STRIDE + ks * 32) >> 4), idesc, (kb | ks) ? 1u : 0u);
-                    } else {
-                        mma_failed = 1;
-                    }
-                    umma_commit(bar_done(s));   // arrives when the MMAs above have completed
+                        for (int ks = 0; ks < 4; ++ks)
+                            umma_tf32_ts(tmem_base + s * GN, s0_at + (kb * 4 + ks) * 8,
+                                         bd + (uint64_t)((kb * R_KB_STRIDE + ks * 32) >> 4), idesc, (kb | ks) ? 1u : 0u);
+                } else {
+                    mma_failed = 1;
                 }
-                if (__shfl_sync(0xffffffffu, mma_failed, 0)) { dead = true; break; }
+                umma_commit(bar_done(s));   // arrives when the MMAs above have completed
+            }
+            return __shfl_sync(0xffffffffu, mma_failed, 0) != 0;
+        };
+        // (request, head, group within the pair) of the group at hand, advanced without divisions
+        int pair = pair_begin, req = pair / a.H, h = pair - req * a.H, gip = g_begin - pair * groups_per_pair;
+        int issued = 0;                               // groups whose MMAs have been issued (first epilogue warp)
+        for (int gcount = 0; gcount < g_end - g_begin && !dead; ++gcount) {
+            const int s = gcount % SLOTS, use = gcount / SLOTS;
+            const int seg = pair - pair_begin;
+            const bool seg_first = gcount == 0 || gip == 0;
+            const bool has_next = gcount + 1 < g_end - g_begin;
+            const bool next_first = gip + 1 == groups_per_pair;      // the next group opens a segment
+            if (warp == FOLD_WARPS && issued == gcount) {
+                if (issue_mma(gcount, seg, seg_first)) { dead = true; break; }
+                ++issued;
             }
             if (!wait_or_abort(bar_done(s), use & 1, abort_flag)) { dead = true; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             float* C_s = reinterpret_cast<float*>(ring + s * SLOT_BYTES + R_BYTES);
-            const int b0 = (gi - pair * groups_per_pair) * GN;
+            const int b0 = gip * GN;
             const uint32_t taddr = tmem_base + s * GN + ((uint32_t)(quad * 32) << 16);
+            float* A_s = reinterpret_cast<float*>(ring + s * SLOT_BYTES);   // the operand rows are dead once the MMAs have completed
             {
-                // accumulator rows (dv) of this thread, all beams of the group, added onto the corr tile in place
+                // accumulator rows (dv) of this thread, all beams of the group, transposed into a tile laid out like
+                // the corr tile, over the slot's operand rows (plain stores: nothing here waits for a shared-memory read)
                 uint32_t v[GN];
 #pragma unroll
                 for (int c0 = 0; c0 < GN; c0 += 16) tmem_ld16(taddr + c0, v + c0);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 const int ip = corr_chunk(i >> 2) * 4 + (i & 3);   // where the corr tile keeps element i of a row
 #pragma unroll
-                for (int j = 0; j < GN; ++j) C_s[j * DV + ip] += __uint_as_float(v[j]);
+                for (int j = 0; j < GN; ++j) A_s[j * DV + ip] = __uint_as_float(v[j]);
             }
             if (bar_or(1, 128, 0)) { dead = true; break; }     // the four epilogue warps: tile complete
-            {
-                // coalesced stores: 16 lanes cover one beam's 128 outputs, 8 elements each
-                const int et = (warp - FOLD_WARPS) * 32 + lane;
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            if (warp == FOLD_WARPS) {
+                // This warp's part of the slot is read out; the next group's MMAs go out now - unless that group
+                // opens a segment whose S_0 this very iteration prepares below (a one-group segment).
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_free(s));
+                if (has_next && !(next_first && seg_first && seg >= 1)) {
+                    if (issue_mma(gcount + 1, seg + (next_first ? 1 : 0), next_first)) { dead = true; break; }
+                    ++issued;
+                }
+            } else {
+                // coalesced stores by the other three warps: 16 lanes cover one beam's 128 outputs, 8 elements each
+                const int et = (warp - FOLD_WARPS - 1) * 32 + lane;
+                OutT* out0 = static_cast<OutT*>(a.out) + (((long long)req * a.W + b0) * a.H + h) * DV;
 #pragma unroll
-                for (int it = 0; it < GN * 16 / 128; ++it) {   // GN * 16 chunks of 16 bytes over 128 threads
-                    const int idx = it * 128 + et, j = idx >> 4, ch = idx & 15;
+                for (int it = 0; it < GN * 16 / 96; ++it) {    // GN * 16 chunks of 16 bytes over 96 threads
+                    const int idx = it * 96 + et, j = idx >> 4, ch = idx & 15;
                     if (b0 + j < a.W) {
-                        const float4 x0 = *reinterpret_cast<const float4*>(C_s + j * DV + corr_chunk(2 * ch) * 4);
-                        const float4 x1 = *reinterpret_cast<const float4*>(C_s + j * DV + corr_chunk(2 * ch + 1) * 4);
-                        const float o[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-                        store8<OutT>(static_cast<OutT*>(a.out) + (((long long)req * a.W + b0 + j) * a.H + h) * DV + ch * 8, o);
+                        const int o0 = j * DV + corr_chunk(2 * ch) * 4, o1 = j * DV + corr_chunk(2 * ch + 1) * 4;
+                        const float4 x0 = *reinterpret_cast<const float4*>(C_s + o0), y0 = *reinterpret_cast<const float4*>(A_s + o0);
+                        const float4 x1 = *reinterpret_cast<const float4*>(C_s + o1), y1 = *reinterpret_cast<const float4*>(A_s + o1);
+                        const float o[8] = {x0.x + y0.x, x0.y + y0.y, x0.z + y0.z, x0.w + y0.w,
+                                            x1.x + y1.x, x1.y + y1.y, x1.z + y1.z, x1.w + y1.w};
+                        store8<OutT>(out0 + (long long)j * a.H * DV + ch * 8, o);
                     }
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_free(s));
             }
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_free(s));
 
             // Past the first group of segment seg >= 1 every MMA of segment seg - 1 has completed and the fold warps
             // have read its staging buffer out (they signal that): both are free for segment seg + 1.
@@ -633,6 +659,11 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 if (!wait_or_abort(bar_sfree((seg + 1) & 1), ((seg - 1) >> 1) & 1, abort_flag)) { dead = true; break; }
                 stage_segment(seg + 1);
                 prepare_s0(seg + 1);
+            }
+            if (++gip == groups_per_pair) {
+                gip = 0;
+                ++pair;
+                if (++h == a.H) { h = 0; ++req; }
             }
         }
         if (dead && lane == 0) *abort_flag = 1;
