@@ -8,10 +8,13 @@
 //     they come from the caller's token tensors and the warp also writes them to the arena.  Results go into a
 //     ring slot in shared memory: the folded query as a row of the K-major 128-byte-swizzled MMA operand
 //     (rounded to TF32), corr as a row of the slot's corr tile.
-//   * 4 EPILOGUE warps (one per tensor-memory lane quadrant).  One lane issues the group's 16 MMAs once all
-//     its rows are written; when they have completed the four warps read the accumulator, add it onto the
-//     corr tile, store the outputs as coalesced 16-byte rows and hand the slot back.  They also prepare the
-//     next segment (below) while the fold warps work on the current one.
+//   * 4 EPILOGUE warps (one per tensor-memory lane quadrant).  One lane of the first issues a group's 16 MMAs
+//     once all its rows are written - one group ahead of the epilogue, so neither the issuing nor the MMAs'
+//     latency lies between two epilogues.  When a group's MMAs have completed the four warps read the
+//     accumulator and transpose it, by plain stores, over the slot's operand rows (dead by then); the other
+//     three warps add that tile to the corr tile and store the outputs as coalesced 16-byte rows while the
+//     first issues the next group; then the slot is handed back.  They also prepare the next segment (below)
+//     while the fold warps work on the current one.
 // Two ring slots (operand rows, corr tile, 48 accumulator columns each) keep the MMA and the epilogue of one
 // group under the folds of the next.  Work = groups of 48 consecutive beams of one (request, head), a
 // contiguous range per CTA chosen on the host; consecutive groups of one head form a segment.  Per segment the
