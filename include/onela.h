@@ -94,7 +94,9 @@ typedef struct onela_config {
     int32_t num_requests; /* request slots */
     int32_t num_layers;   /* GDN layers sharing the ancestry index */
     int32_t num_heads;    /* key heads (and value heads, unless num_v_heads says otherwise) */
-    int32_t dk, dv;       /* head dimensions of k/q and of v/o */
+    int32_t dk, dv;       /* head dimensions of k/q and of v/o: (32, 32), (64, 64), (128, 128), (128, 256), (256, 256),
+                           * (128, 512) or (256, 512), else ONELA_E_UNSUPPORTED; 128 x 128 with bf16 records runs on
+                           * the tensor-core kernel, every other shape on CUDA cores */
     int32_t max_beam;     /* largest beam width W_t */
     int32_t max_steps;    /* largest number of decode calls per request (chain depth) */
     int32_t rec_dtype;    /* dtype of q, k, v: ONELA_DTYPE_* */

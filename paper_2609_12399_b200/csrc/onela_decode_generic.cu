@@ -192,7 +192,7 @@ cudaError_t launch_dims(const DecodeArgs& a, int32_t rec_dtype, int32_t out_dtyp
 bool decode_generic_supported(int32_t dk, int32_t dv, int32_t rec_dtype) {
     (void)rec_dtype;
     return (dk == 32 && dv == 32) || (dk == 64 && dv == 64) || (dk == 128 && dv == 128) ||
-           (dk == 128 && dv == 256) || (dk == 256 && dv == 256);
+           (dk == 128 && dv == 256) || (dk == 256 && dv == 256) || (dk == 128 && dv == 512) || (dk == 256 && dv == 512);
 }
 
 cudaError_t launch_decode_generic(const DecodeArgs& a, int32_t dk, int32_t dv, int32_t rec_dtype,
@@ -203,6 +203,8 @@ cudaError_t launch_decode_generic(const DecodeArgs& a, int32_t dk, int32_t dv, i
     if (dk == 128 && dv == 128) return launch_dims<128, 128>(a, rec_dtype, out_dtype, stream);
     if (dk == 128 && dv == 256) return launch_dims<128, 256>(a, rec_dtype, out_dtype, stream);
     if (dk == 256 && dv == 256) return launch_dims<256, 256>(a, rec_dtype, out_dtype, stream);
+    if (dk == 128 && dv == 512) return launch_dims<128, 512>(a, rec_dtype, out_dtype, stream);
+    if (dk == 256 && dv == 512) return launch_dims<256, 512>(a, rec_dtype, out_dtype, stream);
     *supported = false;
     return cudaErrorInvalidValue;
 }

@@ -147,7 +147,7 @@ def test_depth_one_and_max_depth():
 
 
 @pytest.mark.parametrize("dk,dv,dtype", [(64, 64, "bf16"), (64, 64, "fp32"), (128, 128, "fp32"), (128, 256, "bf16"),
-                                         (256, 256, "bf16"), (32, 32, "bf16")])
+                                         (256, 256, "bf16"), (32, 32, "bf16"), (128, 512, "bf16"), (256, 512, "bf16")])
 def test_other_geometries(dk, dv, dtype):
     wl = CFG1.scaled(H=2, dk=dk, dv=dv, dtype=dtype, W=37, D=3, prompt_len=48, seed=dk + dv)
     _full_check(make_case(wl), "fp32")
