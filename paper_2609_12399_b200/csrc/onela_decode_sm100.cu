@@ -4,7 +4,7 @@
 //   * 12 FOLD warps.  8 lanes own one (beam, head) unit; a warp folds 4 units at a time ("quad"): query
 //     folded through the unit's records newest -> oldest (c = k.r; corr += beta c v; r -= beta c k; decay a
 //     scalar; packed fp32x2 FMAs).  A quad's query and own record arrive through a per-warp stage of 16-byte
-//     async copies, one quad ahead (its lines requested into L2 a quad earlier still); with the append fused in
+//     async copies, one quad ahead; with the append fused in
 //     they come from the caller's token tensors and the warp also writes them to the arena.  Results go into a
 //     ring slot in shared memory: the folded query as a row of the K-major 128-byte-swizzled MMA operand
 //     (rounded to TF32), corr as a row of the slot's corr tile.
@@ -31,6 +31,7 @@
 // records ONELA_E_TIMEOUT and stops working; before returning the CTA waits (bounded) for copies still in
 // flight and frees its tensor memory.
 #include <cstdio>
+#include <mutex>
 
 #include "onela_internal.h"
 #include "onela_layout.cuh"
@@ -289,8 +290,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             u0.gip = g_begin - pair * groups_per_pair;
         }
         // The heads of a quad (own record and query of its units) arrive by 16-byte async copies into the warp's
-        // stage, one quad ahead of their use (each lane copies exactly the chunks it reads back); the lines of the
-        // quad after that are requested into L2; the gates ride in registers.
+        // stage, one quad ahead of their use (each lane copies exactly the chunks it reads back); the gates ride in
+        // registers.  The lines of the FIRST quad are requested into L2 before the launch's dependencies are waited
+        // for (requesting every later quad's lines a quad ahead of its copies as well measured 2 % slower).
         auto request_heads = [&](const Unit& n) {        // the 128-byte lines of a quad's heads, into L2
             if (lane < UPW * 6) {
                 const int un = lane / 6, item = lane % 6;
@@ -304,7 +306,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 asm volatile("prefetch.global.L2 [%0];" ::"l"(p2 + (item & 1) * 128));
             }
         };
-        auto issue_head = [&](const Unit& u, const Unit& n, bool has_next) {
+        auto issue_head = [&](const Unit& u) {
             const uint32_t dst = smem_u32(my_heads);
             const int bb = live_beam(u);
             const long long krow = krow_in(u.req, bb, u.h);
@@ -330,7 +332,6 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
 #pragma unroll
             for (int c = 0; c < NCH; ++c) cp_async16(dst + UPW * REC_BYTES + grp * (DK * 2) + (c * LPU + g) * 16, qr + c * LPU * 16);
             asm volatile("cp.async.commit_group;" ::: "memory");
-            if (has_next) request_heads(n);
         };
         auto load_gate = [&](const Unit& u) {
             const int bb = live_beam(u);
@@ -366,7 +367,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         if (n_quads > 0) request_heads(u0);
         dependency_wait();
         if (n_quads > 0) {
-            issue_head(u0, u1, 1 < n_quads);
+            issue_head(u0);
             gate0 = load_gate(u0);
             if (1 < n_quads) gate1 = load_gate(u1);
             idx_next = load_idx(u0);
@@ -426,7 +427,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 }
             }
             gate0 = gate1;
-            if (k + 1 < n_quads) issue_head(u1, u2, k + 2 < n_quads);   // each lane overwrites only the chunks it has just read
+            if (k + 1 < n_quads) issue_head(u1);   // each lane overwrites only the chunks it has just read
             if (k + 2 < n_quads) gate1 = load_gate(u2);
 
             // lane g keeps the index of level g (position in the staged list for staged levels, arena slot
@@ -742,15 +743,15 @@ int make_partition(int total_groups, int gpp, int sms, Partition* part) {
 template <typename OutT, bool GROUPED>
 cudaError_t launch_ws_t(const DecodeArgs& a, cudaStream_t stream) {
     auto kern = decode_ws_kernel<OutT, GROUPED>;
-    static bool configured = false;
+    static std::once_flag once;                  // host threads may share a context's kernels
+    static cudaError_t configure_error = cudaSuccess;
     static int sms = 148;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-        if (e != cudaSuccess) return e;
+    std::call_once(once, [&]() {
+        configure_error = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         sms = sm_count_ws();
         if (sms > MAX_CTAS) sms = MAX_CTAS;
-        configured = true;
-    }
+    });
+    if (configure_error != cudaSuccess) return configure_error;
     const int groups_per_pair = (a.W + GN - 1) / GN;
     const int total_groups = a.req_count * a.H * groups_per_pair;
     static thread_local Partition part;          // the last launch's partition, reused while the shape stays
