@@ -70,7 +70,7 @@ constexpr int HEADS_TOTAL = FOLD_WARPS * HEAD_BYTES;     // one stage per fold w
 // (what is left of the SM's 256 KiB serves the gathered records as L1).
 constexpr int STAGE_BUF = ONELA_STAGE_BUF;
 constexpr int STAGE_BYTES = 2 * STAGE_BUF * REC_BYTES;
-constexpr int GATE_BYTES = 2 * STAGE_BUF * 8;
+constexpr int GATE_BYTES = (2 * STAGE_BUF * 8 + 127) & ~127;   // padded: the heads' stages behind it stay 128-byte aligned (measured: 1.5 % faster)
 constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + STAGE_BYTES + GATE_BYTES + HEADS_TOTAL + 256 + 1024;
 constexpr uint32_t S0_COL = 128;                 // accumulators of the ring slots in [0, SLOTS * GN); S_0 buffers at 128 and 256
 constexpr uint32_t TMEM_COLS = 512;
@@ -699,15 +699,24 @@ int sm_count_ws() {
     return n;
 }
 
-// Contiguous group ranges for the CTAs.  Starting a segment (a new (request, head): pipeline drained, S_0 reloaded,
-// staging refilled) costs about as much as SEG_COST / GROUP_COST groups, so a CTA's cost is counted as
-// GROUP_COST * groups + SEG_COST * segments and the smallest bound T is searched for which a greedy fill needs no
-// more CTAs than there are SMs.  Returns the number of CTAs used.
-#ifndef ONELA_SEG_COST
-#define ONELA_SEG_COST 3
+// Contiguous group ranges for the CTAs.  A CTA's cost is counted as group_cost * groups + seg_cost * segments (starting
+// a segment: S_0 reloaded, staging refilled, the ring's overlap lost for a moment) and the smallest bound T is searched
+// for which a greedy fill needs no more CTAs than there are SMs.  Returns the number of CTAs used.
+// The costs, in units of ~500 cycles, follow what the kernel measures on the beam-512 stack: a group takes ~4000
+// cycles plus ~500 per chain level beyond the first; starting a segment ~6000 at depth <= 3 (where whole (request,
+// head) pairs per CTA, 128 x 11 groups, beat 141 x 10 groups over two segments by 0.6-1.5 us) and ~3000 deeper (where
+// the shorter CTA wins by 0.6-2.5 us).
+struct PartitionCost {
+    int group, seg;
+};
+PartitionCost partition_cost(int depth) {
+#ifdef ONELA_SEG_COST
+    return {4, ONELA_SEG_COST};
+#else
+    return {8 + (depth > 1 ? depth - 1 : 0), depth <= 3 ? 12 : 6};
 #endif
-constexpr int GROUP_COST = 4, SEG_COST = ONELA_SEG_COST;
-int greedy_fill(int total_groups, int gpp, int limit, int max_ctas, int32_t* begin) {
+}
+int greedy_fill(int total_groups, int gpp, int limit, int max_ctas, PartitionCost c, int32_t* begin) {
     int n = 0, gi = 0;
     while (gi < total_groups) {
         if (n == max_ctas) return max_ctas + 1;
@@ -716,11 +725,11 @@ int greedy_fill(int total_groups, int gpp, int limit, int max_ctas, int32_t* beg
         bool any = false;
         while (gi < total_groups) {
             const int pair_end = (gi / gpp + 1) * gpp;
-            const int room = (limit - cost - SEG_COST) / GROUP_COST;     // groups of this segment that still fit
+            const int room = (limit - cost - c.seg) / c.group;     // groups of this segment that still fit
             if (room <= 0) break;
             const int take = room < pair_end - gi ? room : pair_end - gi;
             gi += take;
-            cost += SEG_COST + take * GROUP_COST;
+            cost += c.seg + take * c.group;
             any = true;
             if (gi < pair_end) break;
         }
@@ -730,14 +739,14 @@ int greedy_fill(int total_groups, int gpp, int limit, int max_ctas, int32_t* beg
     if (begin) begin[n] = total_groups;
     return n;
 }
-int make_partition(int total_groups, int gpp, int sms, Partition* part) {
-    int lo = SEG_COST + GROUP_COST, hi = SEG_COST * (total_groups / gpp + 2) + GROUP_COST * total_groups;
+int make_partition(int total_groups, int gpp, int sms, PartitionCost c, Partition* part) {
+    int lo = c.seg + c.group, hi = c.seg * (total_groups / gpp + 2) + c.group * total_groups;
     while (lo < hi) {
         const int mid = (lo + hi) / 2;
-        if (greedy_fill(total_groups, gpp, mid, sms, nullptr) <= sms) hi = mid;
+        if (greedy_fill(total_groups, gpp, mid, sms, c, nullptr) <= sms) hi = mid;
         else lo = mid + 1;
     }
-    return greedy_fill(total_groups, gpp, lo, sms, part->begin);
+    return greedy_fill(total_groups, gpp, lo, sms, c, part->begin);
 }
 
 template <typename OutT, bool GROUPED>
@@ -755,10 +764,13 @@ cudaError_t launch_ws_t(const DecodeArgs& a, cudaStream_t stream) {
     const int groups_per_pair = (a.W + GN - 1) / GN;
     const int total_groups = a.req_count * a.H * groups_per_pair;
     static thread_local Partition part;          // the last launch's partition, reused while the shape stays
-    static thread_local int part_total = -1, part_gpp = -1, part_sms = -1, part_ctas = 0;
-    if (part_total != total_groups || part_gpp != groups_per_pair || part_sms != sms) {
-        part_ctas = make_partition(total_groups, groups_per_pair, sms, &part);
+    static thread_local int part_total = -1, part_gpp = -1, part_sms = -1, part_group = -1, part_seg = -1, part_ctas = 0;
+    const PartitionCost cost = partition_cost(a.depth);
+    if (part_total != total_groups || part_gpp != groups_per_pair || part_sms != sms || part_group != cost.group ||
+        part_seg != cost.seg) {
+        part_ctas = make_partition(total_groups, groups_per_pair, sms, cost, &part);
         part_total = total_groups; part_gpp = groups_per_pair; part_sms = sms;
+        part_group = cost.group; part_seg = cost.seg;
     }
     // Programmatic dependent launch: this launch's CTAs may start, allocate and read S_0 while the previous
     // kernel of the stream drains; the kernel waits for that kernel's completion before it reads anything else.
