@@ -404,6 +404,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                     cur.q[c] = qv[c * LPU];
                 }
                 cur.own.gate = gate0;
+                // the next quad's copies go out before this quad's stores (each lane overwrites only the chunks it
+                // has just read)
+                if (k + 1 < n_quads) issue_head(u1);
                 if (fused && beam_of(u0) < a.W) {   // the append: this beam's record goes to its arena slot, bit for bit
                     if constexpr (GROUPED) {
                         const long long slot = a.bases.base[u0.req] + bb;
@@ -427,7 +430,6 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 }
             }
             gate0 = gate1;
-            if (k + 1 < n_quads) issue_head(u1);   // each lane overwrites only the chunks it has just read
             if (k + 2 < n_quads) gate1 = load_gate(u2);
 
             // lane g keeps the index of level g (position in the staged list for staged levels, arena slot
@@ -709,12 +711,17 @@ int sm_count_ws() {
 struct PartitionCost {
     int group, seg;
 };
-PartitionCost partition_cost(int depth) {
-#ifdef ONELA_SEG_COST
-    return {4, ONELA_SEG_COST};
-#else
-    return {8 + (depth > 1 ? depth - 1 : 0), depth <= 3 ? 12 : 6};
+#ifndef ONELA_SEG_SHALLOW
+#define ONELA_SEG_SHALLOW 12
 #endif
+#ifndef ONELA_SEG_DEEP
+#define ONELA_SEG_DEEP 6
+#endif
+#ifndef ONELA_SHALLOW_DEPTH
+#define ONELA_SHALLOW_DEPTH 3
+#endif
+PartitionCost partition_cost(int depth) {
+    return {8 + (depth > 1 ? depth - 1 : 0), depth <= ONELA_SHALLOW_DEPTH ? ONELA_SEG_SHALLOW : ONELA_SEG_DEEP};
 }
 int greedy_fill(int total_groups, int gpp, int limit, int max_ctas, PartitionCost c, int32_t* begin) {
     int n = 0, gi = 0;
