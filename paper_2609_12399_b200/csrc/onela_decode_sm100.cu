@@ -32,6 +32,7 @@
 // flight and frees its tensor memory.
 #include <cstdio>
 #include <mutex>
+#include <type_traits>
 
 #include "onela_internal.h"
 #include "onela_layout.cuh"
@@ -113,7 +114,7 @@ struct Partition {
 
 // GROUPED: value head h reads the queries and keys of key head h / g; a.H counts VALUE heads, the record's k lives in
 // the key heads' plane (a.kv) and its v in the value heads' plane (a.vv), 256 bytes each.
-template <typename OutT, bool GROUPED>
+template <typename OutT, bool GROUPED, bool FUSED>
 __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ Partition part,
                                                                int groups_per_pair) {
     extern __shared__ uint8_t smem_raw[];
@@ -172,7 +173,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     const bool single = n_segs == 1;                       // one segment: the two staging buffers serve as one
     const int stage_cap = single ? 2 * STAGE_BUF : STAGE_BUF;
     const int old = a.depth - 1;          // records older than a beam's own: levels old-1 .. 0
-    const bool fused = a.k_in != nullptr;  // append fused in: the newest record comes from the caller's tensors
+    constexpr bool fused = FUSED;          // append fused in: the newest record comes from the caller's tensors
     const char* kv = a.kv;
     const __nv_bfloat16* qbase = static_cast<const __nv_bfloat16*>(a.q);
     // rows of the caller's tensors: q and k have one row per KEY head, v, the gates and the outputs per VALUE head
@@ -257,12 +258,19 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
 
     // How many of the oldest levels of a request's chains fit in `stage_cap` staged records (whole levels only), and
     // how many records that is.  Lane l looks at level l (one load latency for the whole chain); warp-uniform.
-    auto staging_of = [&](int req, int& levels, int& count) {
+    // `sparse` (optional): bit l set when level l has more than W / 4 distinct records, i.e. little sharing - the
+    // levels whose gathered records are worth requesting ahead.
+    auto staging_of = [&](int req, int& levels, int& count, uint32_t* sparse = nullptr) {
         const int32_t* uoff = a.uoff + req * a.uoff_req_stride;
         const int e = (lane < old) ? __ldg(uoff + lane + 1) : 0x7fffffff;
         levels = __popc(__ballot_sync(0xffffffffu, e <= stage_cap));
         count = __shfl_sync(0xffffffffu, e, levels > 0 ? levels - 1 : 0);
         if (levels == 0) count = 0;
+        if (sparse) {
+            int prev = __shfl_up_sync(0xffffffffu, e, 1);
+            if (lane == 0) prev = 0;
+            *sparse = __ballot_sync(0xffffffffu, lane < old && (e - prev) * 4 > a.W);
+        }
     };
 
     if (warp < FOLD_WARPS) {
@@ -341,8 +349,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         };
         // staging layout of the request whose quads are being looked at (the same for all heads of a request)
         int info_req = -1, info_levels = 0, info_count = 0;
+        uint32_t info_sparse = 0;
         auto staged_levels_of = [&](int req) {
-            if (req != info_req) { staging_of(req, info_levels, info_count); info_req = req; }
+            if (req != info_req) { staging_of(req, info_levels, info_count, &info_sparse); info_req = req; }
             return info_levels;
         };
         constexpr int NIDX = LPU >= 8 ? 1 : 8 / LPU;     // the unit's lanes hold the indices of its first 8 levels
@@ -373,157 +382,198 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             idx_next = load_idx(u0);
         }
         put_first_s0();
-        int cur_seg = -1, buf = 0, staged_levels = 0;
+        int cur_seg = -1, buf = 0, staged_levels = 0, n_ahead = 0;
         bool staged_ready = false;
         long long plane_row0 = 0, own_row0 = 0;
         const int32_t *table_r = nullptr, *sidx_r = nullptr;
-        for (int k = 0; k < n_quads && !dead; ++k, u0 = u1, u1 = u2, u2 = next_unit(u2)) {
-            if (u0.seg != cur_seg) {          // entering a segment: nothing to wait for here
-                cur_seg = u0.seg;
-                buf = single ? 0 : (cur_seg & 1);
-                staged_ready = false;
-                staged_levels = staged_levels_of(u0.req);
-                plane_row0 = (long long)u0.h * a.arena_slots;
-                own_row0 = plane_row0 + a.bases.base[u0.req];
-                table_r = a.table + u0.req * a.table_req_stride;
-                sidx_r = a.sidx + u0.req * a.sidx_req_stride;
-            }
-            const bool seg_last = (k + 1 == n_quads) || (u1.seg != cur_seg);
-            const int s = k % SLOTS, use = k / SLOTS;
-            const int u = UPW * warp + grp;                  // row of this unit in the slot
-            const int bb = live_beam(u0);
-            Head cur;
-            {
-                asm volatile("cp.async.wait_group 0;" ::: "memory");
-                const uint4* rec = reinterpret_cast<const uint4*>(my_heads + grp * REC_BYTES) + g;
-                const uint4* qv = reinterpret_cast<const uint4*>(my_heads + UPW * REC_BYTES + grp * (DK * 2)) + g;
-#pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-                    cur.own.k[c] = rec[c * LPU];
-                    cur.own.v[c] = rec[16 + c * LPU];
-                    cur.q[c] = qv[c * LPU];
+        // The loop exists twice, with and without the requests ahead of the gathered records (at its end): where
+        // they are not wanted the loop is exactly the one without them (their mere presence measured 0.7 % slower).
+        auto fold_quads = [&](auto ahead_tag) {
+            constexpr bool AHEAD = decltype(ahead_tag)::value;
+            for (int k = 0; k < n_quads && !dead; ++k, u0 = u1, u1 = u2, u2 = next_unit(u2)) {
+                if (u0.seg != cur_seg) {          // entering a segment: nothing to wait for here
+                    cur_seg = u0.seg;
+                    buf = single ? 0 : (cur_seg & 1);
+                    staged_ready = false;
+                    staged_levels = staged_levels_of(u0.req);
+                    // levels gathered from global memory whose lines are worth requesting ahead (end of the loop)
+                    if (AHEAD) n_ahead = (info_sparse >> staged_levels) ? min(old - staged_levels, NIDX * LPU - staged_levels) : 0;
+                    plane_row0 = (long long)u0.h * a.arena_slots;
+                    own_row0 = plane_row0 + a.bases.base[u0.req];
+                    table_r = a.table + u0.req * a.table_req_stride;
+                    sidx_r = a.sidx + u0.req * a.sidx_req_stride;
                 }
-                cur.own.gate = gate0;
-                // the next quad's copies go out before this quad's stores (each lane overwrites only the chunks it
-                // has just read)
-                if (k + 1 < n_quads) issue_head(u1);
-                if (fused && beam_of(u0) < a.W) {   // the append: this beam's record goes to its arena slot, bit for bit
-                    if constexpr (GROUPED) {
-                        const long long slot = a.bases.base[u0.req] + bb;
-                        uint4* vdst = reinterpret_cast<uint4*>(a.vv_out + ((long long)u0.h * a.arena_slots + slot) * (DV * 2)) + g;
-#pragma unroll
-                        for (int c = 0; c < NCH; ++c) vdst[c * LPU] = cur.own.v[c];
-                        if (u0.h % a.g == 0) {     // the key is stored once per key head: by its first value head
-                            uint4* kdst = reinterpret_cast<uint4*>(a.kv_out + ((long long)key_head(u0.h) * a.arena_slots + slot) * (DK * 2)) + g;
-#pragma unroll
-                            for (int c = 0; c < NCH; ++c) kdst[c * LPU] = cur.own.k[c];
+                const bool seg_last = (k + 1 == n_quads) || (u1.seg != cur_seg);
+                const int s = k % SLOTS, use = k / SLOTS;
+                const int u = UPW * warp + grp;                  // row of this unit in the slot
+                const int bb = live_beam(u0);
+                Head cur;
+                {
+                    asm volatile("cp.async.wait_group 0;" ::: "memory");
+                    const uint4* rec = reinterpret_cast<const uint4*>(my_heads + grp * REC_BYTES) + g;
+                    const uint4* qv = reinterpret_cast<const uint4*>(my_heads + UPW * REC_BYTES + grp * (DK * 2)) + g;
+    #pragma unroll
+                    for (int c = 0; c < NCH; ++c) {
+                        cur.own.k[c] = rec[c * LPU];
+                        cur.own.v[c] = rec[16 + c * LPU];
+                        cur.q[c] = qv[c * LPU];
+                    }
+                    cur.own.gate = gate0;
+                    // the next quad's copies go out before this quad's stores (each lane overwrites only the chunks it
+                    // has just read)
+                    if (k + 1 < n_quads) issue_head(u1);
+                    if (fused && beam_of(u0) < a.W) {   // the append: this beam's record goes to its arena slot, bit for bit
+                        if constexpr (GROUPED) {
+                            const long long slot = a.bases.base[u0.req] + bb;
+                            uint4* vdst = reinterpret_cast<uint4*>(a.vv_out + ((long long)u0.h * a.arena_slots + slot) * (DV * 2)) + g;
+    #pragma unroll
+                            for (int c = 0; c < NCH; ++c) vdst[c * LPU] = cur.own.v[c];
+                            if (u0.h % a.g == 0) {     // the key is stored once per key head: by its first value head
+                                uint4* kdst = reinterpret_cast<uint4*>(a.kv_out + ((long long)key_head(u0.h) * a.arena_slots + slot) * (DK * 2)) + g;
+    #pragma unroll
+                                for (int c = 0; c < NCH; ++c) kdst[c * LPU] = cur.own.k[c];
+                            }
+                        } else {
+                            uint4* dst = reinterpret_cast<uint4*>(a.kv_out + (own_row0 + bb) * REC_BYTES) + g;
+    #pragma unroll
+                            for (int c = 0; c < NCH; ++c) {
+                                dst[c * LPU] = cur.own.k[c];
+                                dst[16 + c * LPU] = cur.own.v[c];
+                            }
                         }
-                    } else {
-                        uint4* dst = reinterpret_cast<uint4*>(a.kv_out + (own_row0 + bb) * REC_BYTES) + g;
-#pragma unroll
-                        for (int c = 0; c < NCH; ++c) {
-                            dst[c * LPU] = cur.own.k[c];
-                            dst[16 + c * LPU] = cur.own.v[c];
+                        if (g == 0) a.gates_out[own_row0 + bb] = gate0;
+                    }
+                }
+                gate0 = gate1;
+                if (k + 2 < n_quads) gate1 = load_gate(u2);
+
+                // lane g keeps the index of level g (position in the staged list for staged levels, arena slot
+                // otherwise); it was fetched while the previous quad was folded, the next quad's is fetched now
+                const Idx my_idx = idx_next;
+                if (k + 1 < n_quads) idx_next = load_idx(u1);
+                auto idx_of = [&](int level) -> int32_t {
+                    int32_t t = 0;
+    #pragma unroll
+                    for (int j = 0; j < NIDX; ++j) {
+                        const int32_t x = __shfl_sync(0xffffffffu, my_idx.v[j], level & (LPU - 1), LPU);
+                        if (j == level / LPU) t = x;
+                    }
+                    return level < NIDX * LPU ? t
+                                              : __ldg((level < staged_levels ? sidx_r : table_r) + (long long)level * a.max_beam + bb);
+                };
+
+                float2 r[4 * NCH], corr[4 * NCH];
+    #pragma unroll
+                for (int c = 0; c < NCH; ++c) unpack8(cur.q[c], r + 4 * c);
+    #pragma unroll
+                for (int e = 0; e < 4 * NCH; ++e) corr[e] = make_float2(0.f, 0.f);
+                float decay = 1.f;
+                L::fold_chain_simple(cur.own, old - 1, staged_levels,
+                              [&](int level) {
+                                  const long long slot = idx_of(level);
+                                  if constexpr (GROUPED) {
+                                      RecT rec;
+                                      const uint4* kp = reinterpret_cast<const uint4*>(k_at(u0.h, slot)) + g;
+                                      const uint4* vp = reinterpret_cast<const uint4*>(v_at(u0.h, slot)) + g;
+    #pragma unroll
+                                      for (int c = 0; c < NCH; ++c) {
+                                          rec.k[c] = __ldg(kp + c * LPU);
+                                          rec.v[c] = __ldg(vp + c * LPU);
+                                      }
+                                      rec.gate = __ldg(a.gates + plane_row0 + slot);
+                                      return rec;
+                                  } else {
+                                      return L::load_global(kv, a.gates, plane_row0 + slot, g);
+                                  }
+                              }, r, corr, decay);
+                // The segment's staging is waited for even when it holds nothing: it keeps this warp from running past
+                // the epilogue warps' preparation of the segment after next (whose barriers share these phases).
+                if (!staged_ready && (staged_levels > 0 || seg_last)) {
+                    if (!wait_or_abort(bar_stage(buf), (single ? 0 : (cur_seg >> 1)) & 1, abort_flag)) { dead = true; break; }
+                    staged_ready = true;
+                }
+                if (staged_levels > 0) {
+                    const uint8_t* st = stage + buf * (STAGE_BUF * REC_BYTES);
+                    const float2* gs = gates_s + buf * STAGE_BUF;
+                    const RecT newest = L::load_shared(st, gs, idx_of(staged_levels - 1), g);
+                    L::fold_chain_simple(newest, staged_levels - 2, 0,
+                                  [&](int level) { return L::load_shared(st, gs, idx_of(level), g); }, r, corr, decay);
+                }
+                if (seg_last) {                    // this warp's last read of the segment's staging buffer
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_sfree(buf));
+                }
+
+                // the slot must have been handed back by the epilogue of its previous use
+                if (use > 0 && !wait_or_abort(bar_free(s), (use - 1) & 1, abort_flag)) { dead = true; break; }
+                uint8_t* R_s = ring + s * SLOT_BYTES;
+                float* C_s = reinterpret_cast<float*>(R_s + R_BYTES);
+                {
+                    // Bank conflicts: the lanes g and g + 4 of a unit own the same chunk positions of two operand rows
+                    // 48 * 128 bytes apart, so the upper four lanes write their two chunks in the opposite order;
+                    // the corr tile (a layout of our own) swaps each pair of 16-byte chunks in every other 128-byte
+                    // stretch of a row instead (corr_chunk; the epilogue reads it the same way).
+                    const int sw = u & 7;
+                    const bool hi = (g >> 2) & 1;
+                    const float2 dc = make_float2(decay, decay);
+    #pragma unroll
+                    for (int c = 0; c < NCH; ++c) {
+                        const int ci = c * LPU + g;                 // elements [8 ci, 8 ci + 8)
+                        const int kb = ci >> 2, ch = 2 * (ci & 3);  // K block of 32 floats; first of two 16-byte chunks
+                        uint8_t* row = R_s + kb * R_KB_STRIDE + u * 128;
+                        float2 x[4];
+    #pragma unroll
+                        for (int e = 0; e < 4; ++e) x[e] = __fmul2_rn(r[4 * c + e], dc);
+                        const float4 lo4 = make_float4(round_tf32(x[0].x), round_tf32(x[0].y), round_tf32(x[1].x), round_tf32(x[1].y));
+                        const float4 hi4 = make_float4(round_tf32(x[2].x), round_tf32(x[2].y), round_tf32(x[3].x), round_tf32(x[3].y));
+                        *reinterpret_cast<float4*>(row + (((ch + (hi ? 1 : 0)) ^ sw) << 4)) = hi ? hi4 : lo4;
+                        *reinterpret_cast<float4*>(row + (((ch + (hi ? 0 : 1)) ^ sw) << 4)) = hi ? lo4 : hi4;
+                        float* crow = C_s + u * DV;
+                        *reinterpret_cast<float4*>(crow + corr_chunk(2 * ci) * 4) =
+                            make_float4(corr[4 * c].x, corr[4 * c].y, corr[4 * c + 1].x, corr[4 * c + 1].y);
+                        *reinterpret_cast<float4*>(crow + corr_chunk(2 * ci + 1) * 4) =
+                            make_float4(corr[4 * c + 2].x, corr[4 * c + 2].y, corr[4 * c + 3].x, corr[4 * c + 3].y);
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_full(s));
+
+                // The next quad's records of the levels that are NOT staged are gathered from global memory in the middle
+                // of its dependent chain.  Where a level has little sharing (most of its records are used by one or two
+                // beams: uniform parents) their lines are requested now, a whole quad ahead - the slot ids have arrived
+                // by now; where many beams share few records the gathers hit L1/L2 anyway and the requests only cost
+                // (measured: +6 % on 8 x 1024 beams with uniform parents, -3 % on the Zipf(1.5) stack if done always).
+                // One request per lane: lane g of a unit asks for line g & 3 of the record of level
+                // old - 1 - 2 p - (g >> 2), newest levels first.  (The segment's own staging layout is used for the
+                // next quad: it differs only across a change of request, and a request is a hint.)
+                if (AHEAD && n_ahead > 0 && k + 1 < n_quads) {
+                    for (int p = 0; 2 * p < n_ahead; ++p) {
+                        const int level = old - 1 - 2 * p - (g >> 2);
+                        const int src = max(level, 0);
+                        int32_t slot = 0;
+    #pragma unroll
+                        for (int j = 0; j < NIDX; ++j) {
+                            const int32_t x = __shfl_sync(0xffffffffu, idx_next.v[j], src & (LPU - 1), LPU);
+                            if (j == src / LPU) slot = x;
+                        }
+                        if (level >= staged_levels && level < NIDX * LPU && ((info_sparse >> level) & 1)) {
+                            const char* line = (g & 2) ? v_at(u1.h, slot) + (g & 1) * 128 : k_at(u1.h, slot) + (g & 1) * 128;
+                            asm volatile("prefetch.global.L2 [%0];" ::"l"(line));
                         }
                     }
-                    if (g == 0) a.gates_out[own_row0 + bb] = gate0;
                 }
             }
-            gate0 = gate1;
-            if (k + 2 < n_quads) gate1 = load_gate(u2);
-
-            // lane g keeps the index of level g (position in the staged list for staged levels, arena slot
-            // otherwise); it was fetched while the previous quad was folded, the next quad's is fetched now
-            const Idx my_idx = idx_next;
-            if (k + 1 < n_quads) idx_next = load_idx(u1);
-            auto idx_of = [&](int level) -> int32_t {
-                int32_t t = 0;
-#pragma unroll
-                for (int j = 0; j < NIDX; ++j) {
-                    const int32_t x = __shfl_sync(0xffffffffu, my_idx.v[j], level & (LPU - 1), LPU);
-                    if (j == level / LPU) t = x;
-                }
-                return level < NIDX * LPU ? t
-                                          : __ldg((level < staged_levels ? sidx_r : table_r) + (long long)level * a.max_beam + bb);
-            };
-
-            float2 r[4 * NCH], corr[4 * NCH];
-#pragma unroll
-            for (int c = 0; c < NCH; ++c) unpack8(cur.q[c], r + 4 * c);
-#pragma unroll
-            for (int e = 0; e < 4 * NCH; ++e) corr[e] = make_float2(0.f, 0.f);
-            float decay = 1.f;
-            L::fold_chain_simple(cur.own, old - 1, staged_levels,
-                          [&](int level) {
-                              const long long slot = idx_of(level);
-                              if constexpr (GROUPED) {
-                                  RecT rec;
-                                  const uint4* kp = reinterpret_cast<const uint4*>(k_at(u0.h, slot)) + g;
-                                  const uint4* vp = reinterpret_cast<const uint4*>(v_at(u0.h, slot)) + g;
-#pragma unroll
-                                  for (int c = 0; c < NCH; ++c) {
-                                      rec.k[c] = __ldg(kp + c * LPU);
-                                      rec.v[c] = __ldg(vp + c * LPU);
-                                  }
-                                  rec.gate = __ldg(a.gates + plane_row0 + slot);
-                                  return rec;
-                              } else {
-                                  return L::load_global(kv, a.gates, plane_row0 + slot, g);
-                              }
-                          }, r, corr, decay);
-            // The segment's staging is waited for even when it holds nothing: it keeps this warp from running past
-            // the epilogue warps' preparation of the segment after next (whose barriers share these phases).
-            if (!staged_ready && (staged_levels > 0 || seg_last)) {
-                if (!wait_or_abort(bar_stage(buf), (single ? 0 : (cur_seg >> 1)) & 1, abort_flag)) { dead = true; break; }
-                staged_ready = true;
-            }
-            if (staged_levels > 0) {
-                const uint8_t* st = stage + buf * (STAGE_BUF * REC_BYTES);
-                const float2* gs = gates_s + buf * STAGE_BUF;
-                const RecT newest = L::load_shared(st, gs, idx_of(staged_levels - 1), g);
-                L::fold_chain_simple(newest, staged_levels - 2, 0,
-                              [&](int level) { return L::load_shared(st, gs, idx_of(level), g); }, r, corr, decay);
-            }
-            if (seg_last) {                    // this warp's last read of the segment's staging buffer
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_sfree(buf));
-            }
-
-            // the slot must have been handed back by the epilogue of its previous use
-            if (use > 0 && !wait_or_abort(bar_free(s), (use - 1) & 1, abort_flag)) { dead = true; break; }
-            uint8_t* R_s = ring + s * SLOT_BYTES;
-            float* C_s = reinterpret_cast<float*>(R_s + R_BYTES);
-            {
-                // Bank conflicts: the lanes g and g + 4 of a unit own the same chunk positions of two operand rows
-                // 48 * 128 bytes apart, so the upper four lanes write their two chunks in the opposite order;
-                // the corr tile (a layout of our own) swaps each pair of 16-byte chunks in every other 128-byte
-                // stretch of a row instead (corr_chunk; the epilogue reads it the same way).
-                const int sw = u & 7;
-                const bool hi = (g >> 2) & 1;
-                const float2 dc = make_float2(decay, decay);
-#pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-                    const int ci = c * LPU + g;                 // elements [8 ci, 8 ci + 8)
-                    const int kb = ci >> 2, ch = 2 * (ci & 3);  // K block of 32 floats; first of two 16-byte chunks
-                    uint8_t* row = R_s + kb * R_KB_STRIDE + u * 128;
-                    float2 x[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) x[e] = __fmul2_rn(r[4 * c + e], dc);
-                    const float4 lo4 = make_float4(round_tf32(x[0].x), round_tf32(x[0].y), round_tf32(x[1].x), round_tf32(x[1].y));
-                    const float4 hi4 = make_float4(round_tf32(x[2].x), round_tf32(x[2].y), round_tf32(x[3].x), round_tf32(x[3].y));
-                    *reinterpret_cast<float4*>(row + (((ch + (hi ? 1 : 0)) ^ sw) << 4)) = hi ? hi4 : lo4;
-                    *reinterpret_cast<float4*>(row + (((ch + (hi ? 0 : 1)) ^ sw) << 4)) = hi ? lo4 : hi4;
-                    float* crow = C_s + u * DV;
-                    *reinterpret_cast<float4*>(crow + corr_chunk(2 * ci) * 4) =
-                        make_float4(corr[4 * c].x, corr[4 * c].y, corr[4 * c + 1].x, corr[4 * c + 1].y);
-                    *reinterpret_cast<float4*>(crow + corr_chunk(2 * ci + 1) * 4) =
-                        make_float4(corr[4 * c + 2].x, corr[4 * c + 2].y, corr[4 * c + 3].x, corr[4 * c + 3].y);
-                }
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_full(s));
+        };
+        // little sharing somewhere in the first request's gathered levels: take the loop that requests lines ahead
+        // (the requests of a batch follow one parent law as a rule; it is a hint either way)
+        bool ahead = false;
+        if (n_quads > 0) {
+            const int sl0 = staged_levels_of(u0.req);
+            ahead = old > sl0 && (info_sparse >> sl0) != 0;
         }
+        if (ahead) fold_quads(std::true_type{});
+        else fold_quads(std::false_type{});
     } else {
         // =============================== EPILOGUE (+ MMA issue, + preparation of the next segments) ===============================
         dependency_wait();
@@ -756,9 +806,9 @@ int make_partition(int total_groups, int gpp, int sms, PartitionCost c, Partitio
     return greedy_fill(total_groups, gpp, lo, sms, c, part->begin);
 }
 
-template <typename OutT, bool GROUPED>
+template <typename OutT, bool GROUPED, bool FUSED>
 cudaError_t launch_ws_t(const DecodeArgs& a, cudaStream_t stream) {
-    auto kern = decode_ws_kernel<OutT, GROUPED>;
+    auto kern = decode_ws_kernel<OutT, GROUPED, FUSED>;
     static std::once_flag once;                  // host threads may share a context's kernels
     static cudaError_t configure_error = cudaSuccess;
     static int sms = 148;
@@ -802,8 +852,15 @@ bool decode_sm100_supported(int32_t dk, int32_t dv, int32_t rec_dtype) {
 }
 
 cudaError_t launch_decode_sm100_ws(const DecodeArgs& a, int32_t out_dtype, bool grouped, cudaStream_t stream) {
-    if (grouped) return out_dtype == ONELA_DTYPE_BF16 ? launch_ws_t<__nv_bfloat16, true>(a, stream) : launch_ws_t<float, true>(a, stream);
-    return out_dtype == ONELA_DTYPE_BF16 ? launch_ws_t<__nv_bfloat16, false>(a, stream) : launch_ws_t<float, false>(a, stream);
+    // one instantiation per (output type, grouped value heads, append fused in): a launch runs only the code it needs
+    const bool fused = a.k_in != nullptr;
+    const bool bf16 = out_dtype == ONELA_DTYPE_BF16;
+    if (grouped) {
+        if (fused) return bf16 ? launch_ws_t<__nv_bfloat16, true, true>(a, stream) : launch_ws_t<float, true, true>(a, stream);
+        return bf16 ? launch_ws_t<__nv_bfloat16, true, false>(a, stream) : launch_ws_t<float, true, false>(a, stream);
+    }
+    if (fused) return bf16 ? launch_ws_t<__nv_bfloat16, false, true>(a, stream) : launch_ws_t<float, false, true>(a, stream);
+    return bf16 ? launch_ws_t<__nv_bfloat16, false, false>(a, stream) : launch_ws_t<float, false, false>(a, stream);
 }
 
 }  // namespace onela
