@@ -809,15 +809,23 @@ int make_partition(int total_groups, int gpp, int sms, PartitionCost c, Partitio
 template <typename OutT, bool GROUPED, bool FUSED>
 cudaError_t launch_ws_t(const DecodeArgs& a, cudaStream_t stream) {
     auto kern = decode_ws_kernel<OutT, GROUPED, FUSED>;
-    static std::once_flag once;                  // host threads may share a context's kernels
-    static cudaError_t configure_error = cudaSuccess;
-    static int sms = 148;
-    std::call_once(once, [&]() {
-        configure_error = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-        sms = sm_count_ws();
-        if (sms > MAX_CTAS) sms = MAX_CTAS;
-    });
-    if (configure_error != cudaSuccess) return configure_error;
+    // One-time set-up per device (function attributes belong to a device's context); host threads may share it.
+    constexpr int MAX_DEVICES = 64;
+    static std::mutex setup_mutex;
+    static int sms_of[MAX_DEVICES] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+    int sms;
+    {
+        std::lock_guard<std::mutex> lock(setup_mutex);
+        if (sms_of[dev] == 0) {
+            const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+            if (e != cudaSuccess) return e;
+            const int n = sm_count_ws();
+            sms_of[dev] = n > MAX_CTAS ? MAX_CTAS : n;
+        }
+        sms = sms_of[dev];
+    }
     const int groups_per_pair = (a.W + GN - 1) / GN;
     const int total_groups = a.req_count * a.H * groups_per_pair;
     static thread_local Partition part;          // the last launch's partition, reused while the shape stays
