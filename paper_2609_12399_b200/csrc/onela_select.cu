@@ -50,9 +50,11 @@ struct SelectShared {
     unsigned int k, count, equal;
 };
 
-// Leaves the k largest composites of src(0 .. n-1) in sh.sel[0 .. k) (unordered); k <= min(n, SEL_CAP).
-template <class Src>
-__device__ void select_topk(const Src& src, uint32_t n, int k, SelectShared& sh) {
+// Leaves the k largest composites of item(0 .. n-1) in sh.sel[0 .. k) (unordered); k <= min(n, SEL_CAP).
+// `item(j, i)` returns composite i = tid + j * SEL_THREADS: from the source itself, or from the thread's registers.
+// MAXJ > 0: at most MAXJ items per thread, loops unrolled (so that a register array can be indexed); 0: any number.
+template <int MAXJ, class Item>
+__device__ void select_passes(const Item& item, uint32_t n, int k, SelectShared& sh) {
     const int tid = threadIdx.x;
     if (tid == 0) { sh.prefix = 0ull; sh.k = (unsigned)k; sh.count = 0u; }
     __syncthreads();
@@ -65,10 +67,10 @@ __device__ void select_topk(const Src& src, uint32_t n, int k, SelectShared& sh)
         const unsigned long long prefix = sh.prefix;
         const unsigned want = sh.k;               // (read here: the bin search below rewrites it)
         const unsigned long long hi_mask = p == 7 ? 0ull : (~0ull << (8 * (p + 1)));
-        for (uint32_t i = tid; i < n_padded; i += SEL_THREADS) {
+        auto count_item = [&](int j, uint32_t i) {
             // whole warps stay in the loop (padding iterations carry no candidate) so the peer vote is complete
             const bool live = i < n;
-            const unsigned long long c = live ? src(i) : 0ull;
+            const unsigned long long c = live ? item(j, i) : 0ull;
             const bool in = live && ((c & hi_mask) == prefix);
             const unsigned bin = (unsigned)(c >> (8 * p)) & 255u;
             // one atomic per distinct bin in the warp: scores cluster, so most lanes share a bin in the early passes
@@ -77,6 +79,15 @@ __device__ void select_topk(const Src& src, uint32_t n, int k, SelectShared& sh)
                 const unsigned peers = __match_any_sync(vote, bin);
                 if ((threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&sh.hist[bin], __popc(peers));
             }
+        };
+        if constexpr (MAXJ > 0) {
+#pragma unroll
+            for (int j = 0; j < MAXJ; ++j) {
+                const uint32_t i = tid + (uint32_t)j * SEL_THREADS;
+                if (i < n_padded) count_item(j, i);
+            }
+        } else {
+            for (uint32_t i = tid; i < n_padded; i += SEL_THREADS) count_item(0, i);
         }
         __syncthreads();
         // the bin that holds the k-th largest: suffix counts over the 256 bins (bin >= b), by the first eight warps
@@ -107,14 +118,42 @@ __device__ void select_topk(const Src& src, uint32_t n, int k, SelectShared& sh)
         if (p == 4 && sh.equal == sh.k) break;
     }
     const unsigned long long threshold = sh.prefix;   // (low bytes zero after an early exit: every equal score is kept)
-    for (uint32_t i = tid; i < n; i += SEL_THREADS) {
-        const unsigned long long c = src(i);
+    auto keep_item = [&](int j, uint32_t i) {
+        const unsigned long long c = item(j, i);
         if (c >= threshold) {
             const unsigned pos = atomicAdd(&sh.count, 1u);
             if (pos < SEL_CAP) sh.sel[pos] = c;
         }
+    };
+    if constexpr (MAXJ > 0) {
+#pragma unroll
+        for (int j = 0; j < MAXJ; ++j) {
+            const uint32_t i = tid + (uint32_t)j * SEL_THREADS;
+            if (i < n) keep_item(j, i);
+        }
+    } else {
+        for (uint32_t i = tid; i < n; i += SEL_THREADS) keep_item(0, i);
     }
     __syncthreads();
+}
+// The passes read every candidate four to eight times.  Up to ITEMS * SEL_THREADS candidates are fetched once, all
+// loads in flight together, and kept in registers (a pass then costs votes and shared-memory atomics only: the
+// merging CTA fell from 48 us to a fraction of that on 16 384 composites); longer lists are re-read from the source.
+template <int ITEMS, class Src>
+__device__ void select_topk(const Src& src, uint32_t n, int k, SelectShared& sh) {
+    if (n <= (uint32_t)ITEMS * SEL_THREADS) {
+        unsigned long long held[ITEMS];
+#pragma unroll
+        for (int j = 0; j < ITEMS; ++j) {
+            const uint32_t i = threadIdx.x + (uint32_t)j * SEL_THREADS;
+            held[j] = i < n ? src(i) : 0ull;
+        }
+        auto item = [&](int j, uint32_t) { return held[j]; };      // j is a compile-time constant in the unrolled loops
+        select_passes<ITEMS>(item, n, k, sh);
+    } else {
+        auto item = [&](int, uint32_t i) { return src(i); };
+        select_passes<0>(item, n, k, sh);
+    }
 }
 
 // Orders sh.sel[0 .. k) best first and writes the survivors out.
@@ -155,7 +194,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_part_kernel(const float* _
     const uint32_t n = min((uint32_t)SEL_PART, N - first);
     const int kp = min((uint32_t)k, n);
     const ScoreSource src{beam_scores + (long long)req * W_prev, cand_logp + (long long)req * W_prev * C, first, C};
-    select_topk(src, n, kp, sh);
+    select_topk<SEL_PART / SEL_THREADS>(src, n, kp, sh);
     unsigned long long* out = scratch + ((long long)req * SEL_PARTS_MAX + part) * SEL_CAP;
     for (int i = threadIdx.x; i < kp; i += SEL_THREADS) out[i] = sh.sel[i];
 }
@@ -171,7 +210,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_merge_kernel(const float* 
     const float* lp = cand_logp + (long long)req * W_prev * C;
     const uint32_t N = (uint32_t)W_prev * (uint32_t)C;
     if (parts == 1) {
-        select_topk(ScoreSource{bs, lp, 0u, C}, N, k, sh);
+        select_topk<SEL_PART / SEL_THREADS>(ScoreSource{bs, lp, 0u, C}, N, k, sh);
     } else {
         // every part but the last left min(k, SEL_PART) composites; read them as one list with gaps skipped
         const uint32_t kp = min((uint32_t)k, (uint32_t)SEL_PART);
@@ -184,7 +223,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_merge_kernel(const float* 
             }
         };
         const Gapped src{scratch + (long long)req * SEL_PARTS_MAX * SEL_CAP, kp};
-        select_topk(src, (uint32_t)(parts - 1) * kp + last_kp, k, sh);
+        select_topk<16>(src, (uint32_t)(parts - 1) * kp + last_kp, k, sh);
     }
     sort_and_emit(sh, k, bs, lp, C, parents + (long long)req * k, codes + (long long)req * k, scores + (long long)req * k);
 }
