@@ -43,8 +43,6 @@ struct ScoreSource {     // composites computed from the caller's scores; item i
 };
 struct SelectShared {
     unsigned int hist[256];
-    unsigned int suffix[256];
-    unsigned int warp_total[8];
     unsigned long long sel[SEL_CAP];
     unsigned long long prefix;
     unsigned int k, count, equal;
@@ -57,13 +55,12 @@ template <int MAXJ, class Item>
 __device__ void select_passes(const Item& item, uint32_t n, int k, SelectShared& sh) {
     const int tid = threadIdx.x;
     if (tid == 0) { sh.prefix = 0ull; sh.k = (unsigned)k; sh.count = 0u; }
+    if (tid < 256) sh.hist[tid] = 0u;
     __syncthreads();
     // after the pass over byte p, sh.prefix holds bytes 7..p of the k-th largest composite and sh.k how many
     // survivors are still to be found among the candidates that share those bytes
     const uint32_t n_padded = (n + SEL_THREADS - 1) / SEL_THREADS * SEL_THREADS;
-    for (int p = 7; p >= 0; --p) {
-        if (tid < 256) sh.hist[tid] = 0u;
-        __syncthreads();
+    for (int p = 7; p >= 0; --p) {             // two block-wide barriers per pass
         const unsigned long long prefix = sh.prefix;
         const unsigned want = sh.k;               // (read here: the bin search below rewrites it)
         const unsigned long long hi_mask = p == 7 ? 0ull : (~0ull << (8 * (p + 1)));
@@ -90,27 +87,30 @@ __device__ void select_passes(const Item& item, uint32_t n, int k, SelectShared&
             for (uint32_t i = tid; i < n_padded; i += SEL_THREADS) count_item(0, i);
         }
         __syncthreads();
-        // the bin that holds the k-th largest: suffix counts over the 256 bins (bin >= b), by the first eight warps
-        if (tid < 256) {
-            unsigned v = sh.hist[tid];
+        // the bin that holds the k-th largest, by the first warp alone: lane l takes bins 8 l .. 8 l + 7, suffix counts
+        // (candidates in bins >= b) across the lanes by shuffles; it also clears the histogram for the next pass
+        if (tid < 32) {
+            unsigned h[8], mine = 0;
+#pragma unroll
+            for (int t = 0; t < 8; ++t) { h[t] = sh.hist[8 * tid + t]; mine += h[t]; }
+#pragma unroll
+            for (int t = 0; t < 8; ++t) sh.hist[8 * tid + t] = 0u;
+            unsigned incl = mine;                                   // counts of lanes >= this one
 #pragma unroll
             for (int off = 1; off < 32; off <<= 1) {
-                const unsigned up = __shfl_down_sync(0xffffffffu, v, off);
-                if ((tid & 31) + off < 32) v += up;
+                const unsigned up = __shfl_down_sync(0xffffffffu, incl, off);
+                if (tid + off < 32) incl += up;
             }
-            if ((tid & 31) == 0) sh.warp_total[tid >> 5] = v;      // lane 0 holds its warp's whole count
-            sh.suffix[tid] = v;
-        }
-        __syncthreads();
-        if (tid < 256) {
-            unsigned higher = 0;
-            for (int w = (tid >> 5) + 1; w < 8; ++w) higher += sh.warp_total[w];
-            const unsigned here = sh.suffix[tid] + higher;                                   // candidates in bins >= tid
-            const unsigned next = here - sh.hist[tid];                                       // ... in bins > tid
-            if (here >= want && next < want) {                                               // exactly one bin qualifies
-                sh.prefix = prefix | ((unsigned long long)tid << (8 * p));
-                sh.k = want - next;
-                sh.equal = sh.hist[tid];
+            unsigned here = incl;                                   // candidates in bins >= 8 tid + t, from t = 0 down
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                const unsigned next = here - h[t];                  // ... in bins > 8 tid + t
+                if (here >= want && next < want) {                  // exactly one bin qualifies
+                    sh.prefix = prefix | ((unsigned long long)(8 * tid + t) << (8 * p));
+                    sh.k = want - next;
+                    sh.equal = h[t];
+                }
+                here = next;
             }
         }
         __syncthreads();
@@ -165,16 +165,28 @@ __device__ void sort_and_emit(SelectShared& sh, int k, const float* bs, const fl
     for (int i = tid; i < n_sort; i += SEL_THREADS)
         if (i >= k) sh.sel[i] = 0ull;
     __syncthreads();
-    for (int size = 2; size <= n_sort; size <<= 1) {        // bitonic sort, descending
-        for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            for (int i = tid; i < n_sort / 2; i += SEL_THREADS) {
-                const int lo = 2 * i - (i & (stride - 1)), hi = lo + stride;
-                const bool desc = (lo & size) == 0;
-                const unsigned long long x = sh.sel[lo], y = sh.sel[hi];
-                if ((x < y) == desc) { sh.sel[lo] = y; sh.sel[hi] = x; }
-            }
+    // Bitonic sort, descending.  Compare-exchange i of a step pairs elements inside the 64-element block i / 32 whenever
+    // the stride is below 64, and thread i (= pair i; n_sort / 2 <= 512 pairs) belongs to warp i / 32: those steps need
+    // the warp only, and a block-wide barrier stands just before and after each run of them.
+    auto exchange = [&](int i, int size, int stride) {
+        const int lo = 2 * i - (i & (stride - 1)), hi = lo + stride;
+        const bool desc = (lo & size) == 0;
+        const unsigned long long x = sh.sel[lo], y = sh.sel[hi];
+        if ((x < y) == desc) { sh.sel[lo] = y; sh.sel[hi] = x; }
+    };
+    static_assert(SEL_CAP / 2 <= SEL_THREADS, "one compare-exchange per thread and step");
+    const bool mine = tid < n_sort / 2;
+    for (int size = 2; size <= n_sort; size <<= 1) {
+        int stride = size >> 1;
+        for (; stride >= 64; stride >>= 1) {                // partners in different 64-element blocks
+            if (mine) exchange(tid, size, stride);
             __syncthreads();
         }
+        for (; stride > 0; stride >>= 1) {                  // partners inside this warp's 64-element block
+            if (mine) exchange(tid, size, stride);
+            __syncwarp();
+        }
+        __syncthreads();
     }
     for (int i = tid; i < k; i += SEL_THREADS) {
         const uint32_t idx = 0xffffffffu - (uint32_t)(sh.sel[i] & 0xffffffffull);
