@@ -145,6 +145,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     ctx = run.ctx
     run.prefill_states()
     S0 = {(r, l): ctx.onela_export_shared_state(r, l) for r in range(wl.R) for l in range(wl.L)}
+    S0_all = torch.stack([torch.stack([S0[(r, l)] for l in range(wl.L)]) for r in range(wl.R)])   # [R][L][H][dv][dk]
     calls = [run.generate_call(t) for t in range(wl.D)]
     outs = run.alloc_outputs()
     torch.cuda.synchronize()
@@ -154,8 +155,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
 
     def generation(decode_events=None, stream=None):
         ctx.onela_reset(stream)
-        for (r, l), S in S0.items():
-            ctx.onela_init_shared_state(r, l, S, stream)
+        ctx.onela_init_shared_states(0, wl.R, S0_all, stream)     # all layers of all requests: one copy
         for call in calls:
             run.run_call(call, outs, stream, decode_events, fused=fused, group_events=True)
 

@@ -132,6 +132,14 @@ onela_status onela_reset(onela_ctx* ctx, void* stream);
 onela_status onela_init_shared_state(onela_ctx* ctx, int32_t request, int32_t layer, const float* S0_dev,
                                      void* stream);
 
+/* The same for ALL layers of req_count consecutive requests in one copy (a serving loop that admits a batch
+ * stores num_layers states per request: one call instead of req_count * num_layers).  S0_dev (device, 16-byte
+ * aligned) is [req_count][num_layers][value heads][dv][dk] fp32; same ownership and restart rule, applied to every
+ * request of the range.  ONELA_E_INVAL for a range outside the request slots or a null / misaligned pointer, and
+ * nothing is copied. */
+onela_status onela_init_shared_states(onela_ctx* ctx, int32_t req_begin, int32_t req_count, const float* S0_dev,
+                                      void* stream);
+
 /* Same store slot, filled by running Eq. 1 from the zero state over n_tokens prompt tokens in fp32:
  * k_dev [n_tokens][H][dk], v_dev [n_tokens][H][dv] in rec_dtype, alpha_dev, beta_dev [n_tokens][H] fp32. */
 onela_status onela_prefill_shared_state(onela_ctx* ctx, int32_t request, int32_t layer, const void* k_dev,

@@ -50,6 +50,7 @@ PROTOTYPES = {
     "onela_destroy": (c_int32, [c_void_p]),
     "onela_reset": (c_int32, [c_void_p, c_void_p]),
     "onela_init_shared_state": (c_int32, [c_void_p, c_int32, c_int32, c_void_p, c_void_p]),
+    "onela_init_shared_states": (c_int32, [c_void_p, c_int32, c_int32, c_void_p, c_void_p]),
     "onela_prefill_shared_state": (c_int32, [c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
                                              c_int32, c_void_p]),
     "onela_export_shared_state": (c_int32, [c_void_p, c_int32, c_int32, c_void_p, c_void_p]),
@@ -193,6 +194,11 @@ class Onela:
         c = self.cfg
         p = self._ptr(S0, torch.float32, (c.value_heads, c.dv, c.dk), "S0")
         _check(self.lib.onela_init_shared_state(self.handle, request, layer, p, self._s(stream)), "onela_init_shared_state")
+
+    def onela_init_shared_states(self, req_begin, req_count, S0, stream=None):
+        c = self.cfg
+        p = self._ptr(S0, torch.float32, (req_count, c.num_layers, c.value_heads, c.dv, c.dk), "S0")
+        _check(self.lib.onela_init_shared_states(self.handle, req_begin, req_count, p, self._s(stream)), "onela_init_shared_states")
 
     def onela_prefill_shared_state(self, request, layer, k, v, alpha, beta, stream=None):
         c = self.cfg

@@ -259,6 +259,25 @@ onela_status onela_init_shared_state(onela_ctx* ctx, int32_t request, int32_t la
     return ONELA_OK;
 }
 
+onela_status onela_init_shared_states(onela_ctx* ctx, int32_t req_begin, int32_t req_count, const float* S0_dev,
+                                      void* stream) {
+    if (!ctx || req_begin < 0 || req_count <= 0 || req_begin > ctx->cfg.num_requests - req_count) return ONELA_E_INVAL;
+    if (!S0_dev || !aligned16(S0_dev)) return ONELA_E_INVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    onela_status st = ctx->prepare(s);
+    if (st != ONELA_OK) return st;
+    if (!ctx->dry()) {
+        // the store keeps a request's layers next to each other and the requests in order: one contiguous range
+        const size_t bytes = (size_t)req_count * ctx->cfg.num_layers * ctx->s0_layer_floats() * sizeof(float);
+        if (cudaMemcpyAsync(ctx->s0_slot(req_begin, 0), S0_dev, bytes, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+            return ONELA_E_CUDA;
+        ctx->launches++;
+    }
+    for (int32_t r = req_begin; r < req_begin + req_count; ++r)
+        for (int32_t l = 0; l < ctx->cfg.num_layers; ++l) finish_state_write(ctx, r, l);
+    return ONELA_OK;
+}
+
 onela_status onela_prefill_shared_state(onela_ctx* ctx, int32_t request, int32_t layer, const void* k_dev,
                                         const void* v_dev, const float* alpha_dev, const float* beta_dev,
                                         int32_t n_tokens, void* stream) {

@@ -296,3 +296,21 @@ def test_init_then_export_round_trip():
     ctx.onela_init_shared_state(0, 0, S.cuda())
     back = ctx.onela_export_shared_state(0, 0).cpu()
     assert torch.equal(back, S)      # the store keeps S_0 bit for bit, on every path
+
+
+def test_batched_state_store_equals_the_single_calls():
+    """All layers of a range of requests in one call: the same bytes in the store as the per-(request, layer) calls,
+    other requests untouched."""
+    R, L, H = 3, 2, 2
+    cfg = P.make_config(R, L, H, 128, 128, 8, 2, "bf16", "fp32", 64)
+    ctx = P.Onela(cfg)
+    S = torch.randn(R, L, H, 128, 128, generator=torch.Generator().manual_seed(7))
+    ctx.onela_init_shared_state(0, 0, (S[0, 0] + 1).cuda())
+    ctx.onela_init_shared_state(0, 1, (S[0, 1] + 1).cuda())
+    ctx.onela_init_shared_states(1, 2, S[1:3].cuda())
+    for r in (1, 2):
+        for l in range(L):
+            assert torch.equal(ctx.onela_export_shared_state(r, l).cpu(), S[r, l])
+    assert torch.equal(ctx.onela_export_shared_state(0, 1).cpu(), S[0, 1] + 1)
+    assert ctx.onela_poll_device_status() == (0, 0)
+

@@ -275,6 +275,27 @@ def test_new_prompt_restarts_a_request():
     assert o.onela_get_step_base(0, 0) == 16      # the arena is append-only: no slot is reused
 
 
+def test_batched_state_store_covers_every_layer_of_the_range():
+    """onela_init_shared_states stores all layers of a range of requests: afterwards each of them may decode on
+    every layer, a request outside the range may not, and a request that had decoded restarts at depth 0."""
+    o = ctx(R=3, L=2, slots=100)
+    for bad in [(-1, 1), (0, 0), (2, 2), (3, 1)]:
+        with raises(binding.E_INVAL):
+            o.onela_init_shared_states(bad[0], bad[1], FAKE)
+    with raises(binding.E_INVAL):
+        o.onela_init_shared_states(0, 2, 0)            # null pointer
+    with raises(binding.E_INVAL):
+        o.onela_init_shared_states(0, 2, FAKE + 4)     # not 16-byte aligned
+    o.onela_init_shared_states(1, 2, FAKE)
+    full_step(o, 1, 2, 8, None, [0, 1])
+    with raises(binding.E_ORDER):
+        o.onela_reorder_beams(0, 1, None, 8)            # request 0 has no state
+    assert o.depth_and_width(1) == (1, 8) and o.depth_and_width(2) == (1, 8)
+    o.onela_init_shared_states(2, 1, FAKE)              # a new prompt in slot 2 only
+    assert o.depth_and_width(2) == (0, 0) and o.depth_and_width(1) == (1, 8)
+    full_step(o, 2, 1, 8, None, [0, 1])
+
+
 def test_released_slots_are_reused_lowest_first():
     o = ctx(R=3, L=1, slots=64, W=8)
     for r in range(3):
