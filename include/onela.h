@@ -147,7 +147,7 @@ onela_status onela_prefill_shared_state(onela_ctx* ctx, int32_t request, int32_t
                                         int32_t n_tokens, void* stream);
 
 /* Read the store slot of (request, layer) back as S0_out_dev [num_heads][dv][dk] fp32 row-major, bit for
- * bit what was stored (the tensor-core kernel rounds S_0 to TF32 only on its way into tensor memory). */
+ * bit what was stored (the tensor-core kernel converts S_0 to scaled fp16 only on its way into tensor memory). */
 onela_status onela_export_shared_state(onela_ctx* ctx, int32_t request, int32_t layer, float* S0_out_dev,
                                        void* stream);
 

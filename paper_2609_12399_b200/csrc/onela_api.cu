@@ -63,6 +63,7 @@ Layout carve(const onela_config& c, char* base) {
     }
     l.select_scratch = reinterpret_cast<unsigned long long*>(
         take((size_t)c.num_requests * ONELA_SELECT_PARTS * ONELA_SELECT_CAP * sizeof(unsigned long long)));
+    l.s0_scale = reinterpret_cast<float*>(take((size_t)c.num_requests * c.num_layers * Hv * sizeof(float)));
     l.total_bytes = off;
     return l;
 }
@@ -88,6 +89,7 @@ struct onela_ctx {
     long long table_req_stride() const { return 2LL * cfg.max_steps * cfg.max_beam; }
     long long s0_layer_floats() const { return (long long)Hv() * cfg.dv * cfg.dk; }
     float* s0_slot(int r, int l) const { return lay.s0 + ((long long)r * cfg.num_layers + l) * s0_layer_floats(); }
+    float* s0_scale_slot(int r, int l) const { return lay.s0_scale + ((long long)r * cfg.num_layers + l) * Hv(); }
     int32_t* table_cur(int r) const {
         const int d = req[r].depth;
         return lay.tables + r * table_req_stride() + (long long)((d - 1) & 1) * cfg.max_steps * cfg.max_beam;
@@ -250,8 +252,8 @@ onela_status onela_init_shared_state(onela_ctx* ctx, int32_t request, int32_t la
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if ((st = ctx->prepare(s)) != ONELA_OK) return st;
     if (!ctx->dry()) {
-        if (launch_store_state(S0_dev, ctx->s0_slot(request, layer), ctx->Hv(), ctx->cfg.dk, ctx->cfg.dv,
-                               s) != cudaSuccess)
+        if (launch_store_state(S0_dev, ctx->s0_slot(request, layer), ctx->s0_scale_slot(request, layer), ctx->Hv(),
+                               ctx->cfg.dk, ctx->cfg.dv, s) != cudaSuccess)
             return ONELA_E_CUDA;
         ctx->launches++;
     }
@@ -268,8 +270,9 @@ onela_status onela_init_shared_states(onela_ctx* ctx, int32_t req_begin, int32_t
     if (st != ONELA_OK) return st;
     if (!ctx->dry()) {
         // the store keeps a request's layers next to each other and the requests in order: one contiguous range
-        const size_t bytes = (size_t)req_count * ctx->cfg.num_layers * ctx->s0_layer_floats() * sizeof(float);
-        if (cudaMemcpyAsync(ctx->s0_slot(req_begin, 0), S0_dev, bytes, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+        if (launch_store_state(S0_dev, ctx->s0_slot(req_begin, 0), ctx->s0_scale_slot(req_begin, 0),
+                               (long long)req_count * ctx->cfg.num_layers * ctx->Hv(), ctx->cfg.dk, ctx->cfg.dv,
+                               s) != cudaSuccess)
             return ONELA_E_CUDA;
         ctx->launches++;
     }
@@ -291,9 +294,9 @@ onela_status onela_prefill_shared_state(onela_ctx* ctx, int32_t request, int32_t
     if ((st = ctx->prepare(s)) != ONELA_OK) return st;
     if (!ctx->dry()) {
         bool supported = true;
-        const cudaError_t e = launch_prefill(k_dev, v_dev, alpha_dev, beta_dev, ctx->s0_slot(request, layer), n_tokens,
-                                             ctx->cfg.num_heads, ctx->cfg.dk, ctx->cfg.dv, ctx->cfg.rec_dtype,
-                                             &supported, s);
+        const cudaError_t e = launch_prefill(k_dev, v_dev, alpha_dev, beta_dev, ctx->s0_slot(request, layer),
+                                             ctx->s0_scale_slot(request, layer), n_tokens, ctx->cfg.num_heads, ctx->cfg.dk,
+                                             ctx->cfg.dv, ctx->cfg.rec_dtype, &supported, s);
         if (!supported) return ONELA_E_UNSUPPORTED;
         if (e != cudaSuccess) return ONELA_E_CUDA;
         ctx->launches++;
@@ -497,6 +500,8 @@ onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count,
     a.table = ctx->table_cur(req_begin);
     a.status = ctx->lay.status;
     a.s0_req_stride = (long long)c.num_layers * ctx->s0_layer_floats();
+    a.s0_scale = ctx->s0_scale_slot(req_begin, layer);
+    a.s0_scale_req_stride = (long long)c.num_layers * ctx->Hv();
     a.table_req_stride = ctx->table_req_stride();
     a.arena_slots = c.arena_slots;
     a.sidx = ctx->lay.sidx + req_begin * ctx->sidx_req_stride();

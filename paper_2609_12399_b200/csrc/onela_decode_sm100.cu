@@ -7,8 +7,8 @@
 //     async copies, one quad ahead; with the append fused in
 //     they come from the caller's token tensors and the warp also writes them to the arena.  Results go into a
 //     ring slot in shared memory: the folded query as a row of the K-major 128-byte-swizzled MMA operand
-//     (rounded to TF32), corr as a row of the slot's corr tile.
-//   * 4 EPILOGUE warps (one per tensor-memory lane quadrant).  One lane of the first issues a group's 16 MMAs
+//     (fp16, times a power of two that keeps the row inside fp16's range), corr as a row of the slot's corr tile.
+//   * 4 EPILOGUE warps (one per tensor-memory lane quadrant).  One lane of the first issues a group's 8 MMAs
 //     once all its rows are written - one group ahead of the epilogue, so neither the issuing nor the MMAs'
 //     latency lies between two epilogues.  When a group's MMAs have completed the four warps read the
 //     accumulator and transpose it, by plain stores, over the slot's operand rows (dead by then); the other
@@ -18,7 +18,7 @@
 // Two ring slots (operand rows, corr tile, 48 accumulator columns each) keep the MMA and the epilogue of one
 // group under the folds of the next.  Work = groups of 48 consecutive beams of one (request, head), a
 // contiguous range per CTA chosen on the host; consecutive groups of one head form a segment.  Per segment the
-// head's S_0 sits in tensor memory (rounded to TF32; it is the MMA's A operand there) and the oldest chain
+// head's S_0 sits in tensor memory (as fp16, scaled by the head's power of two; it is the MMA's A operand there) and the oldest chain
 // levels are staged in shared memory, one 512-byte bulk copy per DISTINCT ancestor record (as many whole levels
 // as fit).  S_0 and the staging area are double-buffered, so a CTA moves from one segment to the next without
 // draining: nothing in the main loop is a CTA-wide barrier.
@@ -56,8 +56,9 @@ constexpr int UPW = 32 / LPU;                       // units a fold warp folds a
 constexpr int NCH = 16 / LPU;                       // 16-byte chunks per lane per 256-byte vector
 constexpr int THREADS = (FOLD_WARPS + 4) * 32;      // + 4 epilogue warps (16 warps: four per SM sub-partition)
 constexpr int GN = FOLD_WARPS * UPW;                // beams per group = MMA N (48)
-constexpr int R_KB_STRIDE = GN * 128;               // bytes between the four 32-float K blocks of the operand
-constexpr int R_BYTES = 4 * R_KB_STRIDE;            // operand rows of a group
+constexpr int R_KB_STRIDE = GN * 128;               // bytes between the two K blocks (64 fp16 each) of the operand
+constexpr int R_BYTES = 4 * R_KB_STRIDE;            // a slot's first tile: the group's operand rows (its first half),
+                                                    // later the transposed accumulators (all of it)
 constexpr int C_BYTES = GN * DV * 4;                // corr tile, row = beam
 constexpr int SLOT_BYTES = R_BYTES + C_BYTES;
 constexpr int SLOTS = 2;
@@ -72,8 +73,10 @@ constexpr int HEADS_TOTAL = FOLD_WARPS * HEAD_BYTES;     // one stage per fold w
 constexpr int STAGE_BUF = ONELA_STAGE_BUF;
 constexpr int STAGE_BYTES = 2 * STAGE_BUF * REC_BYTES;
 constexpr int GATE_BYTES = (2 * STAGE_BUF * 8 + 127) & ~127;   // padded: the heads' stages behind it stay 128-byte aligned (measured: 1.5 % faster)
-constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + STAGE_BYTES + GATE_BYTES + HEADS_TOTAL + 256 + 1024;
-constexpr uint32_t S0_COL = 128;                 // accumulators of the ring slots in [0, SLOTS * GN); S_0 buffers at 128 and 256
+constexpr int INV_BYTES = SLOTS * GN * 4;        // per ring slot and beam: what undoes the operands' scales
+constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + STAGE_BYTES + GATE_BYTES + HEADS_TOTAL + 256 + INV_BYTES + 1024;
+constexpr uint32_t S0_COL = 128;                 // accumulators of the ring slots in [0, SLOTS * GN); S_0 buffers (64 columns) at 128 and 256
+constexpr int R_TARGET = 8;                      // a scaled operand row stays below 2^8 x (decay in [1, 2)): far inside fp16's range
 constexpr uint32_t TMEM_COLS = 512;
 static_assert(SLOTS * GN <= 128, "accumulator columns");
 static_assert(R_BYTES >= C_BYTES, "the accumulators are transposed over the operand rows");
@@ -133,6 +136,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     const uint32_t bar_s0_first = smem_u32(bars + 6 + 3 * SLOTS);   // the first segment's S_0, put there by all warps
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 7 + 3 * SLOTS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    float* inv_s = reinterpret_cast<float*>(heads + HEADS_TOTAL + 256);      // [SLOTS][GN]
     auto bar_s0 = [&](int b) { return smem_u32(bars + b); };
     auto bar_stage = [&](int b) { return smem_u32(bars + 2 + b); };
     auto bar_sfree = [&](int b) { return smem_u32(bars + 4 + b); };
@@ -190,25 +194,27 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     const int grp = lane / LPU, g = lane % LPU;
     bool dead = false;                    // this warp gave up (timeout or abort raised elsewhere)
 
-    // S_0 of a (request, head) goes to tensor memory, rounded to TF32 on the way: it is the MMA's A operand there, so
-    // there is no shared-memory copy of S_0 and no S_0 traffic per MMA.  Row-major fp32 in the store; lane i of
-    // tensor memory holds row i; the 128 columns of buffer `buf` start at S0_COL + 128 buf.  A warp takes the 32
-    // rows of its lane quadrant and the 32-column blocks kb0, kb0 + step, ...; the S_0 after this one is requested
-    // into L2 on the way.
+    // S_0 of a (request, head) goes to tensor memory as fp16 (TF32's mantissa; K = 16 per MMA instead of 8), times
+    // the head's power-of-two scale from the store, which keeps it inside fp16's range whatever the caller's units:
+    // it is the MMA's A operand there, so there is no shared-memory copy of S_0 and no S_0 traffic per MMA.
+    // Row-major fp32 in the store; lane i of tensor memory holds row i, two elements per column; the 64 columns of
+    // buffer `buf` start at S0_COL + 128 buf.  A warp takes the 32 rows of its lane quadrant and the 32-element blocks
+    // kb0, kb0 + step, ...; the S_0 after this one is requested into L2 on the way.
     auto load_s0 = [&](int pair_now, int buf, int kb0, int step, bool has_next) {
         const int quad = warp & 3, i = quad * 32 + lane;
         const int req = pair_now / a.H, h = pair_now - req * a.H;
         const float* row = a.s0 + req * a.s0_req_stride + (long long)h * (DV * DK) + (long long)i * DK;
+        const float sc = __ldg(a.s0_scale + req * a.s0_scale_req_stride + h);
 #pragma unroll 1
         for (int kb = kb0; kb < 4; kb += step) {
-            uint32_t v[32];
+            uint32_t v[16];
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const float4 x = __ldg(reinterpret_cast<const float4*>(row + kb * 32) + c);
-                v[4 * c] = __float_as_uint(round_tf32(x.x)); v[4 * c + 1] = __float_as_uint(round_tf32(x.y));
-                v[4 * c + 2] = __float_as_uint(round_tf32(x.z)); v[4 * c + 3] = __float_as_uint(round_tf32(x.w));
+                v[2 * c] = pack_f16x2(x.x * sc, x.y * sc);
+                v[2 * c + 1] = pack_f16x2(x.z * sc, x.w * sc);
             }
-            tmem_st32(tmem_base + S0_COL + buf * 128 + kb * 32 + ((uint32_t)(quad * 32) << 16), v);
+            tmem_st16(tmem_base + S0_COL + buf * 128 + kb * 16 + ((uint32_t)(quad * 32) << 16), v);
             if (has_next) {
                 const int nreq = (pair_now + 1) / a.H, nh = (pair_now + 1) - nreq * a.H;
                 const float* nrow = a.s0 + nreq * a.s0_req_stride + (long long)nh * (DV * DK) + (long long)i * DK + kb * 32;
@@ -224,8 +230,10 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     static_assert(THREADS >= 512, "the first sixteen warps take one 32-column block of the first S_0 each");
     const bool s0_mine = warp < 16;
     float4 s0_first[8];
+    float s0_first_scale = 1.f;
     if (n_segs > 0 && s0_mine) {
         const int req = pair_begin / a.H, h = pair_begin - req * a.H;
+        s0_first_scale = __ldg(a.s0_scale + req * a.s0_scale_req_stride + h);
         const float* row = a.s0 + req * a.s0_req_stride + (long long)h * (DV * DK) + (long long)((warp & 3) * 32 + lane) * DK + (warp >> 2) * 32;
 #pragma unroll
         for (int c = 0; c < 8; ++c) s0_first[c] = __ldg(reinterpret_cast<const float4*>(row) + c);
@@ -237,13 +245,14 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     }
     auto put_first_s0 = [&]() {
         if (n_segs == 0 || !s0_mine) return;
-        uint32_t v[32];
+        const float sc = s0_first_scale;
+        uint32_t v[16];
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
-            v[4 * c] = __float_as_uint(round_tf32(s0_first[c].x)); v[4 * c + 1] = __float_as_uint(round_tf32(s0_first[c].y));
-            v[4 * c + 2] = __float_as_uint(round_tf32(s0_first[c].z)); v[4 * c + 3] = __float_as_uint(round_tf32(s0_first[c].w));
+            v[2 * c] = pack_f16x2(s0_first[c].x * sc, s0_first[c].y * sc);
+            v[2 * c + 1] = pack_f16x2(s0_first[c].z * sc, s0_first[c].w * sc);
         }
-        tmem_st32(tmem_base + S0_COL + (warp >> 2) * 32 + ((uint32_t)((warp & 3) * 32) << 16), v);
+        tmem_st16(tmem_base + S0_COL + (warp >> 2) * 16 + ((uint32_t)((warp & 3) * 32) << 16), v);
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncwarp();
@@ -383,6 +392,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         }
         put_first_s0();
         int cur_seg = -1, buf = 0, staged_levels = 0, n_ahead = 0;
+        float seg_inv_s0 = 1.f;
         bool staged_ready = false;
         long long plane_row0 = 0, own_row0 = 0;
         const int32_t *table_r = nullptr, *sidx_r = nullptr;
@@ -398,6 +408,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                     staged_levels = staged_levels_of(u0.req);
                     // levels gathered from global memory whose lines are worth requesting ahead (end of the loop)
                     if (AHEAD) n_ahead = (info_sparse >> staged_levels) ? min(old - staged_levels, NIDX * LPU - staged_levels) : 0;
+                    seg_inv_s0 = 1.f / __ldg(a.s0_scale + u0.req * a.s0_scale_req_stride + u0.h);   // a power of two
                     plane_row0 = (long long)u0.h * a.arena_slots;
                     own_row0 = plane_row0 + a.bases.base[u0.req];
                     table_r = a.table + u0.req * a.table_req_stride;
@@ -468,6 +479,25 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     #pragma unroll
                 for (int e = 0; e < 4 * NCH; ++e) corr[e] = make_float2(0.f, 0.f);
                 float decay = 1.f;
+                // The scale of the unit's operand row, from the query's norm: a fold step never lengthens r~ (keys of
+                // norm <= 1, beta in [0, 2]), so |r~| stays below 2^hq, the power of two above |q|; scaled to 2^R_TARGET
+                // it leaves a 2^(15 - R_TARGET)-fold margin to fp16's largest number and over twenty binades below it
+                // before elements turn subnormal.  Taken here, off the end-of-quad path (one shuffle reduction).
+                float q_scale = 1.f, q_inv = 1.f;
+                {
+                    float2 n2 = make_float2(0.f, 0.f);
+    #pragma unroll
+                    for (int e = 0; e < 4 * NCH; ++e) n2 = __ffma2_rn(r[e], r[e], n2);
+                    float norm2 = n2.x + n2.y;
+    #pragma unroll
+                    for (int o = LPU / 2; o > 0; o >>= 1) norm2 += __shfl_xor_sync(0xffffffffu, norm2, o);
+                    const int eb = (int)(__float_as_uint(norm2) >> 23) & 255;      // |q|^2 in [2^(eb-127), 2^(eb-126))
+                    const int hq = (eb - 127 + 2) >> 1;                             // |q| < 2^hq
+                    if (eb > 0 && eb < 255 && hq > -100 && hq < 100) {
+                        q_scale = __uint_as_float((uint32_t)(127 + R_TARGET - hq) << 23);
+                        q_inv = __uint_as_float((uint32_t)(127 + hq - R_TARGET) << 23);
+                    }
+                }
                 L::fold_chain_simple(cur.own, old - 1, staged_levels,
                               [&](int level) {
                                   const long long slot = idx_of(level);
@@ -514,20 +544,26 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                     // the corr tile (a layout of our own) swaps each pair of 16-byte chunks in every other 128-byte
                     // stretch of a row instead (corr_chunk; the epilogue reads it the same way).
                     const int sw = u & 7;
-                    const bool hi = (g >> 2) & 1;
-                    const float2 dc = make_float2(decay, decay);
+                    // The folded query decay * r~ goes out as fp16 times two powers of two: the query's (taken when the
+                    // quad started: |r~| <= |q| < 2^R_TARGET / q_scale) and the one that brings the decay into [1, 2).  The
+                    // epilogue multiplies the accumulator by the reciprocals (and by that of the head's S_0 scale), exactly.
+                    float d_scale, d_inv;
+                    pow2_scale(decay, 0, d_scale, d_inv);
+                    if (g == 0) inv_s[s * GN + u] = (q_inv * d_inv) * seg_inv_s0;
+                    const float dcs = (decay * d_scale) * q_scale;
+                    const float2 dc = make_float2(dcs, dcs);
     #pragma unroll
                     for (int c = 0; c < NCH; ++c) {
                         const int ci = c * LPU + g;                 // elements [8 ci, 8 ci + 8)
-                        const int kb = ci >> 2, ch = 2 * (ci & 3);  // K block of 32 floats; first of two 16-byte chunks
-                        uint8_t* row = R_s + kb * R_KB_STRIDE + u * 128;
                         float2 x[4];
     #pragma unroll
                         for (int e = 0; e < 4; ++e) x[e] = __fmul2_rn(r[4 * c + e], dc);
-                        const float4 lo4 = make_float4(round_tf32(x[0].x), round_tf32(x[0].y), round_tf32(x[1].x), round_tf32(x[1].y));
-                        const float4 hi4 = make_float4(round_tf32(x[2].x), round_tf32(x[2].y), round_tf32(x[3].x), round_tf32(x[3].y));
-                        *reinterpret_cast<float4*>(row + (((ch + (hi ? 1 : 0)) ^ sw) << 4)) = hi ? hi4 : lo4;
-                        *reinterpret_cast<float4*>(row + (((ch + (hi ? 0 : 1)) ^ sw) << 4)) = hi ? lo4 : hi4;
+                        // fp16 operand rows: K blocks of 64 elements (128 bytes, 128-byte swizzle), one 16-byte chunk
+                        // per lane and c; a warp's four rows are 512 consecutive bytes: no bank conflicts
+                        uint8_t* row = R_s + (ci >> 3) * R_KB_STRIDE + u * 128;
+                        *reinterpret_cast<uint4*>(row + (((ci & 7) ^ sw) << 4)) =
+                            make_uint4(pack_f16x2(x[0].x, x[0].y), pack_f16x2(x[1].x, x[1].y), pack_f16x2(x[2].x, x[2].y),
+                                       pack_f16x2(x[3].x, x[3].y));
                         float* crow = C_s + u * DV;
                         *reinterpret_cast<float4*>(crow + corr_chunk(2 * ci) * 4) =
                             make_float4(corr[4 * c].x, corr[4 * c].y, corr[4 * c + 1].x, corr[4 * c + 1].y);
@@ -617,7 +653,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             prepare_s0(1);
         }
 
-        // The first epilogue warp issues a group's 16 MMAs as soon as all its rows are written (never a fold warp:
+        // The first epilogue warp issues a group's 8 MMAs as soon as all its rows are written (never a fold warp:
         // whichever fold warp issued would be the last to finish its next quad).  It does so one group AHEAD: once
         // the tile of group k is complete (the named barrier below) it issues group k + 1 while the other three
         // warps store group k, so neither the issuing nor the MMAs' latency lies between two epilogues.
@@ -632,15 +668,15 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 if (ok && gcount == 0) ok = wait_or_abort(bar_s0_first, 0, abort_flag);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 if (ok) {
-                    constexpr uint32_t idesc = idesc_tf32(GN);
+                    constexpr uint32_t idesc = idesc_f16(GN);
                     const uint64_t bd = umma_desc(smem_u32(ring + s * SLOT_BYTES));
                     const uint32_t s0_at = tmem_base + S0_COL + (seg & 1) * 128;
 #pragma unroll
-                    for (int kb = 0; kb < 4; ++kb)
+                    for (int kb = 0; kb < 2; ++kb)          // K block of 64 elements; 16 elements (32 bytes, 8 columns) per MMA
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks)
-                            umma_tf32_ts(tmem_base + s * GN, s0_at + (kb * 4 + ks) * 8,
-                                         bd + (uint64_t)((kb * R_KB_STRIDE + ks * 32) >> 4), idesc, (kb | ks) ? 1u : 0u);
+                            umma_f16_ts(tmem_base + s * GN, s0_at + (kb * 4 + ks) * 8,
+                                        bd + (uint64_t)((kb * R_KB_STRIDE + ks * 32) >> 4), idesc, (kb | ks) ? 1u : 0u);
                 } else {
                     mma_failed = 1;
                 }
@@ -700,8 +736,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                         const int o0 = j * DV + corr_chunk(2 * ch) * 4, o1 = j * DV + corr_chunk(2 * ch + 1) * 4;
                         const float4 x0 = *reinterpret_cast<const float4*>(C_s + o0), y0 = *reinterpret_cast<const float4*>(A_s + o0);
                         const float4 x1 = *reinterpret_cast<const float4*>(C_s + o1), y1 = *reinterpret_cast<const float4*>(A_s + o1);
-                        const float o[8] = {x0.x + y0.x, x0.y + y0.y, x0.z + y0.z, x0.w + y0.w,
-                                            x1.x + y1.x, x1.y + y1.y, x1.z + y1.z, x1.w + y1.w};
+                        const float w = inv_s[s * GN + j];        // undoes the scales of the beam's operand row and of S_0
+                        const float o[8] = {fmaf(y0.x, w, x0.x), fmaf(y0.y, w, x0.y), fmaf(y0.z, w, x0.z), fmaf(y0.w, w, x0.w),
+                                            fmaf(y1.x, w, x1.x), fmaf(y1.y, w, x1.y), fmaf(y1.z, w, x1.z), fmaf(y1.w, w, x1.w)};
                         store8<OutT>(out0 + (long long)j * a.H * DV + ch * 8, o);
                     }
                 }

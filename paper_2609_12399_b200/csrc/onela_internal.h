@@ -22,6 +22,9 @@ struct Layout {
                        // (grouped value heads: keys only, [layer][key head][arena_slots][dk])
     char* vv;          // grouped value heads only: values [layer][value head][arena_slots][dv]
     unsigned long long* select_scratch;   // [request][ONELA_SELECT_PARTS][ONELA_SELECT_CAP]: partial results of beam selection
+    float* s0_scale;   // [request][layer][head]: the power of two that brings the head's largest |S_0| element into
+                       // [2^11, 2^12) (1 for an all-zero or non-finite state); written with the state, read by the
+                       // tensor-core kernel, whose fp16 operand it keeps in range
     size_t total_bytes;
 };
 
@@ -58,6 +61,9 @@ struct DecodeArgs {
     const char* vv;
     char* vv_out;
     int32_t Hk, g;
+    // tensor-core kernel: per-head operand scale of S_0 (see Layout), entry of (req_begin, layer, head 0)
+    const float* s0_scale;
+    long long s0_scale_req_stride;
 };
 
 // Grouped value heads (Hv = g * Hk): what the grouped decode kernel needs.
@@ -110,12 +116,14 @@ cudaError_t launch_append(const void* k, const void* v, const float* alpha, cons
                           float2* gate_plane, long long arena_slots, int32_t req_count, int32_t W, int32_t H,
                           int32_t dk, int32_t dv, int32_t elem_bytes, const BatchBases& bases,
                           cudaStream_t stream);
-cudaError_t launch_store_state(const float* S0_in, float* slot, int32_t H, int32_t dk, int32_t dv, cudaStream_t stream);
+// copies n_heads states of dv x dk floats and leaves each head's operand scale (see Layout::s0_scale) in scale_out
+cudaError_t launch_store_state(const float* S0_in, float* slot, float* scale_out, long long n_heads, int32_t dk, int32_t dv,
+                               cudaStream_t stream);
 cudaError_t launch_export_state(const float* slot, float* S0_out, int32_t H, int32_t dk, int32_t dv, cudaStream_t stream);
 // returns cudaErrorInvalidValue with *supported = false when (dk, dv, dtype) has no instantiation
 cudaError_t launch_prefill(const void* k, const void* v, const float* alpha, const float* beta, float* slot,
-                           int32_t n_tokens, int32_t H, int32_t dk, int32_t dv, int32_t rec_dtype, bool* supported,
-                           cudaStream_t stream);
+                           float* scale_out, int32_t n_tokens, int32_t H, int32_t dk, int32_t dv, int32_t rec_dtype,
+                           bool* supported, cudaStream_t stream);
 
 // decode kernels
 cudaError_t launch_decode_generic(const DecodeArgs& a, int32_t dk, int32_t dv, int32_t rec_dtype,

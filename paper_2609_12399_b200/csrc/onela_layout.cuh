@@ -1,19 +1,10 @@
-// Device helpers shared by the kernel files: TF32 rounding and bf16 unpacking.
+// Device helpers shared by the kernel files: bf16 unpacking.
 #pragma once
 
 #include <cuda_bf16.h>
 #include <stdint.h>
 
 namespace onela {
-
-// Round to the nearest TF32 value (10 explicit mantissa bits), ties away from zero.  The tensor core
-// reads only the upper 19 bits of an fp32 operand; rounding an operand before it is handed over makes that
-// read unbiased instead of a truncation.
-__device__ __forceinline__ float round_tf32(float x) {
-    uint32_t u;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(x));
-    return __uint_as_float(u);
-}
 
 // Two packed bf16 (little endian: element 0 in the low half) -> two fp32, exactly.
 __device__ __forceinline__ void unpack_bf16x2(uint32_t w, float& lo, float& hi) {

@@ -40,11 +40,46 @@ __device__ __forceinline__ float to_float<float>(float x) { return x; }
 template <>
 __device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
 
+// The operand scale of a head (Layout::s0_scale) from the largest magnitude of its state.
+__device__ __forceinline__ float operand_scale(float peak) {
+    const int eb = (int)(__float_as_uint(peak) >> 23) & 255;          // biased exponent of a non-negative number
+    constexpr int target = 11;                                         // scaled peak in [2^11, 2^12)
+    const bool ok = eb > target + 1 && eb < 255;
+    return ok ? __uint_as_float((uint32_t)(254 + target - eb) << 23) : 1.f;
+}
+// Largest value over the CTA (<= 1024 threads), returned to thread 0.
+__device__ __forceinline__ float block_max(float v) {
+    __shared__ float part[32];
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = v;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        v = threadIdx.x < (blockDim.x + 31) / 32 ? part[threadIdx.x] : 0.f;
+        for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    }
+    return v;
+}
+
+// Copy of the caller's states into the store, one CTA per head, with the head's operand scale as a by-product.
+__global__ void __launch_bounds__(256) store_state_kernel(const float4* __restrict__ in, float4* __restrict__ out,
+                                                          float* __restrict__ scale_out, int32_t vec_per_head) {
+    const long long base = (long long)blockIdx.x * vec_per_head;
+    float peak = 0.f;
+    for (int i = threadIdx.x; i < vec_per_head; i += blockDim.x) {
+        const float4 x = __ldg(in + base + i);
+        out[base + i] = x;
+        peak = fmaxf(fmaxf(peak, fmaxf(fabsf(x.x), fabsf(x.y))), fmaxf(fabsf(x.z), fabsf(x.w)));
+    }
+    peak = block_max(peak);
+    if (threadIdx.x == 0) scale_out[blockIdx.x] = operand_scale(peak);
+}
+
 // Eq. 1 from the zero state over the prompt, one CTA per head, thread i owns row i of S in registers.
 template <int DK, int DV, typename T>
 __global__ void __launch_bounds__(DV) prefill_kernel(const T* __restrict__ k, const T* __restrict__ v,
                                                      const float* __restrict__ alpha, const float* __restrict__ beta,
-                                                     float* __restrict__ slot, int32_t n_tokens, int32_t H) {
+                                                     float* __restrict__ slot, float* __restrict__ scale_out,
+                                                     int32_t n_tokens, int32_t H) {
     __shared__ __align__(16) float k_s[2][DK];
     const int h = blockIdx.x, i = threadIdx.x;
     float S[DK];
@@ -99,19 +134,25 @@ __global__ void __launch_bounds__(DV) prefill_kernel(const T* __restrict__ k, co
         __syncthreads();
     }
     float* dst = slot + (long long)h * DV * DK;
+    float peak = 0.f;
 #pragma unroll
-    for (int j = 0; j < DK; ++j) dst[(long long)i * DK + j] = S[j];
+    for (int j = 0; j < DK; ++j) {
+        dst[(long long)i * DK + j] = S[j];
+        peak = fmaxf(peak, fabsf(S[j]));
+    }
+    peak = block_max(peak);
+    if (i == 0) scale_out[h] = operand_scale(peak);
 }
 
 template <int DK, int DV>
 cudaError_t prefill_dispatch(const void* k, const void* v, const float* alpha, const float* beta, float* slot,
-                             int32_t n_tokens, int32_t H, int32_t rec_dtype, cudaStream_t stream) {
+                             float* scale_out, int32_t n_tokens, int32_t H, int32_t rec_dtype, cudaStream_t stream) {
     if (rec_dtype == ONELA_DTYPE_BF16)
         prefill_kernel<DK, DV, __nv_bfloat16><<<H, DV, 0, stream>>>(
-            static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(v), alpha, beta, slot, n_tokens, H);
+            static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(v), alpha, beta, slot, scale_out, n_tokens, H);
     else
         prefill_kernel<DK, DV, float><<<H, DV, 0, stream>>>(static_cast<const float*>(k), static_cast<const float*>(v),
-                                                           alpha, beta, slot, n_tokens, H);
+                                                           alpha, beta, slot, scale_out, n_tokens, H);
     return cudaGetLastError();
 }
 
@@ -129,8 +170,12 @@ cudaError_t launch_append(const void* k, const void* v, const float* alpha, cons
     return cudaGetLastError();
 }
 
-cudaError_t launch_store_state(const float* S0_in, float* slot, int32_t H, int32_t dk, int32_t dv, cudaStream_t stream) {
-    return cudaMemcpyAsync(slot, S0_in, (size_t)H * dk * dv * sizeof(float), cudaMemcpyDeviceToDevice, stream);
+cudaError_t launch_store_state(const float* S0_in, float* slot, float* scale_out, long long n_heads, int32_t dk, int32_t dv,
+                               cudaStream_t stream) {
+    if (n_heads <= 0 || n_heads > 0x7fffffffLL) return cudaErrorInvalidValue;
+    store_state_kernel<<<(unsigned)n_heads, 256, 0, stream>>>(reinterpret_cast<const float4*>(S0_in), reinterpret_cast<float4*>(slot),
+                                                             scale_out, dk * dv / 4);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_export_state(const float* slot, float* S0_out, int32_t H, int32_t dk, int32_t dv, cudaStream_t stream) {
@@ -138,12 +183,12 @@ cudaError_t launch_export_state(const float* slot, float* S0_out, int32_t H, int
 }
 
 cudaError_t launch_prefill(const void* k, const void* v, const float* alpha, const float* beta, float* slot,
-                           int32_t n_tokens, int32_t H, int32_t dk, int32_t dv, int32_t rec_dtype, bool* supported,
-                           cudaStream_t stream) {
+                           float* scale_out, int32_t n_tokens, int32_t H, int32_t dk, int32_t dv, int32_t rec_dtype,
+                           bool* supported, cudaStream_t stream) {
     *supported = true;
-    if (dk == 32 && dv == 32) return prefill_dispatch<32, 32>(k, v, alpha, beta, slot, n_tokens, H, rec_dtype, stream);
-    if (dk == 64 && dv == 64) return prefill_dispatch<64, 64>(k, v, alpha, beta, slot, n_tokens, H, rec_dtype, stream);
-    if (dk == 128 && dv == 128) return prefill_dispatch<128, 128>(k, v, alpha, beta, slot, n_tokens, H, rec_dtype, stream);
+    if (dk == 32 && dv == 32) return prefill_dispatch<32, 32>(k, v, alpha, beta, slot, scale_out, n_tokens, H, rec_dtype, stream);
+    if (dk == 64 && dv == 64) return prefill_dispatch<64, 64>(k, v, alpha, beta, slot, scale_out, n_tokens, H, rec_dtype, stream);
+    if (dk == 128 && dv == 128) return prefill_dispatch<128, 128>(k, v, alpha, beta, slot, scale_out, n_tokens, H, rec_dtype, stream);
     *supported = false;
     return cudaErrorInvalidValue;
 }

@@ -314,3 +314,22 @@ def test_batched_state_store_equals_the_single_calls():
     assert torch.equal(ctx.onela_export_shared_state(0, 1).cpu(), S[0, 1] + 1)
     assert ctx.onela_poll_device_status() == (0, 0)
 
+
+@pytest.mark.parametrize("s0_unit,q_unit", [(1e-6, 1.0), (3e4, 1.0), (1.0, 1e-5), (1.0, 2e3), (1e-5, 1e-4), (1e4, 50.0)])
+def test_tensor_core_operands_keep_their_precision_at_any_scale(s0_unit, q_unit):
+    """The tensor-core kernel feeds fp16 operands; per-head and per-beam powers of two keep them inside the format's
+    range, so states and queries far from unit scale decode as accurately as unit-scale ones (states of 1e-6 or
+    queries of 1e-5 would otherwise sink into fp16's subnormals, states of 3e4 x 128 terms overflow it)."""
+    wl = CFG1.scaled(H=2, W=70, D=3, prompt_len=48, parents="zipf", zipf_s=1.5, seed=4242)
+    case = make_case(wl)
+    for key in case["S0"]:
+        case["S0"][key] = (case["S0"][key].double() * s0_unit).float()
+    for key in case["q"]:
+        case["q"][key] = (case["q"][key].double() * q_unit).to(case["q"][key].dtype)
+    for fused in (True, False):
+        outs, _, ctx = run_library(case, out_dtype="fp32", fused=fused)
+        assert ctx.onela_uses_tensor_core_path()
+        assert ctx.onela_poll_device_status() == (0, 0)
+        ref, _ = run_oracle(case)
+        for key, o in outs.items():
+            assert rel_l2(o.numpy(), ref[key]).max() <= REL_L2_BAR

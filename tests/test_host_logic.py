@@ -70,7 +70,8 @@ def test_workspace_carve_up_size():
     tables = 4 * 2 * 8 * 512 * 4
     index = 2 * (4 * 8 * 512 * 4) + 4 * 9 * 4          # distinct-record index: positions, slot list, level offsets
     select = 4 * 256 * 1024 * 8                        # beam selection: per request 256 partial lists of 1024 candidates
-    assert s0 + arena + tables + index + select <= n <= s0 + arena + tables + index + select + 9 * 1024
+    scales = 4 * 16 * 32 * 4                           # one operand scale per stored head state
+    assert s0 + arena + tables + index + select + scales <= n <= s0 + arena + tables + index + select + scales + 10 * 1024
 
 
 def test_call_order_is_enforced():
