@@ -42,9 +42,9 @@ UNIT = "decodes/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE fused append + decode launch of the default workload at
 # its deepest call (depth 8, all 4 requests of one layer), from the ncu capture summarised in
-# profiles/decode_ws_kernel_cfg4_ncu.md (69.1 MB read + 12.7 MB written).  The algorithmic bytes of that launch
+# profiles/decode_ws_kernel_cfg4_ncu.md (69.1 MB read + 11.9 MB written).  The algorithmic bytes of that launch
 # are 118.7 MB; of the 50.9 MB it writes, 38 MB were still in L2 when the kernel ended.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 81.8e6
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 81.0e6
 
 
 def workload_by_name(name: str) -> inputs.Workload:
