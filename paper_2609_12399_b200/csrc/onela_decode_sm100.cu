@@ -729,6 +729,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 // coalesced stores by the other three warps: 16 lanes cover one beam's 128 outputs, 8 elements each
                 const int et = (warp - FOLD_WARPS - 1) * 32 + lane;
                 OutT* out0 = static_cast<OutT*>(a.out) + (((long long)req * a.W + b0) * a.H + h) * DV;
+                float w8[GN * 16 / 96];                        // what undoes the scales of each row this thread stores
+#pragma unroll
+                for (int it = 0; it < GN * 16 / 96; ++it) w8[it] = inv_s[s * GN + ((it * 96 + et) >> 4)];
 #pragma unroll
                 for (int it = 0; it < GN * 16 / 96; ++it) {    // GN * 16 chunks of 16 bytes over 96 threads
                     const int idx = it * 96 + et, j = idx >> 4, ch = idx & 15;
@@ -736,7 +739,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                         const int o0 = j * DV + corr_chunk(2 * ch) * 4, o1 = j * DV + corr_chunk(2 * ch + 1) * 4;
                         const float4 x0 = *reinterpret_cast<const float4*>(C_s + o0), y0 = *reinterpret_cast<const float4*>(A_s + o0);
                         const float4 x1 = *reinterpret_cast<const float4*>(C_s + o1), y1 = *reinterpret_cast<const float4*>(A_s + o1);
-                        const float w = inv_s[s * GN + j];        // undoes the scales of the beam's operand row and of S_0
+                        const float w = w8[it];
                         const float o[8] = {fmaf(y0.x, w, x0.x), fmaf(y0.y, w, x0.y), fmaf(y0.z, w, x0.z), fmaf(y0.w, w, x0.w),
                                             fmaf(y1.x, w, x1.x), fmaf(y1.y, w, x1.y), fmaf(y1.z, w, x1.z), fmaf(y1.w, w, x1.w)};
                         store8<OutT>(out0 + (long long)j * a.H * DV + ch * 8, o);
