@@ -4,8 +4,8 @@
 //   * 12 FOLD warps.  8 lanes own one (beam, head) unit; a warp folds 4 units at a time ("quad"): query
 //     folded through the unit's records newest -> oldest (c = k.r; corr += beta c v; r -= beta c k; decay a
 //     scalar; packed fp32x2 FMAs).  A quad's query and own record arrive through a per-warp stage of 16-byte
-//     async copies, one quad ahead; with the append fused in
-//     they come from the caller's token tensors and the warp also writes them to the arena.  Results go into a
+//     async copies, one quad ahead; with the append fused in they come from the caller's token tensors and the
+//     warp also writes them to the arena.  Results go into a
 //     ring slot in shared memory: the folded query as a row of the K-major 128-byte-swizzled MMA operand
 //     (fp16, times a power of two that keeps the row inside fp16's range), corr as a row of the slot's corr tile.
 //   * 4 EPILOGUE warps (one per tensor-memory lane quadrant).  One lane of the first issues a group's 8 MMAs
@@ -18,9 +18,9 @@
 // Two ring slots (operand rows, corr tile, 48 accumulator columns each) keep the MMA and the epilogue of one
 // group under the folds of the next.  Work = groups of 48 consecutive beams of one (request, head), a
 // contiguous range per CTA chosen on the host; consecutive groups of one head form a segment.  Per segment the
-// head's S_0 sits in tensor memory (as fp16, scaled by the head's power of two; it is the MMA's A operand there) and the oldest chain
-// levels are staged in shared memory, one 512-byte bulk copy per DISTINCT ancestor record (as many whole levels
-// as fit).  S_0 and the staging area are double-buffered, so a CTA moves from one segment to the next without
+// head's S_0 sits in tensor memory (as fp16, scaled by the head's power of two; it is the MMA's A operand there)
+// and the oldest chain levels are staged in shared memory, one 512-byte bulk copy per DISTINCT ancestor record (as
+// many whole levels as fit).  S_0 and the staging area are double-buffered, so a CTA moves from one segment to the next without
 // draining: nothing in the main loop is a CTA-wide barrier.
 // A second instantiation (GROUPED) serves grouped value heads: segments are (request, VALUE head), the query and the
 // keys are those of key head h / g, and a record's two halves live in two planes (keys per key head, values per value
@@ -423,7 +423,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                     asm volatile("cp.async.wait_group 0;" ::: "memory");
                     const uint4* rec = reinterpret_cast<const uint4*>(my_heads + grp * REC_BYTES) + g;
                     const uint4* qv = reinterpret_cast<const uint4*>(my_heads + UPW * REC_BYTES + grp * (DK * 2)) + g;
-    #pragma unroll
+#pragma unroll
                     for (int c = 0; c < NCH; ++c) {
                         cur.own.k[c] = rec[c * LPU];
                         cur.own.v[c] = rec[16 + c * LPU];
@@ -437,16 +437,16 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                         if constexpr (GROUPED) {
                             const long long slot = a.bases.base[u0.req] + bb;
                             uint4* vdst = reinterpret_cast<uint4*>(a.vv_out + ((long long)u0.h * a.arena_slots + slot) * (DV * 2)) + g;
-    #pragma unroll
+#pragma unroll
                             for (int c = 0; c < NCH; ++c) vdst[c * LPU] = cur.own.v[c];
                             if (u0.h % a.g == 0) {     // the key is stored once per key head: by its first value head
                                 uint4* kdst = reinterpret_cast<uint4*>(a.kv_out + ((long long)key_head(u0.h) * a.arena_slots + slot) * (DK * 2)) + g;
-    #pragma unroll
+#pragma unroll
                                 for (int c = 0; c < NCH; ++c) kdst[c * LPU] = cur.own.k[c];
                             }
                         } else {
                             uint4* dst = reinterpret_cast<uint4*>(a.kv_out + (own_row0 + bb) * REC_BYTES) + g;
-    #pragma unroll
+#pragma unroll
                             for (int c = 0; c < NCH; ++c) {
                                 dst[c * LPU] = cur.own.k[c];
                                 dst[16 + c * LPU] = cur.own.v[c];
@@ -464,7 +464,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 if (k + 1 < n_quads) idx_next = load_idx(u1);
                 auto idx_of = [&](int level) -> int32_t {
                     int32_t t = 0;
-    #pragma unroll
+#pragma unroll
                     for (int j = 0; j < NIDX; ++j) {
                         const int32_t x = __shfl_sync(0xffffffffu, my_idx.v[j], level & (LPU - 1), LPU);
                         if (j == level / LPU) t = x;
@@ -474,9 +474,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 };
 
                 float2 r[4 * NCH], corr[4 * NCH];
-    #pragma unroll
+#pragma unroll
                 for (int c = 0; c < NCH; ++c) unpack8(cur.q[c], r + 4 * c);
-    #pragma unroll
+#pragma unroll
                 for (int e = 0; e < 4 * NCH; ++e) corr[e] = make_float2(0.f, 0.f);
                 float decay = 1.f;
                 // The scale of the unit's operand row, from the query's norm: a fold step never lengthens r~ (keys of
@@ -486,10 +486,10 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 float q_scale = 1.f, q_inv = 1.f;
                 {
                     float2 n2 = make_float2(0.f, 0.f);
-    #pragma unroll
+#pragma unroll
                     for (int e = 0; e < 4 * NCH; ++e) n2 = __ffma2_rn(r[e], r[e], n2);
                     float norm2 = n2.x + n2.y;
-    #pragma unroll
+#pragma unroll
                     for (int o = LPU / 2; o > 0; o >>= 1) norm2 += __shfl_xor_sync(0xffffffffu, norm2, o);
                     const int eb = (int)(__float_as_uint(norm2) >> 23) & 255;      // |q|^2 in [2^(eb-127), 2^(eb-126))
                     const int hq = (eb - 127 + 2) >> 1;                             // |q| < 2^hq
@@ -505,7 +505,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                                       RecT rec;
                                       const uint4* kp = reinterpret_cast<const uint4*>(k_at(u0.h, slot)) + g;
                                       const uint4* vp = reinterpret_cast<const uint4*>(v_at(u0.h, slot)) + g;
-    #pragma unroll
+#pragma unroll
                                       for (int c = 0; c < NCH; ++c) {
                                           rec.k[c] = __ldg(kp + c * LPU);
                                           rec.v[c] = __ldg(vp + c * LPU);
@@ -552,11 +552,11 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                     if (g == 0) inv_s[s * GN + u] = (q_inv * d_inv) * seg_inv_s0;
                     const float dcs = (decay * d_scale) * q_scale;
                     const float2 dc = make_float2(dcs, dcs);
-    #pragma unroll
+#pragma unroll
                     for (int c = 0; c < NCH; ++c) {
                         const int ci = c * LPU + g;                 // elements [8 ci, 8 ci + 8)
                         float2 x[4];
-    #pragma unroll
+#pragma unroll
                         for (int e = 0; e < 4; ++e) x[e] = __fmul2_rn(r[4 * c + e], dc);
                         // fp16 operand rows: K blocks of 64 elements (128 bytes, 128-byte swizzle), one 16-byte chunk
                         // per lane and c; a warp's four rows are 512 consecutive bytes: no bank conflicts
@@ -588,7 +588,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                         const int level = old - 1 - 2 * p - (g >> 2);
                         const int src = max(level, 0);
                         int32_t slot = 0;
-    #pragma unroll
+#pragma unroll
                         for (int j = 0; j < NIDX; ++j) {
                             const int32_t x = __shfl_sync(0xffffffffu, idx_next.v[j], src & (LPU - 1), LPU);
                             if (j == src / LPU) slot = x;
