@@ -687,23 +687,30 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         // (request, head, group within the pair) of the group at hand, advanced without divisions
         int pair = pair_begin, req = pair / a.H, h = pair - req * a.H, gip = g_begin - pair * groups_per_pair;
         int issued = 0;                               // groups whose MMAs have been issued (first epilogue warp)
-        for (int gcount = 0; gcount < g_end - g_begin && !dead; ++gcount) {
+        // A warp that gives up (`fail`) never leaves on its own: it skips its work, raises the abort flag and keeps
+        // arriving at the iteration's named barrier, whose OR makes all four warps leave in the same iteration.
+        bool fail = false;
+        auto give_up = [&]() {
+            fail = true;
+            if (lane == 0) *abort_flag = 1;
+        };
+        for (int gcount = 0; gcount < g_end - g_begin; ++gcount) {
             const int s = gcount % SLOTS, use = gcount / SLOTS;
             const int seg = pair - pair_begin;
             const bool seg_first = gcount == 0 || gip == 0;
             const bool has_next = gcount + 1 < g_end - g_begin;
             const bool next_first = gip + 1 == groups_per_pair;      // the next group opens a segment
-            if (warp == FOLD_WARPS && issued == gcount) {
-                if (issue_mma(gcount, seg, seg_first)) { dead = true; break; }
+            if (!fail && warp == FOLD_WARPS && issued == gcount) {
+                if (issue_mma(gcount, seg, seg_first)) give_up();
                 ++issued;
             }
-            if (!wait_or_abort(bar_done(s), use & 1, abort_flag)) { dead = true; break; }
+            if (!fail && !wait_or_abort(bar_done(s), use & 1, abort_flag)) give_up();
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             float* C_s = reinterpret_cast<float*>(ring + s * SLOT_BYTES + R_BYTES);
             const int b0 = gip * GN;
             const uint32_t taddr = tmem_base + s * GN + ((uint32_t)(quad * 32) << 16);
             float* A_s = reinterpret_cast<float*>(ring + s * SLOT_BYTES);   // the operand rows are dead once the MMAs have completed
-            {
+            if (!fail) {
                 // accumulator rows (dv) of this thread, all beams of the group, transposed into a tile laid out like
                 // the corr tile, over the slot's operand rows (plain stores: nothing here waits for a shared-memory read)
                 uint32_t v[GN];
@@ -714,7 +721,8 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
 #pragma unroll
                 for (int j = 0; j < GN; ++j) A_s[j * DV + ip] = __uint_as_float(v[j]);
             }
-            if (bar_or(1, 128, 0)) { dead = true; break; }     // the four epilogue warps: tile complete
+            // the four epilogue warps: tile complete - or somebody gave up, and then all four leave here together
+            if (bar_or(1, 128, fail ? 1 : 0)) { dead = true; break; }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             if (warp == FOLD_WARPS) {
                 // This warp's part of the slot is read out; the next group's MMAs go out now - unless that group
@@ -722,7 +730,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_free(s));
                 if (has_next && !(next_first && seg_first && seg >= 1)) {
-                    if (issue_mma(gcount + 1, seg + (next_first ? 1 : 0), next_first)) { dead = true; break; }
+                    if (issue_mma(gcount + 1, seg + (next_first ? 1 : 0), next_first)) give_up();   // carried to the next barrier
                     ++issued;
                 }
             } else {
@@ -750,11 +758,15 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             }
 
             // Past the first group of segment seg >= 1 every MMA of segment seg - 1 has completed and the fold warps
-            // have read its staging buffer out (they signal that): both are free for segment seg + 1.
-            if (seg_first && seg >= 1 && seg + 1 < n_segs) {
-                if (!wait_or_abort(bar_sfree((seg + 1) & 1), ((seg - 1) >> 1) & 1, abort_flag)) { dead = true; break; }
-                stage_segment(seg + 1);
-                prepare_s0(seg + 1);
+            // have read its staging buffer out (they signal that): both are free for segment seg + 1.  (More groups
+            // follow, so a warp that gives up here meets the others at the next iteration's barrier.)
+            if (seg_first && seg >= 1 && seg + 1 < n_segs && !fail) {
+                if (!wait_or_abort(bar_sfree((seg + 1) & 1), ((seg - 1) >> 1) & 1, abort_flag)) {
+                    give_up();
+                } else {
+                    stage_segment(seg + 1);
+                    prepare_s0(seg + 1);
+                }
             }
             if (++gip == groups_per_pair) {
                 gip = 0;
@@ -762,6 +774,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 if (++h == a.H) { h = 0; ++req; }
             }
         }
+        if (fail) dead = true;
         if (dead && lane == 0) *abort_flag = 1;
         // A CTA must not exit with bulk copies still landing in its shared memory: after an abort nobody may have
         // waited for the stagings requested last.
