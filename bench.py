@@ -141,7 +141,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
         wl = wl.scaled(L=args.layers)
     out_dtype = args.out_dtype or wl.dtype
     out_bytes = 4 if out_dtype == "fp32" else 2
-    run = WorkloadRun(wl, dev, out_dtype, flags=(2 if args.force_generic else 0) | (4 if args.delta_records else 0))
+    run = WorkloadRun(wl, dev, out_dtype, flags=(2 if args.force_generic else 0) | (4 if args.delta_records else 0) | (8 if args.shared_chains else 0))
     ctx = run.ctx
     run.prefill_states()
     S0 = {(r, l): ctx.onela_export_shared_state(r, l) for r in range(wl.R) for l in range(wl.L)}
@@ -473,6 +473,7 @@ def main():
     ap.add_argument("--delta-records", action="store_true",
                     help="(alpha, delta, k) records with forward projection replay (Section 3.2) instead of raw records "
                          "with the backward fold: the CUDA-core comparison kernel")
+    ap.add_argument("--shared-chains", action="store_true", help="run the shared-ancestor tensor-core kernel (ONELA_FLAG_SHARED_CHAINS)")
     ap.add_argument("--profile", action="store_true", help="eager generations only, for ncu")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (kernel experiments)")

@@ -89,6 +89,12 @@ typedef int32_t onela_status;
  * delta, so with bf16 records the result drifts from the exact recurrence by about one bf16 rounding per record
  * (the default raw-record format has no such term). */
 #define ONELA_FLAG_GTR_DELTA 4u
+/* Chains that share most of their older records (few distinct ancestors per request: at most 160 distinct older
+ * records, at most 64 of them older than the beams' parents, chains of at most 9 records): onela_decode_step and
+ * onela_append_decode_step apply every level but the newest on the tensor cores (dk = dv = 128, bf16 records, one
+ * key head per value head).  A call whose ancestry does not fit reports ONELA_E_UNSUPPORTED through the sticky
+ * device status word and leaves its outputs unwritten. */
+#define ONELA_FLAG_SHARED_CHAINS 8u
 
 typedef struct onela_config {
     int32_t num_requests; /* request slots */

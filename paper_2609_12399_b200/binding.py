@@ -18,7 +18,7 @@ LIB_PATH = _PKG / "libonela.so"
 OK, E_INVAL, E_CAPACITY, E_ORDER, E_CUDA, E_UNSUPPORTED, E_DEVICE_CHECK, E_TIMEOUT = 0, -1, -2, -3, -4, -5, -6, -7
 DTYPE_F32, DTYPE_BF16 = 0, 1
 MAX_BATCH = 64
-FLAG_DRY_RUN, FLAG_FORCE_GENERIC, FLAG_GTR_DELTA = 1, 2, 4
+FLAG_DRY_RUN, FLAG_FORCE_GENERIC, FLAG_GTR_DELTA, FLAG_SHARED_CHAINS = 1, 2, 4, 8
 
 _TORCH_DTYPE = {DTYPE_F32: torch.float32, DTYPE_BF16: torch.bfloat16}
 _DTYPE_CODE = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16, "fp32": DTYPE_F32, "bf16": DTYPE_BF16}

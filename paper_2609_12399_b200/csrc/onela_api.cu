@@ -53,6 +53,7 @@ Layout carve(const onela_config& c, char* base) {
     l.sidx = reinterpret_cast<int32_t*>(take((size_t)c.num_requests * c.max_steps * c.max_beam * sizeof(int32_t)));
     l.ulist = reinterpret_cast<int32_t*>(take((size_t)c.num_requests * c.max_steps * c.max_beam * sizeof(int32_t)));
     l.uoff = reinterpret_cast<int32_t*>(take((size_t)c.num_requests * (c.max_steps + 1) * sizeof(int32_t)));
+    l.urep = reinterpret_cast<int32_t*>(take((size_t)c.num_requests * c.max_steps * c.max_beam * sizeof(int32_t)));
     l.s0 = reinterpret_cast<float*>(take((size_t)c.num_requests * c.num_layers * Hv * c.dv * c.dk * sizeof(float)));
     l.gates = reinterpret_cast<float2*>(take((size_t)c.num_layers * Hv * (size_t)c.arena_slots * sizeof(float2)));
     if (Hv == (size_t)c.num_heads) {
@@ -367,7 +368,8 @@ onela_status onela_reorder_beams(onela_ctx* ctx, int32_t req_begin, int32_t req_
                              (long long)(depth_old & 1) * c.max_steps * c.max_beam;
         if (launch_dedupe(cur, ctx->table_req_stride(), ctx->lay.sidx + req_begin * ctx->sidx_req_stride(),
                           ctx->sidx_req_stride(), ctx->lay.ulist + req_begin * ctx->sidx_req_stride(),
-                          ctx->sidx_req_stride(), ctx->lay.uoff + req_begin * ctx->uoff_req_stride(),
+                          ctx->sidx_req_stride(), ctx->lay.urep + req_begin * ctx->sidx_req_stride(),
+                          ctx->lay.uoff + req_begin * ctx->uoff_req_stride(),
                           ctx->uoff_req_stride(), req_count, W_new, depth_old + 1, c.max_beam, s) != cudaSuccess)
             return ONELA_E_CUDA;
         ctx->launches++;
@@ -507,6 +509,7 @@ onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count,
     a.sidx = ctx->lay.sidx + req_begin * ctx->sidx_req_stride();
     a.ulist = ctx->lay.ulist + req_begin * ctx->sidx_req_stride();
     a.uoff = ctx->lay.uoff + req_begin * ctx->uoff_req_stride();
+    a.urep = ctx->lay.urep + req_begin * ctx->sidx_req_stride();
     a.sidx_req_stride = ctx->sidx_req_stride();
     a.ulist_req_stride = ctx->sidx_req_stride();
     a.uoff_req_stride = ctx->uoff_req_stride();
@@ -517,7 +520,10 @@ onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count,
     a.max_beam = c.max_beam;
     for (int i = 0; i < req_count; ++i) a.bases.base[i] = ctx->req[req_begin + i].step_base.back();
     bool supported = true;
+    const bool wy = ctx->tensor_core && (c.flags & ONELA_FLAG_SHARED_CHAINS) && !ctx->grouped() && depth >= 2 &&
+                    depth <= WY_MAX_LEVELS + 1;
     const cudaError_t e = ctx->gtr()         ? launch_decode_gtr(a, c.dk, c.dv, c.rec_dtype, c.out_dtype, &supported, s)
+                          : wy               ? launch_decode_wy(a, c.out_dtype, s)
                           : ctx->tensor_core ? launch_decode_sm100_ws(a, c.out_dtype, ctx->grouped(), s)
                                              : launch_decode_generic(a, c.dk, c.dv, c.rec_dtype, c.out_dtype, &supported, s);
     if (!supported) return ONELA_E_UNSUPPORTED;

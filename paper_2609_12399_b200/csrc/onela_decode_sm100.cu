@@ -110,10 +110,8 @@ struct Head {           // what a unit's fold needs first
 
 
 // Contiguous ranges of groups, one per CTA, balanced on the host with the cost of starting a segment counted in.
-constexpr int MAX_CTAS = 160;
-struct Partition {
-    int32_t begin[MAX_CTAS + 1];
-};
+constexpr int MAX_CTAS = DECODE_MAX_CTAS;
+using Partition = DecodePartition;
 
 // GROUPED: value head h reads the queries and keys of key head h / g; a.H counts VALUE heads, the record's k lives in
 // the key heads' plane (a.kv) and its v in the value heads' plane (a.vv), 256 bytes each.
@@ -907,6 +905,10 @@ cudaError_t launch_ws_t(const DecodeArgs& a, cudaStream_t stream) {
 
 }  // namespace
 
+int make_decode_partition(int total_groups, int groups_per_pair, int sms, int group_cost, int seg_cost, DecodePartition* part) {
+    return make_partition(total_groups, groups_per_pair, sms > MAX_CTAS ? MAX_CTAS : sms, PartitionCost{group_cost, seg_cost}, part);
+}
+int decode_sm_count() { return sm_count_ws(); }
 
 bool decode_sm100_supported(int32_t dk, int32_t dv, int32_t rec_dtype) {
     return dk == 128 && dv == 128 && rec_dtype == ONELA_DTYPE_BF16;

@@ -49,10 +49,11 @@ __global__ void __launch_bounds__(256) export_chains_kernel(const int32_t* __res
 // One CTA per request.  For every level older than the beams' own records: mark which slots of that
 // level some live chain refers to (slots of one level of one request are consecutive, so slot - min is a
 // dense key < max_beam), prefix-sum the marks, and emit the distinct slots in increasing order plus each
-// beam's position in the request's concatenated list.
+// beam's position in the request's concatenated list, and for every distinct slot one beam that refers to it.
 __global__ void __launch_bounds__(1024) dedupe_kernel(const int32_t* __restrict__ tables_cur_req0, long long table_req_stride,
                                                       int32_t* __restrict__ sidx_req0, long long sidx_req_stride,
                                                       int32_t* __restrict__ ulist_req0, long long ulist_req_stride,
+                                                      int32_t* __restrict__ urep_req0,
                                                       int32_t* __restrict__ uoff_req0, long long uoff_req_stride,
                                                       int32_t W, int32_t depth, int32_t max_beam) {
     extern __shared__ int32_t marks[];          // [max_beam] marks, then their exclusive prefix sums
@@ -62,6 +63,7 @@ __global__ void __launch_bounds__(1024) dedupe_kernel(const int32_t* __restrict_
     const int32_t* table = tables_cur_req0 + r * table_req_stride;
     int32_t* sidx = sidx_req0 + r * sidx_req_stride;
     int32_t* ulist = ulist_req0 + r * ulist_req_stride;
+    int32_t* urep = urep_req0 + r * ulist_req_stride;
     int32_t* uoff = uoff_req0 + r * uoff_req_stride;
     const int ipt = (max_beam + 1023) / 1024;   // marks per thread in the scan
     int32_t off = 0;
@@ -118,7 +120,11 @@ __global__ void __launch_bounds__(1024) dedupe_kernel(const int32_t* __restrict_
             }
         }
         __syncthreads();
-        for (int b = tid; b < W; b += 1024) sidx[(long long)level * max_beam + b] = off + marks[row[b] - mn];
+        for (int b = tid; b < W; b += 1024) {
+            const int32_t pos_b = off + marks[row[b] - mn];
+            sidx[(long long)level * max_beam + b] = pos_b;
+            urep[pos_b] = b;     // any of the beams that share the record will do: they share all its ancestors
+        }
         off += s_total;
         if (tid == 0) uoff[level + 1] = off;
         __syncthreads();
@@ -129,7 +135,7 @@ __global__ void __launch_bounds__(1024) dedupe_kernel(const int32_t* __restrict_
 
 cudaError_t launch_dedupe(const int32_t* tables_cur_req0, long long table_req_stride, int32_t* sidx_req0,
                           long long sidx_req_stride, int32_t* ulist_req0, long long ulist_req_stride,
-                          int32_t* uoff_req0, long long uoff_req_stride, int32_t req_count, int32_t W,
+                          int32_t* urep_req0, int32_t* uoff_req0, long long uoff_req_stride, int32_t req_count, int32_t W,
                           int32_t depth, int32_t max_beam, cudaStream_t stream) {
     const size_t smem = sizeof(int32_t) * (size_t)max_beam;
     if (smem > 48 * 1024) {
@@ -137,8 +143,8 @@ cudaError_t launch_dedupe(const int32_t* tables_cur_req0, long long table_req_st
         if (e != cudaSuccess) return e;
     }
     dedupe_kernel<<<req_count, 1024, smem, stream>>>(tables_cur_req0, table_req_stride, sidx_req0, sidx_req_stride,
-                                                     ulist_req0, ulist_req_stride, uoff_req0, uoff_req_stride, W, depth,
-                                                     max_beam);
+                                                     ulist_req0, ulist_req_stride, urep_req0, uoff_req0, uoff_req_stride, W,
+                                                     depth, max_beam);
     return cudaGetLastError();
 }
 

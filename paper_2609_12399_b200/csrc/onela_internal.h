@@ -16,6 +16,7 @@ struct Layout {
     int32_t* sidx;     // [request][max_steps][max_beam] per (level, beam): index into the request's distinct-record list
     int32_t* ulist;    // [request][max_steps*max_beam] distinct record slots of the live chains, oldest level first
     int32_t* uoff;     // [request][max_steps+1] start of each level inside ulist (uoff[level+1] = end)
+    int32_t* urep;     // [request][max_steps*max_beam] per distinct record: one live beam whose chain holds it
     float* s0;         // [request][layer][head][dv*dk] fp32
     float2* gates;     // [layer][head][arena_slots] (alpha, beta)
     char* kv;          // [layer][head][arena_slots][dk + dv] in rec_dtype: one row = k | v of one record
@@ -53,6 +54,7 @@ struct DecodeArgs {
     const int32_t* sidx;    // distinct-record index of req_begin (see Layout)
     const int32_t* ulist;
     const int32_t* uoff;
+    const int32_t* urep;
     long long sidx_req_stride, ulist_req_stride, uoff_req_stride;
     int32_t req_count, W, H, depth, max_beam;
     BatchBases bases;
@@ -95,9 +97,10 @@ cudaError_t launch_reorder(int32_t* tables_req0, long long table_req_stride, int
 // Distinct-record index of the CURRENT ancestry table (levels 0 .. depth-2; the newest level is the
 // beams' own records, all distinct): per level the sorted distinct slots and, per beam, where its
 // ancestor sits in the request's concatenated list.  Integer work only.
+// urep: per distinct record, one of the live beams whose chain holds it (all such beams share its older ancestors).
 cudaError_t launch_dedupe(const int32_t* tables_cur_req0, long long table_req_stride, int32_t* sidx_req0,
                           long long sidx_req_stride, int32_t* ulist_req0, long long ulist_req_stride,
-                          int32_t* uoff_req0, long long uoff_req_stride, int32_t req_count, int32_t W,
+                          int32_t* urep_req0, int32_t* uoff_req0, long long uoff_req_stride, int32_t req_count, int32_t W,
                           int32_t depth, int32_t max_beam, cudaStream_t stream);
 cudaError_t launch_export_chains(const int32_t* table_cur, int32_t W, int32_t depth, int32_t max_beam,
                                  int32_t* slots_out, cudaStream_t stream);
@@ -135,5 +138,22 @@ cudaError_t launch_decode_gtr(const DecodeArgs& a, int32_t dk, int32_t dv, int32
                               bool* supported, cudaStream_t stream);
 bool decode_sm100_supported(int32_t dk, int32_t dv, int32_t rec_dtype);
 cudaError_t launch_decode_sm100_ws(const DecodeArgs& a, int32_t out_dtype, bool grouped, cudaStream_t stream);
+
+// Contiguous ranges of beam groups, one per CTA of a persistent decode kernel (host-side partitioner in
+// onela_decode_sm100.cu): CTA c works on groups [begin[c], begin[c + 1]).
+constexpr int DECODE_MAX_CTAS = 160;
+struct DecodePartition {
+    int32_t begin[DECODE_MAX_CTAS + 1];
+};
+// group_cost / seg_cost: relative cost of one group and of starting a (request, head) segment.  Returns the CTA count.
+int make_decode_partition(int total_groups, int groups_per_pair, int sms, int group_cost, int seg_cost, DecodePartition* part);
+int decode_sm_count();
+
+// tcgen05 kernel for chains with heavily shared ancestors (dk = dv = 128, bf16 records, one key head per value head):
+// the older levels of all chains are applied in compact form on the tensor cores (see onela_decode_wy.cu).
+// Usable when every request of the call has at most WY_MAX_NODES distinct older records, at most WY_MAX_DEEP of them
+// older than the beams' parents, and 2 <= depth <= WY_MAX_LEVELS + 1; the kernel checks the first two on the device.
+constexpr int WY_MAX_NODES = 160, WY_MAX_DEEP = 64, WY_MAX_LEVELS = 8;
+cudaError_t launch_decode_wy(const DecodeArgs& a, int32_t out_dtype, cudaStream_t stream);
 
 }  // namespace onela

@@ -12,7 +12,6 @@ namespace sm100 {
 
 constexpr int DK = 128, DV = 128;
 constexpr int REC_BYTES = (DK + DV) * 2;       // 512: k | v in bf16
-constexpr int S0_BYTES = DV * DK * 4;          // 65536
 constexpr int WAIT_LIMIT = 1 << 20;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -96,6 +95,16 @@ __device__ __forceinline__ void umma_f16_ts(uint32_t tmem_d, uint32_t tmem_a, ui
         "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// tcgen05.mma, fp16 operands, A and B both from shared memory (K-major, 128-byte swizzle)
+__device__ __forceinline__ void umma_f16_ss(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 // two fp32 -> packed fp16 (element 0 in the low half), round to nearest even
 __device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
     const __half2 t = __floats2half2_rn(lo, hi);
@@ -108,6 +117,13 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* v) {
         :
         : "r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
         : "memory");
+}
+// Write 8 consecutive columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* v) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 :
+                 : "r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                 : "memory");
 }
 // The power of two that brings a positive magnitude m into [2^target, 2^(target + 1)), and its reciprocal; both 1 when
 // m is zero, subnormal, infinite, NaN or too small for the reciprocal to be a normal number.  Used to keep fp16
@@ -219,29 +235,10 @@ struct Lanes {
             fold_step(rec, r, corr, decay);
         }
     }
-    // Fold `first` (already in registers) and then levels hi .. lo (newest first) fetched by `load`, keeping
-    // one record in flight while the previous one is folded.  Two buffers alternate so no record is moved.
-    template <class LoadFn>
-    static __device__ __forceinline__ void fold_chain(const R& first, int hi, int lo, LoadFn load, float2* r,
-                                                      float2* corr, float& decay) {
-        R A = first, B;
-        int level = hi + 1;   // level of the record held in A
-        while (true) {
-            if (level - 1 >= lo) B = load(level - 1);
-            fold_step(A, r, corr, decay);
-            if (--level < lo) break;
-            if (level - 1 >= lo) A = load(level - 1);
-            fold_step(B, r, corr, decay);
-            if (--level < lo) break;
-        }
-    }
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async8(uint32_t dst, const void* src) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
 }
 
 
