@@ -53,7 +53,6 @@ Layout carve(const onela_config& c, char* base) {
     l.sidx = reinterpret_cast<int32_t*>(take((size_t)c.num_requests * c.max_steps * c.max_beam * sizeof(int32_t)));
     l.ulist = reinterpret_cast<int32_t*>(take((size_t)c.num_requests * c.max_steps * c.max_beam * sizeof(int32_t)));
     l.uoff = reinterpret_cast<int32_t*>(take((size_t)c.num_requests * (c.max_steps + 1) * sizeof(int32_t)));
-    l.urep = reinterpret_cast<int32_t*>(take((size_t)c.num_requests * c.max_steps * c.max_beam * sizeof(int32_t)));
     l.s0 = reinterpret_cast<float*>(take((size_t)c.num_requests * c.num_layers * Hv * c.dv * c.dk * sizeof(float)));
     l.gates = reinterpret_cast<float2*>(take((size_t)c.num_layers * Hv * (size_t)c.arena_slots * sizeof(float2)));
     if (Hv == (size_t)c.num_heads) {
@@ -65,6 +64,9 @@ Layout carve(const onela_config& c, char* base) {
     l.select_scratch = reinterpret_cast<unsigned long long*>(
         take((size_t)c.num_requests * ONELA_SELECT_PARTS * ONELA_SELECT_CAP * sizeof(unsigned long long)));
     l.s0_scale = reinterpret_cast<float*>(take((size_t)c.num_requests * c.num_layers * Hv * sizeof(float)));
+    l.urep = reinterpret_cast<int32_t*>(take((size_t)c.num_requests * c.max_steps * c.max_beam * sizeof(int32_t)));
+    l.sg8 = reinterpret_cast<uint8_t*>(take((size_t)c.num_requests * c.max_steps * sg_row_stride(c.max_beam)));
+    l.unode = reinterpret_cast<uint8_t*>(take((size_t)c.num_requests * ONELA_UNODE_CAP * 16));
     l.total_bytes = off;
     return l;
 }
@@ -77,6 +79,7 @@ struct onela_ctx {
     std::vector<ReqState> req;
     int64_t cursor = 0;        // next free arena slot
     int64_t launches = 0;
+    int64_t decode_mark = -1;  // value of `launches` right after the last decode launch
     bool status_cleared = false;
     bool tensor_core = false;  // decode_step runs the tcgen05 kernel
     int32_t elem_bytes = 4;
@@ -97,6 +100,7 @@ struct onela_ctx {
     }
     long long sidx_req_stride() const { return (long long)cfg.max_steps * cfg.max_beam; }
     long long uoff_req_stride() const { return cfg.max_steps + 1; }
+    long long sg8_req_stride() const { return (long long)cfg.max_steps * sg_row_stride(cfg.max_beam); }
     size_t plane_rows() const { return (size_t)cfg.num_heads * (size_t)cfg.arena_slots; }
     char* kv_plane(int l) const { return lay.kv + (size_t)l * plane_rows() * (cfg.dk + cfg.dv) * elem_bytes; }
     float2* gate_plane(int l) const { return lay.gates + (size_t)l * Hv() * (size_t)cfg.arena_slots; }
@@ -370,7 +374,9 @@ onela_status onela_reorder_beams(onela_ctx* ctx, int32_t req_begin, int32_t req_
                           ctx->sidx_req_stride(), ctx->lay.ulist + req_begin * ctx->sidx_req_stride(),
                           ctx->sidx_req_stride(), ctx->lay.urep + req_begin * ctx->sidx_req_stride(),
                           ctx->lay.uoff + req_begin * ctx->uoff_req_stride(),
-                          ctx->uoff_req_stride(), req_count, W_new, depth_old + 1, c.max_beam, s) != cudaSuccess)
+                          ctx->uoff_req_stride(), ctx->lay.sg8 + req_begin * ctx->sg8_req_stride(), ctx->sg8_req_stride(),
+                          sg_row_stride(c.max_beam), ctx->lay.unode + (size_t)req_begin * ONELA_UNODE_CAP * 16, req_count, W_new,
+                          depth_old + 1, c.max_beam, s) != cudaSuccess)
             return ONELA_E_CUDA;
         ctx->launches++;
     }
@@ -510,6 +516,10 @@ onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count,
     a.ulist = ctx->lay.ulist + req_begin * ctx->sidx_req_stride();
     a.uoff = ctx->lay.uoff + req_begin * ctx->uoff_req_stride();
     a.urep = ctx->lay.urep + req_begin * ctx->sidx_req_stride();
+    a.sg8 = ctx->lay.sg8 + req_begin * ctx->sg8_req_stride();
+    a.unode = ctx->lay.unode + (size_t)req_begin * ONELA_UNODE_CAP * 16;
+    a.sg8_req_stride = ctx->sg8_req_stride();
+    a.sg_stride = sg_row_stride(c.max_beam);
     a.sidx_req_stride = ctx->sidx_req_stride();
     a.ulist_req_stride = ctx->sidx_req_stride();
     a.uoff_req_stride = ctx->uoff_req_stride();
@@ -519,6 +529,7 @@ onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count,
     a.depth = depth;
     a.max_beam = c.max_beam;
     for (int i = 0; i < req_count; ++i) a.bases.base[i] = ctx->req[req_begin + i].step_base.back();
+    a.early_ok = ctx->launches == ctx->decode_mark ? 1 : 0;
     bool supported = true;
     const bool wy = ctx->tensor_core && (c.flags & ONELA_FLAG_SHARED_CHAINS) && !ctx->grouped() && depth >= 2 &&
                     depth <= WY_MAX_LEVELS + 1;
@@ -529,6 +540,7 @@ onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count,
     if (!supported) return ONELA_E_UNSUPPORTED;
     if (e != cudaSuccess) return ONELA_E_CUDA;
     ctx->launches++;
+    ctx->decode_mark = ctx->launches;
     return ONELA_OK;
 }
 

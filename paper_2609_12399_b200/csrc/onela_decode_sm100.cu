@@ -76,7 +76,7 @@ constexpr int GATE_BYTES = (2 * STAGE_BUF * 8 + 127) & ~127;   // padded: the he
 constexpr int INV_BYTES = SLOTS * GN * 4;        // per ring slot and beam: what undoes the operands' scales
 constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + STAGE_BYTES + GATE_BYTES + HEADS_TOTAL + 256 + INV_BYTES + 1024;
 constexpr uint32_t S0_COL = 128;                 // accumulators of the ring slots in [0, SLOTS * GN); S_0 buffers (64 columns) at 128 and 256
-constexpr int R_TARGET = 8;                      // a scaled operand row stays below 2^8 x (decay in [1, 2)): far inside fp16's range
+constexpr int R_TARGET = 8;                      // a scaled operand row's largest element lies in [2^8, 2^9) x (decay in [1, 2)): far inside fp16's range
 constexpr uint32_t TMEM_COLS = 512;
 static_assert(SLOTS * GN <= 128, "accumulator columns");
 static_assert(R_BYTES >= C_BYTES, "the accumulators are transposed over the operand rows");
@@ -477,10 +477,10 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
 #pragma unroll
                 for (int e = 0; e < 4 * NCH; ++e) corr[e] = make_float2(0.f, 0.f);
                 float decay = 1.f;
-                // The scale of the unit's operand row, from the query's norm: a fold step never lengthens r~ (keys of
-                // norm <= 1, beta in [0, 2]), so |r~| stays below 2^hq, the power of two above |q|; scaled to 2^R_TARGET
-                // it leaves a 2^(15 - R_TARGET)-fold margin to fp16's largest number and over twenty binades below it
-                // before elements turn subnormal.  Taken here, off the end-of-quad path (one shuffle reduction).
+                // A first guess at the scale of the unit's operand row, from the query's norm and off the end-of-quad
+                // path (one shuffle reduction): with keys of norm <= 1 and beta in [0, 2] a fold step never lengthens r~,
+                // so |r~| stays below 2^hq, the power of two above |q|, and the guess stands.  Whether it does is checked
+                // on the folded row itself (below).
                 float q_scale = 1.f, q_inv = 1.f;
                 {
                     float2 n2 = make_float2(0.f, 0.f);
@@ -542,9 +542,28 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                     // the corr tile (a layout of our own) swaps each pair of 16-byte chunks in every other 128-byte
                     // stretch of a row instead (corr_chunk; the epilogue reads it the same way).
                     const int sw = u & 7;
-                    // The folded query decay * r~ goes out as fp16 times two powers of two: the query's (taken when the
-                    // quad started: |r~| <= |q| < 2^R_TARGET / q_scale) and the one that brings the decay into [1, 2).  The
-                    // epilogue multiplies the accumulator by the reciprocals (and by that of the head's S_0 scale), exactly.
+                    // The folded query decay * r~ goes out as fp16 times two powers of two: the one that brings the decay into
+                    // [1, 2) and the row's own (the guess taken from |q| when the quad started: |r~| < 2^R_TARGET / q_scale).
+                    // The guess is checked against the folded row: OR-ing the magnitudes' bits bounds the largest one from
+                    // above, and if for any unit of the warp that bound reaches 2^(R_TARGET + 4) after scaling (keys longer
+                    // than 1 or beta outside [0, 2] lengthened r~), the warp takes the row's true largest element instead.
+                    // Either way the row stays far inside fp16's range.  The epilogue multiplies the accumulator by the
+                    // reciprocals (and by that of the head's S_0 scale), exactly.
+                    {
+                        uint32_t orb = 0;
+#pragma unroll
+                        for (int e = 0; e < 4 * NCH; ++e) orb |= __float_as_uint(r[e].x) | __float_as_uint(r[e].y);
+                        const bool suspect = !(__uint_as_float(orb & 0x7fffffffu) * q_scale < (float)(1 << (R_TARGET + 4)));
+                        if (__any_sync(0xffffffffu, suspect)) {
+                            uint32_t mx = 0;
+#pragma unroll
+                            for (int e = 0; e < 4 * NCH; ++e)
+                                mx = max(mx, max(__float_as_uint(r[e].x) & 0x7fffffffu, __float_as_uint(r[e].y) & 0x7fffffffu));
+#pragma unroll
+                            for (int o = LPU / 2; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                            pow2_scale(__uint_as_float(mx), R_TARGET, q_scale, q_inv);
+                        }
+                    }
                     float d_scale, d_inv;
                     pow2_scale(decay, 0, d_scale, d_inv);
                     if (g == 0) inv_s[s * GN + u] = (q_inv * d_inv) * seg_inv_s0;

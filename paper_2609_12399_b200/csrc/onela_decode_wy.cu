@@ -78,14 +78,15 @@ constexpr int HEADS_TOTAL = FOLD_WARPS * HEAD_BYTES;
 static_assert(VS_BYTES <= T_BYTES + W_BYTES, "the node values lie over the transposed tile and the first weight tile");
 static_assert(OFF_T % 1024 == 0 && OFF_W % 1024 == 0 && OFF_A % 1024 == 0 && W_BYTES % 1024 == 0 && R_BYTES % 1024 == 0 &&
               A_KB_STRIDE % 1024 == 0 && R_KB_STRIDE % 1024 == 0, "swizzle atoms");
-static_assert(128 * 128 + A_KB_STRIDE + 128 * 128 <= A_BYTES + HEADS_TOTAL, "second key tile's over-read stays inside shared memory");
+constexpr int HI_ROW0 = 64;                         // nodes 128.. are rows 64.. of the second key tile: tensor-memory lanes 64..95
+static_assert(HI_ROW0 * 128 + A_KB_STRIDE + 128 * 128 <= A_BYTES + HEADS_TOTAL, "second key tile's over-read stays inside shared memory");
 static_assert(128 * 128 <= W_BYTES, "the Gram bounce buffer fits the second weight tile");
 
 struct Misc {
     float2 gates[MAXN];            // (alpha, beta) of the nodes
     float ne[MAXN];                // e_kappa / (S_0 scale)
-    float ld[MAXN][MAXL];          // ld[kappa][l] = k_kappa . k_(ancestor of kappa at level l), l < level(kappa)
-    uint8_t anc[MAXN][MAXL];       // ancestor of kappa at level l
+    alignas(16) float ld[MAXN][MAXL];          // ld[kappa][l] = k_kappa . k_(ancestor of kappa at level l), l < level(kappa)
+    alignas(8) uint8_t anc[MAXN][MAXL];       // ancestor of kappa at level l
     uint8_t lvl[MAXN];
     alignas(16) uint8_t sg[MAXL][MAXW + 64];   // node of beam b's chain at level l (whole request; idle beams shadow the last)
     alignas(16) float gout[SLOTS][MAXL][GN];   // k_node . (operand row of beam u) for the chain nodes of the group's beams
@@ -93,7 +94,7 @@ struct Misc {
     float wt[VSLOTS][GN];                      // fold warps: beta_t c_t
     alignas(16) float cA[VSLOTS][GN];          // solver: coefficient of the S_0 accumulator
     alignas(16) float cB[VSLOTS][GN];          // solver: coefficient of the U accumulator
-    uint32_t umax[8];
+    uint32_t umax[24];
     alignas(8) uint64_t bars[24];
     uint32_t tmem_slot;
     int abort_flag;
@@ -120,9 +121,10 @@ constexpr uint32_t GRAM_HI_COL = 224;               // set-up only: K[128..] K_d
 constexpr uint32_t TMEM_COLS = 512;
 static_assert(VSLOTS * GN <= GLO_COL && ACC2_COL + SLOTS * GN <= S0_COL && U_COL + MAXN / 2 <= 512, "tensor-memory map");
 static_assert(PACC_COL + MAXN <= GRAM_LO_COL && GRAM_LO_COL + MAXD <= GRAM_HI_COL && GRAM_HI_COL + MAXD <= S0_COL, "set-up accumulators");
+static_assert(MAXL == 8, "the solve is written out for eight levels");
 constexpr int R_TARGET = 8;                         // a scaled operand row's largest element lies in [2^8, 2^9)
 constexpr int W_TARGET = 7;
-constexpr int U_TARGET = 11;
+constexpr int U_TARGET = 12;                        // the bound on |u| times the scale lies in [2^12, 2^13)
 
 #ifdef ONELA_WY_TL
 // Debug builds only: clock stamps of CTA 0's role milestones, kept in shared memory and written out when the CTA
@@ -144,6 +146,9 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
     for (int i = 0; i < WAIT_LIMIT; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 63) == 63 && *abort_flag) return false;
+#ifdef ONELA_WY_NAP
+        __nanosleep(ONELA_WY_NAP);
+#endif
     }
     return false;
 }
@@ -426,7 +431,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_wy_kernel(const __grid_cons
         }
     } else {
         // =============================== BACK SIDE: epilogue team and solver team ===============================
-        dependency_wait();
+        // What the set-up reads (index arrays, S_0, records of earlier decode calls) was written at least two launches
+        // ago when the host says so; the epilogue team still waits for the predecessor before its first store.
+        if (!a.early_ok) dependency_wait();
         const bool epi = warp < SOL_WARP0;
         const int quad = warp & 3;                    // tensor-memory lane quadrant of this warp
         const int row_i = quad * 32 + lane;           // tensor-memory lane of this thread
@@ -472,53 +479,49 @@ __global__ void __launch_bounds__(THREADS, 1) decode_wy_kernel(const __grid_cons
             // ---------------- set-up of the segment ----------------
             // Keys and values of the distinct nodes: 16-byte async copies, neighbouring threads neighbouring chunks, every
             // copy of a thread in flight at once; a key chunk lands at its place in the operand tile as bf16 and is turned
-            // into fp16 there by the thread that copied it (same size, same place).
+            // into fp16 there by the thread that copied it (same size, same place).  A node's gates, level and ancestors
+            // come from the byte-sized tables the index kernel left, every beam's chain nodes by 16-byte copies too.
             constexpr int CH_PER_THREAD = MAXN * 16 / 256;
             {
+                const bool mine = tb < n;
+                const int kappa = tb;
                 int32_t nslot[CH_PER_THREAD];
 #pragma unroll
                 for (int it = 0; it < CH_PER_THREAD; ++it) {
                     const int ch = tb + 256 * it;
                     nslot[it] = ch < n * 16 ? __ldg(ulist + (ch >> 4)) : 0;
                 }
+                const int32_t slot = mine ? __ldg(ulist + kappa) : 0;
+                uint4 ninfo = make_uint4(0u, 0u, 0u, 0u);
+                if (mine) ninfo = __ldg(reinterpret_cast<const uint4*>(a.unode + (long long)req * (ONELA_UNODE_CAP * 16)) + kappa);
+                if (seg == 0 || (pair - 1) / a.H != req) {       // (the same for all heads of the request)
+                    const int cpr = (groups_per_pair * GN + 15) >> 4;     // 16-byte chunks per level
+                    const uint8_t* src = a.sg8 + req * a.sg8_req_stride;
+                    for (int idx = tb; idx < m * cpr; idx += 256) {
+                        const int l = idx / cpr, c = idx - l * cpr;
+                        cp_async16(smem_u32(&mi.sg[l][c * 16]), src + (long long)l * a.sg_stride + c * 16);
+                    }
+                }
 #pragma unroll
                 for (int it = 0; it < CH_PER_THREAD; ++it) {
-                    const int ch = tb + 256 * it, kappa = ch >> 4, c = ch & 15;
+                    const int ch = tb + 256 * it, kp = ch >> 4, c = ch & 15;
                     if (ch < n * 16) {
                         const char* src = kv + (plane_row0 + nslot[it]) * REC_BYTES + c * 16;
-                        cp_async16(smem_u32(A_s + (c >> 3) * A_KB_STRIDE + (kappa >> 3) * 1024 + (kappa & 7) * 128 + (((c & 7) ^ (kappa & 7)) << 4)), src);
-                        cp_async16(smem_u32(VS_s + kappa * (DV * 2) + c * 16), src + DK * 2);
+                        cp_async16(smem_u32(A_s + (c >> 3) * A_KB_STRIDE + (kp >> 3) * 1024 + (kp & 7) * 128 + (((c & 7) ^ (kp & 7)) << 4)), src);
+                        cp_async16(smem_u32(VS_s + kp * (DV * 2) + c * 16), src + DK * 2);
                     }
                 }
                 asm volatile("cp.async.commit_group;" ::: "memory");
-            }
-            for (int i = tb; i < MAXN * MAXL; i += 256) (&mi.ld[0][0])[i] = 0.f;
-            if (tb < n) {
-                const int kappa = tb;
-                const int32_t slot = __ldg(ulist + kappa), rp = __ldg(urep + kappa);
-                int lv = 0;
-                for (int l = 1; l < m; ++l) lv += (kappa >= __ldg(uoff + l)) ? 1 : 0;
-                int32_t an[MAXL];
-#pragma unroll
-                for (int l = 0; l < MAXL; ++l) an[l] = l < lv ? __ldg(sidx + (long long)l * a.max_beam + rp) : 0;
-                mi.gates[kappa] = __ldg(a.gates + plane_row0 + slot);
-                mi.lvl[kappa] = (uint8_t)lv;
-#pragma unroll
-                for (int l = 0; l < MAXL; ++l) mi.anc[kappa][l] = (uint8_t)an[l];
-            }
-            // every beam's chain nodes (the same for all heads of the request: rebuilt only when the request changes)
-            if (seg == 0 || (pair - 1) / a.H != req) {
-                const int wpad = (groups_per_pair * GN + 3) & ~3;     // idle beams of the last group shadow the last live beam
-#pragma unroll 2
-                for (int idx = tb; idx < m * (wpad >> 2); idx += 256) {
-                    const int l = idx / (wpad >> 2), b4 = (idx - l * (wpad >> 2)) * 4;
-                    const int32_t* row = sidx + (long long)l * a.max_beam;
-                    uint32_t w = 0;
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) w |= ((uint32_t)__ldg(row + min(b4 + j, a.W - 1)) & 0xffu) << (8 * j);
-                    *reinterpret_cast<uint32_t*>(&mi.sg[l][b4]) = w;
+                TL(15, seg);
+                if (mine) {
+                    mi.gates[kappa] = __ldg(a.gates + plane_row0 + slot);
+                    mi.lvl[kappa] = (uint8_t)(ninfo.z & 0xffu);
+                    *reinterpret_cast<uint2*>(&mi.anc[kappa][0]) = make_uint2(ninfo.x, ninfo.y);
                 }
             }
+            for (int i = tb; i < MAXN * MAXL; i += 256) (&mi.ld[0][0])[i] = 0.f;
+            TL(16, seg);
+            TL(17, seg);
             if (seg >= 1) {     // S_0 of a later segment: every MMA of the previous one has completed (end of the loop)
                 const float* row = a.s0 + req * a.s0_req_stride + (long long)h * (DV * DK) + (long long)row_i * DK;
 #pragma unroll 1
@@ -536,12 +539,14 @@ __global__ void __launch_bounds__(THREADS, 1) decode_wy_kernel(const __grid_cons
             } else if (epi) {
                 put_first_s0();
             }
+            TL(18, seg);
             asm volatile("cp.async.wait_all;" ::: "memory");
+            TL(19, seg);
 #pragma unroll
             for (int it = 0; it < CH_PER_THREAD; ++it) {
-                const int ch = tb + 256 * it, kappa = ch >> 4, c = ch & 15;
+                const int ch = tb + 256 * it, kp = ch >> 4, c = ch & 15;
                 if (ch < n * 16) {
-                    uint4* pk = reinterpret_cast<uint4*>(A_s + (c >> 3) * A_KB_STRIDE + (kappa >> 3) * 1024 + (kappa & 7) * 128 + (((c & 7) ^ (kappa & 7)) << 4));
+                    uint4* pk = reinterpret_cast<uint4*>(A_s + (c >> 3) * A_KB_STRIDE + (kp >> 3) * 1024 + (kp & 7) * 128 + (((c & 7) ^ (kp & 7)) << 4));
                     const uint4 x = *pk;
                     *pk = make_uint4(bf16x2_to_f16x2(x.x), bf16x2_to_f16x2(x.y), bf16x2_to_f16x2(x.z), bf16x2_to_f16x2(x.w));
                 }
@@ -574,7 +579,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_wy_kernel(const __grid_cons
                                 const uint64_t bd = umma_desc(abase + kb * A_KB_STRIDE + ks * 32);
                                 umma_f16_ss(tmem_base + GRAM_LO_COL, bd, bd, idesc_d, (kb | ks) ? 1u : 0u);
                                 if (n > 128)
-                                    umma_f16_ss(tmem_base + GRAM_HI_COL, umma_desc(abase + 128 * 128 + kb * A_KB_STRIDE + ks * 32), bd,
+                                    umma_f16_ss(tmem_base + GRAM_HI_COL, umma_desc(abase + HI_ROW0 * 128 + kb * A_KB_STRIDE + ks * 32), bd,
                                                 idesc_d, (kb | ks) ? 1u : 0u);
                             }
                     }
@@ -594,43 +599,63 @@ __global__ void __launch_bounds__(THREADS, 1) decode_wy_kernel(const __grid_cons
             TL(12, seg);   // set-up MMAs complete
 
             // U = [v_kappa - e_kappa S_0 k_kappa] into tensor memory as fp16 times one power of two: lane = output row,
-            // the two teams take alternate blocks of 16 nodes; first the largest magnitude, then the scaled values
+            // the two teams take alternate blocks of 16 nodes.  The power of two comes from a bound on |u|, the largest
+            // |v| plus the largest |e / scale| times the largest |S_0 k| (one cheap look at each), so U is written in
+            // one pass.
             float u_scale = 1.f, u_inv = 1.f;
             {
-                auto u_block = [&](int c0, float* uval) {
-                    uint32_t p[16];
-                    tmem_ld16(tmem_base + PACC_COL + c0 + lane_bits, p);
+                uint32_t vm = 0, pm = 0, nm = 0;
+                for (int ch = tb; ch < n * 16; ch += 256) {
+                    const uint4 w = *reinterpret_cast<const uint4*>(VS_s + ch * 16);
+                    vm = __vmaxu2(vm, __vmaxu2(__vmaxu2(w.x & 0x7fff7fffu, w.y & 0x7fff7fffu), __vmaxu2(w.z & 0x7fff7fffu, w.w & 0x7fff7fffu)));
+                }
+                vm = max(vm & 0xffffu, vm >> 16) << 16;              // the largest bf16 magnitude, as fp32 bits
+                TL(50, seg);
+                for (int c0 = (bw >> 2) * 16; c0 < n16; c0 += 32) {
+                    uint32_t pv[16];
+                    tmem_ld16(tmem_base + PACC_COL + c0 + lane_bits, pv);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const int kappa = c0 + j;
-                        float uv = 0.f;
-                        if (kappa < n) {
-                            const float v = __uint_as_float((uint32_t)(*reinterpret_cast<const uint16_t*>(VS_s + kappa * (DV * 2) + row_i * 2)) << 16);
-                            uv = fmaf(-mi.ne[kappa], __uint_as_float(p[j]), v);
-                        }
-                        uval[j] = uv;
-                    }
-                };
-                uint32_t mx = 0;
-                for (int c0 = (bw >> 2) * 16; c0 < n16; c0 += 32) {
-                    float uval[16];
-                    u_block(c0, uval);
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) mx = max(mx, __float_as_uint(uval[j]) & 0x7fffffffu);
+                    for (int j = 0; j < 16; ++j)
+                        if (c0 + j < n) pm = max(pm, pv[j] & 0x7fffffffu);
                 }
-                mx = __reduce_max_sync(0xffffffffu, mx);
-                if (lane == 0) mi.umax[bw] = mx;
+                TL(51, seg);
+                if (tb < n) nm = __float_as_uint(mi.ne[tb]) & 0x7fffffffu;
+                vm = __reduce_max_sync(0xffffffffu, vm);
+                pm = __reduce_max_sync(0xffffffffu, pm);
+                nm = __reduce_max_sync(0xffffffffu, nm);
+                if (lane == 0) {
+                    mi.umax[bw] = vm;
+                    mi.umax[8 + bw] = pm;
+                    mi.umax[16 + bw] = nm;
+                }
                 if (!team_sync()) { give_up(); break; }
 #pragma unroll
-                for (int i = 0; i < 8; ++i) mx = max(mx, mi.umax[i]);
-                pow2_scale(__uint_as_float(mx), U_TARGET, u_scale, u_inv);
+                for (int i = 0; i < 8; ++i) {
+                    vm = max(vm, mi.umax[i]);
+                    pm = max(pm, mi.umax[8 + i]);
+                    nm = max(nm, mi.umax[16 + i]);
+                }
+                TL(52, seg);
+                pow2_scale(fmaf(__uint_as_float(nm), __uint_as_float(pm), __uint_as_float(vm)), U_TARGET, u_scale, u_inv);
                 for (int c0 = (bw >> 2) * 16; c0 < n16; c0 += 32) {
-                    float uval[16];
-                    u_block(c0, uval);
+                    uint32_t pv[16];
+                    tmem_ld16(tmem_base + PACC_COL + c0 + lane_bits, pv);
+                    // the nodes' factors and this row's value elements while the accumulator block is on its way
+                    float vv[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int kappa = min(c0 + j, n - 1);
+                        vv[j] = __uint_as_float((uint32_t)(*reinterpret_cast<const uint16_t*>(VS_s + kappa * (DV * 2) + row_i * 2)) << 16);
+                    }
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                     uint32_t w8[8];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) w8[j] = pack_f16x2(uval[2 * j] * u_scale, uval[2 * j + 1] * u_scale);
+                    for (int j = 0; j < 16; j += 2) {
+                        const float u0 = c0 + j < n ? fmaf(-mi.ne[min(c0 + j, n - 1)], __uint_as_float(pv[j]), vv[j]) * u_scale : 0.f;
+                        const float u1 = c0 + j + 1 < n ? fmaf(-mi.ne[min(c0 + j + 1, n - 1)], __uint_as_float(pv[j + 1]), vv[j + 1]) * u_scale : 0.f;
+                        w8[j >> 1] = pack_f16x2(u0, u1);
+                    }
                     tmem_st8(tmem_base + U_COL + (c0 >> 1) + lane_bits, w8);
                 }
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
@@ -639,9 +664,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_wy_kernel(const __grid_cons
             // The chain dot products: a node's row of the Gram block goes through shared memory (as fp16, over the
             // second weight tile, idle now) so that the thread can pick its ancestors' columns.
             if (!epi && nd > 0) {
-                for (int part_hi = 0; part_hi < ((n > 128 && quad == 0) ? 2 : 1); ++part_hi) {
+                for (int part_hi = 0; part_hi < ((n > 128 && quad == 2) ? 2 : 1); ++part_hi) {
                     const int kappa = part_hi ? 128 + lane : row_i;
-                    uint8_t* bounce = slot_W(1) + row_i * 128;     // the thread's own 128 bytes (used twice by the first warp)
+                    uint8_t* bounce = slot_W(1) + row_i * 128;     // the thread's own 128 bytes (used twice by the third warp)
                     const uint32_t col = part_hi ? GRAM_HI_COL : GRAM_LO_COL;
                     for (int c0 = 0; c0 < nd16; c0 += 16) {
                         uint32_t p[16];
@@ -671,6 +696,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_wy_kernel(const __grid_cons
             if (epi) {
                 const int te = tid - EPI_WARP0 * 32;          // 0 .. 127
                 float* T_s = reinterpret_cast<float*>(T_raw);
+                dependency_wait();
                 for (int gi = seg_g0; gi < seg_g1; ++gi, ++gcount) {
                     const int s = gcount % SLOTS, vs = gcount % VSLOTS;
                     const int b0 = (gi - pair * groups_per_pair) * GN;
@@ -728,7 +754,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_wy_kernel(const __grid_cons
                 const int ts = tid - SOL_WARP0 * 32;          // 0 .. 127
                 const int my_lvl = row_i < n ? mi.lvl[row_i] : -1;
                 const int hi_kappa = 128 + lane;
-                const int hi_lvl = (quad == 0 && hi_kappa < n) ? mi.lvl[hi_kappa] : -1;
+                const int hi_lvl = (quad == 2 && hi_kappa < n) ? mi.lvl[hi_kappa] : -1;
                 // [S_0 ; K] . R^T of group gc, by the first lane of the last solver warp (which has no beam to solve for);
                 // true: gave up.  K . R^T has one buffer: the caller has seen the previous group's read out.
                 auto issue_mma1 = [&](int gc) -> bool {
@@ -749,7 +775,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_wy_kernel(const __grid_cons
                                     const uint32_t acc = (kb | ks) ? 1u : 0u;
                                     umma_f16_ss(tmem_base + GLO_COL, umma_desc(abase + kb * A_KB_STRIDE + ks * 32), bd, idesc_g, acc);
                                     if (n > 128)
-                                        umma_f16_ss(tmem_base + GHI_COL, umma_desc(abase + 128 * 128 + kb * A_KB_STRIDE + ks * 32), bd, idesc_g, acc);
+                                        umma_f16_ss(tmem_base + GHI_COL, umma_desc(abase + HI_ROW0 * 128 + kb * A_KB_STRIDE + ks * 32), bd, idesc_g, acc);
                                     umma_f16_ts(tmem_base + ACC1_COL + vs * GN, tmem_base + S0_COL + (kb * 4 + ks) * 8, bd, idesc_g, acc);
                                 }
                         } else {
@@ -791,7 +817,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_wy_kernel(const __grid_cons
                                     if (eq & (0xffu << (8 * j))) mi.gout[s][my_lvl][q4 * 4 + j] = __uint_as_float(x[q4 * 4 + j]);
                             }
                         }
-                        if (n > 128 && quad == 0) {
+                        if (n > 128 && quad == 2) {
 #pragma unroll
                             for (int c0 = 0; c0 < GN; c0 += 16) tmem_ld16(tmem_base + GHI_COL + c0 + lane_bits, x + c0);
                             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -821,49 +847,62 @@ __global__ void __launch_bounds__(THREADS, 1) decode_wy_kernel(const __grid_cons
                         // one beam per thread: the triangular solve along its chain, newest of the older levels first
                         const int u = ts;
                         const float f = mi.fA[vs][u];
-                        // Every load first (levels beyond the chain read the parent's entries and count for nothing: their
-                        // beta is taken as 0), then the arithmetic: no branches, all levels unrolled.
+                        // Levels beyond the chain read the parent's entries and count for nothing (their beta is taken as 0).
+                        // A solved level is taken out of all older levels' right-hand sides at once: its row of chain dot
+                        // products is contiguous (two 16-byte loads).
                         int kap[MAXL];
-                        float2 gt[MAXL];
-                        float gg[MAXL], bcv[MAXL], w[MAXL], ldv[MAXL][MAXL];
 #pragma unroll
                         for (int l = 0; l < MAXL; ++l) kap[l] = mi.sg[min(l, m - 1)][b0 + u];
+                        float2 gt[MAXL];
+                        float gg[MAXL], w[MAXL];
 #pragma unroll
                         for (int l = 0; l < MAXL; ++l) {
                             const float2 gl = mi.gates[kap[l]];
                             const float go = mi.gout[s][min(l, m - 1)][u];
                             gt[l] = l < m ? gl : make_float2(1.f, 0.f);
                             gg[l] = l < m ? go : 0.f;
-#pragma unroll
-                            for (int l2 = l + 1; l2 < MAXL; ++l2) ldv[l2][l] = mi.ld[kap[l2]][l];
                         }
+                        TL(35, gcount);
                         float d = 1.f, wmax = 0.f;
 #pragma unroll
                         for (int l = MAXL - 1; l >= 0; --l) {
-                            float c = gg[l];
-#pragma unroll
-                            for (int l2 = l + 1; l2 < MAXL; ++l2) c = fmaf(-bcv[l2], ldv[l2][l], c);
-                            bcv[l] = gt[l].y * c;
-                            w[l] = bcv[l] * d * f;
+                            const float bc = gt[l].y * gg[l];
+                            w[l] = bc * d * f;
                             wmax = fmaxf(wmax, fabsf(w[l]));
                             d *= gt[l].x;
+                            if (l > 0) {
+                                const float4 r0 = *reinterpret_cast<const float4*>(&mi.ld[kap[l]][0]);
+                                gg[0] = fmaf(-bc, r0.x, gg[0]);
+                                if (l > 1) gg[1] = fmaf(-bc, r0.y, gg[1]);
+                                if (l > 2) gg[2] = fmaf(-bc, r0.z, gg[2]);
+                                if (l > 3) gg[3] = fmaf(-bc, r0.w, gg[3]);
+                                if (l > 4) {
+                                    const float4 r1 = *reinterpret_cast<const float4*>(&mi.ld[kap[l]][4]);
+                                    gg[4] = fmaf(-bc, r1.x, gg[4]);
+                                    if (l > 5) gg[5] = fmaf(-bc, r1.y, gg[5]);
+                                    if (l > 6) gg[6] = fmaf(-bc, r1.z, gg[6]);
+                                }
+                            }
                         }
+                        TL(36, gcount);
                         float w_scale, w_inv;
                         pow2_scale(wmax, W_TARGET, w_scale, w_inv);
                         mi.cA[vs][u] = d * f * inv_s0;
                         mi.cB[vs][u] = w_inv * u_inv;
                         uint8_t* wrow = slot_W(s) + (u >> 3) * 1024 + (u & 7) * 128;
-                        // newest level last: the levels beyond the chain (weight 0) share the parent's place
 #pragma unroll
-                        for (int l = MAXL - 1; l >= 0; --l) {
-                            const int kp = kap[l];
-                            *reinterpret_cast<__half*>(wrow + (kp >> 6) * W_KB_STRIDE + ((((kp & 63) >> 3) ^ (u & 7)) << 4) + (kp & 7) * 2) =
-                                __float2half_rn(w[l] * w_scale);
-                        }
+                        for (int l = 0; l < MAXL; ++l)
+                            if (l < m) {
+                                const int kp = kap[l];
+                                *reinterpret_cast<__half*>(wrow + (kp >> 6) * W_KB_STRIDE + ((((kp & 63) >> 3) ^ (u & 7)) << 4) + (kp & 7) * 2) =
+                                    __float2half_rn(w[l] * w_scale);
+                            }
                     }
+                    TL(37, gcount);
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     TL(33, gcount);   // solver: solved
                     named_bar(3, 64);       // the two solving warps
+                    TL(38, gcount);
                     if (ts == 0) {
                         // the accumulator is free once the epilogue of group gcount - 2 has read it
                         bool ok = true;

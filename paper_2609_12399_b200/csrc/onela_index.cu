@@ -55,6 +55,8 @@ __global__ void __launch_bounds__(1024) dedupe_kernel(const int32_t* __restrict_
                                                       int32_t* __restrict__ ulist_req0, long long ulist_req_stride,
                                                       int32_t* __restrict__ urep_req0,
                                                       int32_t* __restrict__ uoff_req0, long long uoff_req_stride,
+                                                      uint8_t* __restrict__ sg8_req0, long long sg8_req_stride, int32_t sg_stride,
+                                                      uint8_t* __restrict__ unode_req0,
                                                       int32_t W, int32_t depth, int32_t max_beam) {
     extern __shared__ int32_t marks[];          // [max_beam] marks, then their exclusive prefix sums
     __shared__ int32_t warp_part[32];
@@ -129,13 +131,33 @@ __global__ void __launch_bounds__(1024) dedupe_kernel(const int32_t* __restrict_
         if (tid == 0) uoff[level + 1] = off;
         __syncthreads();
     }
+    // Compact copies for the shared-chains decode kernel (meaningful while the request has at most 255 distinct
+    // records; the kernel checks the count): every beam's list position per level as one byte, rows padded with the
+    // last live beam's; and per distinct record its level and its ancestors' list positions (through one of the
+    // beams that hold it).
+    uint8_t* sg8 = sg8_req0 + r * sg8_req_stride;
+    for (int i = tid; i < (depth - 1) * sg_stride; i += 1024) {
+        const int level = i / sg_stride, b = i - level * sg_stride;
+        sg8[i] = (uint8_t)sidx[(long long)level * max_beam + min(b, W - 1)];
+    }
+    uint8_t* unode = unode_req0 + (long long)r * (ONELA_UNODE_CAP * 16);
+    for (int j = tid; j < min(off, ONELA_UNODE_CAP); j += 1024) {
+        int lv = 0;
+        for (int l = 1; l < depth - 1; ++l) lv += (j >= uoff[l]) ? 1 : 0;
+        const int rp = urep[j];
+        uint32_t w[4] = {0u, 0u, (uint32_t)lv, 0u};
+        for (int l = 0; l < min(lv, 8); ++l)
+            w[l >> 2] |= ((uint32_t)sidx[(long long)l * max_beam + rp] & 0xffu) << (8 * (l & 3));
+        reinterpret_cast<uint4*>(unode)[j] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
 }
 
 }  // namespace
 
 cudaError_t launch_dedupe(const int32_t* tables_cur_req0, long long table_req_stride, int32_t* sidx_req0,
                           long long sidx_req_stride, int32_t* ulist_req0, long long ulist_req_stride,
-                          int32_t* urep_req0, int32_t* uoff_req0, long long uoff_req_stride, int32_t req_count, int32_t W,
+                          int32_t* urep_req0, int32_t* uoff_req0, long long uoff_req_stride, uint8_t* sg8_req0,
+                          long long sg8_req_stride, int32_t sg_stride, uint8_t* unode_req0, int32_t req_count, int32_t W,
                           int32_t depth, int32_t max_beam, cudaStream_t stream) {
     const size_t smem = sizeof(int32_t) * (size_t)max_beam;
     if (smem > 48 * 1024) {
@@ -143,8 +165,8 @@ cudaError_t launch_dedupe(const int32_t* tables_cur_req0, long long table_req_st
         if (e != cudaSuccess) return e;
     }
     dedupe_kernel<<<req_count, 1024, smem, stream>>>(tables_cur_req0, table_req_stride, sidx_req0, sidx_req_stride,
-                                                     ulist_req0, ulist_req_stride, urep_req0, uoff_req0, uoff_req_stride, W,
-                                                     depth, max_beam);
+                                                     ulist_req0, ulist_req_stride, urep_req0, uoff_req0, uoff_req_stride, sg8_req0,
+                                                     sg8_req_stride, sg_stride, unode_req0, W, depth, max_beam);
     return cudaGetLastError();
 }
 

@@ -17,6 +17,8 @@ struct Layout {
     int32_t* ulist;    // [request][max_steps*max_beam] distinct record slots of the live chains, oldest level first
     int32_t* uoff;     // [request][max_steps+1] start of each level inside ulist (uoff[level+1] = end)
     int32_t* urep;     // [request][max_steps*max_beam] per distinct record: one live beam whose chain holds it
+    uint8_t* sg8;      // [request][max_steps][sg_stride] sidx as bytes, rows padded with the last live beam's entry
+    uint8_t* unode;    // [request][ONELA_UNODE_CAP][16] per distinct record: ancestors' list positions (bytes 0-7), level (byte 8)
     float* s0;         // [request][layer][head][dv*dk] fp32
     float2* gates;     // [layer][head][arena_slots] (alpha, beta)
     char* kv;          // [layer][head][arena_slots][dk + dv] in rec_dtype: one row = k | v of one record
@@ -55,6 +57,10 @@ struct DecodeArgs {
     const int32_t* ulist;
     const int32_t* uoff;
     const int32_t* urep;
+    const uint8_t* sg8;     // byte copies of sidx and the per-record table (see Layout), of req_begin
+    const uint8_t* unode;
+    long long sg8_req_stride;
+    int32_t sg_stride;
     long long sidx_req_stride, ulist_req_stride, uoff_req_stride;
     int32_t req_count, W, H, depth, max_beam;
     BatchBases bases;
@@ -66,6 +72,10 @@ struct DecodeArgs {
     // tensor-core kernel: per-head operand scale of S_0 (see Layout), entry of (req_begin, layer, head 0)
     const float* s0_scale;
     long long s0_scale_req_stride;
+    // 1 when the launch that precedes this one on the context was a decode launch as well (of another layer or of
+    // this one): nothing that launch wrote is read here except the caller's tensors, so a programmatic dependent
+    // launch may read the index arrays, S_0 and the older records before it waits for its predecessor
+    int32_t early_ok;
 };
 
 // Grouped value heads (Hv = g * Hk): what the grouped decode kernel needs.
@@ -98,9 +108,13 @@ cudaError_t launch_reorder(int32_t* tables_req0, long long table_req_stride, int
 // beams' own records, all distinct): per level the sorted distinct slots and, per beam, where its
 // ancestor sits in the request's concatenated list.  Integer work only.
 // urep: per distinct record, one of the live beams whose chain holds it (all such beams share its older ancestors).
+// sg8 / unode: byte-sized copies for the shared-chains kernel (see Layout).
+#define ONELA_UNODE_CAP 256
+inline int32_t sg_row_stride(int32_t max_beam) { return (max_beam + 64 + 15) & ~15; }
 cudaError_t launch_dedupe(const int32_t* tables_cur_req0, long long table_req_stride, int32_t* sidx_req0,
                           long long sidx_req_stride, int32_t* ulist_req0, long long ulist_req_stride,
-                          int32_t* urep_req0, int32_t* uoff_req0, long long uoff_req_stride, int32_t req_count, int32_t W,
+                          int32_t* urep_req0, int32_t* uoff_req0, long long uoff_req_stride, uint8_t* sg8_req0,
+                          long long sg8_req_stride, int32_t sg_stride, uint8_t* unode_req0, int32_t req_count, int32_t W,
                           int32_t depth, int32_t max_beam, cudaStream_t stream);
 cudaError_t launch_export_chains(const int32_t* table_cur, int32_t W, int32_t depth, int32_t max_beam,
                                  int32_t* slots_out, cudaStream_t stream);

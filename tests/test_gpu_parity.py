@@ -333,3 +333,25 @@ def test_tensor_core_operands_keep_their_precision_at_any_scale(s0_unit, q_unit)
         ref, _ = run_oracle(case)
         for key, o in outs.items():
             assert rel_l2(o.numpy(), ref[key]).max() <= REL_L2_BAR
+
+
+@pytest.mark.parametrize("key_norm,beta_lo,beta_hi", [(2.5, 0.5, 1.0), (1.0, 1.0, 2.0), (3.0, 0.6, 0.9)])
+@pytest.mark.parametrize("flags", [0, P.FLAG_SHARED_CHAINS, P.FLAG_FORCE_GENERIC])
+def test_keys_and_gates_outside_the_stable_range(key_norm, beta_lo, beta_hi, flags):
+    """Eq. 1 puts no bound on k or beta.  With |k| = 2-3 or beta in (1, 2) a fold step lengthens the folded query
+    (by up to |1 - beta |k|^2| per level), so after eight levels it is orders of magnitude longer than q.  The fp16
+    operand rows of the tensor-core kernels take their power-of-two scale from the folded row itself, so these
+    inputs decode at the same bar as normalised ones - on every kernel."""
+    wl = CFG1.scaled(H=2, W=100, D=8, prompt_len=32, parents="zipf", zipf_s=1.5, seed=606)
+    case = make_case(wl)
+    g = torch.Generator().manual_seed(7)
+    for key, tok in case["tok"].items():
+        tok["k"] = (tok["k"].double() * key_norm).to(tok["k"].dtype)
+        tok["beta"] = (beta_lo + (beta_hi - beta_lo) * torch.rand(tok["beta"].shape, generator=g)).float()
+    ref, _ = run_oracle(case)
+    for fused in (True, False):
+        outs, _, ctx = run_library(case, out_dtype="fp32", flags=flags, fused=fused)
+        assert ctx.onela_poll_device_status() == (0, 0)
+        for key, o in outs.items():
+            assert np.isfinite(o.numpy()).all()
+            assert rel_l2(o.numpy(), ref[key]).max() <= REL_L2_BAR, key

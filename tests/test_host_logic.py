@@ -71,7 +71,10 @@ def test_workspace_carve_up_size():
     index = 2 * (4 * 8 * 512 * 4) + 4 * 9 * 4          # distinct-record index: positions, slot list, level offsets
     select = 4 * 256 * 1024 * 8                        # beam selection: per request 256 partial lists of 1024 candidates
     scales = 4 * 16 * 32 * 4                           # one operand scale per stored head state
-    assert s0 + arena + tables + index + select + scales <= n <= s0 + arena + tables + index + select + scales + 10 * 1024
+    # per distinct record one beam that holds it, the per-beam positions again as bytes (rows padded), 16 bytes per record
+    compact = 4 * 8 * 512 * 4 + 4 * 8 * (512 + 64) + 4 * 256 * 16
+    total = s0 + arena + tables + index + select + scales + compact
+    assert total <= n <= total + 13 * 1024
 
 
 def test_call_order_is_enforced():
