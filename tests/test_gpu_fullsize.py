@@ -1,12 +1,14 @@
 """Parity at the benchmark configs' FULL sizes, in the launch configuration bench.py times (all requests
 of a layer in one batched call, the one-launch append_decode_step, bf16 outputs, the tensor-core kernel).
 
-The oracle cannot replay every unit of these sizes in seconds, so it computes a seeded sample of
-(beam, head) units one by one for a few (request, layer) pairs at several call depths; for those pairs
-S_0 comes from the oracle's fp64 prefill of the seeded prompt (all other pairs: the library's own prefill
-kernel), so both sides consume identical inputs.  Integer work is checked everywhere: the ancestry rows of
-every request at every call against Eq. 5.  One more property holds at any size and is checked on every
-unit: the tensor-core kernel and the CUDA-core kernel, which share no device code, agree.
+For the checked (request, layer) pairs the oracle replays EVERY (beam, head) unit of EVERY decode call:
+all of config 2, one pair per request of config 3, first and last layer of every request of config 4.
+S_0 is an input of the decode path: for a few pairs it comes from the oracle's fp64 prefill of the seeded
+prompt, for the others it is read back from the library's store (the prefill kernel's result, itself checked
+against the oracle's prefill elsewhere) and handed to the oracle, so both sides consume identical inputs.
+Integer work is checked everywhere: the ancestry rows of every request at every call against Eq. 5.  One more
+property holds at any size and is checked on every unit of every pair: the tensor-core kernel and the
+CUDA-core kernel, which share no device code, agree.
 """
 import numpy as np
 import pytest
@@ -30,15 +32,19 @@ def _oracle_state(wl, r, l):
     return torch.from_numpy(oracle.prefill(p["k"], p["v"], p["alpha"], p["beta"]).astype(np.float32))
 
 
-def _run_and_check(wl, pairs, check_calls, n_units=384, flags=0, keep_all_outputs=False, fused=True):
+def _run_and_check(wl, oracle_pairs, store_pairs, check_calls, flags=0, keep_calls=(), fused=True):
+    """Run the whole generation; compare every unit of the calls in `check_calls` for the given pairs with the
+    oracle.  `oracle_pairs` take S_0 from the oracle's prefill, `store_pairs` from the library's store."""
     run = WorkloadRun(wl, "cuda", "bf16", flags=flags)
-    S0 = {pr: _oracle_state(wl, *pr) for pr in pairs}
+    S0 = {pr: _oracle_state(wl, *pr) for pr in oracle_pairs}
     run.prefill_states(overrides=S0)
+    for pr in store_pairs:
+        S0[pr] = run.ctx.onela_export_shared_state(*pr).cpu()
+    pairs = list(oracle_pairs) + list(store_pairs)
     outs = run.alloc_outputs()
-    rng = np.random.default_rng(wl.seed)
     hist = {pr: {"tok": [], "par": [None]} for pr in pairs}
     parents_all = {r: [None] for r in range(wl.R)}
-    worst, kept = 0.0, {}
+    worst, kept, units = 0.0, {}, 0
     for t in range(wl.D):
         call = run.generate_call(t)
         run.run_call(call, outs, fused=fused)     # fused: the launch configuration bench.py times
@@ -59,44 +65,57 @@ def _run_and_check(wl, pairs, check_calls, n_units=384, flags=0, keep_all_output
             if t > 0:
                 hist[(r, l)]["par"].append(parents_all[r][t])
             if t in check_calls:
-                beams = rng.integers(0, wl.W, n_units)
-                beams[:4] = [0, wl.W - 1, wl.W // 2, min(wl.W - 1, 47)]        # tile edges
-                heads = rng.integers(0, wl.H, n_units)
-                ref = oracle.decode(S0[(r, l)], hist[(r, l)]["tok"], hist[(r, l)]["par"], lay["q"][r].cpu(),
-                                    sel=(beams, heads))
-                got = outs[l][r].float().cpu().numpy()[beams, heads]
-                e = rel_l2(got, ref)
+                ref = oracle.decode(S0[(r, l)], hist[(r, l)]["tok"], hist[(r, l)]["par"], lay["q"][r].cpu())
+                e = rel_l2(outs[l][r].float().cpu().numpy(), ref)
+                units += e.size
                 worst = max(worst, float(e.max()))
                 assert e.max() <= REL_L2_BAR, f"pair {(r, l)} call {t}: rel-L2 {e.max():.3e}"
-        if keep_all_outputs:
+        if t in keep_calls:
             kept[t] = [o.clone() for o in outs]
         assert torch.isfinite(outs[0].float()).all()
     assert run.ctx.onela_poll_device_status() == (0, 0)
-    return worst, kept, run
+    return worst, kept, run, units
+
+
+def _two_kernels_agree(wl, calls):
+    """Every unit of every (request, layer) pair at the given calls: tensor-core kernel against CUDA-core kernel."""
+    _, tc, run, _ = _run_and_check(wl, [], [], [], keep_calls=calls)
+    assert run.ctx.onela_uses_tensor_core_path()
+    del run
+    _, cc, run2, _ = _run_and_check(wl, [], [], [], flags=P.FLAG_FORCE_GENERIC, keep_calls=calls, fused=False)
+    assert not run2.ctx.onela_uses_tensor_core_path()
+    for t in calls:
+        for l in range(wl.L):
+            assert rel_l2(tc[t][l].float().cpu().numpy(), cc[t][l].float().cpu().numpy()).max() <= REL_L2_BAR, (t, l)
 
 
 def test_config2_beam512_zipf_every_call():
-    """32 heads, beam 512, depth 4, Zipf(1.2) parents, 16384-token prompt; sampled units at every call, and
-    the two kernels against each other on every unit."""
+    """32 heads, beam 512, depth 4, Zipf(1.2) parents, 16384-token prompt: every unit of every call against the
+    oracle (65 536 decodes), and the two kernels against each other on every unit of every call."""
     wl = inputs.WORKLOADS[2]
-    worst, fused, run = _run_and_check(wl, [(0, 0)], range(wl.D), keep_all_outputs=True)
-    assert run.ctx.onela_uses_tensor_core_path()
-    _, generic, run2 = _run_and_check(wl, [(0, 0)], [wl.D - 1], flags=P.FLAG_FORCE_GENERIC, keep_all_outputs=True,
-                                      fused=False)
-    assert not run2.ctx.onela_uses_tensor_core_path()
-    for t in range(wl.D):
-        a, b = fused[t][0].float().cpu().numpy(), generic[t][0].float().cpu().numpy()
-        assert rel_l2(a, b).max() <= REL_L2_BAR
+    worst, _, run, units = _run_and_check(wl, [(0, 0)], [], range(wl.D))
+    assert run.ctx.onela_uses_tensor_core_path() and units == wl.D * wl.W * wl.H
+    del run
+    _two_kernels_agree(wl, list(range(wl.D)))
 
 
 def test_config3_batch8_beam1024():
-    """8 requests in one shared arena, beam 1024, depth 6, uniform parents; fused and separate launches."""
+    """8 requests in one shared arena, beam 1024, depth 6, uniform parents: every unit of every call of every
+    request (fused launches), every unit of two requests with separate append and decode launches, and the two
+    kernels against each other at the deepest call."""
     wl = inputs.WORKLOADS[3]
-    _run_and_check(wl, [(0, 0), (7, 0)], [0, 2, wl.D - 1])
-    _run_and_check(wl, [(3, 0)], [1, wl.D - 1], fused=False)
+    _, _, _, units = _run_and_check(wl, [(0, 0), (7, 0)], [(r, 0) for r in range(1, 7)], range(wl.D))
+    assert units == wl.R * wl.D * wl.W * wl.H
+    _run_and_check(wl, [], [(3, 0), (4, 0)], range(wl.D), fused=False)
+    _two_kernels_agree(wl, [wl.D - 1])
 
 
 def test_config4_stack16_beam512():
-    """16 layers x 4 requests, beam 512, depth 8, Zipf(1.5) parents with heavy duplication."""
+    """16 layers x 4 requests, beam 512, depth 8, Zipf(1.5) parents with heavy duplication: every unit of every
+    call for the first and the last layer of every request (plus one middle layer), and the two kernels against
+    each other on every unit of the deepest call of all 64 (request, layer) pairs."""
     wl = inputs.WORKLOADS[4]
-    _run_and_check(wl, [(0, 0), (3, 15), (1, 7)], [0, 1, 4, wl.D - 1])
+    store = [(r, l) for r in range(wl.R) for l in (0, wl.L - 1) if (r, l) not in ((0, 0), (3, 15))]
+    _, _, _, units = _run_and_check(wl, [(0, 0), (3, 15), (1, 7)], store, range(wl.D))
+    assert units == 9 * wl.D * wl.W * wl.H
+    _two_kernels_agree(wl, [wl.D - 1])

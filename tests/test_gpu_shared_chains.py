@@ -60,3 +60,13 @@ def test_more_than_128_distinct_records():
     worst, counts = _check(wl, "fp32", True)
     assert max(c[0] for c in counts.values()) > 128, counts
     assert worst < 1.5e-3, (worst, counts)
+
+
+def test_full_size_stack_every_unit():
+    """The beam-512 decode stack at full width and depth (4 requests x 32 heads x 512 beams, depth 8, Zipf(1.5)), two
+    layers: every unit of every call from the second on, first and last layer of every request."""
+    from test_gpu_fullsize import _run_and_check
+    wl = CFG4.scaled(L=2)
+    pairs = [(r, l) for r in range(wl.R) for l in range(wl.L)]
+    _, _, run, units = _run_and_check(wl, [], pairs, range(1, wl.D), flags=P.FLAG_SHARED_CHAINS)
+    assert units == len(pairs) * (wl.D - 1) * wl.W * wl.H
