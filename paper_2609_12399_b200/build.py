@@ -36,8 +36,19 @@ def _stale(target: Path, deps) -> bool:
     return any(d.stat().st_mtime > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> Path:
+# A second library for the tests of the bounded waits: the same sources with a short wait limit and a hook that
+# makes one arrival go missing.  The product never loads it.
+TESTHOOKS_LIB = PKG / "libonela_testhooks.so"
+TESTHOOKS_FLAGS = ["-DONELA_TEST_HOOKS", "-DONELA_WAIT_LIMIT=(1<<14)"]
+
+
+def build_testhooks(force: bool = False) -> Path:
+    return build(force=force, lib=TESTHOOKS_LIB, obj_dir=PKG / "build_testhooks", extra=TESTHOOKS_FLAGS)
+
+
+def build(force: bool = False, verbose: bool = False, lib: Path = LIB, obj_dir: Path = OBJ, extra=()) -> Path:
     """Compile every .cu under csrc/ for sm_100a and link libonela.so next to this file."""
+    OBJ, LIB = obj_dir, lib
     OBJ.mkdir(exist_ok=True)
     headers = list(CSRC.glob("*.h")) + list(CSRC.glob("*.cuh")) + list((ROOT / "include").glob("*.h"))
     nvcc = _nvcc()
@@ -45,7 +56,7 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     for src in sources():
         obj = OBJ / (src.stem + ".o")
         if force or _stale(obj, [src, *headers]):
-            cmd = [nvcc, *NVCC_FLAGS, "-c", str(src), "-o", str(obj)]
+            cmd = [nvcc, *NVCC_FLAGS, *extra, "-c", str(src), "-o", str(obj)]
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
             jobs.append(cmd)
@@ -69,3 +80,5 @@ def build(force: bool = False, verbose: bool = False) -> Path:
 if __name__ == "__main__":
     import sys
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    if "--testhooks" in sys.argv:
+        print(build_testhooks(force="--force" in sys.argv))

@@ -87,6 +87,12 @@ static_assert((GN * 16) % 96 == 0, "three storing warps share a group's 16-byte 
 using L = Lanes<LPU>;
 using RecT = L::R;
 
+#ifdef ONELA_TEST_HOOKS
+// Test-hooks build only (a second library that the product never loads): when set, the first fold warp of CTA 0
+// leaves out ONE arrival (its first quad's), so that the wait for that group's rows runs out.
+__device__ int g_hook_drop_full_arrival;
+#endif
+
 // Bounded wait that also gives up as soon as the CTA's abort flag is raised.
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     for (int i = 0; i < WAIT_LIMIT; ++i) {
@@ -590,6 +596,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
                 __syncwarp();
+#ifdef ONELA_TEST_HOOKS
+                if (g_hook_drop_full_arrival && blockIdx.x == 0 && warp == 0 && k == 0) continue;
+#endif
                 if (lane == 0) mbar_arrive(bar_full(s));
 
                 // The next quad's records of the levels that are NOT staged are gathered from global memory in the middle
@@ -923,6 +932,12 @@ cudaError_t launch_ws_t(const DecodeArgs& a, cudaStream_t stream) {
 }
 
 }  // namespace
+
+#ifdef ONELA_TEST_HOOKS
+extern "C" int onela_testhook_drop_full_arrival(int on) {
+    return (int)cudaMemcpyToSymbol(g_hook_drop_full_arrival, &on, sizeof(int));
+}
+#endif
 
 int make_decode_partition(int total_groups, int groups_per_pair, int sms, int group_cost, int seg_cost, DecodePartition* part) {
     return make_partition(total_groups, groups_per_pair, sms > MAX_CTAS ? MAX_CTAS : sms, PartitionCost{group_cost, seg_cost}, part);

@@ -12,7 +12,10 @@ namespace sm100 {
 
 constexpr int DK = 128, DV = 128;
 constexpr int REC_BYTES = (DK + DV) * 2;       // 512: k | v in bf16
-constexpr int WAIT_LIMIT = 1 << 20;
+#ifndef ONELA_WAIT_LIMIT
+#define ONELA_WAIT_LIMIT (1 << 20)
+#endif
+constexpr int WAIT_LIMIT = ONELA_WAIT_LIMIT;     // probes of a barrier before a wait gives up (the test-hooks build uses fewer)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
