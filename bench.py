@@ -40,11 +40,26 @@ from paper_2609_12399_b200 import accounting, inputs, replicas  # noqa: E402
 METRIC = "beam-head GDN decodes/s per layer at beam 512"
 UNIT = "decodes/s"
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of ONE fused append + decode launch of the default workload at
-# its deepest call (depth 8, all 4 requests of one layer), from the ncu capture summarised in
-# profiles/decode_ws_kernel_cfg4_ncu.md (69.1 MB read + 11.9 MB written).  The algorithmic bytes of that launch
-# are 118.7 MB; of the 50.9 MB it writes, 38 MB were still in L2 when the kernel ended.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 81.0e6
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE fused append + decode launch of the default workload at its
+# deepest call, as the latest ncu capture found it: read from the summary that the capture's notes keep under
+# profiles/ (key = value lines, with the commit the capture was taken on), never a constant in this file.
+TRAFFIC_SUMMARY = ROOT / "profiles" / "decode_ws_kernel_cfg4_traffic.txt"
+
+
+def ncu_traffic() -> dict:
+    if not TRAFFIC_SUMMARY.exists():
+        return {"bytes": None, "source": "no capture summary under profiles/"}
+    kv = {}
+    for ln in TRAFFIC_SUMMARY.read_text().splitlines():
+        if "=" in ln and not ln.lstrip().startswith("#"):
+            k, v = ln.split("=", 1)
+            kv[k.strip()] = v.strip()
+    try:
+        total = float(kv["dram_bytes_read"]) + float(kv["dram_bytes_write"])
+    except (KeyError, ValueError):
+        return {"bytes": None, "source": f"{TRAFFIC_SUMMARY.name} is incomplete"}
+    return {"bytes": total, "source": f"profiles/{TRAFFIC_SUMMARY.name}: ncu capture of one launch at depth {kv.get('depth', '?')}, "
+                                      f"kernel source at commit {kv.get('commit', '?')}"}
 
 
 def workload_by_name(name: str) -> inputs.Workload:
@@ -265,10 +280,16 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     else:
         peak, peak_src = FALLBACK_HBM_GBS, "of fallback"
     ms_per_step = ms_total / args.steps
+    traffic = ncu_traffic()
+    default_path = not (args.unfused or args.delta_records or args.force_generic or args.shared_chains) and wl.name.startswith("cfg4")
+    clk = clocks.summary()
+    mhz = clk["sm_mhz"] or 0.0
     line = {
         "metric": METRIC, "value": replicas.aggregate_throughput(units_per_step, ms_per_step, world), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32 fold and corrections; the S_0 contraction on the tensor cores with fp16 operands (11-bit significand, "
+                 "exact power-of-two scales) and f32 accumulation",
         "data": "synthetic",
         "config": {"workload": describe(wl), "step": "one whole generation: reset, store S_0, then per decode call "
                    "reorder + per layer append + decode (one fused launch per layer unless --unfused)", "units_per_step": units_per_step,
@@ -280,14 +301,18 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
                    "tensor_core_path": bool(ctx.onela_uses_tensor_core_path()),
                    "record_format": "(alpha, delta, k), forward projection replay" if args.delta_records
                                     else "(k, v, alpha, beta), backward query fold"},
-        "clocks": {**clocks.summary(), "window": "sampled from the warm-up to the end of the timed legs"},
+        "clocks": {**clk, "window": "sampled from the warm-up to the end of the timed legs"},
         "e2e": {"value": e2e["value"], "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                 "ms_per_step": e2e["ms_per_step"]},
         "gpu_launches": int(launches_per_step * args.steps),
         "roofline": {"bound": "hbm", "achieved": achieved_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": achieved_gbs / peak, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if not (args.unfused or args.delta_records or args.force_generic) else None,
-                     "traffic_note": "ncu DRAM read+write bytes of one launch at the deepest call (depth %d), whose "
-                                     "algorithmic bytes are %.1f MB; see profiles/" % (wl.D, per_depth[-1]["algorithmic"] / 1e6),
+                     "frac": achieved_gbs / peak,
+                     "traffic": traffic["bytes"] if default_path else None,
+                     "traffic_note": "ncu DRAM read+write bytes of one launch at the deepest call (depth %d), whose algorithmic "
+                                     "bytes are %.1f MB (writes still in L2 when the kernel ends are not in it); %s"
+                                     % (wl.D, per_depth[-1]["algorithmic"] / 1e6, traffic["source"]),
+                     "headline": {"deepest_call_frac": per_depth[-1]["algorithmic"] / (ms_depth[-1] * 1e-3) / 1e9 / peak,
+                                  "mean_over_calls_frac": achieved_gbs / peak},
                      "warm_l2": warm,
                      "peak_source": peak_src,
                      "frac_of_nominal_8_tbs": achieved_gbs / 8000.0,   # context: the paper-independent nominal HBM3e figure
@@ -298,13 +323,63 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
                               + ("" if args.unfused else " + the call's records written to the arena"),
                      "undeduplicated_gbs": und_total / (dur_ms.sum() * 1e-3) / 1e9,
                      "per_depth": [{"depth": t + 1, "us": float(ms_depth[t] * 1e3),
+                                    "sm_cycles": float(ms_depth[t] * 1e3 * mhz),     # us x the sampled median SM MHz
                                     "algorithmic_MB": per_depth[t]["algorithmic"] / 1e6,
                                     "frac": per_depth[t]["algorithmic"] / (ms_depth[t] * 1e-3) / 1e9 / peak}
                                    for t in range(wl.D)]},
     }
+    if rank == 0 and world == 1 and default_path and not args.no_secondary:
+        del graph
+        # the other beam-512 config and the large-batch config, in the same run (context, not the bench value)
+        line["secondary"] = [secondary_roofline(n, dev, peak, mhz) for n in ("cfg2", "cfg3")]
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(wl, reps=1, gen_device=dev)
     return line
+
+
+def secondary_roofline(name: str, dev, peak: float, mhz: float, reps: int = 5) -> dict:
+    """The same roofline block for another benchmark config, timed in this run: whole generations launched eagerly
+    with the fused call, one CUDA-event pair around each decode call's launches.  These workloads are smaller than
+    L2, so a buffer larger than L2 is overwritten before every decode call's launches (outside the event pairs)."""
+    from paper_2609_12399_b200.runner import WorkloadRun
+
+    wl = workload_by_name(name)
+    run = WorkloadRun(wl, dev, wl.dtype)
+    ctx = run.ctx
+    run.prefill_states()
+    S0_all = torch.stack([torch.stack([ctx.onela_export_shared_state(r, l) for l in range(wl.L)]) for r in range(wl.R)])
+    calls = [run.generate_call(t) for t in range(wl.D)]
+    outs = run.alloc_outputs()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    per_depth = launch_bytes(wl, 2 if wl.dtype == "bf16" else 4, True)
+    pairs = []
+
+    def generation(record):
+        ctx.onela_reset()
+        ctx.onela_init_shared_states(0, wl.R, S0_all)
+        for call in calls:
+            flush.zero_()
+            run.run_call(call, outs, None, pairs if record else None, fused=True, group_events=True)
+
+    for _ in range(3):
+        generation(False)
+    torch.cuda.synchronize()
+    for _ in range(reps):
+        generation(True)
+    torch.cuda.synchronize()
+    per = pairs[0][2]
+    dur_ms = np.array([a.elapsed_time(b) for a, b, _ in pairs]).reshape(reps, wl.D, -1)
+    ms_depth = dur_ms.mean(axis=(0, 2)) / per
+    alg = sum(d["algorithmic"] for d in per_depth) * dur_ms.shape[2] * per * reps
+    achieved = alg / (dur_ms.sum() * 1e-3) / 1e9
+    units = wl.R * wl.W * wl.H
+    del run, calls, outs, flush
+    return {"workload": describe(wl), "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+            "traffic": None, "l2": "a 256 MiB buffer is overwritten before every decode call (the workload is smaller than L2)",
+            "decodes_per_s": units * wl.L * wl.D / (float(ms_depth.sum()) * 1e-3 * wl.L),
+            "per_depth": [{"depth": t + 1, "us": float(ms_depth[t] * 1e3), "sm_cycles": float(ms_depth[t] * 1e3 * mhz),
+                           "algorithmic_MB": per_depth[t]["algorithmic"] / 1e6,
+                           "frac": per_depth[t]["algorithmic"] / (ms_depth[t] * 1e-3) / 1e9 / peak} for t in range(wl.D)]}
 
 
 def run_e2e(args, run, S0, calls, outs, units_per_step, barrier) -> dict:
@@ -477,12 +552,42 @@ def main():
     ap.add_argument("--profile", action="store_true", help="eager generations only, for ncu")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (kernel experiments)")
+    ap.add_argument("--no-secondary", action="store_true", help="skip the roofline blocks of configs 2 and 3")
+    ap.add_argument("--rank-plumbing-only", action="store_true",
+                    help="no GPU work: every rank reports a made-up time (rank + 1 ms) through the timing protocol over gloo; "
+                         "checks the launch, barrier, max-over-ranks and aggregation logic on a CPU box")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" and not args.profile else args.warmup
 
+    # `--gpus N` on its own starts the N replicas itself: one process per GPU under torch.distributed.run on this
+    # node (a launcher that already set RANK / WORLD_SIZE is left alone).
+    if args.gpus > 1 and "RANK" not in os.environ and args.impl == "ours":
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        os.execv(sys.executable, [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+                                  "--master-addr", "127.0.0.1", "--master-port", str(port), str(Path(__file__).resolve()), *sys.argv[1:]])
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "ours" and world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but the launcher started {world} rank(s)")
+
+    if args.rank_plumbing_only:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        if world > 1:
+            torch.distributed.init_process_group("gloo")
+        replicas.barrier()
+        units = 1000
+        (ms,) = replicas.max_over_ranks([float(rank + 1)])
+        replicas.barrier()
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": replicas.aggregate_throughput(units, ms, world), "unit": UNIT,
+                              "n_gpus": world, "ms_per_step": ms, "scaling": "weak", "rank_plumbing_only": True}), flush=True)
+        if world > 1:
+            torch.distributed.destroy_process_group()
+        return
 
     if args.impl == "reference":
         if rank == 0:

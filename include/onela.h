@@ -2,7 +2,7 @@
  * onela.h - C ABI of the beam-shared Gated DeltaNet (GDN) decode library for NVIDIA B200 (sm_100a).
  *
  * The library holds, for every request, ONE post-prefill recurrent state S_0 per (layer, head)
- * ("stores S_ctx only once", paper Section 3.2), an append-only arena of per-token transition
+ * (the shared context state is kept once, not per beam: paper Section 3.2), an append-only arena of per-token transition
  * records, and an ancestry index that maps every live beam to the records on its lineage
  * (Section 3.3, Eq. 5).  A decode call evaluates the GDN output of Eq. 1,
  *
@@ -45,8 +45,8 @@
  *  - Slot numbering: one bump cursor per context.  reorder_beams over requests [b, b+n) assigns, in
  *    request order, base(req, t) = cursor, cursor += W_new (after a release_request: the lowest released
  *    range that fits, first).  The record of beam i at decode call t lives
- *    at global slot base(req, t) + i in every layer ("written once to the physical slots of the current
- *    decoding step and never relocated", Section 3.3).
+ *    at global slot base(req, t) + i in every layer (a record is written once, at its decode call's slots, and
+ *    never moves afterwards: Section 3.3).
  *  - Batched calls (req_count > 1) need the same beam width and depth on every request of the batch,
  *    and at most ONELA_MAX_BATCH requests.
  */
@@ -175,8 +175,8 @@ onela_status onela_reorder_beams(onela_ctx* ctx, int32_t req_begin, int32_t req_
  * A request slot that is re-initialised WITHOUT being released keeps its old slots occupied until onela_reset. */
 onela_status onela_release_request(onela_ctx* ctx, int32_t request);
 
-/* Global beam selection feeding onela_reorder_beams ("all active beams are expanded over the codebook and the
- * global top-k candidates are retained", Section 2.2): for each request of [req_begin, req_begin+req_count),
+/* Global beam selection feeding onela_reorder_beams (every live beam is extended by every code of the codebook and
+ * the best k of all the candidates survive: Section 2.1): for each request of [req_begin, req_begin+req_count),
  * candidate (p, c) scores beam_scores_dev[req][p] + cand_logp_dev[req][p][c], added in fp32, with p over the
  * W_prev beams of the request's current decode call (W_prev = 1, the root, before the first call) and c over the C
  * codes.  The W_new best are written best first: parents_out_dev [req_count][W_new] int32 (the parent map pi_t in
@@ -208,8 +208,8 @@ onela_status onela_select_beams_static(const float* beam_scores_dev, const float
                                        int32_t W_prev, int32_t C, int32_t W_new, int32_t* parents_out_dev,
                                        int32_t* codes_out_dev, float* scores_out_dev, void* stream);
 
-/* Append this call's transition records for one layer ("appends only the compact record ... rather
- * than writing back a full recurrent state", Section 3.4): k_dev [req_count][W][H][dk],
+/* Append this call's transition records for one layer (a call adds one compact record per beam and head; no full
+ * recurrent state is ever written back: Section 3.4): k_dev [req_count][W][H][dk],
  * v_dev [req_count][W][H][dv] in rec_dtype, alpha_dev, beta_dev [req_count][W][H] fp32.  Values are
  * stored bit-exactly and never modified afterwards. */
 onela_status onela_append_records(onela_ctx* ctx, int32_t req_begin, int32_t req_count, int32_t layer,

@@ -1,7 +1,7 @@
 """Global beam selection, written out plainly (test infrastructure: only tests/, the smoke check and the CPU
 baseline legs of bench.py may import this package; the CUDA path shares no code with it).
 
-Section 2.2 of the paper: at each decoding step all active beams are expanded over the semantic-ID codebook and
+Section 2.1 of the paper: at each decoding step all active beams are expanded over the semantic-ID codebook and
 the global top-k candidates are retained; several survivors may share a parent and other parents disappear, which
 is what defines the parent map pi_t(b) that the ancestry index (Eq. 5) consumes.  The paper fixes nothing else,
 so the reading taken here (and by the library) is:

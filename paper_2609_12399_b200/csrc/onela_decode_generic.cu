@@ -17,31 +17,6 @@ namespace {
 
 constexpr int NB = 32;  // beams per tile
 
-template <typename OutT, int N>
-__device__ __forceinline__ void store_out(OutT* p, const float* x);
-template <>
-__device__ __forceinline__ void store_out<float, 4>(float* p, const float* x) {
-    *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]);
-}
-template <>
-__device__ __forceinline__ void store_out<float, 8>(float* p, const float* x) {
-    reinterpret_cast<float4*>(p)[0] = make_float4(x[0], x[1], x[2], x[3]);
-    reinterpret_cast<float4*>(p)[1] = make_float4(x[4], x[5], x[6], x[7]);
-}
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-    const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<const uint32_t*>(&t);
-}
-template <>
-__device__ __forceinline__ void store_out<__nv_bfloat16, 4>(__nv_bfloat16* p, const float* x) {
-    *reinterpret_cast<uint2*>(p) = make_uint2(pack_bf16x2(x[0], x[1]), pack_bf16x2(x[2], x[3]));
-}
-template <>
-__device__ __forceinline__ void store_out<__nv_bfloat16, 8>(__nv_bfloat16* p, const float* x) {
-    *reinterpret_cast<uint4*>(p) = make_uint4(pack_bf16x2(x[0], x[1]), pack_bf16x2(x[2], x[3]),
-                                              pack_bf16x2(x[4], x[5]), pack_bf16x2(x[6], x[7]));
-}
-
 template <int DK, int DV, typename T, typename OutT, int G>
 __global__ void __launch_bounds__(NB* G) decode_generic_kernel(const DecodeArgs a) {
     constexpr int VEC = Vec16<T>::N;

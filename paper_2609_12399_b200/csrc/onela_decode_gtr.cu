@@ -24,10 +24,6 @@ namespace {
 
 constexpr int NB = 32;  // beams per tile
 
-__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
-    const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<const uint32_t*>(&t);
-}
 // N consecutive elements (one 16-byte vector of T) from fp32
 template <typename T>
 __device__ __forceinline__ void store_vec(T* p, const float* x);
@@ -39,19 +35,6 @@ template <>
 __device__ __forceinline__ void store_vec<__nv_bfloat16>(__nv_bfloat16* p, const float* x) {
     *reinterpret_cast<uint4*>(p) = make_uint4(pack2(x[0], x[1]), pack2(x[2], x[3]), pack2(x[4], x[5]), pack2(x[6], x[7]));
 }
-// VEC consecutive outputs of type OutT from fp32 (VEC = elements of one 16-byte vector of the RECORD type)
-template <typename OutT, int VEC>
-__device__ __forceinline__ void store_out(OutT* p, const float* x) {
-    if constexpr (sizeof(OutT) == 4) {
-#pragma unroll
-        for (int e = 0; e < VEC; e += 4) *reinterpret_cast<float4*>(p + e) = make_float4(x[e], x[e + 1], x[e + 2], x[e + 3]);
-    } else if constexpr (VEC == 8) {
-        *reinterpret_cast<uint4*>(p) = make_uint4(pack2(x[0], x[1]), pack2(x[2], x[3]), pack2(x[4], x[5]), pack2(x[6], x[7]));
-    } else {
-        *reinterpret_cast<uint2*>(p) = make_uint2(pack2(x[0], x[1]), pack2(x[2], x[3]));
-    }
-}
-
 template <int DK, int DV, typename T, typename OutT, int G>
 __global__ void __launch_bounds__(NB* G) decode_gtr_kernel(const DecodeArgs a) {
     constexpr int VEC = Vec16<T>::N;

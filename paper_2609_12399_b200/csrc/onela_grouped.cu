@@ -13,22 +13,6 @@ namespace {
 
 constexpr int NB = 32;  // beams per tile
 
-__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
-    const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<const uint32_t*>(&t);
-}
-template <typename OutT, int VEC>
-__device__ __forceinline__ void store_out(OutT* p, const float* x) {
-    if constexpr (sizeof(OutT) == 4) {
-#pragma unroll
-        for (int e = 0; e < VEC; e += 4) *reinterpret_cast<float4*>(p + e) = make_float4(x[e], x[e + 1], x[e + 2], x[e + 3]);
-    } else if constexpr (VEC == 8) {
-        *reinterpret_cast<uint4*>(p) = make_uint4(pack2(x[0], x[1]), pack2(x[2], x[3]), pack2(x[4], x[5]), pack2(x[6], x[7]));
-    } else {
-        *reinterpret_cast<uint2*>(p) = make_uint2(pack2(x[0], x[1]), pack2(x[2], x[3]));
-    }
-}
-
 template <int DK, int DV, typename T, typename OutT, int G>
 __global__ void __launch_bounds__(NB* G) decode_grouped_kernel(const GroupedArgs a) {
     constexpr int VEC = Vec16<T>::N;

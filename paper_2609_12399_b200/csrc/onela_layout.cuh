@@ -1,4 +1,4 @@
-// Device helpers shared by the kernel files: bf16 unpacking.
+// Device helpers shared by the kernel files: bf16 unpacking and packing, vector stores of fp32 results.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -33,5 +33,23 @@ struct Vec16<__nv_bfloat16> {
         unpack_bf16x2(x.w, out[6], out[7]);
     }
 };
+
+// two fp32 -> two packed bf16 (element 0 in the low half), round to nearest even
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+    const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&t);
+}
+// VEC consecutive outputs of type OutT from fp32 (VEC = 4 or 8: the elements of one 16-byte vector of the record type)
+template <typename OutT, int VEC>
+__device__ __forceinline__ void store_out(OutT* p, const float* x) {
+    if constexpr (sizeof(OutT) == 4) {
+#pragma unroll
+        for (int e = 0; e < VEC; e += 4) *reinterpret_cast<float4*>(p + e) = make_float4(x[e], x[e + 1], x[e + 2], x[e + 3]);
+    } else if constexpr (VEC == 8) {
+        *reinterpret_cast<uint4*>(p) = make_uint4(pack2(x[0], x[1]), pack2(x[2], x[3]), pack2(x[4], x[5]), pack2(x[6], x[7]));
+    } else {
+        *reinterpret_cast<uint2*>(p) = make_uint2(pack2(x[0], x[1]), pack2(x[2], x[3]));
+    }
+}
 
 }  // namespace onela

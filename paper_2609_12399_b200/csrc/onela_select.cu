@@ -1,4 +1,4 @@
-// Global beam selection (Section 2.2: every active beam is expanded over the codebook and the global top-k
+// Global beam selection (Section 2.1: every active beam is expanded over the codebook and the global top-k
 // candidates are kept): from the previous beams' cumulative scores and this step's candidate log-probabilities,
 // the W_new best (parent, code) pairs per request, best first, parents in the form onela_reorder_beams takes - so
 // selection, reorder and the layers' decode launches of a step can run back to back on the device (one CUDA graph).

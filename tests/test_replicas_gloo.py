@@ -50,3 +50,21 @@ def test_single_process_is_identity():
     assert replicas.world() == (0, 1)
     assert replicas.max_over_ranks([1.5, 2.5]) == [1.5, 2.5]
     assert replicas.aggregate_throughput(10, 2.0, 1) == pytest.approx(5000.0)
+
+
+def test_bench_starts_its_own_ranks_and_aggregates_over_them():
+    """`python bench.py --gpus 2` (no launcher around it) starts two ranks itself; the timing protocol takes the
+    slowest rank's time (rank r reports r + 1 ms here) and the value counts both replicas' units.  CPU only."""
+    import json
+    import subprocess
+    import sys
+    from pathlib import Path
+
+    root = Path(__file__).resolve().parent.parent
+    r = subprocess.run([sys.executable, str(root / "bench.py"), "--gpus", "2", "--rank-plumbing-only"], capture_output=True,
+                       text=True, timeout=300, env={k: v for k, v in __import__("os").environ.items()
+                                                    if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")})
+    assert r.returncode == 0, r.stdout + r.stderr
+    line = json.loads([ln for ln in r.stdout.splitlines() if ln.startswith("{")][-1])
+    assert line["n_gpus"] == 2 and line["ms_per_step"] == 2.0
+    assert line["value"] == 2 * 1000 / 2.0e-3

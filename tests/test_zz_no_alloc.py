@@ -3,14 +3,17 @@ handed the whole GPU to its own pool, a plug-in on a borrowed stream where cudaM
 allowed.  It keeps its partial lists in an array built into the library instead of a workspace.
 
 Checked here through the C ABI: its parents, codes and scores equal those of onela_select_beams (the workspace
-version, itself held bit-exact to the selection oracle elsewhere) on two calls in a row with different inputs -
-the second call finds the first call's leftovers in the shared array and must not be disturbed by them - and that
-neither call allocates device memory.  Requests beyond the built-in array's room are refused.
+version) and those of the selection oracle, on two calls in a row with different inputs - the second call finds the
+first call's leftovers in the shared array and must not be disturbed by them - and that no call allocates device
+memory: neither PyTorch's allocator nor the driver's count of free bytes moves (the very first call of a process
+loads the library's device code, so one call is made before the counts are taken).  Requests beyond the built-in
+array's room are refused.
 
 This file sorts last on purpose: a run that stops at the first failure has then run every other test."""
 import pytest
 import torch
 
+import oracle.select
 import paper_2609_12399_b200 as P
 from paper_2609_12399_b200 import binding
 
@@ -41,18 +44,24 @@ def test_static_selection_matches_the_workspace_version_twice_and_allocates_noth
     # first call: many candidates (parts + merge through the built-in array); second: ties, a different width,
     # fewer survivors - it runs over whatever the first call left in the array
     cases = [(_inputs(71, R, W, C), W), (_inputs(72, R, W, C, quant=4), 300)]
+    P.onela_select_beams_static(*cases[0][0], W, *_outputs(R, W))     # module load and the array's address: once per process
+    torch.cuda.synchronize()
     for (bs, lp), W_new in cases:
         want = _outputs(R, W_new)
         ctx.onela_select_beams(0, R, bs, lp, C, W_new, *want)
         got = _outputs(R, W_new)
         torch.cuda.synchronize()
-        before = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+        before = torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), torch.cuda.mem_get_info()[0]
         P.onela_select_beams_static(bs, lp, W_new, *got)
         torch.cuda.synchronize()
-        assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == before
+        assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), torch.cuda.mem_get_info()[0]) == before
         assert torch.equal(got[0], want[0]), "parents"
         assert torch.equal(got[1], want[1]), "codes"
         assert torch.equal(got[2].view(torch.int32), want[2].view(torch.int32)), "scores, bit for bit"
+        for r in range(R):      # and the oracle's selection, request by request
+            op, oc, osc = oracle.select.select_beams(bs[r].cpu().numpy(), lp[r].cpu().numpy(), W_new)
+            assert (got[0][r].cpu().numpy() == op).all() and (got[1][r].cpu().numpy() == oc).all()
+            assert (got[2][r].cpu().numpy().view("int32") == osc.view("int32")).all()
     assert ctx.onela_poll_device_status() == (0, 0)
 
 
