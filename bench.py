@@ -237,7 +237,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
         # ---- B'. the same kernel with a WARM L2 (labelled; not the bench value): the deepest call's decode-only
         # launch repeated on one layer, so S_0, the records, the queries and the outputs stay L2-resident
         warm = None
-        if wl.R <= 8:
+        if wl.R <= 8 and not args.delta_records:
             lay = calls[-1]["layers"][0]
             reps = 20
             for _ in range(3):

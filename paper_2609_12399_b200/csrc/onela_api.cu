@@ -226,8 +226,7 @@ onela_status onela_create(const onela_config* cfg, void* workspace_dev, size_t w
         r.has_state.assign(cfg->num_layers, 0);
         r.appended_depth.assign(cfg->num_layers, -1);
     }
-    ctx->tensor_core = decode_sm100_supported(cfg->dk, cfg->dv, cfg->rec_dtype) &&
-                       !(cfg->flags & (ONELA_FLAG_FORCE_GENERIC | ONELA_FLAG_GTR_DELTA));
+    ctx->tensor_core = decode_sm100_supported(cfg->dk, cfg->dv, cfg->rec_dtype) && !(cfg->flags & ONELA_FLAG_FORCE_GENERIC);
     *out = ctx;
     return ONELA_OK;
 }
@@ -531,11 +530,11 @@ onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count,
     for (int i = 0; i < req_count; ++i) a.bases.base[i] = ctx->req[req_begin + i].step_base.back();
     a.early_ok = ctx->launches == ctx->decode_mark ? 1 : 0;
     bool supported = true;
-    const bool wy = ctx->tensor_core && (c.flags & ONELA_FLAG_SHARED_CHAINS) && !ctx->grouped() && depth >= 2 &&
+    const bool wy = ctx->tensor_core && !ctx->gtr() && (c.flags & ONELA_FLAG_SHARED_CHAINS) && !ctx->grouped() && depth >= 2 &&
                     depth <= WY_MAX_LEVELS + 1;
-    const cudaError_t e = ctx->gtr()         ? launch_decode_gtr(a, c.dk, c.dv, c.rec_dtype, c.out_dtype, &supported, s)
+    const cudaError_t e = ctx->gtr() && !ctx->tensor_core ? launch_decode_gtr(a, c.dk, c.dv, c.rec_dtype, c.out_dtype, &supported, s)
                           : wy               ? launch_decode_wy(a, c.out_dtype, s)
-                          : ctx->tensor_core ? launch_decode_sm100_ws(a, c.out_dtype, ctx->grouped(), s)
+                          : ctx->tensor_core ? launch_decode_sm100_ws(a, c.out_dtype, ctx->grouped(), ctx->gtr(), s)
                                              : launch_decode_generic(a, c.dk, c.dv, c.rec_dtype, c.out_dtype, &supported, s);
     if (!supported) return ONELA_E_UNSUPPORTED;
     if (e != cudaSuccess) return ONELA_E_CUDA;

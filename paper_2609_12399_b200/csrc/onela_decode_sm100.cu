@@ -75,6 +75,14 @@ constexpr int STAGE_BYTES = 2 * STAGE_BUF * REC_BYTES;
 constexpr int GATE_BYTES = (2 * STAGE_BUF * 8 + 127) & ~127;   // padded: the heads' stages behind it stay 128-byte aligned (measured: 1.5 % faster)
 constexpr int INV_BYTES = SLOTS * GN * 4;        // per ring slot and beam: what undoes the operands' scales
 constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + STAGE_BYTES + GATE_BYTES + HEADS_TOTAL + 256 + INV_BYTES + 1024;
+// DELTA instantiation (records (alpha, delta, k), forward projection replay): a beam owns TWO rows of a group - its
+// query and its own key, both projected through the parent state - so a group holds GN / 2 beams; per ring slot the
+// beams' own value rows (raw) and three scalars each (alpha_t, beta_t, k_t . q_t) wait for the epilogue.
+constexpr int DELTA_BEAMS = GN / 2;
+constexpr int DELTA_SLOT_BYTES = DELTA_BEAMS * (DV * 2) + DELTA_BEAMS * 16;
+constexpr int SMEM_BYTES_DELTA = SMEM_BYTES + SLOTS * DELTA_SLOT_BYTES;
+static_assert(SMEM_BYTES_DELTA <= 232448, "shared memory per CTA (delta records)");
+static_assert((DELTA_BEAMS * 16) % 96 == 0, "three storing warps share a delta group's 16-byte chunks evenly");
 constexpr uint32_t S0_COL = 128;                 // accumulators of the ring slots in [0, SLOTS * GN); S_0 buffers (64 columns) at 128 and 256
 constexpr int R_TARGET = 8;                      // a scaled operand row's largest element lies in [2^8, 2^9) x (decay in [1, 2)): far inside fp16's range
 constexpr uint32_t TMEM_COLS = 512;
@@ -121,7 +129,10 @@ using Partition = DecodePartition;
 
 // GROUPED: value head h reads the queries and keys of key head h / g; a.H counts VALUE heads, the record's k lives in
 // the key heads' plane (a.kv) and its v in the value heads' plane (a.vv), 256 bytes each.
-template <typename OutT, bool GROUPED, bool FUSED>
+// DELTA: the arena keeps (alpha_t, delta_t, k_t) (Section 3.2, Eq. 2-4); both projections S q_t and S k_t of the parent
+// state are replayed forward from S_0 . q_t and S_0 . k_t (one MMA set over the 2 x 24 rows of a group), delta_t and
+// o_t are formed in the epilogue and the record is written there; always with the append fused in, never GROUPED.
+template <typename OutT, bool GROUPED, bool FUSED, bool DELTA = false>
 __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ Partition part,
                                                                int groups_per_pair) {
     extern __shared__ uint8_t smem_raw[];
@@ -141,6 +152,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 7 + 3 * SLOTS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     float* inv_s = reinterpret_cast<float*>(heads + HEADS_TOTAL + 256);      // [SLOTS][GN]
+    uint8_t* delta_s = heads + HEADS_TOTAL + 256 + INV_BYTES;                // DELTA: [SLOTS][value rows | scalars]
+    constexpr int BPG = DELTA ? DELTA_BEAMS : GN;                            // beams per group
+    static_assert(!DELTA || (FUSED && !GROUPED), "delta records come with the append fused in, ungrouped");
     auto bar_s0 = [&](int b) { return smem_u32(bars + b); };
     auto bar_stage = [&](int b) { return smem_u32(bars + 2 + b); };
     auto bar_sfree = [&](int b) { return smem_u32(bars + 4 + b); };
@@ -292,7 +306,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         const int n_quads = g_end - g_begin;
         uint8_t* my_heads = heads + warp * HEAD_BYTES;
         struct Unit { int seg, req, h, gip; };           // segment, request, head, group within the (request, head) pair
-        auto beam_of = [&](const Unit& u) { return u.gip * GN + UPW * warp + grp; };
+        auto beam_of = [&](const Unit& u) { return u.gip * BPG + (DELTA ? (UPW * warp + grp) >> 1 : UPW * warp + grp); };
         auto live_beam = [&](const Unit& u) { return min(beam_of(u), a.W - 1); };   // idle units shadow a live beam
         auto next_unit = [&](Unit u) {                   // the quad after u's, without divisions
             if (++u.gip == groups_per_pair) {
@@ -317,7 +331,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         auto request_heads = [&](const Unit& n) {        // the 128-byte lines of a quad's heads, into L2
             if (lane < UPW * 6) {
                 const int un = lane / 6, item = lane % 6;
-                const int b2 = min(n.gip * GN + UPW * warp + un, a.W - 1);
+                const int b2 = min(n.gip * BPG + (DELTA ? (UPW * warp + un) >> 1 : UPW * warp + un), a.W - 1);
                 const long long krow2 = krow_in(n.req, b2, n.h), vrow2 = vrow_in(n.req, b2, n.h);
                 const long long slot2 = a.bases.base[n.req] + b2;
                 const char* p2 = item < 2 ? reinterpret_cast<const char*>(qbase) + krow2 * (DK * 2)
@@ -437,7 +451,15 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                     // the next quad's copies go out before this quad's stores (each lane overwrites only the chunks it
                     // has just read)
                     if (k + 1 < n_quads) issue_head(u1);
-                    if (fused && beam_of(u0) < a.W) {   // the append: this beam's record goes to its arena slot, bit for bit
+                    if (DELTA) {
+                        // the key half of the record and the gates; delta_t follows from the epilogue
+                        if ((grp & 1) == 0 && beam_of(u0) < a.W) {
+                            uint4* dst = reinterpret_cast<uint4*>(a.kv_out + (own_row0 + bb) * REC_BYTES) + g;
+#pragma unroll
+                            for (int c = 0; c < NCH; ++c) dst[c * LPU] = cur.own.k[c];
+                            if (g == 0) a.gates_out[own_row0 + bb] = gate0;
+                        }
+                    } else if (fused && beam_of(u0) < a.W) {   // the append: this beam's record goes to its arena slot, bit for bit
                         if constexpr (GROUPED) {
                             const long long slot = a.bases.base[u0.req] + bb;
                             uint4* vdst = reinterpret_cast<uint4*>(a.vv_out + ((long long)u0.h * a.arena_slots + slot) * (DV * 2)) + g;
@@ -478,8 +500,28 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 };
 
                 float2 r[4 * NCH], corr[4 * NCH];
+                float kq = 0.f;              // DELTA: k_t . q_t
+                if (DELTA) {
+                    float2 kx[4 * NCH];
 #pragma unroll
-                for (int c = 0; c < NCH; ++c) unpack8(cur.q[c], r + 4 * c);
+                    for (int c = 0; c < NCH; ++c) {
+                        unpack8(cur.q[c], r + 4 * c);
+                        unpack8(cur.own.k[c], kx + 4 * c);
+                    }
+                    float2 d2 = make_float2(0.f, 0.f);
+#pragma unroll
+                    for (int e = 0; e < 4 * NCH; ++e) d2 = __ffma2_rn(kx[e], r[e], d2);
+                    kq = d2.x + d2.y;
+#pragma unroll
+                    for (int o = LPU / 2; o > 0; o >>= 1) kq += __shfl_xor_sync(0xffffffffu, kq, o);
+                    if (grp & 1) {           // the odd unit of a beam projects its key
+#pragma unroll
+                        for (int e = 0; e < 4 * NCH; ++e) r[e] = kx[e];
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) unpack8(cur.q[c], r + 4 * c);
+                }
 #pragma unroll
                 for (int e = 0; e < 4 * NCH; ++e) corr[e] = make_float2(0.f, 0.f);
                 float decay = 1.f;
@@ -502,8 +544,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                         q_inv = __uint_as_float((uint32_t)(127 + hq - R_TARGET) << 23);
                     }
                 }
-                L::fold_chain_simple(cur.own, old - 1, staged_levels,
-                              [&](int level) {
+                auto gather = [&](int level) {
                                   const long long slot = idx_of(level);
                                   if constexpr (GROUPED) {
                                       RecT rec;
@@ -519,7 +560,15 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                                   } else {
                                       return L::load_global(kv, a.gates, plane_row0 + slot, g);
                                   }
-                              }, r, corr, decay);
+                              };
+                if (DELTA) {     // the replay runs over the older records only; the beam's own is formed in the epilogue
+                    if (old - 1 >= staged_levels) {
+                        const RecT first = gather(old - 1);
+                        L::template fold_chain_simple<true>(first, old - 2, staged_levels, gather, r, corr, decay);
+                    }
+                } else {
+                    L::fold_chain_simple(cur.own, old - 1, staged_levels, gather, r, corr, decay);
+                }
                 // The segment's staging is waited for even when it holds nothing: it keeps this warp from running past
                 // the epilogue warps' preparation of the segment after next (whose barriers share these phases).
                 if (!staged_ready && (staged_levels > 0 || seg_last)) {
@@ -530,7 +579,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                     const uint8_t* st = stage + buf * (STAGE_BUF * REC_BYTES);
                     const float2* gs = gates_s + buf * STAGE_BUF;
                     const RecT newest = L::load_shared(st, gs, idx_of(staged_levels - 1), g);
-                    L::fold_chain_simple(newest, staged_levels - 2, 0,
+                    L::template fold_chain_simple<DELTA>(newest, staged_levels - 2, 0,
                                   [&](int level) { return L::load_shared(st, gs, idx_of(level), g); }, r, corr, decay);
                 }
                 if (seg_last) {                    // this warp's last read of the segment's staging buffer
@@ -593,6 +642,13 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                         *reinterpret_cast<float4*>(crow + corr_chunk(2 * ci + 1) * 4) =
                             make_float4(corr[4 * c + 2].x, corr[4 * c + 2].y, corr[4 * c + 3].x, corr[4 * c + 3].y);
                     }
+                }
+                if (DELTA && (grp & 1) == 0) {      // what the epilogue needs to form delta_t and o_t of this beam
+                    uint8_t* ds = delta_s + s * DELTA_SLOT_BYTES;
+                    const int bq = u >> 1;
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) *reinterpret_cast<uint4*>(ds + bq * (DV * 2) + (c * LPU + g) * 16) = cur.own.v[c];
+                    if (g == 0) *reinterpret_cast<float4*>(ds + DELTA_BEAMS * (DV * 2) + bq * 16) = make_float4(cur.own.gate.x, cur.own.gate.y, kq, 0.f);
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
                 __syncwarp();
@@ -733,7 +789,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             if (!fail && !wait_or_abort(bar_done(s), use & 1, abort_flag)) give_up();
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             float* C_s = reinterpret_cast<float*>(ring + s * SLOT_BYTES + R_BYTES);
-            const int b0 = gip * GN;
+            const int b0 = gip * BPG;
             const uint32_t taddr = tmem_base + s * GN + ((uint32_t)(quad * 32) << 16);
             float* A_s = reinterpret_cast<float*>(ring + s * SLOT_BYTES);   // the operand rows are dead once the MMAs have completed
             if (!fail) {
@@ -759,6 +815,46 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                     if (issue_mma(gcount + 1, seg + (next_first ? 1 : 0), next_first)) give_up();   // carried to the next barrier
                     ++issued;
                 }
+            } else if constexpr (DELTA) {
+                // Eq. 2 and 4 on the two projections of each beam (rows 2 j and 2 j + 1 of the tile):
+                //   delta_t = beta_t (v_t - alpha_t S_{t-1} k_t) ,  o_t = alpha_t S_{t-1} q_t + delta_t (k_t . q_t) ;
+                // the output row and the record's delta half (in the record dtype) leave as 16-byte stores
+                const int et = (warp - FOLD_WARPS - 1) * 32 + lane;
+                const uint8_t* ds = delta_s + s * DELTA_SLOT_BYTES;
+                OutT* out0 = static_cast<OutT*>(a.out) + (((long long)req * a.W + b0) * a.H + h) * DV;
+                char* rec0 = a.kv_out + ((long long)h * a.arena_slots + a.bases.base[req] + b0) * REC_BYTES + DK * 2;
+#pragma unroll
+                for (int it = 0; it < DELTA_BEAMS * 16 / 96; ++it) {
+                    const int idx = it * 96 + et, j = idx >> 4, ch = idx & 15;
+                    if (b0 + j < a.W) {
+                        const int c0 = corr_chunk(2 * ch) * 4, c1 = corr_chunk(2 * ch + 1) * 4;
+                        const float wq = inv_s[s * GN + 2 * j], wk = inv_s[s * GN + 2 * j + 1];
+                        const float* Aq = A_s + (2 * j) * DV;
+                        const float* Cq = C_s + (2 * j) * DV;
+                        const float4 aq0 = *reinterpret_cast<const float4*>(Aq + c0), aq1 = *reinterpret_cast<const float4*>(Aq + c1);
+                        const float4 cq0 = *reinterpret_cast<const float4*>(Cq + c0), cq1 = *reinterpret_cast<const float4*>(Cq + c1);
+                        const float4 ak0 = *reinterpret_cast<const float4*>(Aq + DV + c0), ak1 = *reinterpret_cast<const float4*>(Aq + DV + c1);
+                        const float4 ck0 = *reinterpret_cast<const float4*>(Cq + DV + c0), ck1 = *reinterpret_cast<const float4*>(Cq + DV + c1);
+                        const float uq[8] = {fmaf(aq0.x, wq, cq0.x), fmaf(aq0.y, wq, cq0.y), fmaf(aq0.z, wq, cq0.z), fmaf(aq0.w, wq, cq0.w),
+                                             fmaf(aq1.x, wq, cq1.x), fmaf(aq1.y, wq, cq1.y), fmaf(aq1.z, wq, cq1.z), fmaf(aq1.w, wq, cq1.w)};
+                        const float uk[8] = {fmaf(ak0.x, wk, ck0.x), fmaf(ak0.y, wk, ck0.y), fmaf(ak0.z, wk, ck0.z), fmaf(ak0.w, wk, ck0.w),
+                                             fmaf(ak1.x, wk, ck1.x), fmaf(ak1.y, wk, ck1.y), fmaf(ak1.z, wk, ck1.z), fmaf(ak1.w, wk, ck1.w)};
+                        const float4 sc = *reinterpret_cast<const float4*>(ds + DELTA_BEAMS * (DV * 2) + j * 16);     // alpha_t, beta_t, k_t . q_t
+                        float2 vx[4];
+                        unpack8(*reinterpret_cast<const uint4*>(ds + j * (DV * 2) + ch * 16), vx);
+                        const float vv[8] = {vx[0].x, vx[0].y, vx[1].x, vx[1].y, vx[2].x, vx[2].y, vx[3].x, vx[3].y};
+                        float dl[8], o[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            dl[e] = sc.y * fmaf(-sc.x, uk[e], vv[e]);
+                            o[e] = fmaf(dl[e], sc.z, sc.x * uq[e]);
+                        }
+                        store8<OutT>(out0 + (long long)j * a.H * DV + ch * 8, o);
+                        store8<__nv_bfloat16>(reinterpret_cast<__nv_bfloat16*>(rec0 + (long long)j * REC_BYTES + ch * 16), dl);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_free(s));
             } else {
                 // coalesced stores by the other three warps: 16 lanes cover one beam's 128 outputs, 8 elements each
                 const int et = (warp - FOLD_WARPS - 1) * 32 + lane;
@@ -885,9 +981,11 @@ int make_partition(int total_groups, int gpp, int sms, PartitionCost c, Partitio
     return greedy_fill(total_groups, gpp, lo, sms, c, part->begin);
 }
 
-template <typename OutT, bool GROUPED, bool FUSED>
+template <typename OutT, bool GROUPED, bool FUSED, bool DELTA = false>
 cudaError_t launch_ws_t(const DecodeArgs& a, cudaStream_t stream) {
-    auto kern = decode_ws_kernel<OutT, GROUPED, FUSED>;
+    auto kern = decode_ws_kernel<OutT, GROUPED, FUSED, DELTA>;
+    constexpr int SMEM_BYTES = DELTA ? SMEM_BYTES_DELTA : onela::SMEM_BYTES;
+    constexpr int GN = DELTA ? DELTA_BEAMS : onela::GN;      // beams per group (a delta-record group has two rows per beam)
     // One-time set-up per device (function attributes belong to a device's context); host threads may share it.
     constexpr int MAX_DEVICES = 64;
     static std::mutex setup_mutex;
@@ -948,10 +1046,14 @@ bool decode_sm100_supported(int32_t dk, int32_t dv, int32_t rec_dtype) {
     return dk == 128 && dv == 128 && rec_dtype == ONELA_DTYPE_BF16;
 }
 
-cudaError_t launch_decode_sm100_ws(const DecodeArgs& a, int32_t out_dtype, bool grouped, cudaStream_t stream) {
+cudaError_t launch_decode_sm100_ws(const DecodeArgs& a, int32_t out_dtype, bool grouped, bool delta_records, cudaStream_t stream) {
     // one instantiation per (output type, grouped value heads, append fused in): a launch runs only the code it needs
     const bool fused = a.k_in != nullptr;
     const bool bf16 = out_dtype == ONELA_DTYPE_BF16;
+    if (delta_records) {
+        if (grouped || !fused) return cudaErrorInvalidValue;
+        return bf16 ? launch_ws_t<__nv_bfloat16, false, true, true>(a, stream) : launch_ws_t<float, false, true, true>(a, stream);
+    }
     if (grouped) {
         if (fused) return bf16 ? launch_ws_t<__nv_bfloat16, true, true>(a, stream) : launch_ws_t<float, true, true>(a, stream);
         return bf16 ? launch_ws_t<__nv_bfloat16, true, false>(a, stream) : launch_ws_t<float, true, false>(a, stream);

@@ -151,7 +151,8 @@ bool decode_generic_supported(int32_t dk, int32_t dv, int32_t rec_dtype);
 cudaError_t launch_decode_gtr(const DecodeArgs& a, int32_t dk, int32_t dv, int32_t rec_dtype, int32_t out_dtype,
                               bool* supported, cudaStream_t stream);
 bool decode_sm100_supported(int32_t dk, int32_t dv, int32_t rec_dtype);
-cudaError_t launch_decode_sm100_ws(const DecodeArgs& a, int32_t out_dtype, bool grouped, cudaStream_t stream);
+// delta_records: the arena keeps (alpha, delta, k) and the launch replays both projections forward (fused append only)
+cudaError_t launch_decode_sm100_ws(const DecodeArgs& a, int32_t out_dtype, bool grouped, bool delta_records, cudaStream_t stream);
 
 // Contiguous ranges of beam groups, one per CTA of a persistent decode kernel (host-side partitioner in
 // onela_decode_sm100.cu): CTA c works on groups [begin[c], begin[c + 1]).

@@ -201,6 +201,9 @@ struct Lanes {
     }
     // One fold step on this lane's elements (packed fp32x2 FMAs), with the LPU-lane dot reduction:
     //   c~ = k . r~ ;  corr += (decay beta c~) v ;  r~ -= (beta c~) k ;  decay *= alpha
+    // REPLAY (records (alpha, delta, k), Eq. 3): the vector is not changed, the record's second half is the stored
+    // update vector delta, taken with the weight decay * (k . r):   corr += (decay c~) delta ;  decay *= alpha
+    template <bool REPLAY = false>
     static __device__ __forceinline__ void fold_step(const R& rec, float2* r, float2* corr, float& decay) {
         float2 kx[NP2];
 #pragma unroll
@@ -214,11 +217,13 @@ struct Lanes {
         float dot = (d0.x + d0.y) + (d1.x + d1.y);
 #pragma unroll
         for (int o = LPU / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-        const float bc = rec.gate.y * dot;
+        const float bc = REPLAY ? dot : rec.gate.y * dot;
         const float wv = decay * bc;
         const float2 nbc2 = make_float2(-bc, -bc), wv2 = make_float2(wv, wv);
+        if (!REPLAY) {
 #pragma unroll
-        for (int e = 0; e < NP2; ++e) r[e] = __ffma2_rn(kx[e], nbc2, r[e]);
+            for (int e = 0; e < NP2; ++e) r[e] = __ffma2_rn(kx[e], nbc2, r[e]);
+        }
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
             float2 vx[4];
@@ -229,13 +234,13 @@ struct Lanes {
         decay *= rec.gate.x;
     }
     // Single-buffered chain: fetch a record, fold it (for sources whose latency is short, or to save registers).
-    template <class LoadFn>
+    template <bool REPLAY = false, class LoadFn>
     static __device__ __forceinline__ void fold_chain_simple(const R& first, int hi, int lo, LoadFn load, float2* r,
                                                              float2* corr, float& decay) {
-        fold_step(first, r, corr, decay);
+        fold_step<REPLAY>(first, r, corr, decay);
         for (int level = hi; level >= lo; --level) {
             const R rec = load(level);
-            fold_step(rec, r, corr, decay);
+            fold_step<REPLAY>(rec, r, corr, decay);
         }
     }
 };

@@ -21,10 +21,13 @@ pytestmark = pytest.mark.gpu
 CFG0, CFG1 = inputs.WORKLOADS[0], inputs.WORKLOADS[1]
 
 
-def _check(case, out_dtype, tight=None, batched=True):
+def _check(case, out_dtype, tight=None, batched=True, cuda_cores=False):
     ref, chains = run_oracle(case)
-    outs, slots, ctx = run_library(case, out_dtype=out_dtype, flags=P.FLAG_GTR_DELTA, batched=batched, fused=True)
-    assert not ctx.onela_uses_tensor_core_path()
+    wl = case["wl"]
+    flags = P.FLAG_GTR_DELTA | (P.FLAG_FORCE_GENERIC if cuda_cores else 0)
+    outs, slots, ctx = run_library(case, out_dtype=out_dtype, flags=flags, batched=batched, fused=True)
+    # 128 x 128 bf16 records: both projections of the parent state run on the tensor cores
+    assert ctx.onela_uses_tensor_core_path() == ((wl.dk, wl.dv, wl.dtype) == (128, 128, "bf16") and not cuda_cores)
     want = expected_slots(case, chains)
     for key in want:
         assert np.array_equal(slots[key], want[key]), f"ancestry rows of {key} differ"
@@ -38,9 +41,18 @@ def test_config0_fp32_records_are_tight():
     assert worst > 0.0
 
 
+@pytest.mark.parametrize("cuda_cores", [False, True])
 @pytest.mark.parametrize("out_dtype", ["fp32", "bf16"])
-def test_config1_bf16_records(out_dtype):
-    _check(make_case(CFG1), out_dtype)
+def test_config1_bf16_records(out_dtype, cuda_cores):
+    _check(make_case(CFG1), out_dtype, cuda_cores=cuda_cores)
+
+
+def test_bf16_records_ragged_beams_many_segments():
+    """Widths that leave the last 24-beam group ragged, several (request, head) segments per CTA, two layers."""
+    wl = CFG1.scaled(R=5, L=2, H=7, W=61, D=5, prompt_len=48, parents="zipf", zipf_s=1.4, seed=64)
+    _check(make_case(wl), "bf16")
+    wl = CFG1.scaled(R=1, L=1, H=2, W=25, D=3, prompt_len=48, seed=65)
+    _check(make_case(wl, widths=[25, 1, 24]), "fp32", batched=False)
 
 
 def test_fp32_records_other_shapes_and_ragged_widths():
@@ -53,6 +65,8 @@ def test_fp32_records_other_shapes_and_ragged_widths():
 def test_bf16_records_deep_chain_with_shared_ancestors():
     wl = CFG1.scaled(R=2, H=4, W=96, D=8, prompt_len=128, parents="zipf", zipf_s=1.5, seed=63)
     worst, _ = _check(make_case(wl), "fp32")
+    assert worst <= REL_L2_BAR
+    worst, _ = _check(make_case(wl), "fp32", cuda_cores=True)
     assert worst <= REL_L2_BAR
 
 
@@ -91,6 +105,45 @@ def test_stored_records_are_key_bytes_and_update_vectors():
                 assert np.linalg.norm(got - delta) <= 2e-5 * max(np.linalg.norm(delta), 1e-3), (t, b, h)
                 assert torch.equal(kv[h, base + b, :128], tk["k"][b, h])
                 assert float(gates[h, base + b, 0]) == a_
+            new[b] = S_new
+        prev = new
+
+
+def test_tensor_core_kernel_stores_key_bytes_and_rounded_update_vectors():
+    """The same check for bf16 records, whose launches run on the tensor cores: the key half bit for bit, the delta half
+    within bf16 rounding of beta_t (v_t - alpha_t S_{t-1} k_t) (states from the fp64 recurrence on the stored inputs)."""
+    wl = CFG1.scaled(R=1, H=2, W=30, D=3, prompt_len=32, seed=66)
+    case = make_case(wl)
+    outs, slots, ctx = run_library(case, out_dtype="fp32", flags=P.FLAG_GTR_DELTA, fused=True)
+    assert ctx.onela_uses_tensor_core_path()
+    c = ctx.cfg
+    al = lambda n: (n + 1023) // 1024 * 1024
+    n_idx = c.num_requests * c.max_steps * c.max_beam * 4
+    off_s0 = al(16) + al(2 * n_idx) + al(n_idx) + al(n_idx) + al(c.num_requests * (c.max_steps + 1) * 4)
+    off_gates = off_s0 + al(c.num_requests * c.num_layers * c.num_heads * c.dv * c.dk * 4)
+    off_kv = off_gates + al(c.num_layers * c.num_heads * c.arena_slots * 8)
+    ws = ctx.workspace[ctx.workspace_ptr - ctx.workspace.data_ptr():]
+    gates = ws[off_gates:off_gates + c.num_heads * c.arena_slots * 8].view(torch.float32).view(c.num_heads, c.arena_slots, 2).cpu()
+    kv = ws[off_kv:off_kv + c.num_heads * c.arena_slots * 512].view(torch.bfloat16).view(c.num_heads, c.arena_slots, 256).cpu()
+    S0 = case["S0"][(0, 0)].double().numpy()
+    prev = None
+    for t in range(wl.D):
+        tk = case["tok"][(0, 0, t)]
+        par = case["parents"][(0, t)]
+        base = ctx.onela_get_step_base(0, t)
+        new = {}
+        for b in range(wl.W):
+            S_par = S0 if t == 0 else prev[int(par[b])]
+            S_new = np.empty_like(S_par)
+            for h in range(wl.H):
+                k = tk["k"][b, h].double().numpy(); v = tk["v"][b, h].double().numpy()
+                a_, b_ = float(tk["alpha"][b, h]), float(tk["beta"][b, h])
+                delta = b_ * (v - a_ * (S_par[h] @ k))
+                S_new[h] = a_ * S_par[h] + np.outer(delta, k)
+                got = kv[h, base + b, 128:].double().numpy()
+                assert np.linalg.norm(got - delta) <= 8e-3 * max(np.linalg.norm(delta), 1e-3), (t, b, h)
+                assert torch.equal(kv[h, base + b, :128], tk["k"][b, h])
+                assert float(gates[h, base + b, 0]) == a_ and float(gates[h, base + b, 1]) == b_
             new[b] = S_new
         prev = new
 

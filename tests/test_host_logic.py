@@ -147,7 +147,9 @@ def test_delta_record_mode_takes_only_the_fused_call():
         with raises(binding.E_UNSUPPORTED):
             P.Onela(bad, device="cpu")
     tc = P.make_config(1, 1, 2, 128, 128, 8, 3, "bf16", "bf16", 64, P.FLAG_DRY_RUN | P.FLAG_GTR_DELTA)
-    assert not P.Onela(tc, device="cpu").onela_uses_tensor_core_path()
+    assert P.Onela(tc, device="cpu").onela_uses_tensor_core_path()        # 128 x 128 bf16: the tcgen05 kernel replays too
+    cc = P.make_config(1, 1, 2, 128, 128, 8, 3, "bf16", "bf16", 64, P.FLAG_DRY_RUN | P.FLAG_GTR_DELTA | P.FLAG_FORCE_GENERIC)
+    assert not P.Onela(cc, device="cpu").onela_uses_tensor_core_path()
 
 
 def test_select_beams_argument_checks():
