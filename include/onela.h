@@ -85,7 +85,8 @@ typedef int32_t onela_status;
  * projection accumulators S q_t and S k_t forward from S_0 through the beam's records (oldest first).  delta_t
  * depends on the parent state, so records can only be produced where the replay runs: in this mode
  * onela_append_decode_step is the one call per layer and decode call; onela_append_records and onela_decode_step
- * return ONELA_E_UNSUPPORTED.  dk == dv in {32, 64, 128}; CUDA cores only.  Later calls replay the ROUNDED
+ * return ONELA_E_UNSUPPORTED.  dk == dv in {32, 64, 128}; 128 x 128 with bf16 records runs on the tensor cores (both
+ * projections S q_t and S k_t of a beam go through S_0 in one MMA set), the rest on CUDA cores.  Later calls replay the ROUNDED
  * delta, so with bf16 records the result drifts from the exact recurrence by about one bf16 rounding per record
  * (the default raw-record format has no such term). */
 #define ONELA_FLAG_GTR_DELTA 4u
@@ -101,8 +102,9 @@ typedef struct onela_config {
     int32_t num_layers;   /* GDN layers sharing the ancestry index */
     int32_t num_heads;    /* key heads (and value heads, unless num_v_heads says otherwise) */
     int32_t dk, dv;       /* head dimensions of k/q and of v/o: (32, 32), (64, 64), (128, 128), (128, 256), (256, 256),
-                           * (128, 512) or (256, 512), else ONELA_E_UNSUPPORTED; 128 x 128 with bf16 records runs on
-                           * the tensor-core kernel, every other shape on CUDA cores */
+                           * (128, 512) or (256, 512), else ONELA_E_UNSUPPORTED; dk = 128 with bf16 records runs on
+                           * the tensor-core kernel at every value width (dv = 256 / 512 as two / four tiles of 128
+                           * outputs that share the key head's fold), every other shape on CUDA cores */
     int32_t max_beam;     /* largest beam width W_t */
     int32_t max_steps;    /* largest number of decode calls per request (chain depth) */
     int32_t rec_dtype;    /* dtype of q, k, v: ONELA_DTYPE_* */
@@ -114,8 +116,8 @@ typedef struct onela_config {
      * states, values, gates and outputs are per value head.  Then q, k are [..][num_heads][dk]; v, alpha, beta, out
      * and S_0 are [..][num_v_heads][..]; a record keeps k once per key head and (v, alpha, beta) per value head
      * (num_heads * dk + num_v_heads * (dv + 8 bytes of gates) per slot instead of num_v_heads * (dk + dv + ..)).
-     * (dk, dv) in {(64, 64), (128, 128), (128, 256)}: 128 x 128 bf16 on the tensor-core kernel, the rest on CUDA
-     * cores; onela_prefill_shared_state and ONELA_FLAG_GTR_DELTA are not available (ONELA_E_UNSUPPORTED). */
+     * (dk, dv) in {(64, 64), (128, 128), (128, 256)}: dk = 128 with bf16 records on the tensor-core kernel, the rest
+     * on CUDA cores; onela_prefill_shared_state and ONELA_FLAG_GTR_DELTA are not available (ONELA_E_UNSUPPORTED). */
     int32_t num_v_heads;
 } onela_config;
 

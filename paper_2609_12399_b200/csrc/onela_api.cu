@@ -495,14 +495,20 @@ onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count,
     a.v_in = v_dev;
     a.alpha_in = alpha_dev;
     a.beta_in = beta_dev;
+    // The tensor-core kernel works on value heads of 128 outputs: a wider value head is cut into tiles = dv / 128 of
+    // them (its instantiation for grouped value heads serves both), addressed through per-slot strides.
+    const int tiles = ctx->tensor_core ? c.dv / 128 : 1;
     a.kv_out = ctx->grouped() ? ctx->k_plane(layer) : ctx->kv_plane(layer);
-    a.vv_out = ctx->grouped() ? ctx->v_plane(layer) : nullptr;
+    a.vv_out = ctx->grouped() ? ctx->v_plane(layer) : (tiles > 1 ? a.kv_out + (size_t)c.dk * ctx->elem_bytes : nullptr);
     a.gates_out = ctx->gate_plane(layer);
     a.s0 = ctx->s0_slot(req_begin, layer);
     a.kv = a.kv_out;
     a.vv = a.vv_out;
     a.Hk = c.num_heads;
-    a.g = ctx->Hv() / c.num_heads;
+    a.g = ctx->Hv() / c.num_heads * tiles;
+    a.tiles = tiles;
+    a.k_stride = (long long)(ctx->grouped() ? c.dk : c.dk + c.dv) * ctx->elem_bytes;
+    a.v_stride = (long long)(ctx->grouped() ? c.dv : c.dk + c.dv) * ctx->elem_bytes;
     a.gates = ctx->gate_plane(layer);
     a.table = ctx->table_cur(req_begin);
     a.status = ctx->lay.status;
@@ -524,17 +530,17 @@ onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count,
     a.uoff_req_stride = ctx->uoff_req_stride();
     a.req_count = req_count;
     a.W = W;
-    a.H = ctx->Hv();
+    a.H = ctx->Hv() * tiles;
     a.depth = depth;
     a.max_beam = c.max_beam;
     for (int i = 0; i < req_count; ++i) a.bases.base[i] = ctx->req[req_begin + i].step_base.back();
     a.early_ok = ctx->launches == ctx->decode_mark ? 1 : 0;
     bool supported = true;
-    const bool wy = ctx->tensor_core && !ctx->gtr() && (c.flags & ONELA_FLAG_SHARED_CHAINS) && !ctx->grouped() && depth >= 2 &&
+    const bool wy = ctx->tensor_core && !ctx->gtr() && (c.flags & ONELA_FLAG_SHARED_CHAINS) && !ctx->grouped() && tiles == 1 && depth >= 2 &&
                     depth <= WY_MAX_LEVELS + 1;
     const cudaError_t e = ctx->gtr() && !ctx->tensor_core ? launch_decode_gtr(a, c.dk, c.dv, c.rec_dtype, c.out_dtype, &supported, s)
                           : wy               ? launch_decode_wy(a, c.out_dtype, s)
-                          : ctx->tensor_core ? launch_decode_sm100_ws(a, c.out_dtype, ctx->grouped(), ctx->gtr(), s)
+                          : ctx->tensor_core ? launch_decode_sm100_ws(a, c.out_dtype, ctx->grouped() || tiles > 1, ctx->gtr(), s)
                                              : launch_decode_generic(a, c.dk, c.dv, c.rec_dtype, c.out_dtype, &supported, s);
     if (!supported) return ONELA_E_UNSUPPORTED;
     if (e != cudaSuccess) return ONELA_E_CUDA;

@@ -199,15 +199,19 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     const char* kv = a.kv;
     const __nv_bfloat16* qbase = static_cast<const __nv_bfloat16*>(a.q);
     // rows of the caller's tensors: q and k have one row per KEY head, v, the gates and the outputs per VALUE head
+    // GROUPED also serves value widths of 256 and 512: a value head is cut into a.tiles value heads of 128 outputs
+    // ("tiles") that share its gates and its S_0 scale; value_head(h) is the head a tile belongs to.
     auto key_head = [&](int h) { return GROUPED ? h / a.g : h; };
+    auto value_head = [&](int h) { return GROUPED ? h / a.tiles : h; };
     auto krow_in = [&](int req, int bb, int h) { return ((long long)req * a.W + bb) * (GROUPED ? a.Hk : a.H) + key_head(h); };
     auto vrow_in = [&](int req, int bb, int h) { return ((long long)req * a.W + bb) * a.H + h; };
     // rows of the arena: ungrouped one 512-byte row (k | v) per (head, slot); grouped a 256-byte row in each plane
     auto k_at = [&](int h, long long slot) {
-        return GROUPED ? kv + ((long long)key_head(h) * a.arena_slots + slot) * (DK * 2) : kv + ((long long)h * a.arena_slots + slot) * REC_BYTES;
+        return GROUPED ? kv + ((long long)key_head(h) * a.arena_slots + slot) * a.k_stride : kv + ((long long)h * a.arena_slots + slot) * REC_BYTES;
     };
     auto v_at = [&](int h, long long slot) {
-        return GROUPED ? a.vv + ((long long)h * a.arena_slots + slot) * (DV * 2) : kv + ((long long)h * a.arena_slots + slot) * REC_BYTES + DK * 2;
+        return GROUPED ? a.vv + ((long long)value_head(h) * a.arena_slots + slot) * a.v_stride + (h - value_head(h) * a.tiles) * (DV * 2)
+                       : kv + ((long long)h * a.arena_slots + slot) * REC_BYTES + DK * 2;
     };
     const int grp = lane / LPU, g = lane % LPU;
     bool dead = false;                    // this warp gave up (timeout or abort raised elsewhere)
@@ -222,7 +226,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         const int quad = warp & 3, i = quad * 32 + lane;
         const int req = pair_now / a.H, h = pair_now - req * a.H;
         const float* row = a.s0 + req * a.s0_req_stride + (long long)h * (DV * DK) + (long long)i * DK;
-        const float sc = __ldg(a.s0_scale + req * a.s0_scale_req_stride + h);
+        const float sc = __ldg(a.s0_scale + req * a.s0_scale_req_stride + value_head(h));
 #pragma unroll 1
         for (int kb = kb0; kb < 4; kb += step) {
             uint32_t v[16];
@@ -251,7 +255,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     float s0_first_scale = 1.f;
     if (n_segs > 0 && s0_mine) {
         const int req = pair_begin / a.H, h = pair_begin - req * a.H;
-        s0_first_scale = __ldg(a.s0_scale + req * a.s0_scale_req_stride + h);
+        s0_first_scale = __ldg(a.s0_scale + req * a.s0_scale_req_stride + value_head(h));
         const float* row = a.s0 + req * a.s0_req_stride + (long long)h * (DV * DK) + (long long)((warp & 3) * 32 + lane) * DK + (warp >> 2) * 32;
 #pragma unroll
         for (int c = 0; c < 8; ++c) s0_first[c] = __ldg(reinterpret_cast<const float4*>(row) + c);
@@ -370,8 +374,8 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         };
         auto load_gate = [&](const Unit& u) {
             const int bb = live_beam(u);
-            if (!fused) return __ldg(a.gates + (long long)u.h * a.arena_slots + a.bases.base[u.req] + bb);
-            const long long in_row = vrow_in(u.req, bb, u.h);
+            if (!fused) return __ldg(a.gates + (long long)value_head(u.h) * a.arena_slots + a.bases.base[u.req] + bb);
+            const long long in_row = GROUPED ? ((long long)u.req * a.W + bb) * (a.H / a.tiles) + value_head(u.h) : vrow_in(u.req, bb, u.h);
             return make_float2(__ldg(a.alpha_in + in_row), __ldg(a.beta_in + in_row));
         };
         // staging layout of the request whose quads are being looked at (the same for all heads of a request)
@@ -426,8 +430,8 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                     staged_levels = staged_levels_of(u0.req);
                     // levels gathered from global memory whose lines are worth requesting ahead (end of the loop)
                     if (AHEAD) n_ahead = (info_sparse >> staged_levels) ? min(old - staged_levels, NIDX * LPU - staged_levels) : 0;
-                    seg_inv_s0 = 1.f / __ldg(a.s0_scale + u0.req * a.s0_scale_req_stride + u0.h);   // a power of two
-                    plane_row0 = (long long)u0.h * a.arena_slots;
+                    seg_inv_s0 = 1.f / __ldg(a.s0_scale + u0.req * a.s0_scale_req_stride + value_head(u0.h));   // a power of two
+                    plane_row0 = (long long)value_head(u0.h) * a.arena_slots;      // row 0 of the head's gate plane
                     own_row0 = plane_row0 + a.bases.base[u0.req];
                     table_r = a.table + u0.req * a.table_req_stride;
                     sidx_r = a.sidx + u0.req * a.sidx_req_stride;
@@ -462,11 +466,11 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                     } else if (fused && beam_of(u0) < a.W) {   // the append: this beam's record goes to its arena slot, bit for bit
                         if constexpr (GROUPED) {
                             const long long slot = a.bases.base[u0.req] + bb;
-                            uint4* vdst = reinterpret_cast<uint4*>(a.vv_out + ((long long)u0.h * a.arena_slots + slot) * (DV * 2)) + g;
+                            uint4* vdst = reinterpret_cast<uint4*>(a.vv_out + (v_at(u0.h, slot) - a.vv)) + g;
 #pragma unroll
                             for (int c = 0; c < NCH; ++c) vdst[c * LPU] = cur.own.v[c];
                             if (u0.h % a.g == 0) {     // the key is stored once per key head: by its first value head
-                                uint4* kdst = reinterpret_cast<uint4*>(a.kv_out + ((long long)key_head(u0.h) * a.arena_slots + slot) * (DK * 2)) + g;
+                                uint4* kdst = reinterpret_cast<uint4*>(a.kv_out + (k_at(u0.h, slot) - kv)) + g;
 #pragma unroll
                                 for (int c = 0; c < NCH; ++c) kdst[c * LPU] = cur.own.k[c];
                             }
@@ -478,7 +482,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                                 dst[16 + c * LPU] = cur.own.v[c];
                             }
                         }
-                        if (g == 0) a.gates_out[own_row0 + bb] = gate0;
+                        if (g == 0 && (!GROUPED || u0.h % a.tiles == 0)) a.gates_out[own_row0 + bb] = gate0;
                     }
                 }
                 gate0 = gate1;
@@ -706,7 +710,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             const int b = single ? 0 : (seg & 1);
             int levels, count;
             staging_of(req, levels, count);
-            const long long plane_row0 = (long long)h * a.arena_slots;
+            const long long plane_row0 = (long long)value_head(h) * a.arena_slots;
             const int li = (warp - FOLD_WARPS) * 32 + lane;
             if (li < count) {
                 const long long slot = __ldg(a.ulist + req * a.ulist_req_stride + li), row = plane_row0 + slot;
@@ -1043,7 +1047,8 @@ int make_decode_partition(int total_groups, int groups_per_pair, int sms, int gr
 int decode_sm_count() { return sm_count_ws(); }
 
 bool decode_sm100_supported(int32_t dk, int32_t dv, int32_t rec_dtype) {
-    return dk == 128 && dv == 128 && rec_dtype == ONELA_DTYPE_BF16;
+    // value widths of 256 and 512 run as two or four value heads of 128 outputs that share the key head's fold
+    return dk == 128 && (dv == 128 || dv == 256 || dv == 512) && rec_dtype == ONELA_DTYPE_BF16;
 }
 
 cudaError_t launch_decode_sm100_ws(const DecodeArgs& a, int32_t out_dtype, bool grouped, bool delta_records, cudaStream_t stream) {

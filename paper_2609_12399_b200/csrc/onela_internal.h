@@ -69,6 +69,11 @@ struct DecodeArgs {
     const char* vv;
     char* vv_out;
     int32_t Hk, g;
+    // ... and value widths of 256 / 512 (grouped or not): every value head is cut into `tiles` heads of 128 outputs, so
+    // H = tiles * (value heads) and g = tiles * (value heads per key head); k_stride / v_stride: bytes between
+    // consecutive slots of a key head's keys and of a value head's values (from kv and vv: one interleaved plane or two)
+    int32_t tiles;
+    long long k_stride, v_stride;
     // tensor-core kernel: per-head operand scale of S_0 (see Layout), entry of (req_begin, layer, head 0)
     const float* s0_scale;
     long long s0_scale_req_stride;

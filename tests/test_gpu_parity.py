@@ -150,7 +150,51 @@ def test_depth_one_and_max_depth():
                                          (256, 256, "bf16"), (32, 32, "bf16"), (128, 512, "bf16"), (256, 512, "bf16")])
 def test_other_geometries(dk, dv, dtype):
     wl = CFG1.scaled(H=2, dk=dk, dv=dv, dtype=dtype, W=37, D=3, prompt_len=48, seed=dk + dv)
-    _full_check(make_case(wl), "fp32")
+    _, ctx = _full_check(make_case(wl), "fp32")
+    # key width 128 with bf16 records runs on the tensor cores at every value width (256 and 512 as two and four
+    # value tiles of 128 outputs); the other shapes on the CUDA-core kernel
+    assert bool(ctx.onela_uses_tensor_core_path()) == (dk == 128 and dtype == "bf16")
+
+
+@pytest.mark.parametrize("dv", [256, 512])
+@pytest.mark.parametrize("fused,out_dtype", [(True, "bf16"), (False, "fp32")])
+def test_wide_values_on_the_tensor_cores(dv, fused, out_dtype):
+    """Value widths 256 and 512 (Section 4.1's operator suite) on the tcgen05 kernel: deeper chains with shared ancestors,
+    several requests and layers, ragged beams; the arena rows hold the appended bytes; and the CUDA-core kernel, which
+    shares no device code, agrees on every unit."""
+    wl = CFG1.scaled(R=2, L=2, H=3, dk=128, dv=dv, W=77, D=5, prompt_len=48, parents="zipf", zipf_s=1.4, seed=900 + dv)
+    case = make_case(wl)
+    ref, chains = run_oracle(case)
+    outs, slots, ctx = run_library(case, out_dtype=out_dtype, fused=fused)
+    assert ctx.onela_uses_tensor_core_path() and ctx.onela_poll_device_status() == (0, 0)
+    check_parity(case, outs, ref)
+    outs_cc, _, ctx_cc = run_library(case, out_dtype=out_dtype, flags=P.FLAG_FORCE_GENERIC, fused=fused)
+    assert not ctx_cc.onela_uses_tensor_core_path()
+    for key in outs:
+        assert rel_l2(outs[key].numpy(), outs_cc[key].double().numpy()).max() <= REL_L2_BAR
+    # the arena rows [k | v] of the last layer, byte for byte
+    c = ctx.cfg
+    al = lambda n: (n + 1023) // 1024 * 1024
+    n_idx = c.num_requests * c.max_steps * c.max_beam * 4
+    off_s0 = al(16) + al(2 * n_idx) + al(n_idx) + al(n_idx) + al(c.num_requests * (c.max_steps + 1) * 4)
+    off_gates = off_s0 + al(c.num_requests * c.num_layers * c.num_heads * c.dv * c.dk * 4)
+    off_kv = off_gates + al(c.num_layers * c.num_heads * c.arena_slots * 8)
+    ws = ctx.workspace[ctx.workspace_ptr - ctx.workspace.data_ptr():]
+    row = 128 + dv
+    lay = wl.L - 1
+    g0 = off_gates + lay * c.num_heads * c.arena_slots * 8
+    k0 = off_kv + lay * c.num_heads * c.arena_slots * row * 2
+    gates = ws[g0:g0 + c.num_heads * c.arena_slots * 8].view(torch.float32).view(c.num_heads, c.arena_slots, 2).cpu()
+    kv = ws[k0:k0 + c.num_heads * c.arena_slots * row * 2].view(torch.bfloat16).view(c.num_heads, c.arena_slots, row).cpu()
+    for r in range(wl.R):
+        for t in range(wl.D):
+            base = ctx.onela_get_step_base(r, t)
+            tk = case["tok"][(r, lay, t)]
+            for h in range(wl.H):
+                assert torch.equal(kv[h, base:base + wl.W, :128], tk["k"][:, h])
+                assert torch.equal(kv[h, base:base + wl.W, 128:], tk["v"][:, h])
+                assert torch.equal(gates[h, base:base + wl.W, 0], tk["alpha"][:, h])
+                assert torch.equal(gates[h, base:base + wl.W, 1], tk["beta"][:, h])
 
 
 def test_alpha1_beta0_reduces_to_matvec_on_gpu():
