@@ -46,12 +46,13 @@ def build_testhooks(force: bool = False) -> Path:
     return build(force=force, lib=TESTHOOKS_LIB, obj_dir=PKG / "build_testhooks", extra=TESTHOOKS_FLAGS)
 
 
-# A third one for looking INSIDE the shared-chains kernel: clock stamps of CTA 0's role milestones (wy_timeline.py).
+# A third one for looking INSIDE the two tensor-core decode kernels: clock stamps of CTA 0's role milestones
+# (timeline.py).
 TIMELINE_LIB = PKG / "libonela_timeline.so"
 
 
 def build_timeline(force: bool = False) -> Path:
-    return build(force=force, lib=TIMELINE_LIB, obj_dir=PKG / "build_timeline", extra=["-DONELA_WY_TL"])
+    return build(force=force, lib=TIMELINE_LIB, obj_dir=PKG / "build_timeline", extra=["-DONELA_WY_TL", "-DONELA_WS_TL"])
 
 
 def build(force: bool = False, verbose: bool = False, lib: Path = LIB, obj_dir: Path = OBJ, extra=()) -> Path:

@@ -74,7 +74,12 @@ constexpr int STAGE_BUF = ONELA_STAGE_BUF;
 constexpr int STAGE_BYTES = 2 * STAGE_BUF * REC_BYTES;
 constexpr int GATE_BYTES = (2 * STAGE_BUF * 8 + 127) & ~127;   // padded: the heads' stages behind it stay 128-byte aligned (measured: 1.5 % faster)
 constexpr int INV_BYTES = SLOTS * GN * 4;        // per ring slot and beam: what undoes the operands' scales
-constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + STAGE_BYTES + GATE_BYTES + HEADS_TOTAL + 256 + INV_BYTES + 1024;
+#ifdef ONELA_WS_TL
+constexpr int TL_EXTRA = 3 * 200 * 8;
+#else
+constexpr int TL_EXTRA = 0;
+#endif
+constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + STAGE_BYTES + GATE_BYTES + HEADS_TOTAL + 256 + INV_BYTES + 1024 + TL_EXTRA;
 // DELTA instantiation (records (alpha, delta, k), forward projection replay): a beam owns TWO rows of a group - its
 // query and its own key, both projected through the parent state - so a group holds GN / 2 beams; per ring slot the
 // beams' own value rows (raw) and three scalars each (alpha_t, beta_t, k_t . q_t) wait for the epilogue.
@@ -94,6 +99,24 @@ static_assert(GN % 16 == 0 && GN >= 16 && GN <= 256, "MMA N");
 static_assert((GN * 16) % 96 == 0, "three storing warps share a group's 16-byte chunks evenly");
 using L = Lanes<LPU>;
 using RecT = L::R;
+
+#ifdef ONELA_WS_TL
+// Debug builds only (the timeline library; never compiled into the product): clock stamps of CTA 0's role milestones,
+// kept in shared memory and written out when the CTA ends.  Roles: fold warp 0, the issuing epilogue warp, a storing one.
+constexpr int TL_CAP = 200;
+__device__ unsigned long long g_ws_tl[3 * TL_CAP];
+__device__ int g_ws_tl_n[3];
+#define TL(ev, g)                                                                                         \
+    do {                                                                                                  \
+        if (lane == 0 && tl_role >= 0 && tl_n < TL_CAP)                                                   \
+            tl_s[tl_role * TL_CAP + tl_n++] = ((unsigned long long)(ev) << 56) | ((unsigned long long)((g) & 0xff) << 48) | \
+                                              ((unsigned long long)clock64() & 0xffffffffffffull);         \
+    } while (0)
+constexpr int TL_BYTES = 3 * TL_CAP * 8;
+#else
+#define TL(ev, g) do { } while (0)
+constexpr int TL_BYTES = 0;
+#endif
 
 #ifdef ONELA_TEST_HOOKS
 // Test-hooks build only (a second library that the product never loads): when set, the first fold warp of CTA 0
@@ -153,6 +176,11 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     float* inv_s = reinterpret_cast<float*>(heads + HEADS_TOTAL + 256);      // [SLOTS][GN]
     uint8_t* delta_s = heads + HEADS_TOTAL + 256 + INV_BYTES;                // DELTA: [SLOTS][value rows | scalars]
+#ifdef ONELA_WS_TL
+    unsigned long long* tl_s = reinterpret_cast<unsigned long long*>(delta_s + (DELTA ? SLOTS * DELTA_SLOT_BYTES : 0));
+    const int tl_role = blockIdx.x != 0 ? -1 : warp == 0 ? 0 : warp == FOLD_WARPS ? 1 : warp == FOLD_WARPS + 1 ? 2 : -1;
+    int tl_n = 0;
+#endif
     constexpr int BPG = DELTA ? DELTA_BEAMS : GN;                            // beams per group
     static_assert(!DELTA || (FUSED && !GROUPED), "delta records come with the append fused in, ungrouped");
     auto bar_s0 = [&](int b) { return smem_u32(bars + b); };
@@ -188,6 +216,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next launch may set itself up under this one
+    TL(1, 0);   // tensor memory allocated, barriers ready
 
     const int g_begin = part.begin[blockIdx.x], g_end = part.begin[blockIdx.x + 1];
     const int pair_begin = g_begin / groups_per_pair;
@@ -412,7 +441,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             if (1 < n_quads) gate1 = load_gate(u1);
             idx_next = load_idx(u0);
         }
+        TL(2, 0);   // dependencies waited for, first heads requested
         put_first_s0();
+        TL(3, 0);   // first S_0 in tensor memory
         int cur_seg = -1, buf = 0, staged_levels = 0, n_ahead = 0;
         float seg_inv_s0 = 1.f;
         bool staged_ready = false;
@@ -442,7 +473,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 const int bb = live_beam(u0);
                 Head cur;
                 {
+                    TL(10, k);  // fold: quad start
                     asm volatile("cp.async.wait_group 0;" ::: "memory");
+                    TL(11, k);  // fold: heads landed
                     const uint4* rec = reinterpret_cast<const uint4*>(my_heads + grp * REC_BYTES) + g;
                     const uint4* qv = reinterpret_cast<const uint4*>(my_heads + UPW * REC_BYTES + grp * (DK * 2)) + g;
 #pragma unroll
@@ -592,7 +625,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 }
 
                 // the slot must have been handed back by the epilogue of its previous use
+                TL(12, k);  // fold: folded
                 if (use > 0 && !wait_or_abort(bar_free(s), (use - 1) & 1, abort_flag)) { dead = true; break; }
+                TL(13, k);  // fold: slot free
                 uint8_t* R_s = ring + s * SLOT_BYTES;
                 float* C_s = reinterpret_cast<float*>(R_s + R_BYTES);
                 {
@@ -660,6 +695,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 if (g_hook_drop_full_arrival && blockIdx.x == 0 && warp == 0 && k == 0) continue;
 #endif
                 if (lane == 0) mbar_arrive(bar_full(s));
+                TL(14, k);  // fold: rows written
 
                 // The next quad's records of the levels that are NOT staged are gathered from global memory in the middle
                 // of its dependent chain.  Where a level has little sharing (most of its records are used by one or two
@@ -747,7 +783,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             const int s = gcount % SLOTS, use = gcount / SLOTS;
             int mma_failed = 0;
             if (lane == 0) {
+                TL(20, gcount);  // issue: waiting for the rows
                 bool ok = wait_or_abort(bar_full(s), use & 1, abort_flag);
+                TL(21, gcount);  // issue: rows complete
                 // segment 0's S_0 has a barrier of its own; segment seg >= 1 is use ((seg + 1) >> 1) - 1 of its
                 // buffer's barrier
                 if (ok && seg_first && seg >= 1) ok = wait_or_abort(bar_s0(seg & 1), (((seg + 1) >> 1) - 1) & 1, abort_flag);
@@ -767,6 +805,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                     mma_failed = 1;
                 }
                 umma_commit(bar_done(s));   // arrives when the MMAs above have completed
+                TL(22, gcount);  // issue: MMAs out
             }
             return __shfl_sync(0xffffffffu, mma_failed, 0) != 0;
         };
@@ -790,7 +829,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 if (issue_mma(gcount, seg, seg_first)) give_up();
                 ++issued;
             }
+            TL(30, gcount);  // epilogue: waiting for the accumulators
             if (!fail && !wait_or_abort(bar_done(s), use & 1, abort_flag)) give_up();
+            TL(31, gcount);  // epilogue: accumulators complete
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             float* C_s = reinterpret_cast<float*>(ring + s * SLOT_BYTES + R_BYTES);
             const int b0 = gip * BPG;
@@ -809,6 +850,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             }
             // the four epilogue warps: tile complete - or somebody gave up, and then all four leave here together
             if (bar_or(1, 128, fail ? 1 : 0)) { dead = true; break; }
+            TL(32, gcount);  // epilogue: tile transposed
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             if (warp == FOLD_WARPS) {
                 // This warp's part of the slot is read out; the next group's MMAs go out now - unless that group
@@ -883,6 +925,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 if (lane == 0) mbar_arrive(bar_free(s));
             }
 
+            TL(33, gcount);  // epilogue: group stored / next group issued
             // Past the first group of segment seg >= 1 every MMA of segment seg - 1 has completed and the fold warps
             // have read its staging buffer out (they signal that): both are free for segment seg + 1.  (More groups
             // follow, so a warp that gives up here meets the others at the next iteration's barrier.)
@@ -914,6 +957,13 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
         if (atomicCAS(a.status, ONELA_OK, ONELA_E_TIMEOUT) == ONELA_OK) a.status[1] = (int32_t)blockIdx.x;
     }
 
+#ifdef ONELA_WS_TL
+    TL(40, 0);  // role done
+    if (lane == 0 && tl_role >= 0) {
+        for (int i = 0; i < tl_n; ++i) g_ws_tl[tl_role * TL_CAP + i] = tl_s[tl_role * TL_CAP + i];
+        g_ws_tl_n[tl_role] = tl_n;
+    }
+#endif
     // nor with the fold warps' own async copies in flight
     asm volatile("cp.async.wait_all;" ::: "memory");
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -1034,6 +1084,17 @@ cudaError_t launch_ws_t(const DecodeArgs& a, cudaStream_t stream) {
 }
 
 }  // namespace
+
+#ifdef ONELA_WS_TL
+extern "C" int onela_debug_ws_timeline(unsigned long long* out_host, int* counts_host) {
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(counts_host, g_ws_tl_n, 3 * sizeof(int));
+    cudaMemcpyFromSymbol(out_host, g_ws_tl, sizeof(unsigned long long) * 3 * TL_CAP);
+    const int zero[3] = {0, 0, 0};
+    cudaMemcpyToSymbol(g_ws_tl_n, zero, sizeof(zero));
+    return TL_CAP;
+}
+#endif
 
 #ifdef ONELA_TEST_HOOKS
 extern "C" int onela_testhook_drop_full_arrival(int on) {
