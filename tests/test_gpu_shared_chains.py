@@ -70,3 +70,11 @@ def test_full_size_stack_every_unit():
     pairs = [(r, l) for r in range(wl.R) for l in range(wl.L)]
     _, _, run, units = _run_and_check(wl, [], pairs, range(1, wl.D), flags=P.FLAG_SHARED_CHAINS)
     assert units == len(pairs) * (wl.D - 1) * wl.W * wl.H
+
+
+def test_more_pairs_than_sms_several_segments_per_cta():
+    """More (request, head) pairs than SMs, so a CTA works through several segments (S_0, the node tables and U are
+    rebuilt between them, the beams' index bytes when the request changes), with a ragged last group."""
+    wl = CFG4.scaled(R=5, L=1, H=34, W=60, D=4, prompt_len=32, seed=77)
+    worst, _ = _check(wl, "fp32", True)
+    assert worst < 1.5e-3
