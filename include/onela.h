@@ -79,7 +79,7 @@ typedef int32_t onela_status;
 
 /* flags */
 #define ONELA_FLAG_DRY_RUN 1u       /* validate and advance host bookkeeping, launch nothing (host-logic tests) */
-#define ONELA_FLAG_FORCE_GENERIC 2u /* use the CUDA-core decode kernel even where the tensor-core kernel applies */
+#define ONELA_FLAG_FORCE_GENERIC 2u /* use the CUDA-core decode kernel (fp32 throughout) even where a tensor-core kernel applies */
 /* Record format and replay order of Section 3.2 (Eq. 2-4): the arena keeps (alpha_t, delta_t, k_t) with
  * delta_t = beta_t (v_t - alpha_t S_{t-1} k_t) in rec_dtype in place of v_t, and a decode call replays the two
  * projection accumulators S q_t and S k_t forward from S_0 through the beam's records (oldest first).  delta_t
@@ -103,8 +103,11 @@ typedef struct onela_config {
     int32_t num_heads;    /* key heads (and value heads, unless num_v_heads says otherwise) */
     int32_t dk, dv;       /* head dimensions of k/q and of v/o: (32, 32), (64, 64), (128, 128), (128, 256), (256, 256),
                            * (128, 512) or (256, 512), else ONELA_E_UNSUPPORTED; dk = 128 with bf16 records runs on
-                           * the tensor-core kernel at every value width (dv = 256 / 512 as two / four tiles of 128
-                           * outputs that share the key head's fold), every other shape on CUDA cores */
+                           * the warp-specialised tensor-core kernel at every value width (dv = 256 / 512 as two / four
+                           * tiles of 128 outputs that share the key head's fold); every other shape from (64, 64) up,
+                           * in either record dtype, on a tiled kernel whose contraction with S_0 runs on the tensor
+                           * cores as well (fp16 operands kept in range by exact powers of two, fp32 accumulation);
+                           * (32, 32) on CUDA cores in fp32 throughout */
     int32_t max_beam;     /* largest beam width W_t */
     int32_t max_steps;    /* largest number of decode calls per request (chain depth) */
     int32_t rec_dtype;    /* dtype of q, k, v: ONELA_DTYPE_* */
@@ -116,8 +119,9 @@ typedef struct onela_config {
      * states, values, gates and outputs are per value head.  Then q, k are [..][num_heads][dk]; v, alpha, beta, out
      * and S_0 are [..][num_v_heads][..]; a record keeps k once per key head and (v, alpha, beta) per value head
      * (num_heads * dk + num_v_heads * (dv + 8 bytes of gates) per slot instead of num_v_heads * (dk + dv + ..)).
-     * (dk, dv) in {(64, 64), (128, 128), (128, 256)}: dk = 128 with bf16 records on the tensor-core kernel, the rest
-     * on CUDA cores; onela_prefill_shared_state and ONELA_FLAG_GTR_DELTA are not available (ONELA_E_UNSUPPORTED). */
+     * (dk, dv) in {(64, 64), (128, 128), (128, 256)}: dk = 128 with bf16 records on the warp-specialised tensor-core
+     * kernel, the rest on the tiled one; onela_prefill_shared_state and ONELA_FLAG_GTR_DELTA are not available
+     * (ONELA_E_UNSUPPORTED). */
     int32_t num_v_heads;
 } onela_config;
 
@@ -255,7 +259,9 @@ onela_status onela_get_step_base(const onela_ctx* ctx, int32_t request, int32_t 
 /* Kernels this context has launched since creation (host counter; for launch accounting). */
 int64_t onela_launch_count(const onela_ctx* ctx);
 
-/* 1 if decode_step of this context runs the tcgen05 tensor-core kernel, 0 if the CUDA-core kernel. */
+/* Which kernel decode_step of this context runs: 1 the warp-specialised tcgen05 kernel (dk = 128, bf16 records),
+ * 2 the tiled tcgen05 kernel (every other shape from 64 x 64 up, either record dtype, grouped value heads or not),
+ * 0 a CUDA-core kernel (dk = dv = 32, ONELA_FLAG_FORCE_GENERIC, delta records at shapes other than 128 x 128 bf16). */
 int32_t onela_uses_tensor_core_path(const onela_ctx* ctx);
 
 const char* onela_status_string(onela_status s);

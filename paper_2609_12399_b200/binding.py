@@ -297,8 +297,9 @@ class Onela:
     def onela_launch_count(self) -> int:
         return int(self.lib.onela_launch_count(self.handle))
 
-    def onela_uses_tensor_core_path(self) -> bool:
-        return bool(self.lib.onela_uses_tensor_core_path(self.handle))
+    def onela_uses_tensor_core_path(self) -> int:
+        """0: CUDA-core kernels; 1: the warp-specialised tcgen05 kernel; 2: the tiled tcgen05 kernel."""
+        return int(self.lib.onela_uses_tensor_core_path(self.handle))
 
     def depth_and_width(self, request):
         return self._width(request)

@@ -81,7 +81,8 @@ struct onela_ctx {
     int64_t launches = 0;
     int64_t decode_mark = -1;  // value of `launches` right after the last decode launch
     bool status_cleared = false;
-    bool tensor_core = false;  // decode_step runs the tcgen05 kernel
+    bool tensor_core = false;  // decode_step runs the warp-specialised tcgen05 kernel
+    bool tiled_tc = false;     // decode_step runs the tiled tcgen05 kernel (the other shapes from 64 x 64 up)
     int32_t elem_bytes = 4;
 
     bool dry() const { return cfg.flags & ONELA_FLAG_DRY_RUN; }
@@ -227,6 +228,8 @@ onela_status onela_create(const onela_config* cfg, void* workspace_dev, size_t w
         r.appended_depth.assign(cfg->num_layers, -1);
     }
     ctx->tensor_core = decode_sm100_supported(cfg->dk, cfg->dv, cfg->rec_dtype) && !(cfg->flags & ONELA_FLAG_FORCE_GENERIC);
+    ctx->tiled_tc = !ctx->tensor_core && decode_tiled_supported(cfg->dk, cfg->dv) &&
+                    !(cfg->flags & (ONELA_FLAG_FORCE_GENERIC | ONELA_FLAG_GTR_DELTA));
     *out = ctx;
     return ONELA_OK;
 }
@@ -465,6 +468,40 @@ onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count,
                            const float* beta_dev, cudaStream_t s) {
     const onela_config& c = ctx->cfg;
     const int32_t depth = ctx->req[req_begin].depth, W = ctx->req[req_begin].W;
+    if (ctx->tiled_tc) {
+        TiledArgs ta{};
+        ta.q = q_dev;
+        ta.out = out_dev;
+        ta.s0 = ctx->s0_slot(req_begin, layer);
+        ta.s0_scale = ctx->s0_scale_slot(req_begin, layer);
+        if (ctx->grouped()) {
+            ta.kplane = ctx->k_plane(layer);
+            ta.vplane = ctx->v_plane(layer);
+            ta.k_stride = c.dk;
+            ta.v_stride = c.dv;
+        } else {      // one plane of k | v rows
+            ta.kplane = ctx->kv_plane(layer);
+            ta.vplane = ctx->kv_plane(layer) + (size_t)c.dk * ctx->elem_bytes;
+            ta.k_stride = ta.v_stride = c.dk + c.dv;
+        }
+        ta.gates = ctx->gate_plane(layer);
+        ta.table = ctx->table_cur(req_begin);
+        ta.status = ctx->lay.status;
+        ta.s0_req_stride = (long long)c.num_layers * ctx->s0_layer_floats();
+        ta.s0_scale_req_stride = (long long)c.num_layers * ctx->Hv();
+        ta.table_req_stride = ctx->table_req_stride();
+        ta.arena_slots = c.arena_slots;
+        ta.req_count = req_count;
+        ta.W = W;
+        ta.Hk = c.num_heads;
+        ta.g = ctx->Hv() / c.num_heads;
+        ta.depth = depth;
+        ta.max_beam = c.max_beam;
+        for (int i = 0; i < req_count; ++i) ta.bases.base[i] = ctx->req[req_begin + i].step_base.back();
+        if (launch_decode_tiled(ta, c.dk, c.dv, c.rec_dtype, c.out_dtype, s) != cudaSuccess) return ONELA_E_CUDA;
+        ctx->launches++;
+        return ONELA_OK;
+    }
     if (ctx->grouped() && !ctx->tensor_core) {
         GroupedArgs ga{};
         ga.q = q_dev;
@@ -673,7 +710,7 @@ onela_status onela_get_step_base(const onela_ctx* ctx, int32_t request, int32_t 
 
 int64_t onela_launch_count(const onela_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
-int32_t onela_uses_tensor_core_path(const onela_ctx* ctx) { return ctx && ctx->tensor_core ? 1 : 0; }
+int32_t onela_uses_tensor_core_path(const onela_ctx* ctx) { return !ctx ? 0 : ctx->tensor_core ? 1 : ctx->tiled_tc ? 2 : 0; }
 
 const char* onela_status_string(onela_status s) {
     switch (s) {

@@ -1,0 +1,298 @@
+// Tiled tcgen05 decode kernel for B200 (sm_100a): the shapes the warp-specialised kernel does not take - key widths
+// 64 and 256, value widths 64 to 512, fp32 records at every width, grouped value heads or not (the operator suite of
+// Section 4.1).  The chain walk is the CUDA-core one (see onela_decode_generic.cu); what moves to the tensor cores is
+// the contraction with S_0, which dominates these shapes (dv x dk multiply-adds per unit against 3 dk per record).
+//
+// One CTA = (request, value head, tile of 32 beams), 8 lanes per (beam, head) unit.
+//   1. Every unit folds its query through its records, newest first:  c = k.r ; corr += beta c v ; r -= beta c k,
+//      the decay a running scalar.  corr stays in registers.
+//   2. The folded queries go to shared memory as rows of the MMA's B operand: fp16, K-major, 128-byte swizzle, each row
+//      times the power of two that brings its largest element into [2^8, 2^9) (exact; undone after the product).
+//   3. Per tile of 128 value rows: the S_0 rows become the A operand the same way (fp16, times the head's power of two
+//      kept with the state), dk / 16 MMAs (M = 128, N = 32, K = 16) accumulate S_0 . r~ in tensor memory, and while
+//      they run the previous tile's accumulator is read back (lane = value row), scaled and added to corr in a
+//      shared-memory tile whose rows the units then store as 16-byte vectors.  Two accumulators alternate.
+// The only wait is for the MMAs' completion; it is bounded, and all threads agree on its outcome before going on
+// (ONELA_E_TIMEOUT in the status word otherwise).
+#include "onela_internal.h"
+#include "onela_layout.cuh"
+#include "onela_sm100.cuh"
+
+namespace onela {
+
+namespace {
+
+using sm100::idesc_f16;
+using sm100::mbar_init;
+using sm100::mbar_wait;
+using sm100::pack_f16x2;
+using sm100::pow2_scale;
+using sm100::smem_u32;
+using sm100::tmem_ld16;
+using sm100::umma_commit;
+using sm100::umma_desc;
+using sm100::umma_f16_ss;
+
+constexpr int NB = 32;                 // beams per CTA = MMA N
+constexpr int G = 8;                   // lanes per unit
+constexpr int THREADS = NB * G;
+constexpr int CP = 128 + 4;            // pitch (floats) of the output tile: conflict-free for both access patterns
+constexpr int ROW_TARGET = 8;          // a scaled operand row's largest element lies in [2^8, 2^9)
+constexpr uint32_t ACC_COLS = 64;      // two accumulators of NB columns
+
+template <int KD, int VD>
+constexpr size_t tiled_smem_bytes() {
+    return 1024 + (size_t)(KD / 64) * 128 * 128 + (size_t)(KD / 64) * NB * 128 + (size_t)NB * CP * 4 + NB * 4 + 64;
+}
+
+template <int KD, int VD, typename T, typename OutT>
+__global__ void __launch_bounds__(THREADS) decode_tiled_kernel(const TiledArgs a) {
+    constexpr int VEC = Vec16<T>::N;
+    constexpr int CK = KD / (G * VEC), CV = VD / (G * VEC);   // 16-byte chunks per lane
+    static_assert(KD % 64 == 0 && VD % 64 == 0 && CK >= 1 && CV >= 1, "whole 64-element K blocks, whole chunks per lane");
+    static_assert(128 % (G * VEC) == 0, "a lane's chunk lies inside one tile of 128 value rows");
+    constexpr int KB = KD / 64;                   // K blocks of 64 fp16 (one 128-byte swizzled row each)
+    constexpr int MT = (VD + 127) / 128;          // tiles of 128 value rows
+    constexpr int A_KB = 128 * 128, R_KB = NB * 128;   // bytes of one K block of the two operands
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    uint8_t* smem = smem_raw + (((raw + 1023u) & ~1023u) - raw);      // swizzle atoms need 1024-byte alignment
+    uint8_t* A_s = smem;                                               // [KB][128 rows][128 bytes]
+    uint8_t* R_s = A_s + KB * A_KB;                                    // [KB][NB rows][128 bytes]
+    float* C_s = reinterpret_cast<float*>(R_s + KB * R_KB);            // [NB][CP]
+    float* inv_s = C_s + NB * CP;                                      // [NB] what undoes a row's scales
+    uint64_t* bar = reinterpret_cast<uint64_t*>(inv_s + NB);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        mbar_init(smem_u32(bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(ACC_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int tile = blockIdx.x, hv = blockIdx.y, req = blockIdx.z;
+    const int hk = hv / a.g, Hv = a.Hk * a.g;
+    const int grp = tid / G, g = tid % G;
+    const int b = tile * NB + grp;
+    const bool active = b < a.W;
+    const int bb = active ? b : a.W - 1;  // idle units shadow a live beam so loads and shuffles stay uniform
+
+    const float* S0h = a.s0 + req * a.s0_req_stride + (long long)hv * VD * KD;
+    const float sc0 = __ldg(a.s0_scale + req * a.s0_scale_req_stride + hv);     // a power of two
+    // S_0 rows [128 mt, 128 mt + 128) -> A operand (rows beyond dv are zero); a warp reads whole rows
+    auto put_A = [&](int mt) {
+        constexpr int CPR = KD / 8;        // 16-byte fp16 chunks per row
+        for (int item = tid; item < 128 * CPR; item += THREADS) {
+            const int row = item / CPR, ch = item % CPR;
+            const int i = mt * 128 + row;
+            uint4 w = make_uint4(0u, 0u, 0u, 0u);
+            if (i < VD) {
+                const float4* p = reinterpret_cast<const float4*>(S0h + (long long)i * KD + ch * 8);
+                const float4 x0 = __ldg(p), x1 = __ldg(p + 1);
+                w = make_uint4(pack_f16x2(x0.x * sc0, x0.y * sc0), pack_f16x2(x0.z * sc0, x0.w * sc0),
+                               pack_f16x2(x1.x * sc0, x1.y * sc0), pack_f16x2(x1.z * sc0, x1.w * sc0));
+            }
+            *reinterpret_cast<uint4*>(A_s + (ch >> 3) * A_KB + row * 128 + (((ch & 7) ^ (row & 7)) << 4)) = w;
+        }
+    };
+    // one thread: the tile's dk / 16 MMAs into accumulator mt & 1, and the commit that completes the barrier's phase
+    auto issue = [&](int mt) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint64_t ad = umma_desc(smem_u32(A_s)), bd = umma_desc(smem_u32(R_s));
+        constexpr uint32_t idesc = idesc_f16(NB);
+#pragma unroll
+        for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+                umma_f16_ss(tmem_base + (mt & 1) * NB, ad + (uint64_t)((kb * A_KB + ks * 32) >> 4),
+                            bd + (uint64_t)((kb * R_KB + ks * 32) >> 4), idesc, (kb | ks) ? 1u : 0u);
+        umma_commit(smem_u32(bar));
+    };
+    put_A(0);        // independent of the fold: its loads are in flight while the chain is walked
+
+    // ---- the fold (Section 3.2's recurrence applied to the query from the newest record back) ----
+    const T* q = static_cast<const T*>(a.q) + (((long long)req * a.W + bb) * a.Hk + hk) * KD;
+    const int32_t* table = a.table + req * a.table_req_stride;
+    const T* kplane = reinterpret_cast<const T*>(a.kplane) + (long long)hk * a.arena_slots * a.k_stride;
+    const T* vplane = reinterpret_cast<const T*>(a.vplane) + (long long)hv * a.arena_slots * a.v_stride;
+    const float2* gates = a.gates + (long long)hv * a.arena_slots;
+
+    float r[CK * VEC], corr[CV * VEC];
+#pragma unroll
+    for (int c = 0; c < CK; ++c) Vec16<T>::load(q + (c * G + g) * VEC, r + c * VEC);
+#pragma unroll
+    for (int e = 0; e < CV * VEC; ++e) corr[e] = 0.f;
+    float decay = 1.f;  // product of the alphas already passed
+    for (int level = a.depth - 1; level >= 0; --level) {
+        const int32_t slot = (level == a.depth - 1) ? a.bases.base[req] + bb : __ldg(table + (long long)level * a.max_beam + bb);
+        const T* krec = kplane + (long long)slot * a.k_stride;
+        const T* vrec = vplane + (long long)slot * a.v_stride;
+        const float2 gate = __ldg(gates + slot);
+        float kx[CK * VEC];
+        float dot = 0.f;
+#pragma unroll
+        for (int c = 0; c < CK; ++c) {
+            Vec16<T>::load(krec + (c * G + g) * VEC, kx + c * VEC);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) dot = fmaf(kx[c * VEC + e], r[c * VEC + e], dot);
+        }
+#pragma unroll
+        for (int off = G / 2; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+        const float bc = gate.y * dot;        // beta_j * (k_j . r~_j)
+        const float wv = decay * bc;
+#pragma unroll
+        for (int c = 0; c < CV; ++c) {
+            float vx[VEC];
+            Vec16<T>::load(vrec + (c * G + g) * VEC, vx);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) corr[c * VEC + e] = fmaf(wv, vx[e], corr[c * VEC + e]);
+        }
+#pragma unroll
+        for (int e = 0; e < CK * VEC; ++e) r[e] = fmaf(-bc, kx[e], r[e]);
+        decay *= gate.x;
+    }
+
+    // ---- the folded query decay * r~ as the unit's operand row ----
+    {
+        float m = 0.f;
+#pragma unroll
+        for (int e = 0; e < CK * VEC; ++e) m = fmaxf(m, fabsf(r[e]));
+#pragma unroll
+        for (int off = G / 2; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+        float sc, inv;
+        pow2_scale(m * fabsf(decay), ROW_TARGET, sc, inv);
+        const float f = decay * sc;
+        if (g == 0) inv_s[grp] = inv / sc0;      // both powers of two
+#pragma unroll
+        for (int c = 0; c < CK; ++c) {
+            const int el0 = (c * G + g) * VEC;   // first element of the chunk
+            uint8_t* p = R_s + (el0 >> 6) * R_KB + grp * 128 + ((((el0 & 63) >> 3) ^ (grp & 7)) << 4) + (el0 & 7) * 2;
+            const float* x = r + c * VEC;
+            if constexpr (VEC == 8) {
+                *reinterpret_cast<uint4*>(p) = make_uint4(pack_f16x2(x[0] * f, x[1] * f), pack_f16x2(x[2] * f, x[3] * f),
+                                                          pack_f16x2(x[4] * f, x[5] * f), pack_f16x2(x[6] * f, x[7] * f));
+            } else {
+                *reinterpret_cast<uint2*>(p) = make_uint2(pack_f16x2(x[0] * f, x[1] * f), pack_f16x2(x[2] * f, x[3] * f));
+            }
+        }
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (tid == 0) issue(0);
+
+    OutT* out = static_cast<OutT*>(a.out) + (((long long)req * a.W + b) * Hv + hv) * VD;
+    const int quad = warp & 3, half = warp >> 2;     // tensor-memory lane quadrant and half of the beams of this warp
+    bool failed = false;
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+        // this tile's part of corr, one row per unit
+#pragma unroll
+        for (int c = 0; c < CV; ++c) {
+            if ((c * G * VEC) / 128 != mt) continue;
+            float* dst = C_s + grp * CP + (c * G + g) * VEC - mt * 128;
+#pragma unroll
+            for (int e = 0; e < VEC; e += 4)
+                *reinterpret_cast<float4*>(dst + e) = make_float4(corr[c * VEC + e], corr[c * VEC + e + 1], corr[c * VEC + e + 2], corr[c * VEC + e + 3]);
+        }
+        const bool ok = mbar_wait(smem_u32(bar), mt & 1);
+        if (__syncthreads_or(ok ? 0 : 1)) { failed = true; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (mt + 1 < MT) {               // the A operand is free: the next tile's rows
+            put_A(mt + 1);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
+        {
+            uint32_t v[16];
+            tmem_ld16(tmem_base + (mt & 1) * NB + half * 16 + ((uint32_t)(quad * 32) << 16), v);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            const int i = quad * 32 + lane;          // value row within the tile
+            if (mt * 128 + i < VD) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    float* cell = C_s + (half * 16 + j) * CP + i;
+                    *cell = fmaf(__uint_as_float(v[j]), inv_s[half * 16 + j], *cell);
+                }
+            }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        if (mt + 1 < MT && tid == 0) issue(mt + 1);
+        if (active) {
+#pragma unroll
+            for (int c = 0; c < CV; ++c) {
+                if ((c * G * VEC) / 128 != mt) continue;
+                const float* src = C_s + grp * CP + (c * G + g) * VEC - mt * 128;
+                float x[VEC];
+#pragma unroll
+                for (int e = 0; e < VEC; e += 4) {
+                    const float4 t = *reinterpret_cast<const float4*>(src + e);
+                    x[e] = t.x; x[e + 1] = t.y; x[e + 2] = t.z; x[e + 3] = t.w;
+                }
+                store_out<OutT, VEC>(out + (c * G + g) * VEC, x);
+            }
+        }
+        if (mt + 1 < MT) __syncthreads();      // the tile is read out before the next corr rows overwrite it
+    }
+    if (failed && tid == 0) {
+        if (atomicCAS(a.status, ONELA_OK, ONELA_E_TIMEOUT) == ONELA_OK) a.status[1] = (int32_t)(blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z));
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(ACC_COLS) : "memory");
+    }
+}
+
+template <int KD, int VD, typename T, typename OutT>
+cudaError_t launch_one(const TiledArgs& a, cudaStream_t stream) {
+    auto kern = decode_tiled_kernel<KD, VD, T, OutT>;
+    constexpr size_t smem = tiled_smem_bytes<KD, VD>();
+    static_assert(smem <= 232448, "shared memory per CTA");
+    if (smem > 48 * 1024) {
+        const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    dim3 grid((a.W + NB - 1) / NB, a.Hk * a.g, a.req_count);
+    kern<<<grid, THREADS, smem, stream>>>(a);
+    return cudaGetLastError();
+}
+
+template <int KD, int VD>
+cudaError_t launch_dims(const TiledArgs& a, int32_t rec_dtype, int32_t out_dtype, cudaStream_t stream) {
+    if (rec_dtype == ONELA_DTYPE_BF16) {
+        return out_dtype == ONELA_DTYPE_BF16 ? launch_one<KD, VD, __nv_bfloat16, __nv_bfloat16>(a, stream)
+                                             : launch_one<KD, VD, __nv_bfloat16, float>(a, stream);
+    }
+    return out_dtype == ONELA_DTYPE_BF16 ? launch_one<KD, VD, float, __nv_bfloat16>(a, stream)
+                                         : launch_one<KD, VD, float, float>(a, stream);
+}
+
+}  // namespace
+
+bool decode_tiled_supported(int32_t dk, int32_t dv) {
+    return (dk == 64 && dv == 64) || (dk == 128 && (dv == 128 || dv == 256 || dv == 512)) || (dk == 256 && (dv == 256 || dv == 512));
+}
+
+cudaError_t launch_decode_tiled(const TiledArgs& a, int32_t dk, int32_t dv, int32_t rec_dtype, int32_t out_dtype,
+                                cudaStream_t stream) {
+    if (dk == 64 && dv == 64) return launch_dims<64, 64>(a, rec_dtype, out_dtype, stream);
+    if (dk == 128 && dv == 128) return launch_dims<128, 128>(a, rec_dtype, out_dtype, stream);
+    if (dk == 128 && dv == 256) return launch_dims<128, 256>(a, rec_dtype, out_dtype, stream);
+    if (dk == 128 && dv == 512) return launch_dims<128, 512>(a, rec_dtype, out_dtype, stream);
+    if (dk == 256 && dv == 256) return launch_dims<256, 256>(a, rec_dtype, out_dtype, stream);
+    if (dk == 256 && dv == 512) return launch_dims<256, 512>(a, rec_dtype, out_dtype, stream);
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace onela

@@ -104,6 +104,28 @@ cudaError_t launch_append_grouped(const void* k, const void* v, const float* alp
                                   int32_t Hk, int32_t g, int32_t dk, int32_t dv, int32_t elem_bytes, const BatchBases& bases,
                                   cudaStream_t stream);
 
+// Tiled tcgen05 decode kernel (onela_decode_tiled.cu): every supported shape from 64 x 64 up in either record dtype,
+// grouped value heads or not.  Keys and values are addressed through planes and per-slot strides, so one struct serves
+// the interleaved arena (kplane = the layer's k | v rows, vplane = kplane + dk elements, both strides dk + dv) and the
+// split one (grouped value heads: two planes, strides dk and dv).
+struct TiledArgs {
+    const void* q;          // [req_count][W][Hk][dk]
+    void* out;              // [req_count][W][Hv][dv]
+    const float* s0;        // store slot of (req_begin, layer): [Hv][dv][dk]
+    const float* s0_scale;  // operand scale of (req_begin, layer, value head 0) (see Layout)
+    const char* kplane;     // key of (key head hk, slot) at kplane + ((hk * arena_slots + slot) * k_stride) elements
+    const char* vplane;     // value of (value head hv, slot) at vplane + ((hv * arena_slots + slot) * v_stride) elements
+    const float2* gates;    // [Hv][arena_slots]
+    const int32_t* table;   // current ancestry buffer of req_begin
+    int32_t* status;
+    long long s0_req_stride, s0_scale_req_stride, table_req_stride, arena_slots, k_stride, v_stride;
+    int32_t req_count, W, Hk, g, depth, max_beam;
+    BatchBases bases;
+};
+bool decode_tiled_supported(int32_t dk, int32_t dv);
+cudaError_t launch_decode_tiled(const TiledArgs& a, int32_t dk, int32_t dv, int32_t rec_dtype, int32_t out_dtype,
+                                cudaStream_t stream);
+
 // index kernels
 cudaError_t launch_reorder(int32_t* tables_req0, long long table_req_stride, int32_t req_count,
                            const int32_t* parents, int32_t W_new, int32_t W_prev, int32_t depth_old,

@@ -40,8 +40,9 @@ def _run(wl, g, out_dtype, fused, tight=None, flags=0):
     case = _grouped_case(wl, g)
     cfg = P.make_config(wl.R, wl.L, Hk, wl.dk, wl.dv, wl.W, wl.D, wl.dtype, out_dtype, wl.R * wl.W * wl.D, flags, num_v_heads=wl.H)
     ctx = P.Onela(cfg, device="cuda")
-    # the tensor-core kernel takes 128 x 128 bf16 records, grouped or not; everything else runs on CUDA cores
-    assert bool(ctx.onela_uses_tensor_core_path()) == (wl.dk == 128 and wl.dtype == "bf16" and not flags)
+    # the warp-specialised tensor-core kernel takes dk = 128 with bf16 records, grouped or not; the tiled one the
+    # other shapes; the CUDA-core kernel runs only when forced
+    assert ctx.onela_uses_tensor_core_path() == (0 if flags else 1 if (wl.dk == 128 and wl.dtype == "bf16") else 2)
     dev = torch.device("cuda")
     for (r, l), S in case["S0"].items():
         ctx.onela_init_shared_state(r, l, S.to(dev))
@@ -86,9 +87,21 @@ def test_grouped_heads_on_the_tensor_core_kernel_many_segments_and_depth():
 
 
 def test_grouped_heads_fp32_is_tight_and_other_shapes():
-    _run(CFG1.scaled(H=4, dtype="fp32", W=33, D=4, prompt_len=48, seed=1310), 2, "fp32", True, tight=5e-6)
-    _run(CFG1.scaled(H=6, dk=64, dv=64, dtype="fp32", W=20, D=3, prompt_len=32, seed=1311), 3, "fp32", False, tight=5e-6)
+    """fp32 records and the 64 x 64 shape: the tiled tensor-core kernel within the bar, the CUDA-core kernel (fp32
+    throughout) within rounding."""
+    for flags, tight in ((0, None), (P.FLAG_FORCE_GENERIC, 5e-6)):
+        _run(CFG1.scaled(H=4, dtype="fp32", W=33, D=4, prompt_len=48, seed=1310), 2, "fp32", True, tight=tight, flags=flags)
+        _run(CFG1.scaled(H=6, dk=64, dv=64, dtype="fp32", W=20, D=3, prompt_len=32, seed=1311), 3, "fp32", False, tight=tight, flags=flags)
     _run(CFG1.scaled(H=4, dk=128, dv=256, W=40, D=3, prompt_len=32, seed=1312), 2, "fp32", True)
+
+
+@pytest.mark.parametrize("dk,dv,dtype,g", [(64, 64, "bf16", 2), (64, 64, "fp32", 4), (128, 128, "fp32", 2), (128, 256, "fp32", 3)])
+def test_grouped_heads_on_the_tiled_tensor_core_kernel(dk, dv, dtype, g):
+    """The shapes the warp-specialised kernel does not take, grouped: deeper chains with shared ancestors, several
+    requests and layers, a ragged last tile of beams, bf16 outputs."""
+    wl = CFG1.scaled(R=2, L=2, H=2 * g, dk=dk, dv=dv, dtype=dtype, W=45, D=5, prompt_len=32, parents="zipf", zipf_s=1.4, seed=1340 + dk + dv)
+    _, ctx, worst = _run(wl, g, "bf16" if dtype == "bf16" else "fp32", dtype == "bf16")
+    assert ctx.onela_uses_tensor_core_path() == 2 and worst <= REL_L2_BAR
 
 
 @pytest.mark.parametrize("fused", [False, True])

@@ -151,9 +151,50 @@ def test_depth_one_and_max_depth():
 def test_other_geometries(dk, dv, dtype):
     wl = CFG1.scaled(H=2, dk=dk, dv=dv, dtype=dtype, W=37, D=3, prompt_len=48, seed=dk + dv)
     _, ctx = _full_check(make_case(wl), "fp32")
-    # key width 128 with bf16 records runs on the tensor cores at every value width (256 and 512 as two and four
-    # value tiles of 128 outputs); the other shapes on the CUDA-core kernel
-    assert bool(ctx.onela_uses_tensor_core_path()) == (dk == 128 and dtype == "bf16")
+    # key width 128 with bf16 records runs on the warp-specialised tensor-core kernel at every value width (256 and 512
+    # as two and four value tiles of 128 outputs); the other shapes from 64 x 64 up on the tiled tensor-core kernel;
+    # 32 x 32 on CUDA cores
+    assert ctx.onela_uses_tensor_core_path() == (1 if (dk == 128 and dtype == "bf16") else 2 if dk >= 64 else 0)
+
+
+@pytest.mark.parametrize("dk,dv,dtype", [(64, 64, "bf16"), (64, 64, "fp32"), (128, 128, "fp32"), (128, 256, "fp32"), (128, 512, "fp32"),
+                                         (256, 256, "bf16"), (256, 256, "fp32"), (256, 512, "bf16"), (256, 512, "fp32")])
+@pytest.mark.parametrize("fused,out_dtype", [(True, "bf16"), (False, "fp32")])
+def test_tiled_tensor_core_kernel(dk, dv, dtype, fused, out_dtype):
+    """Key widths 64 and 256, value widths to 512 and fp32 records (Section 4.1's operator suite) on the tiled tcgen05
+    kernel: deeper chains with shared ancestors, several requests and layers, beam widths with a ragged last tile and
+    more than one tile; every unit against the oracle, and against the CUDA-core kernel, whose contraction shares no
+    code with it."""
+    wl = CFG1.scaled(R=2, L=2, H=3, dk=dk, dv=dv, dtype=dtype, W=77, D=5, prompt_len=48, parents="zipf", zipf_s=1.4, seed=950 + dk + dv)
+    case = make_case(wl)
+    ref, chains = run_oracle(case)
+    outs, slots, ctx = run_library(case, out_dtype=out_dtype, fused=fused)
+    assert ctx.onela_uses_tensor_core_path() == 2 and ctx.onela_poll_device_status() == (0, 0)
+    want = expected_slots(case, chains)
+    for key in want:
+        assert np.array_equal(slots[key], want[key])
+    check_parity(case, outs, ref)
+    outs_cc, _, ctx_cc = run_library(case, out_dtype=out_dtype, flags=P.FLAG_FORCE_GENERIC, fused=fused)
+    assert ctx_cc.onela_uses_tensor_core_path() == 0
+    for key in outs:
+        assert rel_l2(outs[key].numpy(), outs_cc[key].double().numpy()).max() <= REL_L2_BAR
+
+
+def test_tiled_tensor_core_kernel_edge_cases():
+    """A single beam, exactly one full tile of 32 beams, one beam more, depth 1 and a long chain; keys and states far
+    from unit scale (the operand rows' power-of-two scales must absorb them)."""
+    for W, D, seed in ((1, 3, 1), (32, 2, 2), (33, 1, 3), (40, 12, 4)):
+        wl = CFG1.scaled(H=2, dk=256, dv=256, W=W, D=D, prompt_len=32, parents="zipf", zipf_s=1.5, seed=970 + seed)
+        _, ctx = _full_check(make_case(wl), "fp32")
+        assert ctx.onela_uses_tensor_core_path() == 2
+    wl = CFG1.scaled(H=2, dk=64, dv=64, dtype="fp32", W=50, D=4, prompt_len=16, seed=979)
+    case = make_case(wl)
+    for key in case["S0"]:
+        case["S0"][key] = case["S0"][key] * 3.0e4
+    for key in case["q"]:
+        case["q"][key] = case["q"][key] * 1.0e-3
+    _, ctx = _full_check(case, "fp32")
+    assert ctx.onela_uses_tensor_core_path() == 2
 
 
 @pytest.mark.parametrize("dv", [256, 512])
