@@ -46,7 +46,7 @@ constexpr size_t tiled_smem_bytes() {
 }
 
 template <int KD, int VD, typename T, typename OutT>
-__global__ void __launch_bounds__(THREADS) decode_tiled_kernel(const TiledArgs a) {
+__global__ void __launch_bounds__(THREADS, 2) decode_tiled_kernel(const TiledArgs a) {
     constexpr int VEC = Vec16<T>::N;
     constexpr int CK = KD / (G * VEC), CV = VD / (G * VEC);   // 16-byte chunks per lane
     static_assert(KD % 64 == 0 && VD % 64 == 0 && CK >= 1 && CV >= 1, "whole 64-element K blocks, whole chunks per lane");
