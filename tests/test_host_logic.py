@@ -152,6 +152,24 @@ def test_delta_record_mode_takes_only_the_fused_call():
     assert not P.Onela(cc, device="cpu").onela_uses_tensor_core_path()
 
 
+def test_kernel_choice_by_shape_dtype_and_flags():
+    """Which decode kernel a configuration gets (onela_uses_tensor_core_path): 1 the warp-specialised tcgen05 kernel
+    (dk = 128, bf16 records, any supported dv, grouped or not), 2 the tiled tcgen05 kernel (every other shape from
+    64 x 64 up, either record dtype), 0 CUDA cores (32 x 32, the force flag, delta records at the other shapes)."""
+    def kernel(dk, dv, rec, flags=0, hv=0):
+        cfg = P.make_config(1, 1, 2, dk, dv, 8, 3, rec, "fp32", 64, P.FLAG_DRY_RUN | flags, num_v_heads=hv)
+        return P.Onela(cfg, device="cpu").onela_uses_tensor_core_path()
+    for dv in (128, 256, 512):
+        assert kernel(128, dv, "bf16") == 1 and kernel(128, dv, "fp32") == 2
+    for dk, dv in ((64, 64), (256, 256), (256, 512)):
+        assert kernel(dk, dv, "bf16") == 2 and kernel(dk, dv, "fp32") == 2
+        assert kernel(dk, dv, "bf16", P.FLAG_FORCE_GENERIC) == 0
+    assert kernel(32, 32, "fp32") == 0 and kernel(32, 32, "bf16") == 0
+    assert kernel(128, 128, "bf16", P.FLAG_FORCE_GENERIC) == 0
+    assert kernel(64, 64, "fp32", P.FLAG_GTR_DELTA) == 0 and kernel(128, 128, "bf16", P.FLAG_GTR_DELTA) == 1
+    assert kernel(128, 128, "bf16", hv=4) == 1 and kernel(64, 64, "bf16", hv=4) == 2 and kernel(128, 256, "fp32", hv=6) == 2
+
+
 def test_select_beams_argument_checks():
     """Selection reads the request's current beam width (1, the root, before the first call), changes no state,
     and refuses widths it cannot deliver."""
