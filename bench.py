@@ -71,7 +71,8 @@ def workload_by_name(name: str) -> inputs.Workload:
 
 def describe(wl: inputs.Workload) -> str:
     idx = inputs.WORKLOADS.index(wl) if wl in inputs.WORKLOADS else -1
-    return (f"configs[{idx}] {wl.name}: {wl.R} requests x {wl.L} layers x {wl.H} heads, dk=dv={wl.dk}, "
+    dims = f"dk=dv={wl.dk}" if wl.dk == wl.dv else f"dk={wl.dk}, dv={wl.dv}"
+    return (f"configs[{idx}] {wl.name}: {wl.R} requests x {wl.L} layers x {wl.H} heads, {dims}, "
             f"{wl.prompt_len}-token prompts, beam {wl.W}, depth {wl.D}, {wl.parents} parents"
             + (f"(s={wl.zipf_s})" if wl.parents == "zipf" else "") + f", {wl.dtype} records, fp32 S_0")
 
@@ -154,11 +155,20 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     wl = workload_by_name(args.workload)
     if args.layers:
         wl = wl.scaled(L=args.layers)
+    # the other shapes of the operator suite (Section 4.1), on a named workload's beams, depths and parents
+    shape = {k: v for k, v in (("dk", args.dk), ("dv", args.dv), ("dtype", args.rec_dtype)) if v}
+    if shape:
+        wl = wl.scaled(name=wl.name + "_shape", **shape)
     out_dtype = args.out_dtype or wl.dtype
     out_bytes = 4 if out_dtype == "fp32" else 2
     run = WorkloadRun(wl, dev, out_dtype, flags=(2 if args.force_generic else 0) | (4 if args.delta_records else 0) | (8 if args.shared_chains else 0))
     ctx = run.ctx
-    run.prefill_states()
+    if wl.dk == wl.dv and wl.dk in (32, 64, 128):
+        run.prefill_states()
+    else:    # no prefill kernel for this shape: seeded random states of a prefilled state's magnitude
+        gen = torch.Generator(device=dev).manual_seed(wl.seed)
+        run.prefill_states({(r, l): 0.05 * torch.randn((wl.H, wl.dv, wl.dk), generator=gen, device=dev)
+                            for r in range(wl.R) for l in range(wl.L)})
     S0 = {(r, l): ctx.onela_export_shared_state(r, l) for r in range(wl.R) for l in range(wl.L)}
     S0_all = torch.stack([torch.stack([S0[(r, l)] for l in range(wl.L)]) for r in range(wl.R)])   # [R][L][H][dv][dk]
     calls = [run.generate_call(t) for t in range(wl.D)]
@@ -545,6 +555,9 @@ def main():
     ap.add_argument("--settle-seconds", type=float, default=1.0, help="extra untimed warm-up after the W steps")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling)")
     ap.add_argument("--force-generic", action="store_true", help="run the CUDA-core decode kernel")
+    ap.add_argument("--dk", type=int, default=0, help="override the workload's key width (64, 128, 256)")
+    ap.add_argument("--dv", type=int, default=0, help="override the workload's value width (64 ... 512)")
+    ap.add_argument("--rec-dtype", default=None, choices=[None, "bf16", "fp32"], help="override the record dtype")
     ap.add_argument("--delta-records", action="store_true",
                     help="(alpha, delta, k) records with forward projection replay (Section 3.2) instead of raw records "
                          "with the backward fold: the CUDA-core comparison kernel")

@@ -232,7 +232,9 @@ onela_status onela_decode_step(onela_ctx* ctx, int32_t req_begin, int32_t req_co
  * record inside the decode kernel, Section 3.4): the call's records are read from the caller's tensors,
  * folded as each beam's newest record, and written to the arena by the same kernel, so they cross HBM
  * once instead of three times.  Same arguments, checks and call-order rules as the two calls it replaces
- * (it counts as the layer's one append of this decode call; decode_step may still be called afterwards). */
+ * (it counts as the layer's one append of this decode call; decode_step may still be called afterwards).
+ * One launch on both tensor-core kernels; where a CUDA-core kernel runs (dk = dv = 32, ONELA_FLAG_FORCE_GENERIC)
+ * the call is the copy kernel followed by the decode kernel. */
 onela_status onela_append_decode_step(onela_ctx* ctx, int32_t req_begin, int32_t req_count, int32_t layer,
                                       const void* k_dev, const void* v_dev, const float* alpha_dev,
                                       const float* beta_dev, const void* q_dev, void* out_dev, void* stream);

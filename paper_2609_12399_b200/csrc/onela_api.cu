@@ -472,6 +472,10 @@ onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count,
         TiledArgs ta{};
         ta.q = q_dev;
         ta.out = out_dev;
+        ta.k_in = k_dev;
+        ta.v_in = v_dev;
+        ta.alpha_in = alpha_dev;
+        ta.beta_in = beta_dev;
         ta.s0 = ctx->s0_slot(req_begin, layer);
         ta.s0_scale = ctx->s0_scale_slot(req_begin, layer);
         if (ctx->grouped()) {
@@ -628,7 +632,7 @@ onela_status onela_append_decode_step(onela_ctx* ctx, int32_t req_begin, int32_t
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if ((st = ctx->prepare(s)) != ONELA_OK) return st;
     if (!ctx->dry()) {
-        if (ctx->tensor_core || ctx->gtr()) {
+        if (ctx->tensor_core || ctx->tiled_tc || ctx->gtr()) {
             st = launch_decode(ctx, req_begin, req_count, layer, q_dev, out_dev, k_dev, v_dev, alpha_dev, beta_dev, s);
             if (st != ONELA_OK) return st;
         } else {   // shapes without the fused kernel: the copy kernel, then the decode kernel

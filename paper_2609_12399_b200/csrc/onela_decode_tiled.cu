@@ -3,17 +3,20 @@
 // Section 4.1).  The chain walk is the CUDA-core one (see onela_decode_generic.cu); what moves to the tensor cores is
 // the contraction with S_0, which dominates these shapes (dv x dk multiply-adds per unit against 3 dk per record).
 //
-// One CTA = (request, value head, tile of 32 beams), 8 lanes per (beam, head) unit.
+// One CTA = (request, value head, tile of 32 beams - 64 at key width 256), 8 lanes per (beam, head) unit.
 //   1. Every unit folds its query through its records, newest first:  c = k.r ; corr += beta c v ; r -= beta c k,
-//      the decay a running scalar.  corr stays in registers.
+//      the decay a running scalar.  corr stays in registers.  With the append fused in, the newest record comes from
+//      the caller's tensors and the unit also writes it to its arena slot.
 //   2. The folded queries go to shared memory as rows of the MMA's B operand: fp16, K-major, 128-byte swizzle, each row
 //      times the power of two that brings its largest element into [2^8, 2^9) (exact; undone after the product).
 //   3. Per tile of 128 value rows: the S_0 rows become the A operand the same way (fp16, times the head's power of two
-//      kept with the state), dk / 16 MMAs (M = 128, N = 32, K = 16) accumulate S_0 . r~ in tensor memory, and while
+//      kept with the state), dk / 16 MMAs (M = 128, N = beams, K = 16) accumulate S_0 . r~ in tensor memory, and while
 //      they run the previous tile's accumulator is read back (lane = value row), scaled and added to corr in a
 //      shared-memory tile whose rows the units then store as 16-byte vectors.  Two accumulators alternate.
 // The only wait is for the MMAs' completion; it is bounded, and all threads agree on its outcome before going on
 // (ONELA_E_TIMEOUT in the status word otherwise).
+#include <mutex>
+
 #include "onela_internal.h"
 #include "onela_layout.cuh"
 #include "onela_sm100.cuh"
@@ -33,20 +36,30 @@ using sm100::umma_commit;
 using sm100::umma_desc;
 using sm100::umma_f16_ss;
 
-constexpr int NB = 32;                 // beams per CTA = MMA N
 constexpr int G = 8;                   // lanes per unit
-constexpr int THREADS = NB * G;
 constexpr int CP = 128 + 4;            // pitch (floats) of the output tile: conflict-free for both access patterns
 constexpr int ROW_TARGET = 8;          // a scaled operand row's largest element lies in [2^8, 2^9)
-constexpr uint32_t ACC_COLS = 64;      // two accumulators of NB columns
 
+// Beams per CTA (= MMA N; 8 threads each).  Key width 256 takes 64: every CTA turns the whole head's S_0 into its A
+// operand, 128 KB of fp32 from L2 per tile of value rows, and at 32 beams per CTA those reads (1 GB per launch at
+// 256 x 512 with 65 536 units) were what bounded the kernel; one CTA of 512 threads holds as many warps as two of 256.
 template <int KD, int VD>
-constexpr size_t tiled_smem_bytes() {
+__host__ __device__ constexpr int tiled_beams() { return KD * VD >= 128 * 128 ? 64 : 32; }
+template <int KD, int VD>
+__host__ __device__ constexpr size_t tiled_smem_bytes() {
+    constexpr int NB = tiled_beams<KD, VD>();
     return 1024 + (size_t)(KD / 64) * 128 * 128 + (size_t)(KD / 64) * NB * 128 + (size_t)NB * CP * 4 + NB * 4 + 64;
 }
 
+// CTAs per SM the registers are capped for: small CTAs are latency-bound (a string of dependent loads per level, one MMA
+// round trip), so the narrowest shape gets four.
+template <int KD, int VD>
+__host__ __device__ constexpr int tiled_min_ctas() { return KD + VD <= 128 ? 4 : tiled_beams<KD, VD>() == 64 ? 1 : 2; }
+
 template <int KD, int VD, typename T, typename OutT>
-__global__ void __launch_bounds__(THREADS, 2) decode_tiled_kernel(const TiledArgs a) {
+__global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, VD>()) decode_tiled_kernel(const TiledArgs a) {
+    constexpr int NB = tiled_beams<KD, VD>(), THREADS = NB * G;
+    constexpr uint32_t ACC_COLS = 2 * NB;      // two accumulators of NB columns (a power of two >= 32)
     constexpr int VEC = Vec16<T>::N;
     constexpr int CK = KD / (G * VEC), CV = VD / (G * VEC);   // 16-byte chunks per lane
     static_assert(KD % 64 == 0 && VD % 64 == 0 && CK >= 1 && CV >= 1, "whole 64-element K blocks, whole chunks per lane");
@@ -123,9 +136,10 @@ __global__ void __launch_bounds__(THREADS, 2) decode_tiled_kernel(const TiledArg
     // ---- the fold (Section 3.2's recurrence applied to the query from the newest record back) ----
     const T* q = static_cast<const T*>(a.q) + (((long long)req * a.W + bb) * a.Hk + hk) * KD;
     const int32_t* table = a.table + req * a.table_req_stride;
-    const T* kplane = reinterpret_cast<const T*>(a.kplane) + (long long)hk * a.arena_slots * a.k_stride;
-    const T* vplane = reinterpret_cast<const T*>(a.vplane) + (long long)hv * a.arena_slots * a.v_stride;
-    const float2* gates = a.gates + (long long)hv * a.arena_slots;
+    T* kplane = reinterpret_cast<T*>(a.kplane) + (long long)hk * a.arena_slots * a.k_stride;
+    T* vplane = reinterpret_cast<T*>(a.vplane) + (long long)hv * a.arena_slots * a.v_stride;
+    float2* gates = a.gates + (long long)hv * a.arena_slots;
+    const bool fused = a.k_in != nullptr;      // append fused in: the newest record comes from the caller's tensors
 
     float r[CK * VEC], corr[CV * VEC];
 #pragma unroll
@@ -133,33 +147,99 @@ __global__ void __launch_bounds__(THREADS, 2) decode_tiled_kernel(const TiledArg
 #pragma unroll
     for (int e = 0; e < CV * VEC; ++e) corr[e] = 0.f;
     float decay = 1.f;  // product of the alphas already passed
-    for (int level = a.depth - 1; level >= 0; --level) {
-        const int32_t slot = (level == a.depth - 1) ? a.bases.base[req] + bb : __ldg(table + (long long)level * a.max_beam + bb);
-        const T* krec = kplane + (long long)slot * a.k_stride;
-        const T* vrec = vplane + (long long)slot * a.v_stride;
-        const float2 gate = __ldg(gates + slot);
+
+    // Lane g of a unit fetches the slot of the unit's ancestor at level g (the oldest eight levels: one load latency
+    // for the whole chain instead of one per level); deeper levels are looked up when they are reached.
+    const int old = a.depth - 1;           // records older than the beam's own: levels old - 1 .. 0
+    const int32_t my_slot = g < old ? __ldg(table + (long long)g * a.max_beam + bb) : 0;
+    auto slot_of = [&](int level) -> int32_t {       // level < old; unit-uniform
+        const int32_t x = __shfl_sync(0xffffffffu, my_slot, level & (G - 1), G);
+        return level < G ? x : __ldg(table + (long long)level * a.max_beam + bb);
+    };
+    struct Raw { uint4 k[CK], v[CV]; float2 gate; };          // this lane's share of a record, as stored
+    auto fetch = [&](int level) -> Raw {                      // an older record, from the arena
+        const long long slot = slot_of(level);
+        const uint4* kp = reinterpret_cast<const uint4*>(kplane + slot * a.k_stride) + g;
+        const uint4* vp = reinterpret_cast<const uint4*>(vplane + slot * a.v_stride) + g;
+        Raw x;
+#pragma unroll
+        for (int c = 0; c < CK; ++c) x.k[c] = __ldg(kp + c * G);
+#pragma unroll
+        for (int c = 0; c < CV; ++c) x.v[c] = __ldg(vp + c * G);
+        x.gate = __ldg(gates + slot);
+        return x;
+    };
+    auto fold = [&](const Raw& x) {       // c = k . r~ ;  corr += decay beta c v ;  r~ -= beta c k ;  decay *= alpha
         float kx[CK * VEC];
         float dot = 0.f;
 #pragma unroll
         for (int c = 0; c < CK; ++c) {
-            Vec16<T>::load(krec + (c * G + g) * VEC, kx + c * VEC);
+            Vec16<T>::unpack(x.k[c], kx + c * VEC);
 #pragma unroll
             for (int e = 0; e < VEC; ++e) dot = fmaf(kx[c * VEC + e], r[c * VEC + e], dot);
         }
 #pragma unroll
         for (int off = G / 2; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
-        const float bc = gate.y * dot;        // beta_j * (k_j . r~_j)
+        const float bc = x.gate.y * dot;
         const float wv = decay * bc;
 #pragma unroll
         for (int c = 0; c < CV; ++c) {
             float vx[VEC];
-            Vec16<T>::load(vrec + (c * G + g) * VEC, vx);
+            Vec16<T>::unpack(x.v[c], vx);
 #pragma unroll
             for (int e = 0; e < VEC; ++e) corr[c * VEC + e] = fmaf(wv, vx[e], corr[c * VEC + e]);
         }
 #pragma unroll
         for (int e = 0; e < CK * VEC; ++e) r[e] = fmaf(-bc, kx[e], r[e]);
-        decay *= gate.x;
+        decay *= x.gate.x;
+    };
+    // The beam's own record: from its arena slot, or - append fused in - from the caller's tensors, in which case this
+    // unit also writes it to the slot, bit for bit (16-byte vectors; the key once per key head, by its first value
+    // head).  The fold reads the caller's copy, so nothing in this launch reads what another CTA of it writes.
+    Raw cur;
+    {
+        const long long slot = a.bases.base[req] + bb;
+        T* kdst = kplane + slot * a.k_stride;
+        T* vdst = vplane + slot * a.v_stride;
+        const T *ksrc = kdst, *vsrc = vdst;
+        if (fused) {
+            const long long krow = ((long long)req * a.W + bb) * a.Hk + hk, vrow = ((long long)req * a.W + bb) * Hv + hv;
+            ksrc = static_cast<const T*>(a.k_in) + krow * KD;
+            vsrc = static_cast<const T*>(a.v_in) + vrow * VD;
+            cur.gate = make_float2(__ldg(a.alpha_in + vrow), __ldg(a.beta_in + vrow));
+        } else {
+            cur.gate = __ldg(gates + slot);
+        }
+#pragma unroll
+        for (int c = 0; c < CK; ++c) cur.k[c] = __ldg(reinterpret_cast<const uint4*>(ksrc) + c * G + g);
+#pragma unroll
+        for (int c = 0; c < CV; ++c) cur.v[c] = __ldg(reinterpret_cast<const uint4*>(vsrc) + c * G + g);
+        if (fused && active) {
+#pragma unroll
+            for (int c = 0; c < CV; ++c) reinterpret_cast<uint4*>(vdst)[c * G + g] = cur.v[c];
+            if (hv % a.g == 0) {
+#pragma unroll
+                for (int c = 0; c < CK; ++c) reinterpret_cast<uint4*>(kdst)[c * G + g] = cur.k[c];
+            }
+            if (g == 0) gates[slot] = cur.gate;
+        }
+    }
+    // Narrow records are fetched one level ahead of their fold (the chain is a string of dependent loads otherwise);
+    // wide ones would not fit in the registers twice.
+    constexpr bool AHEAD = KD + VD <= 256;
+    if constexpr (AHEAD) {
+        for (int level = old - 1; level >= 0; --level) {
+            const Raw next = fetch(level);
+            fold(cur);
+            cur = next;
+        }
+        fold(cur);
+    } else {
+        fold(cur);
+        for (int level = old - 1; level >= 0; --level) {
+            const Raw x = fetch(level);
+            fold(x);
+        }
     }
 
     // ---- the folded query decay * r~ as the unit's operand row ----
@@ -192,7 +272,7 @@ __global__ void __launch_bounds__(THREADS, 2) decode_tiled_kernel(const TiledArg
     if (tid == 0) issue(0);
 
     OutT* out = static_cast<OutT*>(a.out) + (((long long)req * a.W + b) * Hv + hv) * VD;
-    const int quad = warp & 3, half = warp >> 2;     // tensor-memory lane quadrant and half of the beams of this warp
+    const int quad = warp & 3, half = warp >> 2;     // tensor-memory lane quadrant of this warp, and which 16 beams it takes
     bool failed = false;
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
@@ -257,12 +337,19 @@ __global__ void __launch_bounds__(THREADS, 2) decode_tiled_kernel(const TiledArg
 template <int KD, int VD, typename T, typename OutT>
 cudaError_t launch_one(const TiledArgs& a, cudaStream_t stream) {
     auto kern = decode_tiled_kernel<KD, VD, T, OutT>;
+    constexpr int NB = tiled_beams<KD, VD>(), THREADS = NB * G;
     constexpr size_t smem = tiled_smem_bytes<KD, VD>();
     static_assert(smem <= 232448, "shared memory per CTA");
-    if (smem > 48 * 1024) {
-        const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-    }
+    static std::once_flag once;          // one per instantiation
+    static cudaError_t attr = cudaSuccess;
+    std::call_once(once, [&] {
+        attr = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        // shared memory for the CTAs the registers allow and no more: what is left of the SM's 228 KB serves the fold's
+        // record loads as L1 (asking for all of it made 128 x 128 fp32 14 % slower)
+        constexpr int pct = (int)((tiled_min_ctas<KD, VD>() * (smem + 1024) * 100 + 228 * 1024 - 1) / (228 * 1024));
+        if (attr == cudaSuccess) attr = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, pct > 100 ? 100 : pct);
+    });
+    if (attr != cudaSuccess) return attr;
     dim3 grid((a.W + NB - 1) / NB, a.Hk * a.g, a.req_count);
     kern<<<grid, THREADS, smem, stream>>>(a);
     return cudaGetLastError();

@@ -111,11 +111,15 @@ cudaError_t launch_append_grouped(const void* k, const void* v, const float* alp
 struct TiledArgs {
     const void* q;          // [req_count][W][Hk][dk]
     void* out;              // [req_count][W][Hv][dv]
+    const void* k_in;       // fused append: this call's records [req_count][W][Hk][dk], [..][Hv][dv], gates [..][Hv], which
+    const void* v_in;       //   the launch also writes to their arena slots; null for a plain decode (the newest record
+    const float* alpha_in;  //   is then read from the arena)
+    const float* beta_in;
     const float* s0;        // store slot of (req_begin, layer): [Hv][dv][dk]
     const float* s0_scale;  // operand scale of (req_begin, layer, value head 0) (see Layout)
-    const char* kplane;     // key of (key head hk, slot) at kplane + ((hk * arena_slots + slot) * k_stride) elements
-    const char* vplane;     // value of (value head hv, slot) at vplane + ((hv * arena_slots + slot) * v_stride) elements
-    const float2* gates;    // [Hv][arena_slots]
+    char* kplane;           // key of (key head hk, slot) at kplane + ((hk * arena_slots + slot) * k_stride) elements
+    char* vplane;           // value of (value head hv, slot) at vplane + ((hv * arena_slots + slot) * v_stride) elements
+    float2* gates;          // [Hv][arena_slots]
     const int32_t* table;   // current ancestry buffer of req_begin
     int32_t* status;
     long long s0_req_stride, s0_scale_req_stride, table_req_stride, arena_slots, k_stride, v_stride;

@@ -17,21 +17,21 @@ struct Vec16;  // one 16-byte vector of T, unpacked to fp32
 template <>
 struct Vec16<float> {
     static constexpr int N = 4;
-    static __device__ __forceinline__ void load(const float* p, float* out) {
-        const float4 x = __ldg(reinterpret_cast<const float4*>(p));
-        out[0] = x.x; out[1] = x.y; out[2] = x.z; out[3] = x.w;
+    static __device__ __forceinline__ void unpack(const uint4& x, float* out) {
+        out[0] = __uint_as_float(x.x); out[1] = __uint_as_float(x.y); out[2] = __uint_as_float(x.z); out[3] = __uint_as_float(x.w);
     }
+    static __device__ __forceinline__ void load(const float* p, float* out) { unpack(__ldg(reinterpret_cast<const uint4*>(p)), out); }
 };
 template <>
 struct Vec16<__nv_bfloat16> {
     static constexpr int N = 8;
-    static __device__ __forceinline__ void load(const __nv_bfloat16* p, float* out) {
-        const uint4 x = __ldg(reinterpret_cast<const uint4*>(p));
+    static __device__ __forceinline__ void unpack(const uint4& x, float* out) {
         unpack_bf16x2(x.x, out[0], out[1]);
         unpack_bf16x2(x.y, out[2], out[3]);
         unpack_bf16x2(x.z, out[4], out[5]);
         unpack_bf16x2(x.w, out[6], out[7]);
     }
+    static __device__ __forceinline__ void load(const __nv_bfloat16* p, float* out) { unpack(__ldg(reinterpret_cast<const uint4*>(p)), out); }
 };
 
 // two fp32 -> two packed bf16 (element 0 in the low half), round to nearest even

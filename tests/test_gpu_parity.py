@@ -178,6 +178,29 @@ def test_tiled_tensor_core_kernel(dk, dv, dtype, fused, out_dtype):
     assert ctx_cc.onela_uses_tensor_core_path() == 0
     for key in outs:
         assert rel_l2(outs[key].numpy(), outs_cc[key].double().numpy()).max() <= REL_L2_BAR
+    # the arena rows [k | v] and the gates of every layer hold the appended bytes (with `fused` the decode launch wrote them)
+    c = ctx.cfg
+    al = lambda n: (n + 1023) // 1024 * 1024
+    n_idx = c.num_requests * c.max_steps * c.max_beam * 4
+    off_s0 = al(16) + al(2 * n_idx) + al(n_idx) + al(n_idx) + al(c.num_requests * (c.max_steps + 1) * 4)
+    off_gates = off_s0 + al(c.num_requests * c.num_layers * c.num_heads * c.dv * c.dk * 4)
+    off_kv = off_gates + al(c.num_layers * c.num_heads * c.arena_slots * 8)
+    ws = ctx.workspace[ctx.workspace_ptr - ctx.workspace.data_ptr():]
+    row, eb, td = dk + dv, (2 if dtype == "bf16" else 4), (torch.bfloat16 if dtype == "bf16" else torch.float32)
+    for lay in range(wl.L):
+        g0 = off_gates + lay * c.num_heads * c.arena_slots * 8
+        k0 = off_kv + lay * c.num_heads * c.arena_slots * row * eb
+        gates = ws[g0:g0 + c.num_heads * c.arena_slots * 8].view(torch.float32).view(c.num_heads, c.arena_slots, 2).cpu()
+        kv = ws[k0:k0 + c.num_heads * c.arena_slots * row * eb].view(td).view(c.num_heads, c.arena_slots, row).cpu()
+        for r in range(wl.R):
+            for t in range(wl.D):
+                base = ctx.onela_get_step_base(r, t)
+                tk = case["tok"][(r, lay, t)]
+                for h in range(wl.H):
+                    assert torch.equal(kv[h, base:base + wl.W, :dk], tk["k"][:, h])
+                    assert torch.equal(kv[h, base:base + wl.W, dk:], tk["v"][:, h])
+                    assert torch.equal(gates[h, base:base + wl.W, 0], tk["alpha"][:, h])
+                    assert torch.equal(gates[h, base:base + wl.W, 1], tk["beta"][:, h])
 
 
 def test_tiled_tensor_core_kernel_edge_cases():
