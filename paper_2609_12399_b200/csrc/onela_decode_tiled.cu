@@ -11,8 +11,9 @@
 //      times the power of two that brings its largest element into [2^8, 2^9) (exact; undone after the product).
 //   3. Per tile of 128 value rows: the S_0 rows become the A operand the same way (fp16, times the head's power of two
 //      kept with the state), dk / 16 MMAs (M = 128, N = beams, K = 16) accumulate S_0 . r~ in tensor memory, and while
-//      they run the previous tile's accumulator is read back (lane = value row), scaled and added to corr in a
-//      shared-memory tile whose rows the units then store as 16-byte vectors.  Two accumulators alternate.
+//      they run the next tile's A operand is built and the previous tile's accumulator is read back (lane = value
+//      row), scaled and added to corr in a shared-memory tile whose rows the units then store as 16-byte vectors.  Two
+//      A operands and two accumulators alternate.
 // The only wait is for the MMAs' completion; it is bounded, and all threads agree on its outcome before going on
 // (ONELA_E_TIMEOUT in the status word otherwise).
 #include <mutex>
@@ -47,8 +48,10 @@ template <int KD, int VD>
 __host__ __device__ constexpr int tiled_beams() { return KD * VD >= 128 * 128 ? 64 : 32; }
 template <int KD, int VD>
 __host__ __device__ constexpr size_t tiled_smem_bytes() {
-    constexpr int NB = tiled_beams<KD, VD>();
-    return 1024 + (size_t)(KD / 64) * 128 * 128 + (size_t)(KD / 64) * NB * 128 + (size_t)NB * CP * 4 + NB * 4 + 64;
+    // two A operands where there is a next tile to prepare and the key is narrow (at key width 256 the second buffer
+    // leaves the fold's record loads 34 KB of L1: 89 -> 106 us at 256 x 256)
+    constexpr int NB = tiled_beams<KD, VD>(), ABUF = (VD > 128 && KD <= 128) ? 2 : 1;
+    return 1024 + (size_t)ABUF * (KD / 64) * 128 * 128 + (size_t)(KD / 64) * NB * 128 + (size_t)NB * CP * 4 + NB * 4 + 64;
 }
 
 // CTAs per SM the registers are capped for: small CTAs are latency-bound (a string of dependent loads per level, one MMA
@@ -71,8 +74,9 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     uint8_t* smem = smem_raw + (((raw + 1023u) & ~1023u) - raw);      // swizzle atoms need 1024-byte alignment
-    uint8_t* A_s = smem;                                               // [KB][128 rows][128 bytes]
-    uint8_t* R_s = A_s + KB * A_KB;                                    // [KB][NB rows][128 bytes]
+    constexpr int ABUF = (MT > 1 && KD <= 128) ? 2 : 1;
+    uint8_t* A_s = smem;                                               // [ABUF][KB][128 rows][128 bytes]: tile mt in buffer mt & 1
+    uint8_t* R_s = A_s + ABUF * KB * A_KB;                             // [KB][NB rows][128 bytes]
     float* C_s = reinterpret_cast<float*>(R_s + KB * R_KB);            // [NB][CP]
     float* inv_s = C_s + NB * CP;                                      // [NB] what undoes a row's scales
     uint64_t* bar = reinterpret_cast<uint64_t*>(inv_s + NB);
@@ -104,24 +108,39 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
     const float sc0 = __ldg(a.s0_scale + req * a.s0_scale_req_stride + hv);     // a power of two
     // S_0 rows [128 mt, 128 mt + 128) -> A operand (rows beyond dv are zero); a warp reads whole rows
     auto put_A = [&](int mt) {
+        uint8_t* A_t = A_s + (mt & (ABUF - 1)) * (KB * A_KB);
         constexpr int CPR = KD / 8;        // 16-byte fp16 chunks per row
-        for (int item = tid; item < 128 * CPR; item += THREADS) {
-            const int row = item / CPR, ch = item % CPR;
-            const int i = mt * 128 + row;
-            uint4 w = make_uint4(0u, 0u, 0u, 0u);
-            if (i < VD) {
-                const float4* p = reinterpret_cast<const float4*>(S0h + (long long)i * KD + ch * 8);
-                const float4 x0 = __ldg(p), x1 = __ldg(p + 1);
-                w = make_uint4(pack_f16x2(x0.x * sc0, x0.y * sc0), pack_f16x2(x0.z * sc0, x0.w * sc0),
+        constexpr int ITEMS = 128 * CPR / THREADS, UNR = ITEMS % 4 == 0 ? 4 : 2;
+        static_assert(128 * CPR % THREADS == 0 && ITEMS % UNR == 0, "every thread converts the same number of chunks");
+#pragma unroll 1
+        for (int it = 0; it < ITEMS; it += UNR) {       // UNR chunks' loads in flight together
+            float4 x[UNR][2];
+#pragma unroll
+            for (int u = 0; u < UNR; ++u) {
+                const int item = (it + u) * THREADS + tid, row = item / CPR, ch = item % CPR;
+                const int i = mt * 128 + row;
+                if (i < VD) {
+                    const float4* p = reinterpret_cast<const float4*>(S0h + (long long)i * KD + ch * 8);
+                    x[u][0] = __ldg(p);
+                    x[u][1] = __ldg(p + 1);
+                } else {
+                    x[u][0] = x[u][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UNR; ++u) {
+                const int item = (it + u) * THREADS + tid, row = item / CPR, ch = item % CPR;
+                const float4 x0 = x[u][0], x1 = x[u][1];
+                *reinterpret_cast<uint4*>(A_t + (ch >> 3) * A_KB + row * 128 + (((ch & 7) ^ (row & 7)) << 4)) =
+                    make_uint4(pack_f16x2(x0.x * sc0, x0.y * sc0), pack_f16x2(x0.z * sc0, x0.w * sc0),
                                pack_f16x2(x1.x * sc0, x1.y * sc0), pack_f16x2(x1.z * sc0, x1.w * sc0));
             }
-            *reinterpret_cast<uint4*>(A_s + (ch >> 3) * A_KB + row * 128 + (((ch & 7) ^ (row & 7)) << 4)) = w;
         }
     };
     // one thread: the tile's dk / 16 MMAs into accumulator mt & 1, and the commit that completes the barrier's phase
     auto issue = [&](int mt) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint64_t ad = umma_desc(smem_u32(A_s)), bd = umma_desc(smem_u32(R_s));
+        const uint64_t ad = umma_desc(smem_u32(A_s + (mt & (ABUF - 1)) * (KB * A_KB))), bd = umma_desc(smem_u32(R_s));
         constexpr uint32_t idesc = idesc_f16(NB);
 #pragma unroll
         for (int kb = 0; kb < KB; ++kb)
@@ -285,10 +304,21 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
             for (int e = 0; e < VEC; e += 4)
                 *reinterpret_cast<float4*>(dst + e) = make_float4(corr[c * VEC + e], corr[c * VEC + e + 1], corr[c * VEC + e + 2], corr[c * VEC + e + 3]);
         }
+        if (ABUF == 2 && mt + 1 < MT) {
+            // the next tile's A operand, under this tile's MMAs: its buffer was last read by tile mt - 1, whose
+            // completion every thread has waited for
+            put_A(mt + 1);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
         const bool ok = mbar_wait(smem_u32(bar), mt & 1);
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         if (__syncthreads_or(ok ? 0 : 1)) { failed = true; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (mt + 1 < MT) {               // the A operand is free: the next tile's rows
+        if (ABUF == 2) {
+            // ... and its MMAs, under this tile's epilogue: their accumulator was read out before the barrier that
+            // ended the previous iteration
+            if (mt + 1 < MT && tid == 0) issue(mt + 1);
+        } else if (mt + 1 < MT) {        // one A operand: free now; its MMAs go out after the barrier below
             put_A(mt + 1);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
@@ -307,7 +337,7 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
         }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();
-        if (mt + 1 < MT && tid == 0) issue(mt + 1);
+        if (ABUF == 1 && mt + 1 < MT && tid == 0) issue(mt + 1);
         if (active) {
 #pragma unroll
             for (int c = 0; c < CV; ++c) {
