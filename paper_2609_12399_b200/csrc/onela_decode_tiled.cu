@@ -117,7 +117,9 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
             float4 x[UNR][2];
 #pragma unroll
             for (int u = 0; u < UNR; ++u) {
-                const int item = (it + u) * THREADS + tid, row = item / CPR, ch = item % CPR;
+                // a warp takes one K block (8 chunks = 256 bytes of fp32) of four consecutive rows: whole 128-byte lines
+                // from global memory, 512 consecutive bytes of shared memory (no bank conflicts)
+                const int wi = (it + u) * (THREADS / 32) + warp, row = (wi / KB) * 4 + (lane >> 3), ch = (wi % KB) * 8 + (lane & 7);
                 const int i = mt * 128 + row;
                 if (i < VD) {
                     const float4* p = reinterpret_cast<const float4*>(S0h + (long long)i * KD + ch * 8);
@@ -129,7 +131,7 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
             }
 #pragma unroll
             for (int u = 0; u < UNR; ++u) {
-                const int item = (it + u) * THREADS + tid, row = item / CPR, ch = item % CPR;
+                const int wi = (it + u) * (THREADS / 32) + warp, row = (wi / KB) * 4 + (lane >> 3), ch = (wi % KB) * 8 + (lane & 7);
                 const float4 x0 = x[u][0], x1 = x[u][1];
                 *reinterpret_cast<uint4*>(A_t + (ch >> 3) * A_KB + row * 128 + (((ch & 7) ^ (row & 7)) << 4)) =
                     make_uint4(pack_f16x2(x0.x * sc0, x0.y * sc0), pack_f16x2(x0.z * sc0, x0.w * sc0),
