@@ -322,14 +322,17 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     // levels whose gathered records are worth requesting ahead.
     auto staging_of = [&](int req, int& levels, int& count, uint32_t* sparse = nullptr) {
         const int32_t* uoff = a.uoff + req * a.uoff_req_stride;
-        const int e = (lane < old) ? __ldg(uoff + lane + 1) : 0x7fffffff;
+        // (at most the eight oldest levels, whose list positions a unit's lanes hold: the staged fold then never has to
+        // look an index up in memory)
+        const int e_all = (lane < old) ? __ldg(uoff + lane + 1) : 0x7fffffff;
+        const int e = lane < 8 ? e_all : 0x7fffffff;
         levels = __popc(__ballot_sync(0xffffffffu, e <= stage_cap));
         count = __shfl_sync(0xffffffffu, e, levels > 0 ? levels - 1 : 0);
         if (levels == 0) count = 0;
         if (sparse) {
-            int prev = __shfl_up_sync(0xffffffffu, e, 1);
+            int prev = __shfl_up_sync(0xffffffffu, e_all, 1);
             if (lane == 0) prev = 0;
-            *sparse = __ballot_sync(0xffffffffu, lane < old && (e - prev) * 4 > a.W);
+            *sparse = __ballot_sync(0xffffffffu, lane < old && (e_all - prev) * 4 > a.W);
         }
     };
 
@@ -415,6 +418,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
             return info_levels;
         };
         constexpr int NIDX = LPU >= 8 ? 1 : 8 / LPU;     // the unit's lanes hold the indices of its first 8 levels
+        static_assert(NIDX * LPU >= 8, "staging_of stages up to eight levels: their indices must be among the lanes'");
         struct Idx { int32_t v[NIDX]; };
         auto load_idx = [&](const Unit& u) -> Idx {
             const int sl = staged_levels_of(u.req);
@@ -535,6 +539,18 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                     return level < NIDX * LPU ? t
                                               : __ldg((level < staged_levels ? sidx_r : table_r) + (long long)level * a.max_beam + bb);
                 };
+                // The same for a staged level: always among the lanes' (staging_of stages no level beyond them), so no
+                // branch to the look-up in memory stands in the staged fold - merely being there, never taken, it cost
+                // every level a dozen instructions (2.77 -> 2.5 us per level on the beam-512 stack).
+                auto staged_idx_of = [&](int level) -> int32_t {
+                    int32_t t = 0;
+#pragma unroll
+                    for (int j = 0; j < NIDX; ++j) {
+                        const int32_t x = __shfl_sync(0xffffffffu, my_idx.v[j], level & (LPU - 1), LPU);
+                        if (j == level / LPU) t = x;
+                    }
+                    return t;
+                };
 
                 float2 r[4 * NCH], corr[4 * NCH];
                 float kq = 0.f;              // DELTA: k_t . q_t
@@ -615,9 +631,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 if (staged_levels > 0) {
                     const uint8_t* st = stage + buf * (STAGE_BUF * REC_BYTES);
                     const float2* gs = gates_s + buf * STAGE_BUF;
-                    const RecT newest = L::load_shared(st, gs, idx_of(staged_levels - 1), g);
+                    const RecT newest = L::load_shared(st, gs, staged_idx_of(staged_levels - 1), g);
                     L::template fold_chain_simple<DELTA>(newest, staged_levels - 2, 0,
-                                  [&](int level) { return L::load_shared(st, gs, idx_of(level), g); }, r, corr, decay);
+                                  [&](int level) { return L::load_shared(st, gs, staged_idx_of(level), g); }, r, corr, decay);
                 }
                 if (seg_last) {                    // this warp's last read of the segment's staging buffer
                     __syncwarp();
