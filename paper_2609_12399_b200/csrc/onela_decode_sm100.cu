@@ -543,6 +543,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
                 // branch to the look-up in memory stands in the staged fold - merely being there, never taken, it cost
                 // every level a dozen instructions (2.77 -> 2.5 us per level on the beam-512 stack).
                 auto staged_idx_of = [&](int level) -> int32_t {
+                    if constexpr (NIDX == 1) return __shfl_sync(0xffffffffu, my_idx.v[0], level, LPU);   // level < LPU
                     int32_t t = 0;
 #pragma unroll
                     for (int j = 0; j < NIDX; ++j) {
