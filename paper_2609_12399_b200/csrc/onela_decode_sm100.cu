@@ -106,6 +106,7 @@ using RecT = L::R;
 constexpr int TL_CAP = 200;
 __device__ unsigned long long g_ws_tl[3 * TL_CAP];
 __device__ int g_ws_tl_n[3];
+__device__ int g_ws_tl_cta;                       // the CTA whose roles are stamped
 #define TL(ev, g)                                                                                         \
     do {                                                                                                  \
         if (lane == 0 && tl_role >= 0 && tl_n < TL_CAP)                                                   \
@@ -178,7 +179,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_ws_kernel(const __grid_cons
     uint8_t* delta_s = heads + HEADS_TOTAL + 256 + INV_BYTES;                // DELTA: [SLOTS][value rows | scalars]
 #ifdef ONELA_WS_TL
     unsigned long long* tl_s = reinterpret_cast<unsigned long long*>(delta_s + (DELTA ? SLOTS * DELTA_SLOT_BYTES : 0));
-    const int tl_role = blockIdx.x != 0 ? -1 : warp == 0 ? 0 : warp == FOLD_WARPS ? 1 : warp == FOLD_WARPS + 1 ? 2 : -1;
+    const int tl_role = (int)blockIdx.x != g_ws_tl_cta ? -1 : warp == 0 ? 0 : warp == FOLD_WARPS ? 1 : warp == FOLD_WARPS + 1 ? 2 : -1;
     int tl_n = 0;
 #endif
     constexpr int BPG = DELTA ? DELTA_BEAMS : GN;                            // beams per group
@@ -1103,6 +1104,7 @@ cudaError_t launch_ws_t(const DecodeArgs& a, cudaStream_t stream) {
 }  // namespace
 
 #ifdef ONELA_WS_TL
+extern "C" int onela_debug_ws_timeline_cta(int cta) { return (int)cudaMemcpyToSymbol(g_ws_tl_cta, &cta, sizeof(int)); }
 extern "C" int onela_debug_ws_timeline(unsigned long long* out_host, int* counts_host) {
     cudaDeviceSynchronize();
     cudaMemcpyFromSymbol(counts_host, g_ws_tl_n, 3 * sizeof(int));

@@ -1,6 +1,6 @@
 """Clock-stamped timeline of one CTA of the tensor-core decode kernels.
 
-    python -m paper_2609_12399_b200.timeline [--kernel ws|wy] [--workload cfg2|cfg4] [--depth D]
+    python -m paper_2609_12399_b200.timeline [--kernel ws|wy] [--workload cfg2|cfg4] [--depth D] [--cta C]
 
 Builds a debug copy of the library (`-DONELA_WS_TL -DONELA_WY_TL`: the kernels keep clock64 stamps of CTA 0's role
 milestones in shared memory and write them out when the CTA ends; the product library has no such code), runs the
@@ -33,12 +33,15 @@ def main() -> None:
     ap.add_argument("--kernel", default="ws", choices=["ws", "wy"])
     ap.add_argument("--workload", default="cfg4", choices=["cfg2", "cfg4"])
     ap.add_argument("--depth", type=int, default=0, help="chain depth of the launch to show (default: the deepest)")
+    ap.add_argument("--cta", type=int, default=0, help="ws: the CTA whose roles are stamped (default 0)")
     args = ap.parse_args()
     binding.LIB_PATH = build.build_timeline()
     lib = binding.load_library()
     fn = lib.onela_debug_wy_timeline if args.kernel == "wy" else lib.onela_debug_ws_timeline
     fn.restype = ctypes.c_int
     fn.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
+    if args.kernel == "ws" and args.cta:
+        lib.onela_debug_ws_timeline_cta(ctypes.c_int(args.cta))
     roles = ("fold", "epi", "sol", "iss") if args.kernel == "wy" else ("fold", "issue", "store")
     names = WY_NAMES if args.kernel == "wy" else WS_NAMES
     from .binding import FLAG_SHARED_CHAINS, Onela, make_config
