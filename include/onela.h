@@ -85,8 +85,9 @@ typedef int32_t onela_status;
  * projection accumulators S q_t and S k_t forward from S_0 through the beam's records (oldest first).  delta_t
  * depends on the parent state, so records can only be produced where the replay runs: in this mode
  * onela_append_decode_step is the one call per layer and decode call; onela_append_records and onela_decode_step
- * return ONELA_E_UNSUPPORTED.  dk == dv in {32, 64, 128}; 128 x 128 with bf16 records runs on the tensor cores (both
- * projections S q_t and S k_t of a beam go through S_0 in one MMA set), the rest on CUDA cores.  Later calls replay the ROUNDED
+ * return ONELA_E_UNSUPPORTED.  dk == dv in {32, 64, 128}; from 64 x 64 up both projections S q_t and S k_t of a beam go
+ * through S_0 in one MMA set on the tensor cores (128 x 128 bf16 on the warp-specialised kernel, the rest on the tiled
+ * one), 32 x 32 runs on CUDA cores.  Later calls replay the ROUNDED
  * delta, so with bf16 records the result drifts from the exact recurrence by about one bf16 rounding per record
  * (the default raw-record format has no such term). */
 #define ONELA_FLAG_GTR_DELTA 4u
@@ -263,7 +264,7 @@ int64_t onela_launch_count(const onela_ctx* ctx);
 
 /* Which kernel decode_step of this context runs: 1 the warp-specialised tcgen05 kernel (dk = 128, bf16 records),
  * 2 the tiled tcgen05 kernel (every other shape from 64 x 64 up, either record dtype, grouped value heads or not),
- * 0 a CUDA-core kernel (dk = dv = 32, ONELA_FLAG_FORCE_GENERIC, delta records at shapes other than 128 x 128 bf16). */
+ * 0 a CUDA-core kernel (dk = dv = 32, ONELA_FLAG_FORCE_GENERIC). */
 int32_t onela_uses_tensor_core_path(const onela_ctx* ctx);
 
 const char* onela_status_string(onela_status s);

@@ -228,8 +228,8 @@ onela_status onela_create(const onela_config* cfg, void* workspace_dev, size_t w
         r.appended_depth.assign(cfg->num_layers, -1);
     }
     ctx->tensor_core = decode_sm100_supported(cfg->dk, cfg->dv, cfg->rec_dtype) && !(cfg->flags & ONELA_FLAG_FORCE_GENERIC);
-    ctx->tiled_tc = !ctx->tensor_core && decode_tiled_supported(cfg->dk, cfg->dv) &&
-                    !(cfg->flags & (ONELA_FLAG_FORCE_GENERIC | ONELA_FLAG_GTR_DELTA));
+    ctx->tiled_tc = !ctx->tensor_core && decode_tiled_supported(cfg->dk, cfg->dv) && !(cfg->flags & ONELA_FLAG_FORCE_GENERIC) &&
+                    (!(cfg->flags & ONELA_FLAG_GTR_DELTA) || cfg->dk == cfg->dv);     // delta records: square heads
     *out = ctx;
     return ONELA_OK;
 }
@@ -501,6 +501,7 @@ onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count,
         ta.g = ctx->Hv() / c.num_heads;
         ta.depth = depth;
         ta.max_beam = c.max_beam;
+        ta.delta = ctx->gtr() ? 1 : 0;
         for (int i = 0; i < req_count; ++i) ta.bases.base[i] = ctx->req[req_begin + i].step_base.back();
         if (launch_decode_tiled(ta, c.dk, c.dv, c.rec_dtype, c.out_dtype, s) != cudaSuccess) return ONELA_E_CUDA;
         ctx->launches++;

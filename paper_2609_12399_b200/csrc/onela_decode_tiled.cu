@@ -59,9 +59,16 @@ __host__ __device__ constexpr size_t tiled_smem_bytes() {
 template <int KD, int VD>
 __host__ __device__ constexpr int tiled_min_ctas() { return KD + VD <= 128 ? 4 : tiled_beams<KD, VD>() == 64 ? 1 : 2; }
 
-template <int KD, int VD, typename T, typename OutT>
+// DELTA: the arena keeps (alpha_t, delta_t, k_t) (Section 3.2, Eq. 2-4).  A beam owns TWO rows of the tile - its query
+// and its own key, both projected through the parent state: S_{t-1} x = D S_0 x + sum_j d_j (k_j . x) delta_j, the
+// replay leaving x unchanged - and after the contraction delta_t = beta_t (v_t - alpha_t S_{t-1} k_t) and
+// o_t = alpha_t S_{t-1} q_t + delta_t (k_t . q_t) are formed from the two rows and the record is written; always with
+// the append fused in, dk = dv <= 128.
+template <int KD, int VD, typename T, typename OutT, bool DELTA = false>
 __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, VD>()) decode_tiled_kernel(const TiledArgs a) {
     constexpr int NB = tiled_beams<KD, VD>(), THREADS = NB * G;
+    constexpr int BPT = DELTA ? NB / 2 : NB;          // beams per tile
+    static_assert(!DELTA || (KD == VD && VD <= 128), "delta records: square heads, one tile of value rows");
     constexpr uint32_t ACC_COLS = 2 * NB;      // two accumulators of NB columns (a power of two >= 32)
     constexpr int VEC = Vec16<T>::N;
     constexpr int CK = KD / (G * VEC), CV = VD / (G * VEC);   // 16-byte chunks per lane
@@ -100,7 +107,8 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
     const int tile = blockIdx.x, hv = blockIdx.y, req = blockIdx.z;
     const int hk = hv / a.g, Hv = a.Hk * a.g;
     const int grp = tid / G, g = tid % G;
-    const int b = tile * NB + grp;
+    const int b = tile * BPT + (DELTA ? grp >> 1 : grp);
+    const bool key_row = DELTA && (grp & 1);          // DELTA: the odd row of a beam projects its key
     const bool active = b < a.W;
     const int bb = active ? b : a.W - 1;  // idle units shadow a live beam so loads and shuffles stay uniform
 
@@ -201,7 +209,9 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
         }
 #pragma unroll
         for (int off = G / 2; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
-        const float bc = x.gate.y * dot;
+        // (DELTA, Eq. 3: the record's second half is the stored update vector, taken with the weight decay (k . x); the
+        // projected vector is not changed)
+        const float bc = DELTA ? dot : x.gate.y * dot;
         const float wv = decay * bc;
 #pragma unroll
         for (int c = 0; c < CV; ++c) {
@@ -210,8 +220,10 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
 #pragma unroll
             for (int e = 0; e < VEC; ++e) corr[c * VEC + e] = fmaf(wv, vx[e], corr[c * VEC + e]);
         }
+        if constexpr (!DELTA) {
 #pragma unroll
-        for (int e = 0; e < CK * VEC; ++e) r[e] = fmaf(-bc, kx[e], r[e]);
+            for (int e = 0; e < CK * VEC; ++e) r[e] = fmaf(-bc, kx[e], r[e]);
+        }
         decay *= x.gate.x;
     };
     // The beam's own record: from its arena slot, or - append fused in - from the caller's tensors, in which case this
@@ -235,9 +247,11 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
         for (int c = 0; c < CK; ++c) cur.k[c] = __ldg(reinterpret_cast<const uint4*>(ksrc) + c * G + g);
 #pragma unroll
         for (int c = 0; c < CV; ++c) cur.v[c] = __ldg(reinterpret_cast<const uint4*>(vsrc) + c * G + g);
-        if (fused && active) {
+        if (fused && active && !key_row) {
+            if constexpr (!DELTA) {      // (the delta half of a delta record is written after the contraction)
 #pragma unroll
-            for (int c = 0; c < CV; ++c) reinterpret_cast<uint4*>(vdst)[c * G + g] = cur.v[c];
+                for (int c = 0; c < CV; ++c) reinterpret_cast<uint4*>(vdst)[c * G + g] = cur.v[c];
+            }
             if (hv % a.g == 0) {
 #pragma unroll
                 for (int c = 0; c < CK; ++c) reinterpret_cast<uint4*>(kdst)[c * G + g] = cur.k[c];
@@ -245,10 +259,36 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
             if (g == 0) gates[slot] = cur.gate;
         }
     }
+    float kq = 0.f;          // DELTA: k_t . q_t
+    if constexpr (DELTA) {
+        float kx[CK * VEC];
+#pragma unroll
+        for (int c = 0; c < CK; ++c) {
+            Vec16<T>::unpack(cur.k[c], kx + c * VEC);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) kq = fmaf(kx[c * VEC + e], r[c * VEC + e], kq);
+        }
+#pragma unroll
+        for (int off = G / 2; off > 0; off >>= 1) kq += __shfl_xor_sync(0xffffffffu, kq, off);
+        if (key_row) {
+#pragma unroll
+            for (int e = 0; e < CK * VEC; ++e) r[e] = kx[e];
+        }
+    }
     // Narrow records are fetched one level ahead of their fold (the chain is a string of dependent loads otherwise);
     // wide ones would not fit in the registers twice.
     constexpr bool AHEAD = KD + VD <= 256;
-    if constexpr (AHEAD) {
+    if constexpr (DELTA) {                 // the replay runs over the older records only
+        if (old > 0) {
+            Raw x = fetch(old - 1);
+            for (int level = old - 2; level >= 0; --level) {
+                const Raw next = fetch(level);
+                fold(x);
+                x = next;
+            }
+            fold(x);
+        }
+    } else if constexpr (AHEAD) {
         for (int level = old - 1; level >= 0; --level) {
             const Raw next = fetch(level);
             fold(cur);
@@ -340,7 +380,26 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();
         if (ABUF == 1 && mt + 1 < MT && tid == 0) issue(mt + 1);
-        if (active) {
+        if constexpr (DELTA) {
+            // Eq. 2 and 4 on the beam's two rows (even: S_{t-1} q_t, odd: S_{t-1} k_t), by the even row's lanes:
+            //   delta_t = beta_t (v_t - alpha_t S_{t-1} k_t) ,  o_t = alpha_t S_{t-1} q_t + delta_t (k_t . q_t)
+            if (active && !key_row) {
+                T* ddst = vplane + (long long)(a.bases.base[req] + bb) * a.v_stride;
+#pragma unroll
+                for (int c = 0; c < CV; ++c) {
+                    const float* uq = C_s + grp * CP + (c * G + g) * VEC;
+                    float vx[VEC], dl[VEC], o[VEC];
+                    Vec16<T>::unpack(cur.v[c], vx);
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) {
+                        dl[e] = cur.gate.y * fmaf(-cur.gate.x, uq[CP + e], vx[e]);
+                        o[e] = fmaf(dl[e], kq, cur.gate.x * uq[e]);
+                    }
+                    store_out<OutT, VEC>(out + (c * G + g) * VEC, o);
+                    store_out<T, VEC>(ddst + (c * G + g) * VEC, dl);
+                }
+            }
+        } else if (active) {
 #pragma unroll
             for (int c = 0; c < CV; ++c) {
                 if ((c * G * VEC) / 128 != mt) continue;
@@ -366,35 +425,43 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
     }
 }
 
-template <int KD, int VD, typename T, typename OutT>
+template <int KD, int VD, typename T, typename OutT, bool DELTA = false>
 cudaError_t launch_one(const TiledArgs& a, cudaStream_t stream) {
-    auto kern = decode_tiled_kernel<KD, VD, T, OutT>;
-    constexpr int NB = tiled_beams<KD, VD>(), THREADS = NB * G;
+    auto kern = decode_tiled_kernel<KD, VD, T, OutT, DELTA>;
+    constexpr int NB = tiled_beams<KD, VD>(), THREADS = NB * G, BPT = DELTA ? NB / 2 : NB;
     constexpr size_t smem = tiled_smem_bytes<KD, VD>();
     static_assert(smem <= 232448, "shared memory per CTA");
-    static std::once_flag once;          // one per instantiation
-    static cudaError_t attr = cudaSuccess;
-    std::call_once(once, [&] {
-        attr = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        // shared memory for the CTAs the registers allow and no more: what is left of the SM's 228 KB serves the fold's
-        // record loads as L1 (asking for all of it made 128 x 128 fp32 14 % slower)
-        constexpr int pct = (int)((tiled_min_ctas<KD, VD>() * (smem + 1024) * 100 + 228 * 1024 - 1) / (228 * 1024));
-        if (attr == cudaSuccess) attr = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, pct > 100 ? 100 : pct);
-    });
-    if (attr != cudaSuccess) return attr;
-    dim3 grid((a.W + NB - 1) / NB, a.Hk * a.g, a.req_count);
+    // One-time set-up per instantiation and device (function attributes belong to a device's context).
+    constexpr int MAX_DEVICES = 64;
+    static std::mutex setup_mutex;
+    static bool ready[MAX_DEVICES] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+    {
+        std::lock_guard<std::mutex> lock(setup_mutex);
+        if (!ready[dev]) {
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            // shared memory for the CTAs the registers allow and no more: what is left of the SM's 228 KB serves the
+            // fold's record loads as L1 (asking for all of it made 128 x 128 fp32 14 % slower)
+            constexpr int pct = (int)((tiled_min_ctas<KD, VD>() * (smem + 1024) * 100 + 228 * 1024 - 1) / (228 * 1024));
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, pct > 100 ? 100 : pct);
+            if (e != cudaSuccess) return e;
+            ready[dev] = true;
+        }
+    }
+    dim3 grid((a.W + BPT - 1) / BPT, a.Hk * a.g, a.req_count);
     kern<<<grid, THREADS, smem, stream>>>(a);
     return cudaGetLastError();
 }
 
-template <int KD, int VD>
+template <int KD, int VD, bool DELTA = false>
 cudaError_t launch_dims(const TiledArgs& a, int32_t rec_dtype, int32_t out_dtype, cudaStream_t stream) {
     if (rec_dtype == ONELA_DTYPE_BF16) {
-        return out_dtype == ONELA_DTYPE_BF16 ? launch_one<KD, VD, __nv_bfloat16, __nv_bfloat16>(a, stream)
-                                             : launch_one<KD, VD, __nv_bfloat16, float>(a, stream);
+        return out_dtype == ONELA_DTYPE_BF16 ? launch_one<KD, VD, __nv_bfloat16, __nv_bfloat16, DELTA>(a, stream)
+                                             : launch_one<KD, VD, __nv_bfloat16, float, DELTA>(a, stream);
     }
-    return out_dtype == ONELA_DTYPE_BF16 ? launch_one<KD, VD, float, __nv_bfloat16>(a, stream)
-                                         : launch_one<KD, VD, float, float>(a, stream);
+    return out_dtype == ONELA_DTYPE_BF16 ? launch_one<KD, VD, float, __nv_bfloat16, DELTA>(a, stream)
+                                         : launch_one<KD, VD, float, float, DELTA>(a, stream);
 }
 
 }  // namespace
@@ -405,6 +472,12 @@ bool decode_tiled_supported(int32_t dk, int32_t dv) {
 
 cudaError_t launch_decode_tiled(const TiledArgs& a, int32_t dk, int32_t dv, int32_t rec_dtype, int32_t out_dtype,
                                 cudaStream_t stream) {
+    if (a.delta) {       // (alpha, delta, k) records: square heads, the append fused in
+        if (!a.k_in || a.g != 1) return cudaErrorInvalidValue;
+        if (dk == 64 && dv == 64) return launch_dims<64, 64, true>(a, rec_dtype, out_dtype, stream);
+        if (dk == 128 && dv == 128) return launch_dims<128, 128, true>(a, rec_dtype, out_dtype, stream);
+        return cudaErrorInvalidValue;
+    }
     if (dk == 64 && dv == 64) return launch_dims<64, 64>(a, rec_dtype, out_dtype, stream);
     if (dk == 128 && dv == 128) return launch_dims<128, 128>(a, rec_dtype, out_dtype, stream);
     if (dk == 128 && dv == 256) return launch_dims<128, 256>(a, rec_dtype, out_dtype, stream);

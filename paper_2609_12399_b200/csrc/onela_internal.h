@@ -124,6 +124,7 @@ struct TiledArgs {
     int32_t* status;
     long long s0_req_stride, s0_scale_req_stride, table_req_stride, arena_slots, k_stride, v_stride;
     int32_t req_count, W, Hk, g, depth, max_beam;
+    int32_t delta;          // 1: the arena keeps (alpha, delta, k) records and the launch replays both projections forward
     BatchBases bases;
 };
 bool decode_tiled_supported(int32_t dk, int32_t dv);

@@ -26,8 +26,9 @@ def _check(case, out_dtype, tight=None, batched=True, cuda_cores=False):
     wl = case["wl"]
     flags = P.FLAG_GTR_DELTA | (P.FLAG_FORCE_GENERIC if cuda_cores else 0)
     outs, slots, ctx = run_library(case, out_dtype=out_dtype, flags=flags, batched=batched, fused=True)
-    # 128 x 128 bf16 records: both projections of the parent state run on the tensor cores
-    assert ctx.onela_uses_tensor_core_path() == ((wl.dk, wl.dv, wl.dtype) == (128, 128, "bf16") and not cuda_cores)
+    # both projections of the parent state run on the tensor cores: 128 x 128 bf16 records on the warp-specialised kernel,
+    # the other shapes from 64 x 64 up on the tiled one; 32 x 32 and the forced path on CUDA cores
+    assert ctx.onela_uses_tensor_core_path() == (0 if cuda_cores or wl.dk < 64 else 1 if (wl.dk, wl.dtype) == (128, "bf16") else 2)
     want = expected_slots(case, chains)
     for key in want:
         assert np.array_equal(slots[key], want[key]), f"ancestry rows of {key} differ"
@@ -55,11 +56,26 @@ def test_bf16_records_ragged_beams_many_segments():
     _check(make_case(wl, widths=[25, 1, 24]), "fp32", batched=False)
 
 
-def test_fp32_records_other_shapes_and_ragged_widths():
+@pytest.mark.parametrize("cuda_cores", [False, True])
+def test_fp32_records_other_shapes_and_ragged_widths(cuda_cores):
+    """fp32 records: within rounding on the CUDA cores (fp32 throughout), within the bar on the tiled tensor-core kernel
+    (fp16 operands of the two projections)."""
+    tight = 5e-6 if cuda_cores else None
     wl = CFG1.scaled(R=2, L=2, H=3, dk=64, dv=64, dtype="fp32", W=37, D=4, prompt_len=48, parents="zipf", zipf_s=1.3, seed=61)
-    _check(make_case(wl), "fp32", tight=5e-6)
+    _check(make_case(wl), "fp32", tight=tight, cuda_cores=cuda_cores)
     wl = CFG1.scaled(R=1, L=1, H=2, dtype="fp32", W=50, D=5, prompt_len=64, seed=62)
-    _check(make_case(wl, widths=[50, 7, 33, 64, 20]), "fp32", tight=5e-6, batched=False)
+    _check(make_case(wl, widths=[50, 7, 33, 64, 20]), "fp32", tight=tight, batched=False, cuda_cores=cuda_cores)
+
+
+@pytest.mark.parametrize("dk,dtype,out_dtype", [(64, "bf16", "bf16"), (64, "bf16", "fp32"), (64, "fp32", "bf16"), (128, "fp32", "fp32")])
+def test_delta_records_on_the_tiled_tensor_core_kernel(dk, dtype, out_dtype):
+    """Deeper chains with shared ancestors, several requests and layers, a ragged last tile (16 or 32 beams per tile:
+    two rows each) and a single beam; the stored records are the caller's key bytes and
+    delta_t = beta_t (v_t - alpha_t S_{t-1} k_t) from the oracle's states."""
+    wl = CFG1.scaled(R=2, L=2, H=3, dk=dk, dv=dk, dtype=dtype, W=45, D=6, prompt_len=48, parents="zipf", zipf_s=1.4, seed=66 + dk)
+    worst, ctx = _check(make_case(wl), out_dtype)
+    assert ctx.onela_uses_tensor_core_path() == 2 and worst <= REL_L2_BAR
+    _check(make_case(CFG1.scaled(R=1, L=1, H=2, dk=dk, dv=dk, dtype=dtype, W=33, D=3, prompt_len=32, seed=67), widths=[33, 1, 17]), out_dtype, batched=False)
 
 
 def test_bf16_records_deep_chain_with_shared_ancestors():
@@ -70,12 +86,15 @@ def test_bf16_records_deep_chain_with_shared_ancestors():
     assert worst <= REL_L2_BAR
 
 
-def test_stored_records_are_key_bytes_and_update_vectors():
+@pytest.mark.parametrize("cuda_cores,tol", [(True, 2e-5), (False, 2e-3)])
+def test_stored_records_are_key_bytes_and_update_vectors(cuda_cores, tol):
     """The arena holds (k_t bit for bit | delta_t), gates (alpha_t, beta_t); delta_t is checked against
-    beta_t (v_t - alpha_t S_{t-1} k_t) with S_{t-1} the parent beam's state from the fp64 full-state recurrence."""
+    beta_t (v_t - alpha_t S_{t-1} k_t) with S_{t-1} the parent beam's state from the fp64 full-state recurrence:
+    within fp32 rounding on the CUDA cores, within the fp16 operands' rounding on the tiled tensor-core kernel."""
     wl = CFG1.scaled(R=1, H=2, dtype="fp32", W=12, D=3, prompt_len=32, seed=64)
     case = make_case(wl)
-    outs, slots, ctx = run_library(case, out_dtype="fp32", flags=P.FLAG_GTR_DELTA, fused=True)
+    outs, slots, ctx = run_library(case, out_dtype="fp32", flags=P.FLAG_GTR_DELTA | (P.FLAG_FORCE_GENERIC if cuda_cores else 0), fused=True)
+    assert ctx.onela_uses_tensor_core_path() == (0 if cuda_cores else 2)
     c = ctx.cfg
     al = lambda n: (n + 1023) // 1024 * 1024
     n_idx = c.num_requests * c.max_steps * c.max_beam * 4
@@ -102,7 +121,7 @@ def test_stored_records_are_key_bytes_and_update_vectors():
                 delta = b_ * (v - a_ * (S_par[h] @ k))
                 S_new[h] = a_ * S_par[h] + np.outer(delta, k)     # Eq. 1 in the paper's record form
                 got = kv[h, base + b, 128:].double().numpy()
-                assert np.linalg.norm(got - delta) <= 2e-5 * max(np.linalg.norm(delta), 1e-3), (t, b, h)
+                assert np.linalg.norm(got - delta) <= tol * max(np.linalg.norm(delta), 1e-3), (t, b, h)
                 assert torch.equal(kv[h, base + b, :128], tk["k"][b, h])
                 assert float(gates[h, base + b, 0]) == a_
             new[b] = S_new

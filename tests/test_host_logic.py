@@ -155,7 +155,7 @@ def test_delta_record_mode_takes_only_the_fused_call():
 def test_kernel_choice_by_shape_dtype_and_flags():
     """Which decode kernel a configuration gets (onela_uses_tensor_core_path): 1 the warp-specialised tcgen05 kernel
     (dk = 128, bf16 records, any supported dv, grouped or not), 2 the tiled tcgen05 kernel (every other shape from
-    64 x 64 up, either record dtype), 0 CUDA cores (32 x 32, the force flag, delta records at the other shapes)."""
+    64 x 64 up, either record dtype, raw or delta records), 0 CUDA cores (32 x 32, the force flag)."""
     def kernel(dk, dv, rec, flags=0, hv=0):
         cfg = P.make_config(1, 1, 2, dk, dv, 8, 3, rec, "fp32", 64, P.FLAG_DRY_RUN | flags, num_v_heads=hv)
         return P.Onela(cfg, device="cpu").onela_uses_tensor_core_path()
@@ -166,7 +166,9 @@ def test_kernel_choice_by_shape_dtype_and_flags():
         assert kernel(dk, dv, "bf16", P.FLAG_FORCE_GENERIC) == 0
     assert kernel(32, 32, "fp32") == 0 and kernel(32, 32, "bf16") == 0
     assert kernel(128, 128, "bf16", P.FLAG_FORCE_GENERIC) == 0
-    assert kernel(64, 64, "fp32", P.FLAG_GTR_DELTA) == 0 and kernel(128, 128, "bf16", P.FLAG_GTR_DELTA) == 1
+    assert kernel(64, 64, "fp32", P.FLAG_GTR_DELTA) == 2 and kernel(128, 128, "bf16", P.FLAG_GTR_DELTA) == 1
+    assert kernel(128, 128, "fp32", P.FLAG_GTR_DELTA) == 2 and kernel(32, 32, "fp32", P.FLAG_GTR_DELTA) == 0
+    assert kernel(64, 64, "bf16", P.FLAG_GTR_DELTA | P.FLAG_FORCE_GENERIC) == 0
     assert kernel(128, 128, "bf16", hv=4) == 1 and kernel(64, 64, "bf16", hv=4) == 2 and kernel(128, 256, "fp32", hv=6) == 2
 
 
