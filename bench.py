@@ -341,19 +341,24 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> dict:
     if rank == 0 and world == 1 and default_path and not args.no_secondary:
         del graph
         # the other beam-512 config and the large-batch config, in the same run (context, not the bench value)
-        line["secondary"] = [secondary_roofline(n, dev, peak, mhz) for n in ("cfg2", "cfg3")]
+        # configs 2 and 3 as they are (one layer: every launch alone after a flushed L2), and config 2's launch as a
+        # decoder's layer loop issues it (16 layers back to back)
+        line["secondary"] = [secondary_roofline("cfg2", dev, peak, mhz), secondary_roofline("cfg2", dev, peak, mhz, layers=16),
+                             secondary_roofline("cfg3", dev, peak, mhz)]
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(wl, reps=1, gen_device=dev)
     return line
 
 
-def secondary_roofline(name: str, dev, peak: float, mhz: float, reps: int = 5) -> dict:
+def secondary_roofline(name: str, dev, peak: float, mhz: float, reps: int = 5, layers: int = 0) -> dict:
     """The same roofline block for another benchmark config, timed in this run: whole generations launched eagerly
     with the fused call, one CUDA-event pair around each decode call's launches.  These workloads are smaller than
     L2, so a buffer larger than L2 is overwritten before every decode call's launches (outside the event pairs)."""
     from paper_2609_12399_b200.runner import WorkloadRun
 
     wl = workload_by_name(name)
+    if layers:     # the same launch over a decoder's layers, back to back: each starts under its predecessor's tail
+        wl = wl.scaled(name=f"{wl.name}_x{layers}layers", L=layers, prompt_len=min(wl.prompt_len, 1024))
     run = WorkloadRun(wl, dev, wl.dtype)
     ctx = run.ctx
     run.prefill_states()
@@ -369,6 +374,9 @@ def secondary_roofline(name: str, dev, peak: float, mhz: float, reps: int = 5) -
         ctx.onela_init_shared_states(0, wl.R, S0_all)
         for call in calls:
             flush.zero_()
+            if wl.L > 1:
+                torch.cuda._sleep(int(1.0e6))     # ~0.5 ms of spin: the call's launches queue up behind it, so the event
+                                                  # pair times them back to back, not the host's launch rate
             run.run_call(call, outs, None, pairs if record else None, fused=True, group_events=True)
 
     for _ in range(3):
@@ -385,7 +393,7 @@ def secondary_roofline(name: str, dev, peak: float, mhz: float, reps: int = 5) -
     units = wl.R * wl.W * wl.H
     del run, calls, outs, flush
     return {"workload": describe(wl), "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-            "traffic": None, "l2": "a 256 MiB buffer is overwritten before every decode call (the workload is smaller than L2)",
+            "traffic": None, "l2": "a 256 MiB buffer is overwritten before every decode call's launches (one layer of these workloads is smaller than L2)",
             "decodes_per_s": units * wl.L * wl.D / (float(ms_depth.sum()) * 1e-3 * wl.L),
             "per_depth": [{"depth": t + 1, "us": float(ms_depth[t] * 1e3), "sm_cycles": float(ms_depth[t] * 1e3 * mhz),
                            "algorithmic_MB": per_depth[t]["algorithmic"] / 1e6,
