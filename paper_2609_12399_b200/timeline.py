@@ -34,6 +34,9 @@ def main() -> None:
     ap.add_argument("--workload", default="cfg4", choices=["cfg2", "cfg4"])
     ap.add_argument("--depth", type=int, default=0, help="chain depth of the launch to show (default: the deepest)")
     ap.add_argument("--cta", type=int, default=0, help="ws: the CTA whose roles are stamped (default 0)")
+    ap.add_argument("--layers", type=int, default=1,
+                    help="launch the call over this many layers back to back and show the LAST launch (its start then "
+                         "overlaps its predecessor's tail, as in a decoder's layer loop)")
     args = ap.parse_args()
     binding.LIB_PATH = build.build_timeline()
     lib = binding.load_library()
@@ -46,7 +49,7 @@ def main() -> None:
     names = WY_NAMES if args.kernel == "wy" else WS_NAMES
     from .binding import FLAG_SHARED_CHAINS, Onela, make_config
 
-    wl = inputs.WORKLOADS[int(args.workload[3])].scaled(L=1, prompt_len=64)
+    wl = inputs.WORKLOADS[int(args.workload[3])].scaled(L=max(1, args.layers), prompt_len=64)
     depth_show = args.depth or wl.D
     dev = torch.device("cuda")
     cfg = make_config(wl.R, wl.L, wl.H, wl.dk, wl.dv, wl.W, wl.D, wl.dtype, "bf16", wl.R * wl.W * wl.D,
@@ -54,7 +57,8 @@ def main() -> None:
     ctx = Onela(cfg, device="cuda")
     S0 = torch.randn(wl.R * wl.H, wl.dv, wl.dk, device=dev, generator=torch.Generator(device=dev).manual_seed(1)) * 0.1
     for r in range(wl.R):
-        ctx.onela_init_shared_state(r, 0, S0[r * wl.H:(r + 1) * wl.H].contiguous())
+        for l in range(wl.L):
+            ctx.onela_init_shared_state(r, l, S0[r * wl.H:(r + 1) * wl.H].contiguous())
     buf = (ctypes.c_ulonglong * 800)()
     cnt = (ctypes.c_int * 4)()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
@@ -65,11 +69,14 @@ def main() -> None:
         tk = {nm: torch.stack([inputs.decode_token(wl, r, 0, t, beams=beams, device=dev)[nm] for r in range(wl.R)])
               for nm in ("k", "v", "alpha", "beta")}
         q = torch.stack([inputs.decode_query(wl, r, 0, t, beams=beams, device=dev) for r in range(wl.R)])
-        out = torch.empty((wl.R, wl.W, wl.H, wl.dv), dtype=torch.bfloat16, device=dev)
+        outs = [torch.empty((wl.R, wl.W, wl.H, wl.dv), dtype=torch.bfloat16, device=dev) for _ in range(wl.L)]
         flush.zero_()                                   # cold L2, as in the benchmark's timing of these workloads
         torch.cuda.synchronize()
         fn(buf, cnt)                                    # clears the stamps of earlier launches
-        ctx.onela_append_decode_step(0, wl.R, 0, tk["k"], tk["v"], tk["alpha"], tk["beta"], q, out)
+        if wl.L > 1:
+            torch.cuda._sleep(int(2.0e6))               # the layers' launches queue up behind a short spin
+        for l in range(wl.L):                           # (every layer gets the same seeded token: timing only)
+            ctx.onela_append_decode_step(0, wl.R, l, tk["k"], tk["v"], tk["alpha"], tk["beta"], q, outs[l])
         torch.cuda.synchronize()
         cap = fn(buf, cnt)
         if t + 1 != depth_show:
