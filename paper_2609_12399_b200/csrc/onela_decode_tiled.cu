@@ -46,6 +46,12 @@ constexpr int ROW_TARGET = 8;          // a scaled operand row's largest element
 // 256 x 512 with 65 536 units) were what bounded the kernel; one CTA of 512 threads holds as many warps as two of 256.
 template <int KD, int VD>
 __host__ __device__ constexpr int tiled_beams() { return KD * VD >= 128 * 128 ? 64 : 32; }
+#ifdef ONELA_TEST_HOOKS
+// Test-hooks build only (a second library that the product never loads): when set, CTA (0, 0, 0) leaves out its first
+// tile's MMAs and their commit, so that the wait for them runs out.
+__device__ int g_hook_tiled_skip_issue;
+#endif
+
 template <int KD, int VD>
 __host__ __device__ constexpr size_t tiled_smem_bytes() {
     // two A operands where there is a next tile to prepare and the key is narrow (at key width 256 the second buffer
@@ -330,7 +336,11 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+#ifdef ONELA_TEST_HOOKS
+    if (tid == 0 && !(g_hook_tiled_skip_issue && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)) issue(0);
+#else
     if (tid == 0) issue(0);
+#endif
 
     OutT* out = static_cast<OutT*>(a.out) + (((long long)req * a.W + b) * Hv + hv) * VD;
     const int quad = warp & 3, half = warp >> 2;     // tensor-memory lane quadrant of this warp, and which 16 beams it takes
@@ -465,6 +475,12 @@ cudaError_t launch_dims(const TiledArgs& a, int32_t rec_dtype, int32_t out_dtype
 }
 
 }  // namespace
+
+#ifdef ONELA_TEST_HOOKS
+extern "C" int onela_testhook_tiled_skip_issue(int on) {
+    return (int)cudaMemcpyToSymbol(g_hook_tiled_skip_issue, &on, sizeof(int));
+}
+#endif
 
 bool decode_tiled_supported(int32_t dk, int32_t dv) {
     return (dk == 64 && dv == 64) || (dk == 128 && (dv == 128 || dv == 256 || dv == 512)) || (dk == 256 && (dv == 256 || dv == 512));
