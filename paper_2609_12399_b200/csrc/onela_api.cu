@@ -37,6 +37,13 @@ bool config_sane(const onela_config* c) {
     return true;
 }
 
+// Whether decode_step of this configuration runs the tiled tcgen05 kernel (the other shapes from 64 x 64 up).
+bool uses_tiled_kernel(const onela_config& c) {
+    const bool forced = c.flags & ONELA_FLAG_FORCE_GENERIC;
+    if (forced || decode_sm100_supported(c.dk, c.dv, c.rec_dtype)) return false;
+    return decode_tiled_supported(c.dk, c.dv) && (!(c.flags & ONELA_FLAG_GTR_DELTA) || c.dk == c.dv);   // delta records: square heads
+}
+
 // Carve the workspace.  `base` may be null (size query only).
 Layout carve(const onela_config& c, char* base) {
     const size_t es = c.rec_dtype == ONELA_DTYPE_BF16 ? 2 : 4;
@@ -67,6 +74,8 @@ Layout carve(const onela_config& c, char* base) {
     l.urep = reinterpret_cast<int32_t*>(take((size_t)c.num_requests * c.max_steps * c.max_beam * sizeof(int32_t)));
     l.sg8 = reinterpret_cast<uint8_t*>(take((size_t)c.num_requests * c.max_steps * sg_row_stride(c.max_beam)));
     l.unode = reinterpret_cast<uint8_t*>(take((size_t)c.num_requests * ONELA_UNODE_CAP * 16));
+    if (uses_tiled_kernel(c))
+        l.s0_f16 = reinterpret_cast<uint16_t*>(take((size_t)c.num_requests * c.num_layers * Hv * s0_f16_head_bytes(c.dk, c.dv)));
     l.total_bytes = off;
     return l;
 }
@@ -95,6 +104,15 @@ struct onela_ctx {
     long long s0_layer_floats() const { return (long long)Hv() * cfg.dv * cfg.dk; }
     float* s0_slot(int r, int l) const { return lay.s0 + ((long long)r * cfg.num_layers + l) * s0_layer_floats(); }
     float* s0_scale_slot(int r, int l) const { return lay.s0_scale + ((long long)r * cfg.num_layers + l) * Hv(); }
+    uint16_t* s0_f16_slot(int r, int l) const {       // tiled kernel's operand copy of (request, layer, head 0)
+        return lay.s0_f16 + ((long long)r * cfg.num_layers + l) * Hv() * (long long)(s0_f16_head_bytes(cfg.dk, cfg.dv) / 2);
+    }
+    // after a state write: the tiled kernel's operand copy of the n_heads states from (r, l) on
+    cudaError_t pack_states(int r, int l, long long n_heads, cudaStream_t s) {
+        if (!tiled_tc) return cudaSuccess;
+        launches++;
+        return launch_pack_state(s0_slot(r, l), s0_scale_slot(r, l), s0_f16_slot(r, l), n_heads, cfg.dk, cfg.dv, s);
+    }
     int32_t* table_cur(int r) const {
         const int d = req[r].depth;
         return lay.tables + r * table_req_stride() + (long long)((d - 1) & 1) * cfg.max_steps * cfg.max_beam;
@@ -228,8 +246,7 @@ onela_status onela_create(const onela_config* cfg, void* workspace_dev, size_t w
         r.appended_depth.assign(cfg->num_layers, -1);
     }
     ctx->tensor_core = decode_sm100_supported(cfg->dk, cfg->dv, cfg->rec_dtype) && !(cfg->flags & ONELA_FLAG_FORCE_GENERIC);
-    ctx->tiled_tc = !ctx->tensor_core && decode_tiled_supported(cfg->dk, cfg->dv) && !(cfg->flags & ONELA_FLAG_FORCE_GENERIC) &&
-                    (!(cfg->flags & ONELA_FLAG_GTR_DELTA) || cfg->dk == cfg->dv);     // delta records: square heads
+    ctx->tiled_tc = uses_tiled_kernel(*cfg);
     *out = ctx;
     return ONELA_OK;
 }
@@ -263,6 +280,7 @@ onela_status onela_init_shared_state(onela_ctx* ctx, int32_t request, int32_t la
                                ctx->cfg.dk, ctx->cfg.dv, s) != cudaSuccess)
             return ONELA_E_CUDA;
         ctx->launches++;
+        if (ctx->pack_states(request, layer, ctx->Hv(), s) != cudaSuccess) return ONELA_E_CUDA;
     }
     finish_state_write(ctx, request, layer);
     return ONELA_OK;
@@ -282,6 +300,7 @@ onela_status onela_init_shared_states(onela_ctx* ctx, int32_t req_begin, int32_t
                                s) != cudaSuccess)
             return ONELA_E_CUDA;
         ctx->launches++;
+        if (ctx->pack_states(req_begin, 0, (long long)req_count * ctx->cfg.num_layers * ctx->Hv(), s) != cudaSuccess) return ONELA_E_CUDA;
     }
     for (int32_t r = req_begin; r < req_begin + req_count; ++r)
         for (int32_t l = 0; l < ctx->cfg.num_layers; ++l) finish_state_write(ctx, r, l);
@@ -307,6 +326,7 @@ onela_status onela_prefill_shared_state(onela_ctx* ctx, int32_t request, int32_t
         if (!supported) return ONELA_E_UNSUPPORTED;
         if (e != cudaSuccess) return ONELA_E_CUDA;
         ctx->launches++;
+        if (ctx->pack_states(request, layer, ctx->Hv(), s) != cudaSuccess) return ONELA_E_CUDA;
     }
     finish_state_write(ctx, request, layer);
     return ONELA_OK;
@@ -478,6 +498,8 @@ onela_status launch_decode(onela_ctx* ctx, int32_t req_begin, int32_t req_count,
         ta.beta_in = beta_dev;
         ta.s0 = ctx->s0_slot(req_begin, layer);
         ta.s0_scale = ctx->s0_scale_slot(req_begin, layer);
+        ta.s0_f16 = reinterpret_cast<const char*>(ctx->s0_f16_slot(req_begin, layer));
+        ta.s0_f16_req_stride = (long long)c.num_layers * ctx->Hv() * (long long)s0_f16_head_bytes(c.dk, c.dv);
         if (ctx->grouped()) {
             ta.kplane = ctx->k_plane(layer);
             ta.vplane = ctx->v_plane(layer);

@@ -26,7 +26,9 @@ namespace onela {
 
 namespace {
 
+using sm100::bulk_load;
 using sm100::idesc_f16;
+using sm100::mbar_expect_tx;
 using sm100::mbar_init;
 using sm100::mbar_wait;
 using sm100::pack_f16x2;
@@ -92,12 +94,15 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
     uint8_t* R_s = A_s + ABUF * KB * A_KB;                             // [KB][NB rows][128 bytes]
     float* C_s = reinterpret_cast<float*>(R_s + KB * R_KB);            // [NB][CP]
     float* inv_s = C_s + NB * CP;                                      // [NB] what undoes a row's scales
-    uint64_t* bar = reinterpret_cast<uint64_t*>(inv_s + NB);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar + 1);
+    uint64_t* bar = reinterpret_cast<uint64_t*>(inv_s + NB);          // a tile's MMAs complete
+    uint64_t* abar = bar + 1;                                          // [2] an A operand has landed
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(abar + 2);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
         mbar_init(smem_u32(bar), 1);
+        mbar_init(smem_u32(abar), 1);
+        mbar_init(smem_u32(abar + 1), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
@@ -118,43 +123,28 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
     const bool active = b < a.W;
     const int bb = active ? b : a.W - 1;  // idle units shadow a live beam so loads and shuffles stay uniform
 
-    const float* S0h = a.s0 + req * a.s0_req_stride + (long long)hv * VD * KD;
     const float sc0 = __ldg(a.s0_scale + req * a.s0_scale_req_stride + hv);     // a power of two
-    // S_0 rows [128 mt, 128 mt + 128) -> A operand (rows beyond dv are zero); a warp reads whole rows
-    auto put_A = [&](int mt) {
-        uint8_t* A_t = A_s + (mt & (ABUF - 1)) * (KB * A_KB);
-        constexpr int CPR = KD / 8;        // 16-byte fp16 chunks per row
-        constexpr int ITEMS = 128 * CPR / THREADS, UNR = ITEMS % 4 == 0 ? 4 : 2;
-        static_assert(128 * CPR % THREADS == 0 && ITEMS % UNR == 0, "every thread converts the same number of chunks");
-#pragma unroll 1
-        for (int it = 0; it < ITEMS; it += UNR) {       // UNR chunks' loads in flight together
-            float4 x[UNR][2];
+    // The A operand of tile mt (S_0 rows [128 mt, 128 mt + 128), rows beyond dv zero): the store keeps every state as
+    // this kernel's operand as well - fp16, times the head's scale, in 16 KB tiles of 128 rows x 64 columns laid out
+    // as the MMA reads them - so a tile is dk / 64 bulk copies of 16 KB, requested by one thread, landing on a barrier
+    // of their own while the CTA does something else (the fold; the previous tile's epilogue).
+    const char* A_src = a.s0_f16 + req * a.s0_f16_req_stride + (long long)hv * ((long long)MT * KB * A_KB);
+    int a_loads = 0, a_waits = 0;         // thread 0: A operands requested / waited for
+    auto load_A = [&](int mt) {           // thread 0 only
+        const uint32_t ab = smem_u32(abar + (mt & (ABUF - 1)));
+        mbar_expect_tx(ab, KB * A_KB);
 #pragma unroll
-            for (int u = 0; u < UNR; ++u) {
-                // a warp takes one K block (8 chunks = 256 bytes of fp32) of four consecutive rows: whole 128-byte lines
-                // from global memory, 512 consecutive bytes of shared memory (no bank conflicts)
-                const int wi = (it + u) * (THREADS / 32) + warp, row = (wi / KB) * 4 + (lane >> 3), ch = (wi % KB) * 8 + (lane & 7);
-                const int i = mt * 128 + row;
-                if (i < VD) {
-                    const float4* p = reinterpret_cast<const float4*>(S0h + (long long)i * KD + ch * 8);
-                    x[u][0] = __ldg(p);
-                    x[u][1] = __ldg(p + 1);
-                } else {
-                    x[u][0] = x[u][1] = make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < UNR; ++u) {
-                const int wi = (it + u) * (THREADS / 32) + warp, row = (wi / KB) * 4 + (lane >> 3), ch = (wi % KB) * 8 + (lane & 7);
-                const float4 x0 = x[u][0], x1 = x[u][1];
-                *reinterpret_cast<uint4*>(A_t + (ch >> 3) * A_KB + row * 128 + (((ch & 7) ^ (row & 7)) << 4)) =
-                    make_uint4(pack_f16x2(x0.x * sc0, x0.y * sc0), pack_f16x2(x0.z * sc0, x0.w * sc0),
-                               pack_f16x2(x1.x * sc0, x1.y * sc0), pack_f16x2(x1.z * sc0, x1.w * sc0));
-            }
-        }
+        for (int kb = 0; kb < KB; ++kb)
+            bulk_load(smem_u32(A_s + (mt & (ABUF - 1)) * (KB * A_KB) + kb * A_KB), A_src + ((long long)mt * KB + kb) * A_KB, A_KB, ab);
+        ++a_loads;
     };
-    // one thread: the tile's dk / 16 MMAs into accumulator mt & 1, and the commit that completes the barrier's phase
+    // one thread: once the tile's A operand has landed, its dk / 16 MMAs into accumulator mt & 1 and the commit that
+    // completes the barrier's phase (if the operand does not land in time nothing is issued, and the CTA's wait for the
+    // MMAs runs out in turn)
     auto issue = [&](int mt) {
+        const bool landed = mbar_wait(smem_u32(abar + (mt & (ABUF - 1))), (ABUF == 2 ? mt >> 1 : mt) & 1);
+        ++a_waits;
+        if (!landed) return;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint64_t ad = umma_desc(smem_u32(A_s + (mt & (ABUF - 1)) * (KB * A_KB))), bd = umma_desc(smem_u32(R_s));
         constexpr uint32_t idesc = idesc_f16(NB);
@@ -166,7 +156,7 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
                             bd + (uint64_t)((kb * R_KB + ks * 32) >> 4), idesc, (kb | ks) ? 1u : 0u);
         umma_commit(smem_u32(bar));
     };
-    put_A(0);        // independent of the fold: its loads are in flight while the chain is walked
+    if (tid == 0) load_A(0);        // in flight while the chain is walked
 
     // ---- the fold (Section 3.2's recurrence applied to the query from the newest record back) ----
     const T* q = static_cast<const T*>(a.q) + (((long long)req * a.W + bb) * a.Hk + hk) * KD;
@@ -356,11 +346,10 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
             for (int e = 0; e < VEC; e += 4)
                 *reinterpret_cast<float4*>(dst + e) = make_float4(corr[c * VEC + e], corr[c * VEC + e + 1], corr[c * VEC + e + 2], corr[c * VEC + e + 3]);
         }
-        if (ABUF == 2 && mt + 1 < MT) {
+        if (ABUF == 2 && mt + 1 < MT && tid == 0) {
             // the next tile's A operand, under this tile's MMAs: its buffer was last read by tile mt - 1, whose
-            // completion every thread has waited for
-            put_A(mt + 1);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            // completion this thread has waited for
+            load_A(mt + 1);
         }
         const bool ok = mbar_wait(smem_u32(bar), mt & 1);
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -370,9 +359,8 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
             // ... and its MMAs, under this tile's epilogue: their accumulator was read out before the barrier that
             // ended the previous iteration
             if (mt + 1 < MT && tid == 0) issue(mt + 1);
-        } else if (mt + 1 < MT) {        // one A operand: free now; its MMAs go out after the barrier below
-            put_A(mt + 1);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        } else if (mt + 1 < MT && tid == 0) {        // one A operand: free now; its MMAs go out after the barrier below
+            load_A(mt + 1);
         }
         {
             uint32_t v[16];
@@ -424,6 +412,12 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
             }
         }
         if (mt + 1 < MT) __syncthreads();      // the tile is read out before the next corr rows overwrite it
+    }
+    if (tid == 0) {
+        // a CTA must not exit with bulk copies still landing in its shared memory: after a wait ran out nobody may
+        // have waited for the A operand requested last (requests use the two barriers in turn, in order)
+        for (; a_waits < a_loads; ++a_waits)
+            mbar_wait(smem_u32(abar + (a_waits & (ABUF - 1))), (ABUF == 2 ? a_waits >> 1 : a_waits) & 1);
     }
     if (failed && tid == 0) {
         if (atomicCAS(a.status, ONELA_OK, ONELA_E_TIMEOUT) == ONELA_OK) a.status[1] = (int32_t)(blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z));

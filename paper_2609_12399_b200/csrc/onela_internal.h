@@ -28,8 +28,14 @@ struct Layout {
     float* s0_scale;   // [request][layer][head]: the power of two that brings the head's largest |S_0| element into
                        // [2^11, 2^12) (1 for an all-zero or non-finite state); written with the state, read by the
                        // tensor-core kernel, whose fp16 operand it keeps in range
+    uint16_t* s0_f16;  // configurations of the tiled tensor-core kernel only: [request][layer][head] the state as that
+                       // kernel's MMA operand - fp16, times the head's operand scale, value rows padded to a multiple
+                       // of 128, in tiles of 128 rows x 64 columns (16 KB, rows of 128 bytes, 16-byte chunks swizzled
+                       // by the row) in the order [tile of rows][tile of columns]; written with the state
     size_t total_bytes;
 };
+// bytes of one head's operand copy (see Layout::s0_f16)
+inline size_t s0_f16_head_bytes(int32_t dk, int32_t dv) { return (size_t)((dv + 127) / 128) * 128 * (size_t)dk * 2; }
 
 struct BatchBases {
     int32_t base[ONELA_MAX_BATCH];  // first slot of this call's records, per request of the batch
@@ -117,6 +123,8 @@ struct TiledArgs {
     const float* beta_in;
     const float* s0;        // store slot of (req_begin, layer): [Hv][dv][dk]
     const float* s0_scale;  // operand scale of (req_begin, layer, value head 0) (see Layout)
+    const char* s0_f16;     // operand copy of (req_begin, layer, value head 0) (see Layout::s0_f16)
+    long long s0_f16_req_stride;   // bytes between consecutive requests' copies (same layer)
     char* kplane;           // key of (key head hk, slot) at kplane + ((hk * arena_slots + slot) * k_stride) elements
     char* vplane;           // value of (value head hv, slot) at vplane + ((hv * arena_slots + slot) * v_stride) elements
     float2* gates;          // [Hv][arena_slots]
@@ -168,6 +176,9 @@ cudaError_t launch_append(const void* k, const void* v, const float* alpha, cons
 // copies n_heads states of dv x dk floats and leaves each head's operand scale (see Layout::s0_scale) in scale_out
 cudaError_t launch_store_state(const float* S0_in, float* slot, float* scale_out, long long n_heads, int32_t dk, int32_t dv,
                                cudaStream_t stream);
+// the tiled kernel's operand copy of n_heads stored states (see Layout::s0_f16), from the store slots and their scales
+cudaError_t launch_pack_state(const float* slot, const float* scale, uint16_t* dst, long long n_heads, int32_t dk, int32_t dv,
+                              cudaStream_t stream);
 cudaError_t launch_export_state(const float* slot, float* S0_out, int32_t H, int32_t dk, int32_t dv, cudaStream_t stream);
 // returns cudaErrorInvalidValue with *supported = false when (dk, dv, dtype) has no instantiation
 cudaError_t launch_prefill(const void* k, const void* v, const float* alpha, const float* beta, float* slot,

@@ -4,6 +4,8 @@
 //  - store_state / prefill: fill the store slot of one (request, layer) with S_0 (Section 3.2: the
 //    post-prefill state is stored once per request), either from a caller tensor or by running Eq. 1
 //    from the zero state over the prompt.
+#include <cuda_fp16.h>
+
 #include "onela_internal.h"
 #include "onela_layout.cuh"
 
@@ -167,6 +169,37 @@ cudaError_t launch_append(const void* k, const void* v, const float* alpha, cons
     append_kernel<<<grid, warps_per_block * 32, 0, stream>>>(static_cast<const char*>(k), static_cast<const char*>(v),
                                                              alpha, beta, kv_plane, gate_plane, arena_slots, W, H,
                                                              dk * elem_bytes, dv * elem_bytes, bases);
+    return cudaGetLastError();
+}
+
+// One CTA per head: the stored state as the tiled tensor-core kernel's A operand (see Layout::s0_f16).  The rounding
+// is the one that kernel would do itself (x * scale to the nearest fp16), so results do not depend on who converts.
+__global__ void __launch_bounds__(256) pack_state_f16_kernel(const float* __restrict__ slot, const float* __restrict__ scale,
+                                                             uint16_t* __restrict__ dst, int32_t dk, int32_t dv) {
+    const long long head = blockIdx.x;
+    const float* S = slot + head * (long long)dv * dk;
+    const float sc = scale[head];
+    const int cpr = dk / 8, kb_n = dk / 64, rows = (dv + 127) / 128 * 128;     // 16-byte chunks per row, column tiles, padded rows
+    char* out = reinterpret_cast<char*>(dst) + head * (long long)rows * dk * 2;
+    for (int item = threadIdx.x; item < rows * cpr; item += blockDim.x) {
+        const int i = item / cpr, ch = item - i * cpr;
+        uint4 w = make_uint4(0u, 0u, 0u, 0u);
+        if (i < dv) {
+            const float4* p = reinterpret_cast<const float4*>(S + (long long)i * dk + ch * 8);
+            const float4 x0 = __ldg(p), x1 = __ldg(p + 1);
+            const __half2 h0 = __floats2half2_rn(x0.x * sc, x0.y * sc), h1 = __floats2half2_rn(x0.z * sc, x0.w * sc);
+            const __half2 h2 = __floats2half2_rn(x1.x * sc, x1.y * sc), h3 = __floats2half2_rn(x1.z * sc, x1.w * sc);
+            w = make_uint4(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1),
+                           *reinterpret_cast<const uint32_t*>(&h2), *reinterpret_cast<const uint32_t*>(&h3));
+        }
+        const int mt = i >> 7, row = i & 127, kb = ch >> 3, c8 = ch & 7;
+        *reinterpret_cast<uint4*>(out + ((long long)(mt * kb_n + kb) * 128 + row) * 128 + ((c8 ^ (row & 7)) << 4)) = w;
+    }
+}
+
+cudaError_t launch_pack_state(const float* slot, const float* scale, uint16_t* dst, long long n_heads, int32_t dk, int32_t dv,
+                              cudaStream_t stream) {
+    pack_state_f16_kernel<<<(unsigned)n_heads, 256, 0, stream>>>(slot, scale, dst, dk, dv);
     return cudaGetLastError();
 }
 
