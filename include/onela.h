@@ -251,8 +251,9 @@ onela_status onela_export_chains(onela_ctx* ctx, int32_t request, int32_t* slots
 onela_status onela_poll_device_status(onela_ctx* ctx, int32_t* code_host, int32_t* detail_host);
 
 /* Resident bytes (host bookkeeping; Section 4.4 reports the same three quantities): the stored S_0
- * matrices, the records appended so far (slots * heads * record bytes * layers), and the live
- * ancestry rows. */
+ * matrices (fp32; configurations of the tiled tensor-core kernel keep every state a second time as that kernel's
+ * fp16 operand, half as many bytes again, not counted here), the records appended so far (slots * heads * record
+ * bytes * layers), and the live ancestry rows. */
 onela_status onela_get_stats(const onela_ctx* ctx, int64_t* s0_bytes_host, int64_t* arena_bytes_used_host,
                              int64_t* index_bytes_host);
 
