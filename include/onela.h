@@ -25,7 +25,7 @@
  *    host object released by onela_destroy(), which never touches the workspace.
  *  - `stream` is a cudaStream_t passed as void*.  Every call is asynchronous and ordered on that
  *    stream; inputs may be reused as soon as the stream has passed the call.  Only
- *    onela_poll_device_status() synchronises.  The tensor-core decode kernel is launched with programmatic
+ *    onela_poll_device_status() synchronises.  The warp-specialised tensor-core decode kernel is launched with programmatic
  *    stream serialisation: it may start while the previous kernel of the stream drains, but it reads only its
  *    own shared-state store before it has waited for that kernel's completion, so stream order holds for every
  *    tensor the caller passes.  A caller kernel that follows it AND is itself launched with programmatic stream
