@@ -261,8 +261,10 @@ def test_wide_values_on_the_tensor_cores(dv, fused, out_dtype):
                 assert torch.equal(gates[h, base:base + wl.W, 1], tk["beta"][:, h])
 
 
-def test_alpha1_beta0_reduces_to_matvec_on_gpu():
-    wl = CFG1.scaled(H=2, W=64, D=3, prompt_len=64)
+@pytest.mark.parametrize("dk,dv,dtype", [(128, 128, "bf16"), (64, 64, "bf16"), (256, 512, "fp32")])
+def test_alpha1_beta0_reduces_to_matvec_on_gpu(dk, dv, dtype):
+    """On both tensor-core kernels (the second and third shapes run the tiled one)."""
+    wl = CFG1.scaled(H=2, dk=dk, dv=dv, dtype=dtype, W=64, D=3, prompt_len=64)
     case = make_case(wl)
     for tk in case["tok"].values():
         tk["alpha"].fill_(1.0)
@@ -273,8 +275,9 @@ def test_alpha1_beta0_reduces_to_matvec_on_gpu():
         assert rel_l2(o.numpy(), want).max() <= REL_L2_BAR
 
 
-def test_shared_chains_give_identical_outputs_on_gpu():
-    wl = CFG1.scaled(H=2, W=64, D=3, prompt_len=64)
+@pytest.mark.parametrize("dk,dv,dtype", [(128, 128, "bf16"), (64, 64, "fp32"), (256, 256, "bf16")])
+def test_shared_chains_give_identical_outputs_on_gpu(dk, dv, dtype):
+    wl = CFG1.scaled(H=2, dk=dk, dv=dv, dtype=dtype, W=64, D=3, prompt_len=64)
     case = make_case(wl)
     case["parents"][(0, 2)] = torch.full((64,), 5, dtype=torch.int32)
     for n in ("k", "v", "alpha", "beta"):
@@ -423,12 +426,13 @@ def test_batched_state_store_equals_the_single_calls():
     assert ctx.onela_poll_device_status() == (0, 0)
 
 
+@pytest.mark.parametrize("dk,dv,dtype", [(128, 128, "bf16"), (256, 256, "fp32")])
 @pytest.mark.parametrize("s0_unit,q_unit", [(1e-6, 1.0), (3e4, 1.0), (1.0, 1e-5), (1.0, 2e3), (1e-5, 1e-4), (1e4, 50.0)])
-def test_tensor_core_operands_keep_their_precision_at_any_scale(s0_unit, q_unit):
+def test_tensor_core_operands_keep_their_precision_at_any_scale(s0_unit, q_unit, dk, dv, dtype):
     """The tensor-core kernel feeds fp16 operands; per-head and per-beam powers of two keep them inside the format's
     range, so states and queries far from unit scale decode as accurately as unit-scale ones (states of 1e-6 or
     queries of 1e-5 would otherwise sink into fp16's subnormals, states of 3e4 x 128 terms overflow it)."""
-    wl = CFG1.scaled(H=2, W=70, D=3, prompt_len=48, parents="zipf", zipf_s=1.5, seed=4242)
+    wl = CFG1.scaled(H=2, dk=dk, dv=dv, dtype=dtype, W=70, D=3, prompt_len=48, parents="zipf", zipf_s=1.5, seed=4242)
     case = make_case(wl)
     for key in case["S0"]:
         case["S0"][key] = (case["S0"][key].double() * s0_unit).float()
@@ -441,6 +445,23 @@ def test_tensor_core_operands_keep_their_precision_at_any_scale(s0_unit, q_unit)
         ref, _ = run_oracle(case)
         for key, o in outs.items():
             assert rel_l2(o.numpy(), ref[key]).max() <= REL_L2_BAR
+
+
+@pytest.mark.parametrize("key_norm,beta_lo,beta_hi", [(2.5, 0.5, 1.0), (1.0, 1.0, 2.0), (3.0, 0.6, 0.9)])
+def test_keys_and_gates_outside_the_stable_range_on_the_tiled_kernel(key_norm, beta_lo, beta_hi):
+    """The same inputs through the tiled tensor-core kernel (its operand rows are scaled by their exact largest element)."""
+    wl = CFG1.scaled(H=2, dk=64, dv=64, dtype="fp32", W=100, D=8, prompt_len=32, parents="zipf", zipf_s=1.5, seed=607)
+    case = make_case(wl)
+    g = torch.Generator().manual_seed(8)
+    for key, tok in case["tok"].items():
+        tok["k"] = (tok["k"].double() * key_norm).to(tok["k"].dtype)
+        tok["beta"] = (beta_lo + (beta_hi - beta_lo) * torch.rand(tok["beta"].shape, generator=g)).float()
+    ref, _ = run_oracle(case)
+    outs, _, ctx = run_library(case, out_dtype="fp32", fused=True)
+    assert ctx.onela_uses_tensor_core_path() == 2 and ctx.onela_poll_device_status() == (0, 0)
+    for key, o in outs.items():
+        assert np.isfinite(o.numpy()).all()
+        assert rel_l2(o.numpy(), ref[key]).max() <= REL_L2_BAR, key
 
 
 @pytest.mark.parametrize("key_norm,beta_lo,beta_hi", [(2.5, 0.5, 1.0), (1.0, 1.0, 2.0), (3.0, 0.6, 0.9)])
