@@ -177,13 +177,12 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
     // for the whole chain instead of one per level); deeper levels are looked up when they are reached.
     const int old = a.depth - 1;           // records older than the beam's own: levels old - 1 .. 0
     const int32_t my_slot = g < old ? __ldg(table + (long long)g * a.max_beam + bb) : 0;
-    auto slot_of = [&](int level) -> int32_t {       // level < old; unit-uniform
-        const int32_t x = __shfl_sync(0xffffffffu, my_slot, level & (G - 1), G);
-        return level < G ? x : __ldg(table + (long long)level * a.max_beam + bb);
-    };
+    // (two look-ups, used by two runs of the chain walk: one loop with a branch between them costs every level a
+    // dozen instructions, taken or not)
+    auto slot_near = [&](int level) -> int32_t { return __shfl_sync(0xffffffffu, my_slot, level, G); };          // level < G
+    auto slot_far = [&](int level) -> int32_t { return __ldg(table + (long long)level * a.max_beam + bb); };    // level >= G
     struct Raw { uint4 k[CK], v[CV]; float2 gate; };          // this lane's share of a record, as stored
-    auto fetch = [&](int level) -> Raw {                      // an older record, from the arena
-        const long long slot = slot_of(level);
+    auto fetch_slot = [&](long long slot) -> Raw {            // an older record, from the arena
         const uint4* kp = reinterpret_cast<const uint4*>(kplane + slot * a.k_stride) + g;
         const uint4* vp = reinterpret_cast<const uint4*>(vplane + slot * a.v_stride) + g;
         Raw x;
@@ -274,27 +273,42 @@ __global__ void __launch_bounds__(tiled_beams<KD, VD>() * G, tiled_min_ctas<KD, 
     // Narrow records are fetched one level ahead of their fold (the chain is a string of dependent loads otherwise);
     // wide ones would not fit in the registers twice.
     constexpr bool AHEAD = KD + VD <= 256;
-    if constexpr (DELTA) {                 // the replay runs over the older records only
+    const int near_top = min(old, G) - 1;        // levels near_top .. 0: slots among the lanes'; old - 1 .. G: in memory
+    if constexpr (DELTA) {                       // the replay runs over the older records only
         if (old > 0) {
-            Raw x = fetch(old - 1);
-            for (int level = old - 2; level >= 0; --level) {
-                const Raw next = fetch(level);
+            Raw x = old > G ? fetch_slot(slot_far(old - 1)) : fetch_slot(slot_near(old - 1));
+            for (int level = old - 2; level >= G; --level) {
+                const Raw next = fetch_slot(slot_far(level));
+                fold(x);
+                x = next;
+            }
+            for (int level = min(old - 2, near_top); level >= 0; --level) {
+                const Raw next = fetch_slot(slot_near(level));
                 fold(x);
                 x = next;
             }
             fold(x);
         }
     } else if constexpr (AHEAD) {
-        for (int level = old - 1; level >= 0; --level) {
-            const Raw next = fetch(level);
+        for (int level = old - 1; level >= G; --level) {
+            const Raw next = fetch_slot(slot_far(level));
+            fold(cur);
+            cur = next;
+        }
+        for (int level = near_top; level >= 0; --level) {
+            const Raw next = fetch_slot(slot_near(level));
             fold(cur);
             cur = next;
         }
         fold(cur);
     } else {
         fold(cur);
-        for (int level = old - 1; level >= 0; --level) {
-            const Raw x = fetch(level);
+        for (int level = old - 1; level >= G; --level) {
+            const Raw x = fetch_slot(slot_far(level));
+            fold(x);
+        }
+        for (int level = near_top; level >= 0; --level) {
+            const Raw x = fetch_slot(slot_near(level));
             fold(x);
         }
     }
